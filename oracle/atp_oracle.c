@@ -1,0 +1,446 @@
+/*
+ * CPU oracle for the ATP (attention on top principal keys) prefill path.
+ *
+ * TEST INFRASTRUCTURE ONLY. This file is the slow, plain, double-precision
+ * statement of what the path computes; it exists so that tests and the
+ * benchmark's CPU baseline have something to compare and time against. It
+ * shares no code with the CUDA library and the library never calls it.
+ *
+ * Everything is row-major, double precision, naive loops. No BLAS / LAPACK.
+ * OpenMP is used only over independent work (disjoint Jacobi pairs, output
+ * rows); results do not depend on the thread count.
+ *
+ * What each function follows (paper sections / equations):
+ *   oracle_svd_jacobi        SVD of the hidden state, Eq. 3
+ *   oracle_principal_basis   X = U X', X' = [sigma_1 v_1 .. sigma_r v_r], Eq. 5 and Sec. 4.2;
+ *                            it is also the minimiser of Eq. 9 (Eckart-Young)
+ *   oracle_attention         Q,K,V = U {Q',K',V'} (Eq. 6), then attention of every query on the
+ *                            r principal keys/values: the procedure of Eq. 1 with K', V' in place
+ *                            of K, V (Sec. 4.1 closing paragraph, Fig. 2 caption)
+ *   oracle_lowrank_linear    linear layers applied to the r-row representation (Sec. 1, Sec. 4.3)
+ *   oracle_norm              the "Norm" box of Fig. 3 (RMSNorm / LayerNorm, unit gain)
+ *   oracle_alternating_svd   Algorithm 1 (appendix B), the paper's own approximate extraction
+ *   oracle_svd_entropy       Eq. 4
+ *
+ * Parity status: every function here is pinned by tests/test_oracle_pins.py
+ * (closed forms, planted spectra, Eckart-Young, reduction to textbook
+ * attention, brute force on tiny inputs, LAPACK cross-check). The one value
+ * that stays unpinned end to end is O on inputs whose cut r falls inside a
+ * cluster of equal singular values: there the basis itself is not unique
+ * ("parity unpinned" for that case only; stage-wise parity still holds).
+ */
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+#include <stdint.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define ORACLE_API __attribute__((visibility("default")))
+
+ORACLE_API int oracle_num_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* ------------------------------------------------------------------ */
+/* One-sided (Hestenes) Jacobi SVD, Eq. 3.                            */
+/*                                                                    */
+/* Works on n "vectors" a_0..a_{n-1} of length m held as the rows of  */
+/* A (n x m). Plane rotations are applied to pairs of vectors until   */
+/* all pairs are orthogonal; the same rotations are accumulated in G  */
+/* (n x n, starts as identity, row i follows vector i). At the end    */
+/* a_i = sigma_i * w_i with w_i orthonormal and row i of G is the     */
+/* matching singular vector on the other side.                        */
+/* ------------------------------------------------------------------ */
+static int jacobi_rows(double *A, double *G, int n, int m, double tol, int max_sweeps)
+{
+    int np = n + (n & 1);              /* pad to even for the round-robin schedule */
+    int *idx = (int *)malloc(sizeof(int) * np);
+    for (int i = 0; i < np; ++i) idx[i] = i;
+    int sweeps = 0;
+    for (; sweeps < max_sweeps; ++sweeps) {
+        double worst = 0.0;
+        /* largest squared norm: vectors far below it are treated as zero */
+        double nmax = 0.0;
+        for (int i = 0; i < n; ++i) {
+            double s = 0.0;
+            for (int k = 0; k < m; ++k) s += A[(size_t)i * m + k] * A[(size_t)i * m + k];
+            if (s > nmax) nmax = s;
+        }
+        double tiny = nmax * 1e-300;
+        for (int round = 0; round < np - 1; ++round) {
+#pragma omp parallel for schedule(dynamic, 4) reduction(max : worst)
+            for (int t = 0; t < np / 2; ++t) {
+                int p = idx[t], q = idx[np - 1 - t];
+                if (p >= n || q >= n) continue;
+                if (p > q) { int tmp = p; p = q; q = tmp; }
+                double *ap = A + (size_t)p * m, *aq = A + (size_t)q * m;
+                double alpha = 0.0, beta = 0.0, gamma = 0.0;
+                for (int k = 0; k < m; ++k) {
+                    alpha += ap[k] * ap[k];
+                    beta += aq[k] * aq[k];
+                    gamma += ap[k] * aq[k];
+                }
+                if (alpha <= tiny || beta <= tiny) continue;   /* a zero vector is orthogonal to all */
+                double off = fabs(gamma) / sqrt(alpha * beta);
+                if (off > worst) worst = off;
+                if (off < tol) continue;
+                double zeta = (beta - alpha) / (2.0 * gamma);
+                double tt = (zeta >= 0 ? 1.0 : -1.0) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
+                double c = 1.0 / sqrt(1.0 + tt * tt), s = c * tt;
+                for (int k = 0; k < m; ++k) {
+                    double x = ap[k], y = aq[k];
+                    ap[k] = c * x - s * y;
+                    aq[k] = s * x + c * y;
+                }
+                double *gp = G + (size_t)p * n, *gq = G + (size_t)q * n;
+                for (int k = 0; k < n; ++k) {
+                    double x = gp[k], y = gq[k];
+                    gp[k] = c * x - s * y;
+                    gq[k] = s * x + c * y;
+                }
+            }
+            /* rotate the schedule: position 0 fixed, the rest shift by one */
+            int last = idx[np - 1];
+            for (int i = np - 1; i > 1; --i) idx[i] = idx[i - 1];
+            idx[1] = last;
+        }
+        if (worst < tol) { ++sweeps; break; }
+    }
+    free(idx);
+    return sweeps;
+}
+
+/*
+ * X (L x d) = U diag(S) Vt, n = min(L, d); U is L x n, Vt is n x d, S descending.
+ * Returns the number of sweeps used (60 if the tolerance was not met).
+ * Singular vectors that belong to sigma = 0 are completed to an orthonormal set.
+ */
+ORACLE_API int oracle_svd_jacobi(const double *X, int L, int d, double *U, double *S, double *Vt)
+{
+    int n = L < d ? L : d;
+    int m = L < d ? d : L;
+    /* vectors to rotate: rows of X if L <= d, else rows of X^T (columns of X) */
+    double *A = (double *)malloc(sizeof(double) * (size_t)n * m);
+    double *G = (double *)calloc((size_t)n * n, sizeof(double));
+    if (L <= d) {
+        memcpy(A, X, sizeof(double) * (size_t)L * d);
+    } else {
+        for (int i = 0; i < L; ++i)
+            for (int j = 0; j < d; ++j) A[(size_t)j * L + i] = X[(size_t)i * d + j];
+    }
+    for (int i = 0; i < n; ++i) G[(size_t)i * n + i] = 1.0;
+    int sweeps = jacobi_rows(A, G, n, m, 1e-14, 60);
+
+    double *sig = (double *)malloc(sizeof(double) * n);
+    int *ord = (int *)malloc(sizeof(int) * n);
+    for (int i = 0; i < n; ++i) {
+        double s = 0.0;
+        for (int k = 0; k < m; ++k) s += A[(size_t)i * m + k] * A[(size_t)i * m + k];
+        sig[i] = sqrt(s);
+        ord[i] = i;
+    }
+    /* sort descending (stable insertion sort) */
+    for (int i = 1; i < n; ++i) {
+        int o = ord[i], j = i - 1;
+        while (j >= 0 && sig[ord[j]] < sig[o]) { ord[j + 1] = ord[j]; --j; }
+        ord[j + 1] = o;
+    }
+    double smax = n > 0 ? sig[ord[0]] : 0.0;
+    /* W rows: normalised rotated vectors (length m); zero ones completed by Gram-Schmidt.
+       Gc rows: the accumulated rotations in sorted order; they are orthonormal already. */
+    double *W = (double *)malloc(sizeof(double) * (size_t)n * m);
+    for (int a = 0; a < n; ++a) {
+        int i = ord[a];
+        double *w = W + (size_t)a * m;
+        S[a] = sig[i];
+        if (sig[i] > smax * 1e-150 && sig[i] > 0.0) {
+            for (int k = 0; k < m; ++k) w[k] = A[(size_t)i * m + k] / sig[i];
+        } else {
+            S[a] = 0.0;
+            /* try unit vectors until one has a component outside the span found so far;
+               zero vectors sort last, so every earlier row of W is already final */
+            for (int e = 0; e < m; ++e) {
+                for (int k = 0; k < m; ++k) w[k] = (k == e) ? 1.0 : 0.0;
+                for (int rep = 0; rep < 2; ++rep)
+                    for (int b = 0; b < a; ++b) {
+                        double *wb = W + (size_t)b * m, dot = 0.0;
+                        for (int k = 0; k < m; ++k) dot += wb[k] * w[k];
+                        for (int k = 0; k < m; ++k) w[k] -= dot * wb[k];
+                    }
+                double nr = 0.0;
+                for (int k = 0; k < m; ++k) nr += w[k] * w[k];
+                nr = sqrt(nr);
+                if (nr > 0.5 / sqrt((double)m + 1.0)) {
+                    for (int k = 0; k < m; ++k) w[k] /= nr;
+                    break;
+                }
+            }
+        }
+    }
+    /* map back: L <= d: W rows are v_i (length d), G rows are u_i (length L = n)
+                 L >  d: W rows are u_i (length L), G rows are v_i (length d = n) */
+    if (L <= d) {
+        for (int a = 0; a < n; ++a) {
+            for (int k = 0; k < d; ++k) Vt[(size_t)a * d + k] = W[(size_t)a * m + k];
+            for (int k = 0; k < L; ++k) U[(size_t)k * n + a] = G[(size_t)ord[a] * n + k];
+        }
+    } else {
+        for (int a = 0; a < n; ++a) {
+            for (int k = 0; k < L; ++k) U[(size_t)k * n + a] = W[(size_t)a * m + k];
+            for (int k = 0; k < d; ++k) Vt[(size_t)a * d + k] = G[(size_t)ord[a] * n + k];
+        }
+    }
+    free(A); free(G); free(sig); free(ord); free(W);
+    return sweeps;
+}
+
+/* ------------------------------------------------------------------ */
+/* Principal basis: Eq. 5 with U = first r left singular vectors and   */
+/* X' = U^T X = [sigma_1 v_1; ...; sigma_r v_r] (Sec. 4.2).            */
+/* Sign convention (the paper fixes none): each column of U_r is       */
+/* flipped so that its entries sum to >= 0 (the zeroth-order weight    */
+/* 1.U of Eq. 8 is then non-negative); when that sum is within         */
+/* 1e-6*sqrt(L) of zero the largest-magnitude entry of the matching    */
+/* row of X_r is made positive instead.                                */
+/* sigma_all (nullable) receives all min(L,d) singular values.         */
+/* ------------------------------------------------------------------ */
+ORACLE_API int oracle_principal_basis(const double *X, int L, int d, int r, double *U_r, double *X_r,
+                                      double *sigma, double *sigma_all)
+{
+    int n = L < d ? L : d;
+    if (r < 1 || r > n) return -1;
+    double *U = (double *)malloc(sizeof(double) * (size_t)L * n);
+    double *S = (double *)malloc(sizeof(double) * n);
+    double *Vt = (double *)malloc(sizeof(double) * (size_t)n * d);
+    int sweeps = oracle_svd_jacobi(X, L, d, U, S, Vt);
+    for (int i = 0; i < L; ++i)
+        for (int a = 0; a < r; ++a) U_r[(size_t)i * r + a] = U[(size_t)i * n + a];
+    if (sigma) for (int a = 0; a < r; ++a) sigma[a] = S[a];
+    if (sigma_all) for (int a = 0; a < n; ++a) sigma_all[a] = S[a];
+    /* X_r = U_r^T X, written as the product it is defined by */
+#pragma omp parallel for schedule(static)
+    for (int a = 0; a < r; ++a) {
+        double *row = X_r + (size_t)a * d;
+        for (int k = 0; k < d; ++k) row[k] = 0.0;
+        for (int i = 0; i < L; ++i) {
+            double u = U_r[(size_t)i * r + a];
+            const double *x = X + (size_t)i * d;
+            for (int k = 0; k < d; ++k) row[k] += u * x[k];
+        }
+    }
+    for (int a = 0; a < r; ++a) {
+        double sum = 0.0;
+        for (int i = 0; i < L; ++i) sum += U_r[(size_t)i * r + a];
+        int flip;
+        if (fabs(sum) >= 1e-6 * sqrt((double)L)) {
+            flip = sum < 0.0;
+        } else {
+            double best = 0.0; int bk = 0;
+            for (int k = 0; k < d; ++k)
+                if (fabs(X_r[(size_t)a * d + k]) > best) { best = fabs(X_r[(size_t)a * d + k]); bk = k; }
+            flip = X_r[(size_t)a * d + bk] < 0.0;
+        }
+        if (flip) {
+            for (int i = 0; i < L; ++i) U_r[(size_t)i * r + a] = -U_r[(size_t)i * r + a];
+            for (int k = 0; k < d; ++k) X_r[(size_t)a * d + k] = -X_r[(size_t)a * d + k];
+        }
+    }
+    free(U); free(S); free(Vt);
+    return sweeps;
+}
+
+/* C (M x N) = A (M x K) * B (K x N), all row-major */
+static void matmul(const double *A, const double *B, double *C, int M, int K, int N)
+{
+#pragma omp parallel for schedule(static)
+    for (int i = 0; i < M; ++i) {
+        double *c = C + (size_t)i * N;
+        for (int j = 0; j < N; ++j) c[j] = 0.0;
+        for (int k = 0; k < K; ++k) {
+            double a = A[(size_t)i * K + k];
+            const double *b = B + (size_t)k * N;
+            for (int j = 0; j < N; ++j) c[j] += a * b[j];
+        }
+    }
+}
+
+/* ------------------------------------------------------------------ */
+/* Attention of all L queries on the r principal keys / values.        */
+/*   Q' = X_r W_Q, K' = X_r W_K, V' = X_r W_V                (Eq. 6)   */
+/*   Q  = U_r Q'        (q_mode 0, Eq. 6)   or   Q = X W_Q  (q_mode 1) */
+/*   per head h (column block of width d_h = dp / heads):              */
+/*   O_h = Softmax(Q_h K'_h^T * scale) V'_h   (Eq. 1 on r keys)        */
+/* scale <= 0 selects 1/sqrt(d_h). X may be NULL when q_mode == 0.     */
+/* ------------------------------------------------------------------ */
+ORACLE_API int oracle_attention(const double *X, const double *U_r, const double *X_r,
+                                const double *W_Q, const double *W_K, const double *W_V,
+                                int L, int d, int dp, int r, int heads, int q_mode, double scale,
+                                double *O)
+{
+    if (heads < 1 || dp % heads != 0) return -1;
+    if (q_mode == 1 && !X) return -1;
+    int dh = dp / heads;
+    if (scale <= 0.0) scale = 1.0 / sqrt((double)dh);
+    double *Qp = (double *)malloc(sizeof(double) * (size_t)r * dp);
+    double *Kp = (double *)malloc(sizeof(double) * (size_t)r * dp);
+    double *Vp = (double *)malloc(sizeof(double) * (size_t)r * dp);
+    double *Q = (double *)malloc(sizeof(double) * (size_t)L * dp);
+    matmul(X_r, W_K, Kp, r, d, dp);
+    matmul(X_r, W_V, Vp, r, d, dp);
+    if (q_mode == 0) {
+        matmul(X_r, W_Q, Qp, r, d, dp);
+        matmul(U_r, Qp, Q, L, r, dp);
+    } else {
+        matmul(X, W_Q, Q, L, d, dp);
+    }
+#pragma omp parallel
+    {
+        double *s = (double *)malloc(sizeof(double) * (size_t)r);
+#pragma omp for schedule(static) collapse(2)
+        for (int l = 0; l < L; ++l) {
+            for (int h = 0; h < heads; ++h) {
+                const double *q = Q + (size_t)l * dp + (size_t)h * dh;
+                double mx = -INFINITY;
+                for (int i = 0; i < r; ++i) {
+                    const double *k = Kp + (size_t)i * dp + (size_t)h * dh;
+                    double acc = 0.0;
+                    for (int c = 0; c < dh; ++c) acc += q[c] * k[c];
+                    s[i] = acc * scale;
+                    if (s[i] > mx) mx = s[i];
+                }
+                double den = 0.0;
+                for (int i = 0; i < r; ++i) { s[i] = exp(s[i] - mx); den += s[i]; }
+                double *o = O + (size_t)l * dp + (size_t)h * dh;
+                for (int c = 0; c < dh; ++c) o[c] = 0.0;
+                for (int i = 0; i < r; ++i) {
+                    double p = s[i] / den;
+                    const double *v = Vp + (size_t)i * dp + (size_t)h * dh;
+                    for (int c = 0; c < dh; ++c) o[c] += p * v[c];
+                }
+            }
+        }
+        free(s);
+    }
+    free(Qp); free(Kp); free(Vp); free(Q);
+    return 0;
+}
+
+static double gelu_erf(double x) { return 0.5 * x * (1.0 + erf(x / sqrt(2.0))); }
+static double silu(double x) { return x / (1.0 + exp(-x)); }
+
+/* ------------------------------------------------------------------ */
+/* Low-rank linear layer: Y = act(U_r (X_r W) + bias)                  */
+/*   act 0: none, 1: GELU (erf form), 2: SwiGLU with a second weight   */
+/*   W_gate: Y = silu(U_r X_r W_gate) * (U_r X_r W)                    */
+/* bias (length d_out) and W_gate are nullable.                        */
+/* ------------------------------------------------------------------ */
+ORACLE_API int oracle_lowrank_linear(const double *U_r, const double *X_r, const double *W,
+                                     const double *bias, const double *W_gate, int act,
+                                     int L, int r, int d_in, int d_out, double *Y)
+{
+    if (act == 2 && !W_gate) return -1;
+    double *T = (double *)malloc(sizeof(double) * (size_t)r * d_out);
+    matmul(X_r, W, T, r, d_in, d_out);
+    matmul(U_r, T, Y, L, r, d_out);
+    if (bias)
+        for (int i = 0; i < L; ++i)
+            for (int j = 0; j < d_out; ++j) Y[(size_t)i * d_out + j] += bias[j];
+    if (act == 1) {
+        for (size_t i = 0; i < (size_t)L * d_out; ++i) Y[i] = gelu_erf(Y[i]);
+    } else if (act == 2) {
+        double *Gt = (double *)malloc(sizeof(double) * (size_t)L * d_out);
+        matmul(X_r, W_gate, T, r, d_in, d_out);
+        matmul(U_r, T, Gt, L, r, d_out);
+        for (size_t i = 0; i < (size_t)L * d_out; ++i) Y[i] = silu(Gt[i]) * Y[i];
+        free(Gt);
+    }
+    free(T);
+    return 0;
+}
+
+/* ------------------------------------------------------------------ */
+/* "Norm" box of Fig. 3, unit gain, optional residual added first.     */
+/*   kind 0: RMSNorm  x / sqrt(mean(x^2) + eps)                        */
+/*   kind 1: LayerNorm (x - mean) / sqrt(var + eps)                    */
+/* ------------------------------------------------------------------ */
+ORACLE_API int oracle_norm(const double *X, const double *residual, int kind, double eps,
+                           int L, int d, double *Y)
+{
+    for (int i = 0; i < L; ++i) {
+        const double *x = X + (size_t)i * d;
+        double *y = Y + (size_t)i * d;
+        for (int k = 0; k < d; ++k) y[k] = x[k] + (residual ? residual[(size_t)i * d + k] : 0.0);
+        double mean = 0.0;
+        if (kind == 1) {
+            for (int k = 0; k < d; ++k) mean += y[k];
+            mean /= d;
+        }
+        double var = 0.0;
+        for (int k = 0; k < d; ++k) var += (y[k] - mean) * (y[k] - mean);
+        var /= d;
+        double inv = 1.0 / sqrt(var + eps);
+        for (int k = 0; k < d; ++k) y[k] = (y[k] - mean) * inv;
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------ */
+/* Algorithm 1 (appendix B): alternating rank-1 fits with deflation.   */
+/* For each component: `inner` rounds of u = X v / |v|^2,              */
+/* v = X^T u / |u|^2 starting from the given v0 (r x d, row i is the   */
+/* start for component i), then X <- X - u v^T. After the rounds the   */
+/* pair is rescaled so that u has unit norm and the scale sits in v    */
+/* (Sec. 4.2: sigma is fused into v). Outputs U (L x r), Xp (r x d).   */
+/* ------------------------------------------------------------------ */
+ORACLE_API int oracle_alternating_svd(const double *X, int L, int d, int r, const double *v0,
+                                      int inner, double *U, double *Xp)
+{
+    double *R = (double *)malloc(sizeof(double) * (size_t)L * d);
+    double *u = (double *)malloc(sizeof(double) * L);
+    double *v = (double *)malloc(sizeof(double) * d);
+    memcpy(R, X, sizeof(double) * (size_t)L * d);
+    for (int i = 0; i < r; ++i) {
+        for (int k = 0; k < d; ++k) v[k] = v0[(size_t)i * d + k];
+        for (int l = 0; l < L; ++l) u[l] = 0.0;
+        for (int j = 0; j < inner; ++j) {
+            double vv = 0.0;
+            for (int k = 0; k < d; ++k) vv += v[k] * v[k];
+            for (int l = 0; l < L; ++l) {
+                double acc = 0.0;
+                for (int k = 0; k < d; ++k) acc += R[(size_t)l * d + k] * v[k];
+                u[l] = vv > 0.0 ? acc / vv : 0.0;
+            }
+            double uu = 0.0;
+            for (int l = 0; l < L; ++l) uu += u[l] * u[l];
+            for (int k = 0; k < d; ++k) v[k] = 0.0;
+            for (int l = 0; l < L; ++l)
+                for (int k = 0; k < d; ++k) v[k] += R[(size_t)l * d + k] * u[l];
+            for (int k = 0; k < d; ++k) v[k] = uu > 0.0 ? v[k] / uu : 0.0;
+        }
+        for (int l = 0; l < L; ++l)
+            for (int k = 0; k < d; ++k) R[(size_t)l * d + k] -= u[l] * v[k];
+        double un = 0.0;
+        for (int l = 0; l < L; ++l) un += u[l] * u[l];
+        un = sqrt(un);
+        for (int l = 0; l < L; ++l) U[(size_t)l * r + i] = un > 0.0 ? u[l] / un : 0.0;
+        for (int k = 0; k < d; ++k) Xp[(size_t)i * d + k] = v[k] * un;
+    }
+    free(R); free(u); free(v);
+    return 0;
+}
+
+/* Eq. 4: mu = -log2( sum_i sbar_i^2 ), sbar_i = sigma_i / sum_j sigma_j. */
+ORACLE_API double oracle_svd_entropy(const double *sigma, int n)
+{
+    double tot = 0.0, acc = 0.0;
+    for (int i = 0; i < n; ++i) tot += sigma[i];
+    if (tot <= 0.0) return 0.0;
+    for (int i = 0; i < n; ++i) acc += (sigma[i] / tot) * (sigma[i] / tot);
+    return -log2(acc);
+}
