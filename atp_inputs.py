@@ -100,6 +100,8 @@ def finish(x, dtype):
     """Round once to the workload dtype; keep as float64 for the oracle."""
     if dtype == "bf16":
         return round_to_bf16(x).astype(np.float64)
+    if dtype == "f64":
+        return np.asarray(x, dtype=np.float64)
     return np.asarray(x, dtype=np.float32).astype(np.float64)
 
 
