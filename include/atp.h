@@ -1,0 +1,174 @@
+/*
+ * libatp -- the per-layer prefill hot path of ATP (attention on top principal keys)
+ * for NVIDIA B200 (sm_100a).
+ *
+ * The three main calls follow the paper's statement of the problem:
+ *
+ *   atp_principal_basis(X, r)                     -> (U_r, X_r)   Eq. 3, Eq. 5, Sec. 4.2, Eq. 9
+ *   atp_attention(X, U_r, X_r, W_Q, W_K, W_V, h)  -> O            Eq. 6, Eq. 1 on r principal keys
+ *   atp_lowrank_linear(U_r, X_r, W)               -> Y            Sec. 4.3 (linear layers on the
+ *                                                                 r-row representation)
+ *   atp_input_norm(X [, residual])                -> X_n          the "Norm" box of Fig. 3
+ *
+ * General conventions
+ *   - Plain C ABI. Every matrix is row-major with a leading dimension `ld` in elements.
+ *   - Every `data` pointer is DEVICE memory owned by the caller; every pointer inside
+ *     `atp_seqs` and every options struct is HOST memory, read during the call only.
+ *   - The library allocates no tensors. Scratch memory is a caller-owned device buffer handed
+ *     over with atp_set_workspace(); its required size comes from atp_workspace_bytes().
+ *     atp_create() allocates one small device status word and a pinned staging page, freed by
+ *     atp_destroy().
+ *   - Calls only enqueue work on the context's stream (atp_set_stream) and return; they never
+ *     synchronise, except atp_poll_device_status().
+ *   - Errors the host can detect are returned at once and nothing is launched. Conditions only
+ *     the device can see (a Jacobi iteration that hit its sweep limit, a bounded wait that ran
+ *     out, a value outside the representable range) are recorded in the status word and read
+ *     back by atp_poll_device_status(); no kernel traps or spins without bound.
+ *   - dtype ATP_BF16 needs 16-byte aligned base pointers and `ld` a multiple of 8; otherwise
+ *     ATP_ERR_INVALID_ARG is returned.
+ *
+ * Batches and ragged lengths: several independent sequences are packed row-wise.
+ *   X, U_r, O, Y hold sum(L_b) rows; sequence b owns rows [row_off[b], row_off[b+1]).
+ *   X_r holds sum(r_b) rows;         sequence b owns rows [rank_off[b], rank_off[b+1]).
+ *   U_r has at least max(r_b) columns; sequence b uses the first r_b of them.
+ *   sigma holds sum(r_b) floats laid out like the rows of X_r.
+ * batch = 1 with row_off = {0, L} is the plain (X, r) call of the paper.
+ */
+#ifndef ATP_H_
+#define ATP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    ATP_OK = 0,
+    ATP_ERR_INVALID_ARG = 1,
+    ATP_ERR_INVALID_RANK = 2,
+    ATP_ERR_UNSUPPORTED_DTYPE = 3,
+    ATP_ERR_WORKSPACE_TOO_SMALL = 4,
+    ATP_ERR_CUDA = 5,
+    ATP_ERR_NOT_CONVERGED = 6,
+    ATP_ERR_TIMEOUT = 7,
+    ATP_ERR_RANGE = 8
+} atp_status;
+
+typedef enum { ATP_F32 = 0, ATP_BF16 = 1 } atp_dtype;
+
+/* Device matrix, row-major; element (i, j) lives at data + (i*ld + j) * sizeof(dtype). */
+typedef struct {
+    void *data;
+    atp_dtype dtype;
+    int64_t rows, cols, ld;
+} atp_mat;
+
+/* Packed batch description; all three arrays are HOST memory. */
+typedef struct {
+    int32_t batch;
+    const int32_t *row_off;   /* batch + 1 entries: rows of X / U_r / O / Y per sequence */
+    const int32_t *rank;      /* batch entries: r_b                                       */
+    const int32_t *rank_off;  /* batch + 1 entries: rows of X_r per sequence               */
+} atp_seqs;
+
+typedef enum { ATP_OP_BASIS = 0, ATP_OP_ATTENTION = 1, ATP_OP_LINEAR = 2, ATP_OP_NORM = 3 } atp_op;
+typedef enum { ATP_Q_LOWRANK = 0, ATP_Q_FULL = 1 } atp_q_mode;
+typedef enum { ATP_ACT_NONE = 0, ATP_ACT_GELU = 1, ATP_ACT_SWIGLU = 2 } atp_act;
+typedef enum { ATP_NORM_RMS = 0, ATP_NORM_LAYER = 1 } atp_norm_kind;
+
+/* Options. Set struct_size = sizeof(the struct); a NULL options pointer selects the defaults
+ * (every numeric field below also treats 0 / negative as "default" where noted). */
+typedef struct {
+    uint32_t struct_size;
+    int32_t oversample;    /* extra columns of the range finder; < 0: default 64              */
+    int32_t power_iters;   /* subspace (power) iterations;        < 0: default 2              */
+    int32_t max_sweeps;    /* Jacobi sweep limit;                 <= 0: default 16            */
+    uint64_t seed;         /* seed of the +-1 test matrix                                      */
+} atp_basis_opts;
+
+typedef struct {
+    uint32_t struct_size;
+    int32_t q_mode;        /* atp_q_mode; LOWRANK: Q = U_r (X_r W_Q) (Eq. 6); FULL: Q = X W_Q  */
+    float scale;           /* logit scale; <= 0: 1/sqrt(d_h)                                   */
+} atp_attn_opts;
+
+typedef struct {
+    uint32_t struct_size;
+    int32_t act;           /* atp_act                                                          */
+    const float *bias;     /* device, d_out floats, nullable; added before the activation      */
+    const atp_mat *W_gate; /* host struct, device data; required for ATP_ACT_SWIGLU            */
+} atp_linear_opts;
+
+typedef struct atp_ctx atp_ctx;
+
+/* Context: binds a CUDA device; holds the stream, the workspace pointer and the status word. */
+atp_status atp_create(atp_ctx **ctx, int device);
+atp_status atp_destroy(atp_ctx *ctx);
+/* cuda_stream is a cudaStream_t (NULL = default stream). */
+atp_status atp_set_stream(atp_ctx *ctx, void *cuda_stream);
+/* Scratch bytes `op` needs for this batch (d = columns of X / X_r; d_out = columns of the widest
+ * weight the call will see, i.e. d' for attention, d_out for a linear layer, ignored otherwise). */
+atp_status atp_workspace_bytes(atp_ctx *ctx, int op, const atp_seqs *seqs, int64_t d, int64_t d_out,
+                               atp_dtype dtype, size_t *bytes);
+/* dev_ptr: device memory, 256-byte aligned, stays owned by the caller. Contents are scratch. */
+atp_status atp_set_workspace(atp_ctx *ctx, void *dev_ptr, size_t bytes);
+
+/*
+ * Norm box of Fig. 3 (unit gain): Y = norm(X + residual). RMSNorm x/sqrt(mean(x^2)+eps) or
+ * LayerNorm (x-mean)/sqrt(var+eps), row by row, statistics in fp32. residual is nullable.
+ * Y may alias X. All three share shape (rows x cols) and dtype.
+ */
+atp_status atp_input_norm(atp_ctx *ctx, const atp_mat *X, const atp_mat *residual, int kind, float eps,
+                          atp_mat *Y);
+
+/*
+ * Principal basis (Eq. 3, Eq. 5, Sec. 4.2): for every sequence b, the top-r_b left singular
+ * vectors U_r (L_b x r_b, orthonormal columns) and X_r = U_r^T X = [sigma_1 v_1; ..; sigma_r v_r]
+ * (r_b x d), components sorted by sigma descending, i.e. the minimiser of Eq. 9. Computed by a
+ * randomised range finder with subspace iteration, block Gram-Schmidt orthonormalisation and a
+ * one-sided Jacobi rotation of the projected rows (not by a full SVD), so the subspace is the
+ * optimal one up to the range finder's error; opts->power_iters trades passes over X for that.
+ * Sign of each component: sum of the column of U_r >= 0; if that sum is within 1e-6*sqrt(L_b) of
+ * zero, the largest-magnitude entry of the row of X_r is positive.
+ *   X      in   sum(L_b) x d                      (f32 or bf16)
+ *   U_r    out  sum(L_b) x (>= max r_b), same dtype as X; columns >= r_b of a sequence untouched
+ *   X_r    out  sum(r_b) x d, same dtype as X
+ *   sigma  out  device, sum(r_b) floats, nullable
+ * Requires 1 <= r_b <= min(L_b, d) (else ATP_ERR_INVALID_RANK).
+ */
+atp_status atp_principal_basis(atp_ctx *ctx, const atp_mat *X, const atp_seqs *seqs,
+                               const atp_basis_opts *opts, atp_mat *U_r, atp_mat *X_r, float *sigma);
+
+/*
+ * Attention of all queries on the r principal keys and values (Eq. 6, then the procedure of
+ * Eq. 1 with K', V' in place of K, V; Fig. 2): Q' = X_r W_Q, K' = X_r W_K, V' = X_r W_V,
+ * Q = U_r Q' (or X W_Q with q_mode FULL), and per head h (column block of width d'/heads)
+ * O_h = Softmax(Q_h K'_h^T * scale) V'_h over the r_b keys of the sequence. No mask.
+ *   X    in  sum(L_b) x d, nullable unless q_mode == ATP_Q_FULL
+ *   W_*  in  d x d' each (so that X W matches Eq. 2); heads must divide d'
+ *   O    out sum(L_b) x d', same dtype as U_r
+ */
+atp_status atp_attention(atp_ctx *ctx, const atp_mat *X, const atp_mat *U_r, const atp_mat *X_r,
+                         const atp_mat *W_Q, const atp_mat *W_K, const atp_mat *W_V, int heads,
+                         const atp_seqs *seqs, const atp_attn_opts *opts, atp_mat *O);
+
+/*
+ * Linear layer through the low-rank representation (Sec. 4.3): Y = act(U_r (X_r W) + bias);
+ * with ATP_ACT_SWIGLU, Y = silu(U_r (X_r W_gate)) * (U_r (X_r W)). GELU is the erf form.
+ *   W  in  d_in x d_out;  Y out sum(L_b) x d_out, same dtype as U_r
+ */
+atp_status atp_lowrank_linear(atp_ctx *ctx, const atp_mat *U_r, const atp_mat *X_r, const atp_mat *W,
+                              const atp_seqs *seqs, const atp_linear_opts *opts, atp_mat *Y);
+
+/* Synchronises the stream, returns and clears the device-side status (ATP_OK if none). */
+atp_status atp_poll_device_status(atp_ctx *ctx);
+/* Number of kernels this context has launched since creation (for accounting). */
+int64_t atp_launch_count(const atp_ctx *ctx);
+const char *atp_status_string(atp_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ATP_H_ */

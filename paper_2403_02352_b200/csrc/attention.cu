@@ -1,0 +1,232 @@
+// atp_attention: Eq. 6 projections of the r-row representation, then attention of every query
+// on the r principal keys/values (the procedure of Eq. 1 with K', V' in place of K, V).
+#include "gemm_simt.cuh"
+#include <math.h>
+
+constexpr int ATT_MAX_BATCH = 32;
+struct AttnSeq { const float *Q, *K, *V; void *O; int L, r; };
+struct AttnBatch { AttnSeq s[ATT_MAX_BATCH]; int count; };
+
+// One CTA: 64 queries of one head of one sequence; keys in blocks of 64; online softmax in fp32.
+// Shared: Qt[dh][68], Kt[dh][68] (transposed tiles), Vs[64][dh], Ps[64][65].
+template <typename TO>
+__global__ void __launch_bounds__(256)
+attn_simt_kernel(const __grid_constant__ AttnBatch batch, int dh, int ldq, int ldkv, int ldo, float scale)
+{
+    extern __shared__ __align__(16) float smem[];
+    const AttnSeq &sq = batch.s[blockIdx.z];
+    const int q0 = blockIdx.x * 64;
+    if (q0 >= sq.L) return;
+    const int head = blockIdx.y;
+    float *Qt = smem;                       // dh x 68
+    float *Kt = Qt + (size_t)dh * 68;       // dh x 68
+    float *Vs = Kt + (size_t)dh * 68;       // 64 x dh
+    float *Ps = Vs + (size_t)64 * dh;       // 64 x 65
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    const int hoff = head * dh;
+
+    for (int e = tid; e < 64 * dh; e += 256) {
+        int row = e / dh, c = e - row * dh;
+        float v = 0.f;
+        if (q0 + row < sq.L) v = sq.Q[(size_t)(q0 + row) * ldq + hoff + c];
+        Qt[c * 68 + row] = v;
+    }
+    float m_run[4], l_run[4], acc[4][8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        m_run[i] = -INFINITY; l_run[i] = 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
+    }
+    const int ncol = dh / 16;               // columns of O per thread (dh is a multiple of 16)
+
+    for (int k0 = 0; k0 < sq.r; k0 += 64) {
+        __syncthreads();                    // previous block's Vs / Ps / Kt no longer in use
+        for (int e = tid; e < 64 * dh; e += 256) {
+            int row = e / dh, c = e - row * dh;
+            float kv = 0.f, vv = 0.f;
+            if (k0 + row < sq.r) {
+                kv = sq.K[(size_t)(k0 + row) * ldkv + hoff + c];
+                vv = sq.V[(size_t)(k0 + row) * ldkv + hoff + c];
+            }
+            Kt[c * 68 + row] = kv;
+            Vs[row * dh + c] = vv;
+        }
+        __syncthreads();
+        float s[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) s[i][j] = 0.f;
+        for (int c = 0; c < dh; ++c) {
+            float4 a = *(const float4 *)&Qt[c * 68 + ty * 4];
+            float4 b = *(const float4 *)&Kt[c * 68 + tx * 4];
+            float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) s[i][j] = fmaf(av[i], bv[j], s[i][j]);
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float mx = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                s[i][j] = (k0 + tx * 4 + j < sq.r) ? s[i][j] * scale : -INFINITY;
+                mx = fmaxf(mx, s[i][j]);
+            }
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            float m_new = fmaxf(m_run[i], mx);          // finite: every block holds at least one valid key
+            float alpha = expf(m_run[i] - m_new);       // exp(-inf) = 0 on the first block
+            float sum = 0.f;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                float p = expf(s[i][j] - m_new);
+                Ps[(ty * 4 + i) * 65 + tx * 4 + j] = p;
+                sum += p;
+            }
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+            l_run[i] = l_run[i] * alpha + sum;
+            m_run[i] = m_new;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[i][j] *= alpha;
+        }
+        __syncthreads();
+        for (int k = 0; k < 64; ++k) {
+            float p[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) p[i] = Ps[(ty * 4 + i) * 65 + k];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (j < ncol) {
+                    float v = Vs[k * dh + tx + 16 * j];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) acc[i][j] = fmaf(p[i], v, acc[i][j]);
+                }
+            }
+        }
+    }
+    TO *O = (TO *)sq.O;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        int row = q0 + ty * 4 + i;
+        if (row >= sq.L) continue;
+        float inv = 1.f / l_run[i];
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            if (j < ncol) O[(size_t)row * ldo + hoff + tx + 16 * j] = from_f32<TO>(acc[i][j] * inv);
+    }
+}
+
+struct AttnPlan { float *Qp, *Kp, *Vp, *Q; };
+static void plan_attn(Arena &ar, int64_t tr, int64_t tl, int64_t dp, AttnPlan &p)
+{
+    p.Qp = ar.take<float>((size_t)tr * dp);
+    p.Kp = ar.take<float>((size_t)tr * dp);
+    p.Vp = ar.take<float>((size_t)tr * dp);
+    p.Q = ar.take<float>((size_t)tl * dp);
+}
+size_t attention_workspace_bytes(const std::vector<SeqDims> &seqs, int64_t dp)
+{
+    int64_t tr = 0, tl = 0;
+    for (auto &s : seqs) { tr += s.r; tl += s.L; }
+    Arena ar(nullptr, (size_t)-1);
+    AttnPlan p;
+    plan_attn(ar, tr, tl, dp, p);
+    return ar.off;
+}
+
+template <typename T>
+static atp_status attention_impl(atp_ctx *ctx, const atp_mat *X, const atp_mat *U_r, const atp_mat *X_r,
+                                 const atp_mat *WQ, const atp_mat *WK, const atp_mat *WV, int heads,
+                                 const std::vector<SeqDims> &seqs, int q_mode, float scale, atp_mat *O)
+{
+    const int d = (int)X_r->cols, dp = (int)WQ->cols, dh = dp / heads;
+    int64_t tr = 0, tl = 0;
+    for (auto &s : seqs) { tr += s.r; tl += s.L; }
+    Arena ar(ctx->workspace, ctx->workspace_bytes);
+    AttnPlan pl;
+    plan_attn(ar, tr, tl, dp, pl);
+    if (ar.overflow || !ctx->workspace) return ATP_ERR_WORKSPACE_TOO_SMALL;
+    atp_status st;
+    GemmEpi store{EPI_STORE, nullptr};
+    {   // Q', K', V' = X_r W (Eq. 6), all sequences at once
+        GemmBatch b; b.count = (q_mode == ATP_Q_LOWRANK) ? 3 : 2;
+        const atp_mat *Ws[3] = {WK, WV, WQ};
+        float *outs[3] = {pl.Kp, pl.Vp, pl.Qp};
+        for (int i = 0; i < b.count; ++i)
+            b.p[i] = GemmProblem{X_r->data, Ws[i]->data, outs[i], nullptr, (int)tr, dp, d, (int)X_r->ld, (int)Ws[i]->ld, dp, 0};
+        if ((st = launch_gemm_simt<T, T, float, false>(ctx, b, store)) != ATP_OK) return st;
+    }
+    if (q_mode == ATP_Q_LOWRANK) {      // Q = U_r Q'
+        std::vector<GemmProblem> ps;
+        for (auto &s : seqs)
+            if (s.L > 0)
+                ps.push_back(GemmProblem{(const T *)U_r->data + (size_t)s.row0 * U_r->ld, pl.Qp + (size_t)s.rank0 * dp,
+                                         pl.Q + (size_t)s.row0 * dp, nullptr, s.L, dp, s.r, (int)U_r->ld, dp, dp, 0});
+        st = for_each_chunk(ps, [&](const GemmBatch &b) { return launch_gemm_simt<T, float, float, false>(ctx, b, store); });
+        if (st != ATP_OK) return st;
+    } else {                            // Q = X W_Q
+        GemmBatch b; b.count = 1;
+        b.p[0] = GemmProblem{X->data, WQ->data, pl.Q, nullptr, (int)tl, dp, d, (int)X->ld, (int)WQ->ld, dp, 0};
+        if ((st = launch_gemm_simt<T, T, float, false>(ctx, b, store)) != ATP_OK) return st;
+    }
+    size_t smem = ((size_t)dh * 68 * 2 + (size_t)64 * dh + 64 * 65) * sizeof(float);
+    ATP_CUDA_OK(ctx, cudaFuncSetAttribute(attn_simt_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    for (size_t i = 0; i < seqs.size(); i += ATT_MAX_BATCH) {
+        AttnBatch ab; ab.count = 0; int maxL = 0;
+        for (size_t j = i; j < seqs.size() && ab.count < ATT_MAX_BATCH; ++j) {
+            const SeqDims &s = seqs[j];
+            if (s.L == 0) continue;
+            ab.s[ab.count++] = AttnSeq{pl.Q + (size_t)s.row0 * dp, pl.Kp + (size_t)s.rank0 * dp, pl.Vp + (size_t)s.rank0 * dp,
+                                       (T *)O->data + (size_t)s.row0 * O->ld, s.L, s.r};
+            if (s.L > maxL) maxL = s.L;
+        }
+        if (ab.count == 0) continue;
+        dim3 grid(ceil_div(maxL, 64), heads, ab.count);
+        attn_simt_kernel<T><<<grid, 256, smem, ctx->stream>>>(ab, dh, dp, dp, (int)O->ld, scale);
+        ATP_LAUNCHED(ctx);
+    }
+    return ATP_OK;
+}
+
+extern "C" atp_status atp_attention(atp_ctx *ctx, const atp_mat *X, const atp_mat *U_r, const atp_mat *X_r,
+                                    const atp_mat *W_Q, const atp_mat *W_K, const atp_mat *W_V, int heads,
+                                    const atp_seqs *seqs, const atp_attn_opts *opts, atp_mat *O)
+{
+    if (!ctx) return ATP_ERR_INVALID_ARG;
+    atp_status st;
+    if ((st = check_mat(U_r)) != ATP_OK || (st = check_mat(X_r)) != ATP_OK || (st = check_mat(W_Q)) != ATP_OK ||
+        (st = check_mat(W_K)) != ATP_OK || (st = check_mat(W_V)) != ATP_OK || (st = check_mat(O)) != ATP_OK)
+        return st;
+    int q_mode = ATP_Q_LOWRANK; float scale = 0.f;
+    if (opts) {
+        if (opts->struct_size < sizeof(atp_attn_opts)) return ATP_ERR_INVALID_ARG;
+        q_mode = opts->q_mode; scale = opts->scale;
+    }
+    if (q_mode != ATP_Q_LOWRANK && q_mode != ATP_Q_FULL) return ATP_ERR_INVALID_ARG;
+    if (q_mode == ATP_Q_FULL) {
+        if (!X || (st = check_mat(X)) != ATP_OK) return st != ATP_OK ? st : ATP_ERR_INVALID_ARG;
+        if (X->rows != U_r->rows || X->cols != X_r->cols || X->dtype != X_r->dtype) return ATP_ERR_INVALID_ARG;
+    }
+    const atp_dtype dt = X_r->dtype;
+    if (U_r->dtype != dt || W_Q->dtype != dt || W_K->dtype != dt || W_V->dtype != dt || O->dtype != dt)
+        return ATP_ERR_UNSUPPORTED_DTYPE;
+    const int64_t d = X_r->cols, dp = W_Q->cols;
+    if (W_Q->rows != d || W_K->rows != d || W_V->rows != d || W_K->cols != dp || W_V->cols != dp) return ATP_ERR_INVALID_ARG;
+    if (heads < 1 || dp % heads != 0) return ATP_ERR_INVALID_ARG;
+    const int64_t dh = dp / heads;
+    if (dh % 16 != 0 || dh > 128) return ATP_ERR_INVALID_ARG;     // head widths 16..128 in steps of 16
+    std::vector<SeqDims> sd;
+    if ((st = check_seqs(seqs, sd, U_r->rows)) != ATP_OK) return st;
+    int64_t tr = 0; int maxr = 0;
+    for (auto &s : sd) { tr += s.r; if (s.r > maxr) maxr = s.r; }
+    if (X_r->rows != tr || U_r->cols < maxr || O->rows != U_r->rows || O->cols != dp) return ATP_ERR_INVALID_ARG;
+    if (U_r->rows == 0) return ATP_OK;
+    if (!(scale > 0.f)) scale = 1.0f / sqrtf((float)dh);
+    ATP_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+    if (dt == ATP_F32) return attention_impl<float>(ctx, X, U_r, X_r, W_Q, W_K, W_V, heads, sd, q_mode, scale, O);
+    return attention_impl<__nv_bfloat16>(ctx, X, U_r, X_r, W_Q, W_K, W_V, heads, sd, q_mode, scale, O);
+}

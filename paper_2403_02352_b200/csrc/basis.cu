@@ -1,0 +1,768 @@
+// atp_principal_basis: top-r left singular vectors U_r and X_r = U_r^T X (Eq. 3, Eq. 5, Sec. 4.2),
+// i.e. the minimiser of Eq. 9, computed as
+//   1. randomised range finder  Y = X Omega  (+-1 test matrix) with subspace (power) iterations
+//      Z = orth(X^T Y), Y = orth(X Z), each orthonormalised by block Gram-Schmidt (two passes)
+//      with a Cholesky-QR of every 64-column panel (Gram matrix and Cholesky factor in fp64);
+//   2. projection  B = Y^T X  (r~ x d);
+//   3. one-sided block Jacobi on the rows of B (pairs of 32-row blocks, round-robin order): the
+//      rotated rows are sigma_i v_i^T and the accumulated rotations turn Y into singular vectors;
+//   4. sort by sigma, fix signs, write U_r = Y W and X_r.
+#include "gemm_simt.cuh"
+#include <math.h>
+#include <algorithm>
+
+constexpr int PB = 64;            // orthonormalisation panel width
+constexpr int GRAM_ROWS = 512;    // rows per CTA of the panel Gram kernel
+constexpr int BJ = 32;            // Jacobi block height (pairs are 64 rows)
+constexpr int BMAX = 32;          // sequences per launch
+
+// ------------------------------------------------------------------------------------------------
+__global__ void fill_omega_kernel(float *om, size_t n, uint64_t seed)
+{
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+        om[i] = (mix64(seed, i) & 1) ? 1.f : -1.f;
+}
+
+struct PanelSeq { float *P; int n, pb, ld; double *gpart; float *rinv; int *flags; };
+struct PanelBatch { PanelSeq s[BMAX]; int count; };
+
+// Partial Gram matrices of a panel: G_chunk = P_chunk^T P_chunk, fp64 accumulation.
+__global__ void __launch_bounds__(256) panel_gram_kernel(const __grid_constant__ PanelBatch batch)
+{
+    const PanelSeq &sq = batch.s[blockIdx.y];
+    const int r0 = blockIdx.x * GRAM_ROWS;
+    if (sq.pb <= 0 || r0 >= sq.n) return;
+    const int r1 = min(sq.n, r0 + GRAM_ROWS);
+    __shared__ __align__(16) float Ps[32][PB + 4];
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    double acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.0;
+    for (int rr = r0; rr < r1; rr += 32) {
+        for (int e = tid; e < 32 * PB; e += 256) {
+            int row = e >> 6, c = e & 63;
+            float v = 0.f;
+            if (rr + row < r1 && c < sq.pb) v = sq.P[(size_t)(rr + row) * sq.ld + c];
+            Ps[row][c] = v;
+        }
+        __syncthreads();
+#pragma unroll 4
+        for (int k = 0; k < 32; ++k) {
+            float4 a = *(const float4 *)&Ps[k][ty * 4];
+            float4 b = *(const float4 *)&Ps[k][tx * 4];
+            double av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fma(av[i], bv[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+    double *dst = sq.gpart + (size_t)blockIdx.x * PB * PB;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) dst[(ty * 4 + i) * PB + tx * 4 + j] = acc[i][j];
+}
+
+// Sums the partial Gram matrices in order, scales to unit diagonal, Cholesky-factors in fp64 and
+// writes Rinv (pb x pb, fp32) such that P * Rinv has orthonormal columns. A column whose scaled
+// pivot falls below 1e-10 (its part outside the span of the earlier columns is below 1e-5 of its
+// norm) is flagged as dependent: its Rinv column is zero and the apply kernel replaces it by a
+// pseudo-random vector, which the second Gram-Schmidt pass orthonormalises.
+__global__ void __launch_bounds__(256) panel_chol_kernel(const __grid_constant__ PanelBatch batch)
+{
+    const PanelSeq &sq = batch.s[blockIdx.x];
+    const int n = sq.pb;
+    if (n <= 0) return;
+    extern __shared__ double chol_sm[];
+    double (*G)[PB + 1] = (double (*)[PB + 1])chol_sm;
+    double (*Li)[PB + 1] = (double (*)[PB + 1])(chol_sm + PB * (PB + 1));
+    __shared__ double dsc[PB];
+    __shared__ int dep[PB];
+    const int tid = threadIdx.x;
+    const int nchunks = (sq.n + GRAM_ROWS - 1) / GRAM_ROWS;
+    for (int e = tid; e < PB * PB; e += 256) {
+        double s = 0.0;
+        for (int c = 0; c < nchunks; ++c) s += sq.gpart[(size_t)c * PB * PB + e];
+        G[e >> 6][e & 63] = s;
+    }
+    __syncthreads();
+    if (tid < PB) { dsc[tid] = (tid < n && G[tid][tid] > 0.0) ? sqrt(G[tid][tid]) : 0.0; dep[tid] = 0; }
+    __syncthreads();
+    for (int e = tid; e < PB * PB; e += 256) {
+        int i = e >> 6, j = e & 63;
+        double den = dsc[i] * dsc[j];
+        G[i][j] = den > 0.0 ? G[i][j] / den : 0.0;
+    }
+    __syncthreads();
+    for (int j = 0; j < n; ++j) {
+        double piv = G[j][j];
+        bool bad = !(piv > 1e-10);
+        double ljj = bad ? 1.0 : sqrt(piv);
+        __syncthreads();
+        if (tid == 0) { G[j][j] = ljj; if (bad) dep[j] = 1; }
+        for (int i = j + 1 + tid; i < n; i += 256) G[i][j] = bad ? 0.0 : G[i][j] / ljj;
+        __syncthreads();
+        // trailing update of the lower triangle
+        int m = n - j - 1;
+        for (int e = tid; e < m * m; e += 256) {
+            int a = e / m, b = e - a * m;
+            if (b <= a) G[j + 1 + a][j + 1 + b] -= G[j + 1 + a][j] * G[j + 1 + b][j];
+        }
+        __syncthreads();
+    }
+    // Li = inverse of the lower-triangular factor, one column per thread
+    if (tid < n) {
+        int c = tid;
+        for (int i = 0; i < n; ++i) {
+            double x = 0.0;
+            if (i >= c) {
+                x = (i == c) ? 1.0 : 0.0;
+                for (int k = c; k < i; ++k) x -= G[i][k] * Li[k][c];
+                x /= G[i][i];
+            }
+            Li[i][c] = x;
+        }
+    }
+    __syncthreads();
+    for (int e = tid; e < PB * PB; e += 256) {
+        int k = e >> 6, c = e & 63;      // Rinv[k][c] = Li[c][k] / dsc[k]
+        double v = 0.0;
+        if (k < n && c < n && !dep[c] && !dep[k] && dsc[k] > 0.0) v = Li[c][k] / dsc[k];
+        sq.rinv[e] = (float)v;
+    }
+    if (tid < PB) sq.flags[tid] = (tid < n) ? dep[tid] : 0;
+}
+
+// P <- P * Rinv in place (each CTA owns 64 rows); flagged columns are refilled with hash noise.
+__global__ void __launch_bounds__(256) panel_apply_kernel(const __grid_constant__ PanelBatch batch, uint64_t seed)
+{
+    const PanelSeq &sq = batch.s[blockIdx.y];
+    const int r0 = blockIdx.x * 64;
+    if (sq.pb <= 0 || r0 >= sq.n) return;
+    __shared__ __align__(16) float Rs[PB][PB + 4];
+    __shared__ float Ts[64][PB + 1];
+    __shared__ int fl[PB];
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    for (int e = tid; e < PB * PB; e += 256) Rs[e >> 6][e & 63] = sq.rinv[e];
+    if (tid < PB) fl[tid] = sq.flags[tid];
+    for (int e = tid; e < 64 * PB; e += 256) {
+        int row = e >> 6, c = e & 63;
+        float v = 0.f;
+        if (r0 + row < sq.n && c < sq.pb) v = sq.P[(size_t)(r0 + row) * sq.ld + c];
+        Ts[row][c] = v;
+    }
+    __syncthreads();
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+    for (int k = 0; k < PB; ++k) {
+        float4 b = *(const float4 *)&Rs[k][tx * 4];
+        float bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float a = Ts[ty * 4 + i][k];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a, bv[j], acc[i][j]);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        int row = r0 + ty * 4 + i;
+        if (row >= sq.n) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            int c = tx * 4 + j;
+            if (c >= sq.pb) continue;
+            float v = acc[i][j];
+            if (fl[c]) v = hash_uniform(seed, ((uint64_t)blockIdx.y << 40) ^ ((uint64_t)row << 8) ^ (uint64_t)c);
+            sq.P[(size_t)row * sq.ld + c] = v;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// One-sided block Jacobi on the rows of BW = [B | Wt] (r~ x (d + r~)); only the first d columns
+// enter the inner products, all d + r~ columns are rotated.
+struct JacSeq { float *BW; int rt, d, ld, nb; unsigned *maxoff; int *conv; };
+struct JacBatch { JacSeq s[BMAX]; int count; };
+
+__global__ void init_w_kernel(const __grid_constant__ JacBatch batch)
+{
+    const JacSeq &sq = batch.s[blockIdx.y];
+    size_t n = (size_t)sq.rt * sq.rt;
+    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
+        int i = (int)(e / sq.rt), k = (int)(e - (size_t)i * sq.rt);
+        sq.BW[(size_t)i * sq.ld + sq.d + k] = (i == k) ? 1.f : 0.f;
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) { *sq.maxoff = 0u; *sq.conv = 0; }
+}
+
+__device__ __forceinline__ void rr_pair(int nb, int step, int t, int &I, int &J)
+{
+    // round-robin tournament of nb (even) players, round `step` in [0, nb-1), table t in [0, nb/2)
+    int m = nb - 1;
+    if (t == 0) { I = m; J = step % m; }
+    else { I = (step + t) % m; J = (step - t + m) % m; }
+    if (I > J) { int x = I; I = J; J = x; }
+}
+
+__global__ void __launch_bounds__(256)
+jacobi_pair_kernel(const __grid_constant__ JacBatch batch, int step, float tol_rot, float tol_skip)
+{
+    const JacSeq &sq = batch.s[blockIdx.y];
+    if (*sq.conv) return;
+    const int npairs = sq.nb / 2;
+    if ((int)blockIdx.x >= npairs) return;
+    int I, J;
+    rr_pair(sq.nb, step % (sq.nb - 1), blockIdx.x, I, J);
+    __shared__ float G[64][65];
+    __shared__ float Vt[64][65];
+    __shared__ __align__(16) float St[32][68];     // phase 1: transposed column tile; phase 3: reused as input tile
+    float (*Tl)[65] = G;                           // phase 3 input tile (G is dead by then)
+    __shared__ float cs[32], sn[32];
+    __shared__ int pp[32], qq[32];
+    __shared__ float red[8];
+    __shared__ int rotated;
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    auto grow = [&](int i) -> int {     // global row of local row i, or -1
+        int g = (i < 32) ? I * BJ + i : J * BJ + (i - 32);
+        return (g < sq.rt) ? g : -1;
+    };
+    // ---- phase 1: G = S S^T over the first d columns (tile sums in fp32, running sum in fp64)
+    double acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.0;
+    for (int c0 = 0; c0 < sq.d; c0 += 32) {
+        for (int e = tid; e < 64 * 32; e += 256) {
+            int row = e >> 5, c = e & 31;
+            int g = grow(row);
+            float v = 0.f;
+            if (g >= 0 && c0 + c < sq.d) v = sq.BW[(size_t)g * sq.ld + c0 + c];
+            St[c][row] = v;
+        }
+        __syncthreads();
+        float part[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) part[i][j] = 0.f;
+#pragma unroll 8
+        for (int c = 0; c < 32; ++c) {
+            float4 a = *(const float4 *)&St[c][ty * 4];
+            float4 b = *(const float4 *)&St[c][tx * 4];
+            float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) part[i][j] = fmaf(av[i], bv[j], part[i][j]);
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i][j] += (double)part[i][j];
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            G[ty * 4 + i][tx * 4 + j] = (float)acc[i][j];
+            Vt[ty * 4 + i][tx * 4 + j] = (ty * 4 + i == tx * 4 + j) ? 1.f : 0.f;
+        }
+    __syncthreads();
+    // largest scaled off-diagonal entry of this pair
+    float mo = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            int a = ty * 4 + i, b = tx * 4 + j;
+            if (a != b) {
+                float den = sqrtf(G[a][a] * G[b][b]);
+                if (den > 0.f) mo = fmaxf(mo, fabsf(G[a][b]) / den);
+            }
+        }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mo = fmaxf(mo, __shfl_xor_sync(0xffffffffu, mo, o));
+    if ((tid & 31) == 0) red[tid >> 5] = mo;
+    __syncthreads();
+    mo = red[0];
+#pragma unroll
+    for (int w = 1; w < 8; ++w) mo = fmaxf(mo, red[w]);
+    if (tid == 0) atomicMax(sq.maxoff, __float_as_uint(mo));
+    if (mo <= tol_skip) return;
+
+    // ---- phase 2: diagonalise G by cyclic two-sided Jacobi, accumulating the row operations in Vt
+    for (int sweep = 0; sweep < 12; ++sweep) {
+        if (tid == 0) rotated = 0;
+        __syncthreads();
+        for (int st = 0; st < 63; ++st) {
+            if (tid < 32) {
+                int p, q;
+                rr_pair(64, st, tid, p, q);
+                float gpp = G[p][p], gqq = G[q][q], gpq = G[p][q];
+                float c = 1.f, s = 0.f;
+                if (fabsf(gpq) > tol_rot * sqrtf(gpp * gqq) && gpq != 0.f) {
+                    float zeta = (gqq - gpp) / (2.f * gpq);
+                    float t = copysignf(1.f, zeta) / (fabsf(zeta) + sqrtf(1.f + zeta * zeta));
+                    c = rsqrtf(1.f + t * t);
+                    s = c * t;
+                    rotated = 1;
+                }
+                cs[tid] = c; sn[tid] = s; pp[tid] = p; qq[tid] = q;
+            }
+            __syncthreads();
+            // G <- J^T G J on 2x2 blocks (row pair a, column pair b); Vt rows rotate like G rows
+#pragma unroll
+            for (int it = 0; it < 4; ++it) {
+                int idx = tid + it * 256;
+                int a = idx >> 5, b = idx & 31;
+                int pa = pp[a], qa = qq[a], pb_ = pp[b], qb = qq[b];
+                float ca = cs[a], sa = sn[a], cb = cs[b], sb = sn[b];
+                float g00 = G[pa][pb_], g01 = G[pa][qb], g10 = G[qa][pb_], g11 = G[qa][qb];
+                float r00 = ca * g00 - sa * g10, r01 = ca * g01 - sa * g11;
+                float r10 = sa * g00 + ca * g10, r11 = sa * g01 + ca * g11;
+                G[pa][pb_] = cb * r00 - sb * r01; G[pa][qb] = sb * r00 + cb * r01;
+                G[qa][pb_] = cb * r10 - sb * r11; G[qa][qb] = sb * r10 + cb * r11;
+            }
+#pragma unroll
+            for (int it = 0; it < 8; ++it) {
+                int idx = tid + it * 256;
+                int a = idx >> 6, col = idx & 63;
+                int pa = pp[a], qa = qq[a];
+                float ca = cs[a], sa = sn[a];
+                float x = Vt[pa][col], y = Vt[qa][col];
+                Vt[pa][col] = ca * x - sa * y;
+                Vt[qa][col] = sa * x + ca * y;
+            }
+            __syncthreads();
+        }
+        if (!rotated) break;
+        __syncthreads();
+    }
+    // ---- phase 3: rows <- Vt * rows over all d + r~ columns
+    const int ncols = sq.d + sq.rt;
+    for (int c0 = 0; c0 < ncols; c0 += 64) {
+        for (int e = tid; e < 64 * 64; e += 256) {
+            int row = e >> 6, c = e & 63;
+            int g = grow(row);
+            float v = 0.f;
+            if (g >= 0 && c0 + c < ncols) v = sq.BW[(size_t)g * sq.ld + c0 + c];
+            Tl[row][c] = v;
+        }
+        __syncthreads();
+        float out[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) out[i][j] = 0.f;
+        for (int k = 0; k < 64; ++k) {
+            float bv[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) bv[j] = Tl[k][tx + 16 * j];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                float a = Vt[ty * 4 + i][k];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) out[i][j] = fmaf(a, bv[j], out[i][j]);
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            int g = grow(ty * 4 + i);
+            if (g < 0) continue;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                int c = c0 + tx + 16 * j;
+                if (c < ncols) sq.BW[(size_t)g * sq.ld + c] = out[i][j];
+            }
+        }
+    }
+}
+
+__global__ void jacobi_sweep_end_kernel(const __grid_constant__ JacBatch batch, float tol_conv, int last, int *dev_status)
+{
+    int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= batch.count) return;
+    const JacSeq &sq = batch.s[b];
+    if (!*sq.conv) {
+        float mo = __uint_as_float(*sq.maxoff);
+        if (mo <= tol_conv) *sq.conv = 1;
+        else if (last) raise_status(dev_status, ATP_ERR_NOT_CONVERGED);
+    }
+    *sq.maxoff = 0u;
+}
+
+// ------------------------------------------------------------------------------------------------
+struct FinSeq {
+    const float *BW; const float *Y; float *sig; int *ord; float *tsum; float *Wsel;
+    void *Xr; float *sigma_out; int rt, r, d, ld, L, ldy, ldxr;
+};
+struct FinBatch { FinSeq s[BMAX]; int count; };
+
+// Row norms of B (= singular values) and their descending order. One CTA per sequence.
+__global__ void __launch_bounds__(1024) sigma_sort_kernel(const __grid_constant__ FinBatch batch)
+{
+    const FinSeq &sq = batch.s[blockIdx.x];
+    extern __shared__ float sh[];
+    int npow = 1;
+    while (npow < sq.rt) npow <<= 1;
+    float *key = sh;
+    int *idx = (int *)(sh + npow);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (int i = warp; i < npow; i += 32) {
+        float s = -1.f;
+        if (i < sq.rt) {
+            double acc = 0.0;
+            float part = 0.f;
+            for (int c = lane; c < sq.d; c += 32) { float v = sq.BW[(size_t)i * sq.ld + c]; part = fmaf(v, v, part); }
+            acc = part;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+            s = (float)sqrt(acc);
+        }
+        if (lane == 0) { key[i] = s; idx[i] = i; }
+    }
+    __syncthreads();
+    for (int k = 2; k <= npow; k <<= 1)
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int i = tid; i < npow; i += 1024) {
+                int l = i ^ j;
+                if (l > i) {
+                    bool desc = ((i & k) == 0);
+                    float ki = key[i], kl = key[l];
+                    int ii = idx[i], il = idx[l];
+                    bool i_first = (ki > kl) || (ki == kl && ii < il);   // order wanted in a descending run
+                    if (desc ? !i_first : i_first) { key[i] = kl; key[l] = ki; idx[i] = il; idx[l] = ii; }
+                }
+            }
+            __syncthreads();
+        }
+    for (int i = tid; i < sq.rt; i += 1024) { sq.sig[i] = key[i]; sq.ord[i] = idx[i]; }
+}
+
+// Column sums of Y (L x r~): t[k] = sum_l Y[l][k].
+__global__ void colsum_kernel(const __grid_constant__ FinBatch batch)
+{
+    const FinSeq &sq = batch.s[blockIdx.y];
+    int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= sq.rt) return;
+    float s = 0.f;
+    for (int l = 0; l < sq.L; ++l) s += sq.Y[(size_t)l * sq.ldy + k];
+    sq.tsum[k] = s;
+}
+
+// One CTA per kept component: sign rule, then X_r row, Wsel column and sigma.
+template <typename T>
+__global__ void __launch_bounds__(256) select_kernel(const __grid_constant__ FinBatch batch)
+{
+    const FinSeq &sq = batch.s[blockIdx.y];
+    const int a = blockIdx.x;
+    if (a >= sq.r) return;
+    const int i = sq.ord[a];
+    const float *row = sq.BW + (size_t)i * sq.ld;
+    __shared__ float redf[8];
+    __shared__ int redi[8];
+    __shared__ float sgn_s;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    float s = 0.f;
+    for (int k = tid; k < sq.rt; k += 256) s = fmaf(sq.tsum[k], row[sq.d + k], s);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) redf[warp] = s;
+    __syncthreads();
+    if (tid == 0) {
+        float tot = 0.f;
+        for (int w = 0; w < 8; ++w) tot += redf[w];
+        sgn_s = tot;
+    }
+    __syncthreads();
+    float colsum = sgn_s;
+    __syncthreads();
+    float sgn;
+    if (fabsf(colsum) >= 1e-6f * sqrtf((float)sq.L)) {
+        sgn = colsum < 0.f ? -1.f : 1.f;
+    } else {      // fall back to the largest-magnitude entry of the row (first one on ties)
+        float best = -1.f; int bi = 0x7fffffff;
+        for (int c = tid; c < sq.d; c += 256) {
+            float v = fabsf(row[c]);
+            if (v > best) { best = v; bi = c; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            float ob = __shfl_xor_sync(0xffffffffu, best, o);
+            int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (ob > best || (ob == best && oi < bi)) { best = ob; bi = oi; }
+        }
+        if (lane == 0) { redf[warp] = best; redi[warp] = bi; }
+        __syncthreads();
+        if (tid == 0) {
+            float b = redf[0]; int bi2 = redi[0];
+            for (int w = 1; w < 8; ++w)
+                if (redf[w] > b || (redf[w] == b && redi[w] < bi2)) { b = redf[w]; bi2 = redi[w]; }
+            sgn_s = (bi2 < sq.d && row[bi2] < 0.f) ? -1.f : 1.f;
+        }
+        __syncthreads();
+        sgn = sgn_s;
+    }
+    T *xr = (T *)sq.Xr + (size_t)a * sq.ldxr;
+    for (int c = tid; c < sq.d; c += 256) xr[c] = from_f32<T>(sgn * row[c]);
+    for (int k = tid; k < sq.rt; k += 256) sq.Wsel[(size_t)k * sq.r + a] = sgn * row[sq.d + k];
+    if (tid == 0 && sq.sigma_out) sq.sigma_out[a] = sq.sig[a];
+}
+
+// ------------------------------------------------------------------------------------------------
+struct SeqPlan {
+    SeqDims dims; int rt, npanel_L, npanel_d;
+    float *Y, *Z, *BW, *Wsel, *tsum, *sig, *Cc, *rinv; double *gpart; int *ord, *flags, *conv; unsigned *maxoff;
+};
+struct BasisPlan {
+    std::vector<SeqPlan> seqs; float *omega; float *part; size_t part_stride; int rtmax; int splits;
+};
+
+constexpr size_t CHOL_SMEM = 2 * PB * (PB + 1) * sizeof(double);
+
+static int pick_splits(int K) { int s = K / 1024; return s < 1 ? 1 : (s > 16 ? 16 : s); }
+
+static void plan_basis(Arena &ar, const std::vector<SeqDims> &sd, int d, int oversample, BasisPlan &bp)
+{
+    bp.seqs.clear(); bp.rtmax = 0;
+    int maxdim = d; size_t maxpart = 0;
+    for (auto &s : sd) {
+        SeqPlan p; p.dims = s;
+        int m = std::min(s.L, d);
+        p.rt = std::min(m, s.r + oversample);
+        if (s.L == 0) p.rt = 0;
+        bp.rtmax = std::max(bp.rtmax, p.rt);
+        maxdim = std::max(maxdim, s.L);
+        bp.seqs.push_back(p);
+    }
+    bp.omega = ar.take<float>((size_t)d * bp.rtmax);
+    bp.splits = pick_splits(maxdim);
+    for (auto &p : bp.seqs) {
+        int L = p.dims.L, rt = p.rt;
+        p.Y = ar.take<float>((size_t)L * rt);
+        p.Z = ar.take<float>((size_t)d * rt);
+        p.BW = ar.take<float>((size_t)rt * (d + rt));
+        p.Wsel = ar.take<float>((size_t)rt * p.dims.r);
+        p.tsum = ar.take<float>(rt);
+        p.sig = ar.take<float>(rt);
+        p.ord = ar.take<int>(rt);
+        p.Cc = ar.take<float>((size_t)rt * PB);
+        p.rinv = ar.take<float>(PB * PB);
+        p.flags = ar.take<int>(PB);
+        p.gpart = ar.take<double>((size_t)ceil_div(std::max(std::max(L, d), 1), GRAM_ROWS) * PB * PB);
+        p.maxoff = ar.take<unsigned>(1);
+        p.conv = ar.take<int>(1);
+        maxpart = std::max(maxpart, (size_t)rt * PB);
+    }
+    bp.part_stride = maxpart;
+    bp.part = ar.take<float>((size_t)bp.splits * std::min<size_t>(bp.seqs.size(), BMAX) * maxpart);
+}
+
+size_t basis_workspace_bytes(const std::vector<SeqDims> &sd, int d, int oversample)
+{
+    Arena ar(nullptr, (size_t)-1);
+    BasisPlan bp;
+    plan_basis(ar, sd, d, oversample, bp);
+    return ar.off;
+}
+
+// Orthonormalise the columns of M_b (n_b x rt_b, ld = rt_b) for the sequences [i0, i1).
+static atp_status orthonormalise(atp_ctx *ctx, BasisPlan &bp, size_t i0, size_t i1, bool z_side, int d, uint64_t seed)
+{
+    int maxpan = 0, maxn = 0;
+    for (size_t i = i0; i < i1; ++i) {
+        maxpan = std::max(maxpan, ceil_div(bp.seqs[i].rt, PB));
+        maxn = std::max(maxn, z_side ? d : bp.seqs[i].dims.L);
+    }
+    atp_status st;
+    ATP_CUDA_OK(ctx, cudaFuncSetAttribute(panel_chol_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHOL_SMEM));
+    for (int pj = 0; pj < maxpan; ++pj) {
+        const int j0 = pj * PB;
+        for (int rep = 0; rep < 2; ++rep) {
+            GemmBatch proj, upd; PanelBatch pb;
+            proj.count = upd.count = pb.count = (int)(i1 - i0);
+            for (size_t i = i0; i < i1; ++i) {
+                SeqPlan &p = bp.seqs[i];
+                float *M = z_side ? p.Z : p.Y;
+                int n = z_side ? d : p.dims.L;
+                int w = std::min(PB, p.rt - j0);
+                if (w <= 0 || n <= 0) { w = 0; n = 0; }
+                int k = (int)(i - i0);
+                // C = Qprev^T P  (j0 x w), then P -= Qprev C
+                proj.p[k] = GemmProblem{M, M + j0, p.Cc, nullptr, w > 0 ? j0 : 0, w, n, p.rt, p.rt, PB, 0};
+                upd.p[k] = GemmProblem{M, p.Cc, M + j0, M + j0, n, w, w > 0 ? j0 : 0, p.rt, PB, p.rt, p.rt};
+                pb.s[k] = PanelSeq{M + j0, n, w, p.rt, p.gpart, p.rinv, p.flags};
+            }
+            if (j0 > 0) {
+                if ((st = launch_gemm_simt<float, float, float, true>(ctx, proj, GemmEpi{EPI_STORE, nullptr}, bp.splits, bp.part,
+                                                                      bp.part_stride)) != ATP_OK) return st;
+                if ((st = launch_gemm_simt<float, float, float, false>(ctx, upd, GemmEpi{EPI_D_MINUS, nullptr})) != ATP_OK) return st;
+            }
+            panel_gram_kernel<<<dim3(ceil_div(maxn, GRAM_ROWS), pb.count), 256, 0, ctx->stream>>>(pb);
+            ATP_LAUNCHED(ctx);
+            panel_chol_kernel<<<pb.count, 256, CHOL_SMEM, ctx->stream>>>(pb);
+            ATP_LAUNCHED(ctx);
+            panel_apply_kernel<<<dim3(ceil_div(maxn, 64), pb.count), 256, 0, ctx->stream>>>(
+                pb, seed + 7919ull * (uint64_t)(pj * 2 + rep) + (z_side ? 104729ull : 0ull));
+            ATP_LAUNCHED(ctx);
+        }
+    }
+    return ATP_OK;
+}
+
+template <typename T>
+static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<SeqDims> &sd, int oversample,
+                             int power_iters, int max_sweeps, uint64_t seed, atp_mat *U_r, atp_mat *X_r, float *sigma)
+{
+    const int d = (int)X->cols;
+    Arena ar(ctx->workspace, ctx->workspace_bytes);
+    BasisPlan bp;
+    plan_basis(ar, sd, d, oversample, bp);
+    if (ar.overflow || !ctx->workspace) return ATP_ERR_WORKSPACE_TOO_SMALL;
+    atp_status st;
+    {
+        size_t n = (size_t)d * bp.rtmax;
+        fill_omega_kernel<<<(unsigned)std::min<size_t>((n + 255) / 256, 4096), 256, 0, ctx->stream>>>(bp.omega, n, seed);
+        ATP_LAUNCHED(ctx);
+    }
+    const float tol_conv = (X->dtype == ATP_F32) ? 1e-6f : 3e-5f;
+    const float tol_rot = tol_conv * 0.25f;
+    GemmEpi store{EPI_STORE, nullptr};
+
+    for (size_t i0 = 0; i0 < bp.seqs.size(); i0 += BMAX) {
+        const size_t i1 = std::min(bp.seqs.size(), i0 + BMAX);
+        const int cnt = (int)(i1 - i0);
+        auto Xb = [&](const SeqPlan &p) { return (const T *)X->data + (size_t)p.dims.row0 * X->ld; };
+        GemmBatch g; g.count = cnt;
+        // Y = X Omega
+        for (size_t i = i0; i < i1; ++i) {
+            SeqPlan &p = bp.seqs[i];
+            g.p[i - i0] = GemmProblem{Xb(p), bp.omega, p.Y, nullptr, p.dims.L, p.rt, d, (int)X->ld, bp.rtmax, p.rt, 0};
+        }
+        if ((st = launch_gemm_simt<T, float, float, false>(ctx, g, store)) != ATP_OK) return st;
+        if ((st = orthonormalise(ctx, bp, i0, i1, false, d, seed)) != ATP_OK) return st;
+        for (int it = 0; it < power_iters; ++it) {
+            // Z = X^T Y ; orth ; Y = X Z ; orth
+            for (size_t i = i0; i < i1; ++i) {
+                SeqPlan &p = bp.seqs[i];
+                g.p[i - i0] = GemmProblem{Xb(p), p.Y, p.Z, nullptr, p.rt > 0 ? d : 0, p.rt, p.dims.L, (int)X->ld, p.rt, p.rt, 0};
+            }
+            if ((st = launch_gemm_simt<T, float, float, true>(ctx, g, store)) != ATP_OK) return st;
+            if ((st = orthonormalise(ctx, bp, i0, i1, true, d, seed + 1000003ull * (it + 1))) != ATP_OK) return st;
+            for (size_t i = i0; i < i1; ++i) {
+                SeqPlan &p = bp.seqs[i];
+                g.p[i - i0] = GemmProblem{Xb(p), p.Z, p.Y, nullptr, p.dims.L, p.rt, d, (int)X->ld, p.rt, p.rt, 0};
+            }
+            if ((st = launch_gemm_simt<T, float, float, false>(ctx, g, store)) != ATP_OK) return st;
+            if ((st = orthonormalise(ctx, bp, i0, i1, false, d, seed + 2000003ull * (it + 1))) != ATP_OK) return st;
+        }
+        // B = Y^T X into BW[:, :d]; Wt = I
+        JacBatch jb; jb.count = cnt; FinBatch fb; fb.count = cnt;
+        int maxnb = 2, maxrt = 0, maxr = 0;
+        for (size_t i = i0; i < i1; ++i) {
+            SeqPlan &p = bp.seqs[i];
+            int k = (int)(i - i0);
+            g.p[k] = GemmProblem{p.Y, Xb(p), p.BW, nullptr, p.rt, p.rt > 0 ? d : 0, p.dims.L, p.rt, (int)X->ld, d + p.rt, 0};
+            int nb = ceil_div(std::max(p.rt, 1), BJ); nb += nb & 1;
+            jb.s[k] = JacSeq{p.BW, p.rt, d, d + p.rt, nb, p.maxoff, p.conv};
+            fb.s[k] = FinSeq{p.BW, p.Y, p.sig, p.ord, p.tsum, p.Wsel,
+                             (T *)X_r->data + (size_t)p.dims.rank0 * X_r->ld, sigma ? sigma + p.dims.rank0 : nullptr,
+                             p.rt, p.dims.r, d, d + p.rt, p.dims.L, p.rt, (int)X_r->ld};
+            maxnb = std::max(maxnb, nb); maxrt = std::max(maxrt, p.rt); maxr = std::max(maxr, p.dims.r);
+        }
+        if (maxrt == 0) continue;
+        if ((st = launch_gemm_simt<float, T, float, true>(ctx, g, store)) != ATP_OK) return st;
+        init_w_kernel<<<dim3(64, cnt), 256, 0, ctx->stream>>>(jb);
+        ATP_LAUNCHED(ctx);
+        for (int sw = 0; sw < max_sweeps; ++sw) {
+            for (int step = 0; step < maxnb - 1; ++step) {
+                jacobi_pair_kernel<<<dim3(maxnb / 2, cnt), 256, 0, ctx->stream>>>(jb, step, tol_rot, tol_rot);
+                ATP_LAUNCHED(ctx);
+            }
+            jacobi_sweep_end_kernel<<<1, BMAX, 0, ctx->stream>>>(jb, tol_conv, sw == max_sweeps - 1, ctx->dev_status);
+            ATP_LAUNCHED(ctx);
+        }
+        int npow = 1; while (npow < maxrt) npow <<= 1;
+        size_t sm = (size_t)npow * 8;
+        if (sm > 48 * 1024) ATP_CUDA_OK(ctx, cudaFuncSetAttribute(sigma_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm));
+        sigma_sort_kernel<<<cnt, 1024, sm, ctx->stream>>>(fb);
+        ATP_LAUNCHED(ctx);
+        colsum_kernel<<<dim3(ceil_div(maxrt, 128), cnt), 128, 0, ctx->stream>>>(fb);
+        ATP_LAUNCHED(ctx);
+        select_kernel<T><<<dim3(maxr, cnt), 256, 0, ctx->stream>>>(fb);
+        ATP_LAUNCHED(ctx);
+        // U_r = Y Wsel
+        for (size_t i = i0; i < i1; ++i) {
+            SeqPlan &p = bp.seqs[i];
+            g.p[i - i0] = GemmProblem{p.Y, p.Wsel, (T *)U_r->data + (size_t)p.dims.row0 * U_r->ld, nullptr,
+                                      p.dims.L, p.dims.r, p.rt, p.rt, p.dims.r, (int)U_r->ld, 0};
+        }
+        if ((st = launch_gemm_simt<float, float, T, false>(ctx, g, store)) != ATP_OK) return st;
+    }
+    return ATP_OK;
+}
+
+extern "C" atp_status atp_principal_basis(atp_ctx *ctx, const atp_mat *X, const atp_seqs *seqs,
+                                          const atp_basis_opts *opts, atp_mat *U_r, atp_mat *X_r, float *sigma)
+{
+    if (!ctx) return ATP_ERR_INVALID_ARG;
+    atp_status st;
+    if ((st = check_mat(X)) != ATP_OK || (st = check_mat(U_r)) != ATP_OK || (st = check_mat(X_r)) != ATP_OK) return st;
+    int oversample = 64, power_iters = 2, max_sweeps = 16; uint64_t seed = 0x243F6A8885A308D3ull;
+    if (opts) {
+        if (opts->struct_size < sizeof(atp_basis_opts)) return ATP_ERR_INVALID_ARG;
+        if (opts->oversample >= 0) oversample = opts->oversample;
+        if (opts->power_iters >= 0) power_iters = opts->power_iters;
+        if (opts->max_sweeps > 0) max_sweeps = opts->max_sweeps;
+        seed ^= opts->seed * 0x9E3779B97F4A7C15ull;
+    }
+    if (oversample > 4096 || power_iters > 64 || max_sweeps > 200) return ATP_ERR_INVALID_ARG;
+    if (U_r->dtype != X->dtype || X_r->dtype != X->dtype) return ATP_ERR_UNSUPPORTED_DTYPE;
+    std::vector<SeqDims> sd;
+    if ((st = check_seqs(seqs, sd, X->rows)) != ATP_OK) return st;
+    int64_t tr = 0; int maxr = 0;
+    for (auto &s : sd) {
+        if (s.r > X->cols) return ATP_ERR_INVALID_RANK;
+        if (std::min<int64_t>(s.L, X->cols) > 4096 && s.r + oversample > 4096) return ATP_ERR_INVALID_RANK;   // sort buffer limit
+        tr += s.r; maxr = std::max(maxr, s.r);
+    }
+    if (U_r->rows != X->rows || U_r->cols < maxr || X_r->rows != tr || X_r->cols != X->cols) return ATP_ERR_INVALID_ARG;
+    if (X->rows == 0) return ATP_OK;
+    ATP_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+    if (X->dtype == ATP_F32) return basis_impl<float>(ctx, X, sd, oversample, power_iters, max_sweeps, seed, U_r, X_r, sigma);
+    return basis_impl<__nv_bfloat16>(ctx, X, sd, oversample, power_iters, max_sweeps, seed, U_r, X_r, sigma);
+}
+
+// ------------------------------------------------------------------------------------------------
+size_t linear_workspace_bytes(const std::vector<SeqDims> &seqs, int64_t d_out);
+size_t attention_workspace_bytes(const std::vector<SeqDims> &seqs, int64_t dp);
+
+extern "C" atp_status atp_workspace_bytes(atp_ctx *ctx, int op, const atp_seqs *seqs, int64_t d, int64_t d_out,
+                                          atp_dtype dtype, size_t *bytes)
+{
+    if (!ctx || !bytes) return ATP_ERR_INVALID_ARG;
+    if (dtype != ATP_F32 && dtype != ATP_BF16) return ATP_ERR_UNSUPPORTED_DTYPE;
+    *bytes = 0;
+    if (op == ATP_OP_NORM) return ATP_OK;
+    std::vector<SeqDims> sd;
+    atp_status st = check_seqs(seqs, sd, -1);
+    if (st != ATP_OK) return st;
+    if (d < 1 || d > 0x7fffffff) return ATP_ERR_INVALID_ARG;
+    switch (op) {
+        case ATP_OP_BASIS: *bytes = basis_workspace_bytes(sd, (int)d, 64) + 256; return ATP_OK;
+        case ATP_OP_ATTENTION: if (d_out < 1) return ATP_ERR_INVALID_ARG; *bytes = attention_workspace_bytes(sd, d_out) + 256; return ATP_OK;
+        case ATP_OP_LINEAR: if (d_out < 1) return ATP_ERR_INVALID_ARG; *bytes = linear_workspace_bytes(sd, d_out) + 256; return ATP_OK;
+        default: return ATP_ERR_INVALID_ARG;
+    }
+}

@@ -1,0 +1,76 @@
+// Shared declarations of libatp: context, launch helpers, dtype conversion, counter-based hash.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+#include <vector>
+#include "atp.h"
+
+struct atp_ctx {
+    int device = 0;
+    cudaStream_t stream = nullptr;
+    void *workspace = nullptr;
+    size_t workspace_bytes = 0;
+    int *dev_status = nullptr;       // one word, sticky: first non-zero atp_status raised on device
+    int64_t launches = 0;
+    cudaError_t last_cuda = cudaSuccess;
+    int sm_count = 148;
+};
+
+#define ATP_CUDA_OK(ctx, expr)                                   \
+    do {                                                         \
+        cudaError_t e__ = (expr);                                \
+        if (e__ != cudaSuccess) { (ctx)->last_cuda = e__; return ATP_ERR_CUDA; } \
+    } while (0)
+
+// After a kernel launch: count it and surface launch-configuration errors.
+#define ATP_LAUNCHED(ctx)                                        \
+    do {                                                         \
+        (ctx)->launches++;                                       \
+        cudaError_t e__ = cudaGetLastError();                    \
+        if (e__ != cudaSuccess) { (ctx)->last_cuda = e__; return ATP_ERR_CUDA; } \
+    } while (0)
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// Bump allocator over the caller's workspace (host-side bookkeeping only).
+struct Arena {
+    char *base; size_t cap; size_t off = 0; bool overflow = false;
+    Arena(void *b, size_t c) : base((char *)b), cap(c) {}
+    template <typename T> T *take(size_t n) {
+        off = align_up(off, 256);
+        size_t bytes = n * sizeof(T);
+        T *p = (T *)(base ? base + off : nullptr);
+        off += bytes;
+        if (off > cap) overflow = true;
+        return p;
+    }
+};
+
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// splitmix64 finaliser used as a counter-based generator: value = mix(seed, counter).
+__host__ __device__ __forceinline__ uint64_t mix64(uint64_t seed, uint64_t ctr) {
+    uint64_t z = seed + 0x9E3779B97F4A7C15ull * (ctr + 1);
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+__device__ __forceinline__ float hash_uniform(uint64_t seed, uint64_t ctr) {   // in (-1, 1)
+    return ((float)(mix64(seed, ctr) >> 40) + 0.5f) * (2.0f / 16777216.0f) - 1.0f;
+}
+
+__device__ __forceinline__ void raise_status(int *dev_status, int code) { atomicCAS(dev_status, 0, code); }
+
+static inline size_t dtype_size(atp_dtype t) { return t == ATP_BF16 ? 2 : 4; }
+
+// Per-sequence sizes of a packed batch, host side.
+struct SeqDims { int row0, L, r, rank0; };
+atp_status check_seqs(const atp_seqs *s, std::vector<SeqDims> &out, int64_t total_rows_expected);
+atp_status check_mat(const atp_mat *m, bool need_data = true);
