@@ -44,6 +44,13 @@
 extern "C" {
 #endif
 
+/* Exported symbols (the library is built with hidden default visibility). */
+#if defined(__GNUC__)
+#define ATP_API __attribute__((visibility("default")))
+#else
+#define ATP_API
+#endif
+
 typedef enum {
     ATP_OK = 0,
     ATP_ERR_INVALID_ARG = 1,
@@ -104,23 +111,23 @@ typedef struct {
 typedef struct atp_ctx atp_ctx;
 
 /* Context: binds a CUDA device; holds the stream, the workspace pointer and the status word. */
-atp_status atp_create(atp_ctx **ctx, int device);
-atp_status atp_destroy(atp_ctx *ctx);
+ATP_API atp_status atp_create(atp_ctx **ctx, int device);
+ATP_API atp_status atp_destroy(atp_ctx *ctx);
 /* cuda_stream is a cudaStream_t (NULL = default stream). */
-atp_status atp_set_stream(atp_ctx *ctx, void *cuda_stream);
+ATP_API atp_status atp_set_stream(atp_ctx *ctx, void *cuda_stream);
 /* Scratch bytes `op` needs for this batch (d = columns of X / X_r; d_out = columns of the widest
  * weight the call will see, i.e. d' for attention, d_out for a linear layer, ignored otherwise). */
-atp_status atp_workspace_bytes(atp_ctx *ctx, int op, const atp_seqs *seqs, int64_t d, int64_t d_out,
+ATP_API atp_status atp_workspace_bytes(atp_ctx *ctx, int op, const atp_seqs *seqs, int64_t d, int64_t d_out,
                                atp_dtype dtype, size_t *bytes);
 /* dev_ptr: device memory, 256-byte aligned, stays owned by the caller. Contents are scratch. */
-atp_status atp_set_workspace(atp_ctx *ctx, void *dev_ptr, size_t bytes);
+ATP_API atp_status atp_set_workspace(atp_ctx *ctx, void *dev_ptr, size_t bytes);
 
 /*
  * Norm box of Fig. 3 (unit gain): Y = norm(X + residual). RMSNorm x/sqrt(mean(x^2)+eps) or
  * LayerNorm (x-mean)/sqrt(var+eps), row by row, statistics in fp32. residual is nullable.
  * Y may alias X. All three share shape (rows x cols) and dtype.
  */
-atp_status atp_input_norm(atp_ctx *ctx, const atp_mat *X, const atp_mat *residual, int kind, float eps,
+ATP_API atp_status atp_input_norm(atp_ctx *ctx, const atp_mat *X, const atp_mat *residual, int kind, float eps,
                           atp_mat *Y);
 
 /*
@@ -138,7 +145,7 @@ atp_status atp_input_norm(atp_ctx *ctx, const atp_mat *X, const atp_mat *residua
  *   sigma  out  device, sum(r_b) floats, nullable
  * Requires 1 <= r_b <= min(L_b, d) (else ATP_ERR_INVALID_RANK).
  */
-atp_status atp_principal_basis(atp_ctx *ctx, const atp_mat *X, const atp_seqs *seqs,
+ATP_API atp_status atp_principal_basis(atp_ctx *ctx, const atp_mat *X, const atp_seqs *seqs,
                                const atp_basis_opts *opts, atp_mat *U_r, atp_mat *X_r, float *sigma);
 
 /*
@@ -150,7 +157,7 @@ atp_status atp_principal_basis(atp_ctx *ctx, const atp_mat *X, const atp_seqs *s
  *   W_*  in  d x d' each (so that X W matches Eq. 2); heads must divide d'
  *   O    out sum(L_b) x d', same dtype as U_r
  */
-atp_status atp_attention(atp_ctx *ctx, const atp_mat *X, const atp_mat *U_r, const atp_mat *X_r,
+ATP_API atp_status atp_attention(atp_ctx *ctx, const atp_mat *X, const atp_mat *U_r, const atp_mat *X_r,
                          const atp_mat *W_Q, const atp_mat *W_K, const atp_mat *W_V, int heads,
                          const atp_seqs *seqs, const atp_attn_opts *opts, atp_mat *O);
 
@@ -159,14 +166,14 @@ atp_status atp_attention(atp_ctx *ctx, const atp_mat *X, const atp_mat *U_r, con
  * with ATP_ACT_SWIGLU, Y = silu(U_r (X_r W_gate)) * (U_r (X_r W)). GELU is the erf form.
  *   W  in  d_in x d_out;  Y out sum(L_b) x d_out, same dtype as U_r
  */
-atp_status atp_lowrank_linear(atp_ctx *ctx, const atp_mat *U_r, const atp_mat *X_r, const atp_mat *W,
+ATP_API atp_status atp_lowrank_linear(atp_ctx *ctx, const atp_mat *U_r, const atp_mat *X_r, const atp_mat *W,
                               const atp_seqs *seqs, const atp_linear_opts *opts, atp_mat *Y);
 
 /* Synchronises the stream, returns and clears the device-side status (ATP_OK if none). */
-atp_status atp_poll_device_status(atp_ctx *ctx);
+ATP_API atp_status atp_poll_device_status(atp_ctx *ctx);
 /* Number of kernels this context has launched since creation (for accounting). */
-int64_t atp_launch_count(const atp_ctx *ctx);
-const char *atp_status_string(atp_status s);
+ATP_API int64_t atp_launch_count(const atp_ctx *ctx);
+ATP_API const char *atp_status_string(atp_status s);
 
 #ifdef __cplusplus
 }

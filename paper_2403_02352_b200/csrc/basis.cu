@@ -313,7 +313,7 @@ jacobi_pair_kernel(const __grid_constant__ JacBatch batch, int step, float tol_r
                 if (fabsf(gpq) > tol_rot * sqrtf(gpp * gqq) && gpq != 0.f) {
                     float zeta = (gqq - gpp) / (2.f * gpq);
                     float t = copysignf(1.f, zeta) / (fabsf(zeta) + sqrtf(1.f + zeta * zeta));
-                    c = rsqrtf(1.f + t * t);
+                    c = 1.f / sqrtf(1.f + t * t);
                     s = c * t;
                     rotated = 1;
                 }

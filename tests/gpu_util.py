@@ -1,0 +1,60 @@
+"""Helpers shared by the GPU parity tests: tensor conversion, error metric, basis invariants."""
+import math
+
+import numpy as np
+import torch
+
+TOL = {"f32": 1e-4, "bf16": 2e-2}          # max relative error bars for O and Y (max|G-R| / max|R|)
+
+
+def tdtype(dtype):
+    return torch.float32 if dtype == "f32" else torch.bfloat16
+
+
+def to_dev(a, dtype, ld_multiple=8):
+    """numpy (float64 holding values of `dtype`) -> CUDA tensor; rows padded so that ld % 8 == 0."""
+    a = np.asarray(a, dtype=np.float64)
+    rows, cols = a.shape
+    ld = (cols + ld_multiple - 1) // ld_multiple * ld_multiple
+    t = torch.zeros((rows, ld), dtype=tdtype(dtype), device="cuda")
+    t[:, :cols] = torch.from_numpy(a).to(tdtype(dtype))
+    return t[:, :cols]
+
+
+def to_np(t):
+    return t.detach().float().cpu().double().numpy()
+
+
+def rel_err(G, R):
+    den = np.abs(R).max()
+    return float(np.abs(G - R).max() / (den if den > 0 else 1.0))
+
+
+def basis_invariants(X, U, Xr, sig):
+    """T1 quantities of one sequence (all float64 numpy)."""
+    r = U.shape[1]
+    s_true = np.linalg.svd(X, compute_uv=False)
+    out = {}
+    out["orth"] = float(np.abs(U.T @ U - np.eye(r)).max())
+    out["xr_vs_utx"] = float(np.abs(Xr - U.T @ X).max() / s_true[0])
+    # quality of the subspace alone: project X on an exactly orthonormalised copy of U
+    Qu, _ = np.linalg.qr(U)
+    res_sub = math.sqrt(max(np.linalg.norm(X) ** 2 - np.linalg.norm(Qu.T @ X) ** 2, 0.0))
+    opt = math.sqrt(float((s_true[r:] ** 2).sum()))
+    out["opt"] = opt
+    out["res_sub"] = res_sub
+    out["res_ratio"] = res_sub / opt if opt > 1e-12 * s_true[0] else 1.0 + res_sub / s_true[0]
+    out["res_pair"] = float(np.linalg.norm(X - U @ Xr))
+    G = Xr @ Xr.T
+    dg = np.sqrt(np.maximum(np.diag(G), 0))
+    den = np.outer(dg, dg)
+    den[den < (1e-12 * s_true[0]) ** 2] = np.inf
+    off = np.abs(G - np.diag(np.diag(G))) / den
+    out["offdiag"] = float(off.max())
+    out["energy_rel"] = float(abs(np.linalg.norm(Xr) ** 2 - (s_true[:r] ** 2).sum()) / (s_true ** 2).sum())
+    rn = np.linalg.norm(Xr, axis=1)
+    out["sigma_vs_rows"] = float(np.abs(sig - rn).max() / s_true[0])
+    out["sorted"] = bool(np.all(np.diff(sig) <= 1e-6 * s_true[0]))
+    out["sigma_rel"] = np.abs(sig - s_true[:r]) / s_true[0]
+    out["s_true"] = s_true
+    return out

@@ -1,0 +1,43 @@
+"""The C-ABI library loads and exports every symbol include/atp.h declares (no compute calls)."""
+import ctypes
+import os
+import re
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "atp.h")).read()
+    return sorted(set(re.findall(r"ATP_API[^;(]*?\b(atp_\w+)\s*\(", text)))
+
+
+def test_header_declares_the_paper_calls():
+    names = declared_symbols()
+    for must in ("atp_principal_basis", "atp_attention", "atp_lowrank_linear", "atp_input_norm",
+                 "atp_create", "atp_destroy", "atp_workspace_bytes", "atp_set_workspace", "atp_poll_device_status"):
+        assert must in names
+
+
+def test_library_exports_every_declared_symbol():
+    from paper_2403_02352_b200 import build
+    lib = ctypes.CDLL(build.build())
+    for name in declared_symbols():
+        assert hasattr(lib, name), name
+
+
+def test_binding_lists_the_same_symbols():
+    import paper_2403_02352_b200 as pkg
+    assert sorted(pkg.exported_symbols) == declared_symbols()
+    pkg.binding.lib.atp_status_string.restype = ctypes.c_char_p
+    assert pkg.binding.status_string(0) == "ok"
+    assert "rank" in pkg.binding.status_string(2)
+
+
+def test_no_fallback_without_cuda():
+    import pytest
+    import torch
+    import paper_2403_02352_b200 as pkg
+    if torch.cuda.is_available():
+        pytest.skip("CUDA present")
+    with pytest.raises(RuntimeError):
+        pkg.Context(0)
