@@ -1,0 +1,307 @@
+#!/usr/bin/env python
+"""Benchmark of the ATP prefill hot path on B200: one "step" is one pass of the whole layer
+(Norm -> basis -> attention on r principal keys -> output projection and FFN through the low-rank
+representation) over one batch of synthetic sequences.
+
+    python bench.py --gpus 1 --steps K --warmup W [--workload NAME] [--rank R]
+    python bench.py --impl reference ...      # the CPU oracle, timed on the host cores
+
+Prints one JSON line (rank 0). With N > 1 ranks (torchrun) every rank processes its own batch of
+independent sequences (no data-path collective): weak scaling.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+import atp_inputs as ai  # noqa: E402
+
+WORKLOADS = {
+    # name: (builder, kwargs, layer composition)
+    "bert_large_bf16": dict(build=lambda r, seed: ai.bert_large_bf16(r=r or 256, seed=seed), default_rank=256),
+    "bert_base_fp32": dict(build=lambda r, seed: ai.bert_base_fp32(r=r or 128, seed=seed - 2000), default_rank=128),
+    "llama7b_bf16": dict(build=lambda r, seed: ai.llama7b_bf16(r=r or 1024, seed=seed + 1000), default_rank=1024),
+    "long_context_bf16": dict(build=lambda r, seed: ai.long_context_bf16(r=r or 1024, seed=seed + 2000), default_rank=1024),
+    "serving_bf16": dict(build=lambda r, seed: ai.serving_batch_bf16(seed=seed + 3000), default_rank=0),
+}
+POST_NORM = {"gelu": "layer", "swiglu": "rms", None: "layer"}
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        m = json.load(open(p))
+        return dict(hbm_gbs=m["hbm_gbs"], bf16_tflops=m["bf16_tflops_sustained"], source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1400.0, source="fallback")
+
+
+FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # 148 SMs x 128 FMA lanes x 2 flop x max SM clock
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return None
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except Exception:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return None
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_step(w, seq_index):
+    import oracle
+    s = w.seqs[seq_index]
+    return oracle.layer_forward(s.X, w.weights, s.r, w.heads, ffn=w.ffn, input_norm=w.input_norm,
+                                post_norm=POST_NORM[w.ffn])
+
+
+def run_reference(args):
+    """The CPU oracle as it stands, on the host cores; each step is one sequence of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    w = WORKLOADS[args.workload]["build"](args.rank, args.seed)
+    nseq = len(w.seqs)
+    for i in range(args.warmup):
+        oracle_step(w, i % nseq)
+    t0 = time.perf_counter()
+    toks = 0
+    for i in range(args.steps):
+        oracle_step(w, i % nseq)
+        toks += w.seqs[i % nseq].X.shape[0]
+    dt = time.perf_counter() - t0
+    val = toks / dt
+    sample = f"one sequence of the batch per step ({w.seqs[0].X.shape[0]} tokens), full layer"
+    line = {"impl": "reference", "metric": "ATP layer prefill tokens/sec", "value": val, "unit": "tokens/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "sequences_per_step": 1, "heads": w.heads, "d": w.d, "rank": w.ranks[0]},
+            "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="bert_large_bf16", choices=sorted(WORKLOADS))
+    ap.add_argument("--rank", type=int, default=0, help="number of principal keys r (0: the workload's default)")
+    ap.add_argument("--seed", type=int, default=2000)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--power-iters", type=int, default=-1)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        if args.steps == 20 and args.warmup == 3:
+            args.steps, args.warmup = 3, 1
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+    import paper_2403_02352_b200 as atp          # raises if libatp.so is missing: no fallback
+    from paper_2403_02352_b200.layer import AtpLayer
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+    args.warmup = max(args.warmup, 3)
+
+    w = WORKLOADS[args.workload]["build"](args.rank, args.seed + 17 * rank)   # every rank: its own sequences
+    tdt = torch.float32 if w.dtype == "f32" else torch.bfloat16
+
+    def dev_mat(a, pin=False):
+        t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(tdt)
+        return t.pin_memory() if pin else t.to(dev)
+
+    weights = {k: dev_mat(v) for k, v in w.weights.items()}
+    Xpacked, row_off, rank_arr, rank_off = ai.pack(w.seqs)
+    lengths, ranks = w.lengths, w.ranks
+    tokens = int(sum(lengths))
+    x_bytes = Xpacked.size * (4 if w.dtype == "f32" else 2)
+    # rotating input sets: the same sequences with rows cyclically shifted per set would change the
+    # problem; instead each set is an independent copy placed at a different address, and the L2 is
+    # flushed between steps, so that no step finds its inputs or weights cached.
+    nsets = max(2, min(8, int(300e6 // max(x_bytes, 1)) + 1))
+    Xsets = [dev_mat(Xpacked) for _ in range(nsets)]
+    Xhost = dev_mat(Xpacked, pin=True)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    ctx = atp.Context(local)
+    layer = AtpLayer(ctx, weights, lengths, ranks, w.heads, ffn=w.ffn, input_norm=w.input_norm,
+                     post_norm=POST_NORM[w.ffn], power_iters=args.power_iters)
+    out_rows, out_cols = None, None
+
+    def step(i):
+        return layer.forward(Xsets[i % nsets])
+
+    for i in range(args.warmup):
+        y = step(i)
+    ctx.poll()
+    out_shape = tuple(y.shape)
+    Yhost = torch.empty(out_shape, dtype=tdt).pin_memory()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-timed region: K steps, CUDA events per step, L2 flushed between steps
+    sampler = ClockSampler(local) if rank == 0 else None
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    launches0 = ctx.launches
+    barrier()
+    if sampler:
+        sampler.start()
+    for i in range(args.steps):
+        flush.zero_()
+        evs[i][0].record()
+        step(i)
+        evs[i][1].record()
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    launches = (ctx.launches - launches0)
+    ctx.poll()
+    ms = sum(a.elapsed_time(b) for a, b in evs)
+    if world > 1:
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    value = world * tokens * args.steps / (ms / 1e3)
+
+    # ---- end to end: pinned host input -> device, layer, result -> host, every step
+    xd = torch.empty_like(Xsets[0])
+    e2e_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    barrier()
+    for i in range(args.steps):
+        flush.zero_()
+        e2e_ev[i][0].record()
+        xd.copy_(Xhost, non_blocking=True)
+        yy = layer.forward(xd)
+        Yhost.copy_(yy, non_blocking=True)
+        e2e_ev[i][1].record()
+    barrier()
+    ms_e2e = sum(a.elapsed_time(b) for a, b in e2e_ev)
+    if world > 1:
+        t = torch.tensor([ms_e2e], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item())
+    e2e = {"value": world * tokens * args.steps / (ms_e2e / 1e3), "unit": "tokens/s",
+           "h2d_bytes_per_step": int(x_bytes), "d2h_bytes_per_step": int(Yhost.numel() * Yhost.element_size())}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- per-kernel times (event pair around every launch; separate pass, not the timed one)
+    pk = peaks()
+    ctx.profile_start()
+    nprof = 2
+    for i in range(nprof):
+        flush.zero_()
+        step(i)
+    prof = ctx.profile_stop()
+    total_ms = sum(v["ms"] for v in prof.values()) or 1.0
+    dom_name, dom = max(prof.items(), key=lambda kv: kv[1]["ms"])
+    per_launch_s = dom["ms"] / 1e3 / max(dom["launches"], 1)
+    ridge = pk["bf16_tflops"] * 1e12 / (pk["hbm_gbs"] * 1e9)
+    if dom_name.endswith("_simt") or dom_name.startswith("jacobi"):
+        bound, peak, unit = "alu", FP32_ALU_TFLOPS, "TFLOP/s"
+        achieved = dom["flops"] / max(dom["launches"], 1) / per_launch_s / 1e12
+    elif dom["flops"] > 0 and dom["flops"] / max(dom["bytes"], 1.0) > ridge:
+        bound, peak, unit = "tensor", pk["bf16_tflops"], "TFLOP/s"
+        achieved = dom["flops"] / max(dom["launches"], 1) / per_launch_s / 1e12
+    else:
+        bound, peak, unit = "hbm", pk["hbm_gbs"], "GB/s"
+        achieved = dom["bytes"] / max(dom["launches"], 1) / per_launch_s / 1e9
+    roofline = {"kernel": dom_name, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
+                "frac": achieved / peak, "traffic": None, "peak_source": pk["source"],
+                "share_of_step": dom["ms"] / total_ms,
+                "kernels": {k: {"launches": v["launches"] // nprof, "ms_per_step": v["ms"] / nprof,
+                                "share": v["ms"] / total_ms} for k, v in sorted(prof.items(), key=lambda kv: -kv[1]["ms"])}}
+
+    # ---- CPU baseline: the oracle on a bounded sample of the same workload
+    cpu = None
+    if not args.no_cpu_baseline and world == 1:
+        import oracle
+        t0 = time.perf_counter()
+        n = 0
+        toks = 0
+        while n < len(w.seqs) and (time.perf_counter() - t0 < 15.0 or n == 0):
+            oracle_step(w, n)
+            toks += w.seqs[n].X.shape[0]
+            n += 1
+        dt = time.perf_counter() - t0
+        cpu = {"value": toks / dt, "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle",
+               "sample": f"{n} of {len(w.seqs)} sequences ({toks} tokens), full layer, {dt:.1f} s"}
+
+    line = {"metric": "ATP layer prefill tokens/sec", "value": value, "unit": "tokens/s", "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
+            "config": {"workload": w.name, "batch": len(lengths), "tokens_per_step_per_gpu": tokens, "d": w.d,
+                       "heads": w.heads, "rank": ranks[0] if len(set(ranks)) == 1 else "L_b/4",
+                       "ffn": w.ffn, "d_ff": w.d_ff, "input_norm": w.input_norm,
+                       "layer": "basis+attention" + ("+W_O" if "W_O" in w.weights else "") + ("+FFN" if w.ffn else ""),
+                       "l2": "flushed between steps (256 MiB memset), %d rotating input copies" % nsets,
+                       "parallelism": f"dp{world} (independent sequences per rank)"},
+            "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

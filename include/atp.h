@@ -175,6 +175,17 @@ ATP_API atp_status atp_poll_device_status(atp_ctx *ctx);
 ATP_API int64_t atp_launch_count(const atp_ctx *ctx);
 ATP_API const char *atp_status_string(atp_status s);
 
+/*
+ * Per-kernel timing (tracing aid, not part of the paper's method). Between start and stop every
+ * kernel launch of this context is bracketed by a pair of CUDA events on the context's stream,
+ * which slows the calls down: never leave it on while measuring throughput. stop synchronises and
+ * writes one text line per kernel name into buf (host memory, cap bytes, always NUL-terminated):
+ *   "<name> <launches> <total ms> <algorithmic flops> <algorithmic bytes>\n"
+ * *needed (nullable) receives the size a complete report takes.
+ */
+ATP_API atp_status atp_profile_start(atp_ctx *ctx);
+ATP_API atp_status atp_profile_stop(atp_ctx *ctx, char *buf, size_t cap, size_t *needed);
+
 #ifdef __cplusplus
 }
 #endif

@@ -121,3 +121,34 @@ def svd_entropy(sigma) -> float:
     """Eq. 4 with log base 2."""
     sigma = _c(sigma)
     return float(_load().oracle_svd_entropy(_p(sigma), sigma.shape[0]))
+
+
+def layer_forward(X, weights, r, heads, ffn=None, input_norm=None, post_norm="layer", stages=None):
+    """One ATP layer (Fig. 3) for a single sequence, composed from the functions above: Norm,
+    basis, attention on r principal keys, then output projection and FeedForward, each linear layer
+    applied to the principal basis of its own input (same r). `stages` (a dict) receives the
+    intermediate results when given. Returns the layer output."""
+    st = {} if stages is None else stages
+    Xin = norm(X, kind=input_norm) if input_norm else np.asarray(X, dtype=np.float64)
+    U, Xr, _ = principal_basis(Xin, r)
+    O = attention(Xin, U, Xr, weights["W_Q"], weights["W_K"], weights["W_V"], heads)
+    st.update(Xin=Xin, U=U, Xr=Xr, O=O)
+    if "W_O" not in weights:
+        return O
+    Uo, Or, _ = principal_basis(O, r)
+    A = lowrank_linear(Uo, Or, weights["W_O"])
+    st.update(A=A)
+    if not ffn:
+        return A
+    H = norm(X, residual=A, kind=post_norm)
+    Uh, Hr, _ = principal_basis(H, r)
+    if ffn == "gelu":
+        F = lowrank_linear(Uh, Hr, weights["W_1"], act="gelu")
+        Uf, Fr, _ = principal_basis(F, r)
+        Y = lowrank_linear(Uf, Fr, weights["W_2"])
+    else:
+        F = lowrank_linear(Uh, Hr, weights["W_up"], W_gate=weights["W_gate"], act="swiglu")
+        Uf, Fr, _ = principal_basis(F, r)
+        Y = lowrank_linear(Uf, Fr, weights["W_down"])
+    st.update(H=H, F=F, Y=Y)
+    return Y

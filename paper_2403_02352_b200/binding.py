@@ -22,7 +22,7 @@ NORM = {"rms": 0, "layer": 1}
 exported_symbols = (
     "atp_create", "atp_destroy", "atp_set_stream", "atp_workspace_bytes", "atp_set_workspace",
     "atp_input_norm", "atp_principal_basis", "atp_attention", "atp_lowrank_linear",
-    "atp_poll_device_status", "atp_launch_count", "atp_status_string",
+    "atp_poll_device_status", "atp_launch_count", "atp_status_string", "atp_profile_start", "atp_profile_stop",
 )
 
 
@@ -73,6 +73,8 @@ def _load():
     lib.atp_workspace_bytes.argtypes = [C.c_void_p, C.c_int, C.POINTER(Seqs), C.c_int64, C.c_int64, C.c_int,
                                         C.POINTER(C.c_size_t)]
     lib.atp_poll_device_status.argtypes = [C.c_void_p]
+    lib.atp_profile_start.argtypes = [C.c_void_p]
+    lib.atp_profile_stop.argtypes = [C.c_void_p, C.c_char_p, C.c_size_t, C.POINTER(C.c_size_t)]
     lib.atp_input_norm.argtypes = [C.c_void_p, C.POINTER(Mat), C.POINTER(Mat), C.c_int, C.c_float, C.POINTER(Mat)]
     lib.atp_principal_basis.argtypes = [C.c_void_p, C.POINTER(Mat), C.POINTER(Seqs), C.POINTER(BasisOpts),
                                         C.POINTER(Mat), C.POINTER(Mat), C.c_void_p]
@@ -187,6 +189,19 @@ class Context:
     def poll(self):
         """Synchronise and raise if a kernel recorded a device-side condition."""
         _check(lib.atp_poll_device_status(self._h), "device status")
+
+    def profile_start(self):
+        _check(lib.atp_profile_start(self._h), "atp_profile_start")
+
+    def profile_stop(self):
+        """Returns {kernel name: dict(launches, ms, flops, bytes)} for the launches since profile_start."""
+        buf = C.create_string_buffer(1 << 16)
+        _check(lib.atp_profile_stop(self._h, buf, len(buf), None), "atp_profile_stop")
+        out = {}
+        for line in buf.value.decode().splitlines():
+            name, n, ms, fl, by = line.split()
+            out[name] = dict(launches=int(n), ms=float(ms), flops=float(fl), bytes=float(by))
+        return out
 
     @property
     def launches(self) -> int:

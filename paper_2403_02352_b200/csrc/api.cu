@@ -1,6 +1,9 @@
 // Context management, argument validation, status handling and the Norm box of Fig. 3.
 #include "common.cuh"
 #include <new>
+#include <string>
+#include <string.h>
+#include <stdio.h>
 
 atp_status check_mat(const atp_mat *m, bool need_data)
 {
@@ -97,6 +100,46 @@ atp_status atp_poll_device_status(atp_ctx *ctx)
 
 int64_t atp_launch_count(const atp_ctx *ctx) { return ctx ? ctx->launches : -1; }
 
+atp_status atp_profile_start(atp_ctx *ctx)
+{
+    if (!ctx) return ATP_ERR_INVALID_ARG;
+    ctx->profiling = true;
+    return ATP_OK;
+}
+
+atp_status atp_profile_stop(atp_ctx *ctx, char *buf, size_t cap, size_t *needed)
+{
+    if (!ctx) return ATP_ERR_INVALID_ARG;
+    ctx->profiling = false;
+    ATP_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+    ATP_CUDA_OK(ctx, cudaStreamSynchronize(ctx->stream));
+    struct Agg { const char *name; long n; double ms, flops, bytes; };
+    std::vector<Agg> agg;
+    for (auto &r : ctx->recs) {
+        float ms = 0.f;
+        cudaEventElapsedTime(&ms, r.a, r.b);
+        cudaEventDestroy(r.a); cudaEventDestroy(r.b);
+        size_t i = 0;
+        for (; i < agg.size(); ++i) if (!strcmp(agg[i].name, r.name)) break;
+        if (i == agg.size()) agg.push_back(Agg{r.name, 0, 0, 0, 0});
+        agg[i].n++; agg[i].ms += ms; agg[i].flops += r.flops; agg[i].bytes += r.bytes;
+    }
+    ctx->recs.clear();
+    std::string out;
+    char line[256];
+    for (auto &a : agg) {
+        snprintf(line, sizeof line, "%s %ld %.6f %.6e %.6e\n", a.name, a.n, a.ms, a.flops, a.bytes);
+        out += line;
+    }
+    if (needed) *needed = out.size() + 1;
+    if (buf && cap > 0) {
+        size_t n = out.size() < cap - 1 ? out.size() : cap - 1;
+        memcpy(buf, out.data(), n);
+        buf[n] = 0;
+    }
+    return ATP_OK;
+}
+
 const char *atp_status_string(atp_status s)
 {
     switch (s) {
@@ -177,6 +220,7 @@ extern "C" atp_status atp_input_norm(atp_ctx *ctx, const atp_mat *X, const atp_m
     ATP_CUDA_OK(ctx, cudaSetDevice(ctx->device));
     int rows = (int)X->rows, cols = (int)X->cols;
     dim3 grid(ceil_div(rows, 8));
+    ATP_KERNEL(ctx, "norm", 0, (double)rows * cols * dtype_size(X->dtype) * (residual ? 3 : 2));
     if (X->dtype == ATP_F32)
         norm_kernel<float><<<grid, 256, 0, ctx->stream>>>((const float *)X->data, residual ? (const float *)residual->data : nullptr,
                                                           (float *)Y->data, rows, cols, (int)X->ld, residual ? (int)residual->ld : 0,

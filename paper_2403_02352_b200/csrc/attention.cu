@@ -176,16 +176,19 @@ static atp_status attention_impl(atp_ctx *ctx, const atp_mat *X, const atp_mat *
     size_t smem = ((size_t)dh * 68 * 2 + (size_t)64 * dh + 64 * 65) * sizeof(float);
     ATP_CUDA_OK(ctx, cudaFuncSetAttribute(attn_simt_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     for (size_t i = 0; i < seqs.size(); i += ATT_MAX_BATCH) {
-        AttnBatch ab; ab.count = 0; int maxL = 0;
+        AttnBatch ab; ab.count = 0; int maxL = 0; double fl = 0, by = 0;
         for (size_t j = i; j < seqs.size() && ab.count < ATT_MAX_BATCH; ++j) {
             const SeqDims &s = seqs[j];
             if (s.L == 0) continue;
             ab.s[ab.count++] = AttnSeq{pl.Q + (size_t)s.row0 * dp, pl.Kp + (size_t)s.rank0 * dp, pl.Vp + (size_t)s.rank0 * dp,
                                        (T *)O->data + (size_t)s.row0 * O->ld, s.L, s.r};
             if (s.L > maxL) maxL = s.L;
+            fl += 4.0 * s.L * s.r * dp;
+            by += (2.0 * s.r * dp + s.L * dp) * sizeof(float) + (double)s.L * dp * sizeof(T);
         }
         if (ab.count == 0) continue;
         dim3 grid(ceil_div(maxL, 64), heads, ab.count);
+        ATP_KERNEL(ctx, "attn_simt", fl, by);
         attn_simt_kernel<T><<<grid, 256, smem, ctx->stream>>>(ab, dh, dp, dp, (int)O->ld, scale);
         ATP_LAUNCHED(ctx);
     }

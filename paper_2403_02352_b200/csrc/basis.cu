@@ -609,10 +609,13 @@ static atp_status orthonormalise(atp_ctx *ctx, BasisPlan &bp, size_t i0, size_t 
                                                                       bp.part_stride)) != ATP_OK) return st;
                 if ((st = launch_gemm_simt<float, float, float, false>(ctx, upd, GemmEpi{EPI_D_MINUS, nullptr})) != ATP_OK) return st;
             }
+            ATP_KERNEL(ctx, "panel_gram", 0, 0);
             panel_gram_kernel<<<dim3(ceil_div(maxn, GRAM_ROWS), pb.count), 256, 0, ctx->stream>>>(pb);
             ATP_LAUNCHED(ctx);
+            ATP_KERNEL(ctx, "panel_chol", 0, 0);
             panel_chol_kernel<<<pb.count, 256, CHOL_SMEM, ctx->stream>>>(pb);
             ATP_LAUNCHED(ctx);
+            ATP_KERNEL(ctx, "panel_apply", 0, 0);
             panel_apply_kernel<<<dim3(ceil_div(maxn, 64), pb.count), 256, 0, ctx->stream>>>(
                 pb, seed + 7919ull * (uint64_t)(pj * 2 + rep) + (z_side ? 104729ull : 0ull));
             ATP_LAUNCHED(ctx);
@@ -633,6 +636,7 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
     atp_status st;
     {
         size_t n = (size_t)d * bp.rtmax;
+        ATP_KERNEL(ctx, "fill_omega", 0, 0);
         fill_omega_kernel<<<(unsigned)std::min<size_t>((n + 255) / 256, 4096), 256, 0, ctx->stream>>>(bp.omega, n, seed);
         ATP_LAUNCHED(ctx);
     }
@@ -683,23 +687,29 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
         }
         if (maxrt == 0) continue;
         if ((st = launch_gemm_simt<float, T, float, true>(ctx, g, store)) != ATP_OK) return st;
+        ATP_KERNEL(ctx, "init_w", 0, 0);
         init_w_kernel<<<dim3(64, cnt), 256, 0, ctx->stream>>>(jb);
         ATP_LAUNCHED(ctx);
         for (int sw = 0; sw < max_sweeps; ++sw) {
             for (int step = 0; step < maxnb - 1; ++step) {
+                ATP_KERNEL(ctx, "jacobi_pair", 0, 0);
                 jacobi_pair_kernel<<<dim3(maxnb / 2, cnt), 256, 0, ctx->stream>>>(jb, step, tol_rot, tol_rot);
                 ATP_LAUNCHED(ctx);
             }
+            ATP_KERNEL(ctx, "jacobi_sweep_end", 0, 0);
             jacobi_sweep_end_kernel<<<1, BMAX, 0, ctx->stream>>>(jb, tol_conv, sw == max_sweeps - 1, ctx->dev_status);
             ATP_LAUNCHED(ctx);
         }
         int npow = 1; while (npow < maxrt) npow <<= 1;
         size_t sm = (size_t)npow * 8;
         if (sm > 48 * 1024) ATP_CUDA_OK(ctx, cudaFuncSetAttribute(sigma_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm));
+        ATP_KERNEL(ctx, "sigma_sort", 0, 0);
         sigma_sort_kernel<<<cnt, 1024, sm, ctx->stream>>>(fb);
         ATP_LAUNCHED(ctx);
+        ATP_KERNEL(ctx, "colsum", 0, 0);
         colsum_kernel<<<dim3(ceil_div(maxrt, 128), cnt), 128, 0, ctx->stream>>>(fb);
         ATP_LAUNCHED(ctx);
+        ATP_KERNEL(ctx, "select", 0, 0);
         select_kernel<T><<<dim3(maxr, cnt), 256, 0, ctx->stream>>>(fb);
         ATP_LAUNCHED(ctx);
         // U_r = Y Wsel

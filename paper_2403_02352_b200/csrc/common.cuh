@@ -7,7 +7,13 @@
 #include <vector>
 #include "atp.h"
 
+// One record per kernel launch while profiling is on (see atp_profile_start).
+struct ProfRec { const char *name; cudaEvent_t a, b; double flops, bytes; };
+
 struct atp_ctx {
+    bool profiling = false;
+    bool prof_open = false;
+    std::vector<ProfRec> recs;
     int device = 0;
     cudaStream_t stream = nullptr;
     void *workspace = nullptr;
@@ -24,10 +30,27 @@ struct atp_ctx {
         if (e__ != cudaSuccess) { (ctx)->last_cuda = e__; return ATP_ERR_CUDA; } \
     } while (0)
 
+// Before a kernel launch: name it and state its algorithmic work (used only while profiling).
+static inline void prof_begin(atp_ctx *ctx, const char *name, double flops, double bytes)
+{
+    if (!ctx->profiling) return;
+    ProfRec r{name, nullptr, nullptr, flops, bytes};
+    if (cudaEventCreate(&r.a) != cudaSuccess || cudaEventCreate(&r.b) != cudaSuccess) return;
+    cudaEventRecord(r.a, ctx->stream);
+    ctx->recs.push_back(r);
+    ctx->prof_open = true;
+}
+static inline void prof_end(atp_ctx *ctx)
+{
+    if (ctx->prof_open) { cudaEventRecord(ctx->recs.back().b, ctx->stream); ctx->prof_open = false; }
+}
+#define ATP_KERNEL(ctx, name, flops, bytes) prof_begin((ctx), (name), (double)(flops), (double)(bytes))
+
 // After a kernel launch: count it and surface launch-configuration errors.
 #define ATP_LAUNCHED(ctx)                                        \
     do {                                                         \
         (ctx)->launches++;                                       \
+        prof_end(ctx);                                           \
         cudaError_t e__ = cudaGetLastError();                    \
         if (e__ != cudaSuccess) { (ctx)->last_cuda = e__; return ATP_ERR_CUDA; } \
     } while (0)

@@ -157,12 +157,20 @@ static atp_status launch_gemm_simt(atp_ctx *ctx, const GemmBatch &batch, GemmEpi
     }
     if (maxM == 0 || maxN == 0 || batch.count == 0) return ATP_OK;
     if (splits < 1 || !part) splits = 1;
+    double flops = 0, bytes = 0;
+    for (int i = 0; i < batch.count; ++i) {
+        const GemmProblem &q = batch.p[i];
+        flops += 2.0 * q.M * q.N * q.K;
+        bytes += (double)q.M * q.K * sizeof(TA) + (double)q.K * q.N * sizeof(TB) + (double)q.M * q.N * sizeof(TC);
+    }
     dim3 grid(ceil_div(maxN, 64), ceil_div(maxM, 64), batch.count * splits);
+    ATP_KERNEL(ctx, "gemm_simt", flops, bytes);
     gemm_simt_kernel<TA, TB, TC, TRANS_A><<<grid, 256, 0, ctx->stream>>>(batch, epi, splits, part, part_stride);
     ATP_LAUNCHED(ctx);
     if (splits > 1) {
         int blocks = ceil_div(maxM * maxN, 256);
         if (blocks > 1024) blocks = 1024;
+        ATP_KERNEL(ctx, "gemm_splitk_reduce", 0, 0);
         gemm_splitk_reduce_kernel<TC><<<dim3(blocks, batch.count), 256, 0, ctx->stream>>>(batch, splits, part, part_stride);
         ATP_LAUNCHED(ctx);
     }

@@ -1,0 +1,98 @@
+"""One ATP layer as a sequence of C-ABI calls (Fig. 3): Norm -> basis -> attention on r principal
+keys -> output projection and FeedForward through the low-rank representation.
+
+The composition for the linear layers follows the paper's remark that the next stage "first attains
+principal components" of its input: every linear layer sees (U_r, X_r) of its own input, with the
+same rank r. All buffers are allocated once, here; forward() only issues library calls.
+"""
+from __future__ import annotations
+
+from typing import Dict, Optional, Sequence
+
+import torch
+
+from . import binding as B
+
+
+class AtpLayer:
+    def __init__(self, ctx: B.Context, weights: Dict[str, torch.Tensor], lengths: Sequence[int], ranks: Sequence[int],
+                 heads: int, ffn: Optional[str] = None, input_norm: Optional[str] = None, post_norm: str = "layer",
+                 blocks: str = "auto", power_iters: int = -1, oversample: int = -1, seed: int = 0):
+        self.ctx, self.w = ctx, weights
+        self.lengths, self.ranks = [int(x) for x in lengths], [int(x) for x in ranks]
+        self.heads, self.ffn, self.input_norm, self.post_norm = heads, ffn, input_norm, post_norm
+        self.power_iters, self.oversample, self.seed = power_iters, oversample, seed
+        self.has_wo = "W_O" in weights
+        self.dtype = weights["W_Q"].dtype
+        self.device = weights["W_Q"].device
+        self.d = weights["W_Q"].shape[0]
+        self.dp = weights["W_Q"].shape[1]
+        self.d_ff = 0
+        if ffn == "gelu":
+            self.d_ff = weights["W_1"].shape[1]
+        elif ffn == "swiglu":
+            self.d_ff = weights["W_up"].shape[1]
+        rows, tr, maxr = sum(self.lengths), sum(self.ranks), max(self.ranks)
+        ldu = (maxr + 7) // 8 * 8
+
+        def buf(r, c):
+            return torch.empty((r, (c + 7) // 8 * 8), dtype=self.dtype, device=self.device)[:, :c]
+
+        def basis_out(cols):
+            return (torch.zeros((rows, ldu), dtype=self.dtype, device=self.device)[:, :maxr], buf(tr, cols),
+                    torch.empty(tr, dtype=torch.float32, device=self.device))
+
+        self.Xn = buf(rows, self.d) if input_norm else None
+        self.bX = basis_out(self.d)
+        self.O = buf(rows, self.dp)
+        if self.has_wo:
+            self.bO = basis_out(self.dp)
+            self.A = buf(rows, self.d)
+        if ffn:
+            self.H = buf(rows, self.d)
+            self.bH = basis_out(self.d)
+            self.F = buf(rows, self.d_ff)
+            self.bF = basis_out(self.d_ff)
+            self.Y = buf(rows, self.d)
+        # one workspace large enough for every call of the layer
+        sd = B.SeqDesc(self.lengths, self.ranks)
+        dt = B._dt(weights["W_Q"])
+        need = max(ctx.workspace_bytes(B.OP_BASIS, sd, max(self.d, self.dp, self.d_ff), 0, dt),
+                   ctx.workspace_bytes(B.OP_ATTENTION, sd, self.d, self.dp, dt),
+                   ctx.workspace_bytes(B.OP_LINEAR, sd, max(self.d, self.d_ff), max(self.d, self.d_ff), dt))
+        ctx.ensure_workspace(need)
+
+    def _basis(self, X, out):
+        return B.atp_principal_basis(self.ctx, X, self.lengths, self.ranks, oversample=self.oversample,
+                                     power_iters=self.power_iters, seed=self.seed, out=out, auto_workspace=False)
+
+    def _linear(self, basis, W, out, act=None, W_gate=None):
+        return B.atp_lowrank_linear(self.ctx, basis[0], basis[1], W, self.lengths, self.ranks, act=act, W_gate=W_gate,
+                                    out=out, auto_workspace=False)
+
+    def forward(self, X: torch.Tensor) -> torch.Tensor:
+        """Returns the layer output (Y with an FFN, else the projected attention output, else O)."""
+        c, w = self.ctx, self.w
+        Xin = X
+        if self.input_norm:
+            Xin = B.atp_input_norm(c, X, None, kind=self.input_norm, out=self.Xn)
+        self._basis(Xin, self.bX)
+        B.atp_attention(c, Xin, self.bX[0], self.bX[1], w["W_Q"], w["W_K"], w["W_V"], self.heads, self.lengths,
+                        self.ranks, out=self.O, auto_workspace=False)
+        if not self.has_wo:
+            return self.O
+        self._basis(self.O, self.bO)
+        self._linear(self.bO, w["W_O"], self.A)
+        if not self.ffn:
+            return self.A
+        B.atp_input_norm(c, X, self.A, kind=self.post_norm, out=self.H)        # H = Norm(X + A)
+        self._basis(self.H, self.bH)
+        if self.ffn == "gelu":
+            self._linear(self.bH, w["W_1"], self.F, act="gelu")
+            self._basis(self.F, self.bF)
+            self._linear(self.bF, w["W_2"], self.Y)
+        else:
+            self._linear(self.bH, w["W_up"], self.F, act="swiglu", W_gate=w["W_gate"])
+            self._basis(self.F, self.bF)
+            self._linear(self.bF, w["W_down"], self.Y)
+        return self.Y
