@@ -60,7 +60,8 @@ typedef enum {
     ATP_ERR_CUDA = 5,
     ATP_ERR_NOT_CONVERGED = 6,
     ATP_ERR_TIMEOUT = 7,
-    ATP_ERR_RANGE = 8
+    ATP_ERR_RANGE = 8,
+    ATP_ERR_STATIC_SCRATCH_LIMIT = 9
 } atp_status;
 
 typedef enum { ATP_F32 = 0, ATP_BF16 = 1 } atp_dtype;
@@ -185,6 +186,31 @@ ATP_API const char *atp_status_string(atp_status s);
  */
 ATP_API atp_status atp_profile_start(atp_ctx *ctx);
 ATP_API atp_status atp_profile_stop(atp_ctx *ctx, char *buf, size_t cap, size_t *needed);
+
+/*
+ * Low-rank linear layer without any allocation (the paper has no counterpart: this entry point
+ * exists for deployment, not for the method). It computes what atp_lowrank_linear computes,
+ * Y = act(U_r (X_r W) + bias) with act NONE or GELU, for callers that may not allocate device
+ * memory at all: code running inside another program's memory pool, or a latency-critical loop
+ * where cudaMalloc / cudaFree are forbidden. Such callers cannot use atp_create (it allocates a
+ * status word) nor supply a workspace, so this call takes no context: it runs on the device that
+ * is current, on the given stream (cudaStream_t, NULL = default), and keeps its intermediate
+ * X_r W in a fixed buffer of ATP_STATIC_SCRATCH_BYTES that is part of the library image. Every GPU
+ * that loads the library holds that buffer until the process exits.
+ *   - It calls no cudaMalloc, cudaFree or other allocating routine; inputs and outputs are the
+ *     caller's, as in atp_lowrank_linear (same layouts, same dtype rules). SwiGLU is not offered.
+ *   - Limit: sum(r_b) * d_out * 4 bytes must fit in ATP_STATIC_SCRATCH_BYTES, otherwise
+ *     ATP_ERR_STATIC_SCRATCH_LIMIT is returned and nothing is launched.
+ *   - The first call on each device looks up the buffer's device address; make that first call
+ *     before starting any stream capture on that device.
+ *   - All calls share the one buffer, and it keeps whatever the previous call left in it. The
+ *     intermediate is rewritten in full before it is read, so no clearing is needed, but two calls
+ *     that overlap on the GPU (different streams, no ordering between them) race on it: order them.
+ */
+#define ATP_STATIC_SCRATCH_BYTES (8u << 20)
+ATP_API atp_status atp_lowrank_linear_static(void *cuda_stream, const atp_mat *U_r, const atp_mat *X_r,
+                                             const atp_mat *W, const atp_seqs *seqs, const atp_linear_opts *opts,
+                                             atp_mat *Y);
 
 #ifdef __cplusplus
 }

@@ -12,7 +12,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libatp.so")
 
 OK, ERR_INVALID_ARG, ERR_INVALID_RANK, ERR_UNSUPPORTED_DTYPE, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, \
-    ERR_NOT_CONVERGED, ERR_TIMEOUT, ERR_RANGE = range(9)
+    ERR_NOT_CONVERGED, ERR_TIMEOUT, ERR_RANGE, ERR_STATIC_SCRATCH_LIMIT = range(10)
+STATIC_SCRATCH_BYTES = 8 << 20
 F32, BF16 = 0, 1
 OP_BASIS, OP_ATTENTION, OP_LINEAR, OP_NORM = 0, 1, 2, 3
 Q_LOWRANK, Q_FULL = 0, 1
@@ -23,6 +24,7 @@ exported_symbols = (
     "atp_create", "atp_destroy", "atp_set_stream", "atp_workspace_bytes", "atp_set_workspace",
     "atp_input_norm", "atp_principal_basis", "atp_attention", "atp_lowrank_linear",
     "atp_poll_device_status", "atp_launch_count", "atp_status_string", "atp_profile_start", "atp_profile_stop",
+    "atp_lowrank_linear_static",
 )
 
 
@@ -83,6 +85,8 @@ def _load():
                                   C.POINTER(Mat)]
     lib.atp_lowrank_linear.argtypes = [C.c_void_p, C.POINTER(Mat), C.POINTER(Mat), C.POINTER(Mat), C.POINTER(Seqs),
                                        C.POINTER(LinearOpts), C.POINTER(Mat)]
+    lib.atp_lowrank_linear_static.argtypes = [C.c_void_p, C.POINTER(Mat), C.POINTER(Mat), C.POINTER(Mat),
+                                              C.POINTER(Seqs), C.POINTER(LinearOpts), C.POINTER(Mat)]
     return lib
 
 
@@ -282,3 +286,17 @@ def atp_lowrank_linear(ctx: Context, U_r, X_r, W, lengths, ranks, bias=None, act
     _check(lib.atp_lowrank_linear(ctx._h, C.byref(ms[0]), C.byref(ms[1]), C.byref(ms[2]), C.byref(sd.c), C.byref(opts),
                                   C.byref(ms[3])), "atp_lowrank_linear")
     return Y
+
+
+def atp_lowrank_linear_static(U_r, X_r, W, lengths, ranks, out, bias=None, act=None, stream=None):
+    """Y = act(U_r (X_r W) + bias) through the entry point that allocates nothing: no context, no
+    workspace; the intermediate lives in a fixed buffer inside the library (see include/atp.h for
+    the size limit and the rules on overlapping calls). `out` must be supplied by the caller."""
+    sd = SeqDesc(lengths, ranks)
+    opts = LinearOpts(C.sizeof(LinearOpts), ACT[act], C.c_void_p(bias.data_ptr()) if bias is not None else None, None)
+    ms = [mat(t) for t in (U_r, X_r, W, out)]
+    s = torch.cuda.current_stream(U_r.device).cuda_stream if stream is None else stream
+    with torch.cuda.device(U_r.device):
+        _check(lib.atp_lowrank_linear_static(C.c_void_p(s), C.byref(ms[0]), C.byref(ms[1]), C.byref(ms[2]),
+                                             C.byref(sd.c), C.byref(opts), C.byref(ms[3])), "atp_lowrank_linear_static")
+    return out

@@ -152,6 +152,8 @@ const char *atp_status_string(atp_status s)
         case ATP_ERR_NOT_CONVERGED: return "Jacobi iteration hit its sweep limit";
         case ATP_ERR_TIMEOUT: return "a bounded device-side wait ran out";
         case ATP_ERR_RANGE: return "value outside the representable range";
+        case ATP_ERR_STATIC_SCRATCH_LIMIT:
+            return "problem exceeds the fixed scratch buffer of atp_lowrank_linear_static (sum(r) * d_out * 4 bytes > ATP_STATIC_SCRATCH_BYTES)";
     }
     return "unknown status";
 }

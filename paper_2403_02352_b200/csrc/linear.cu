@@ -103,3 +103,70 @@ extern "C" atp_status atp_lowrank_linear(atp_ctx *ctx, const atp_mat *U_r, const
     if (U_r->dtype == ATP_F32) return linear_impl<float>(ctx, U_r, X_r, W, sd, act, bias, Wg, Y);
     return linear_impl<__nv_bfloat16>(ctx, U_r, X_r, W, sd, act, bias, Wg, Y);
 }
+
+// ------------------------------------------------------------------------------------------------
+// Low-rank linear layer for callers that cannot allocate device memory.
+//
+// The regular call keeps its intermediate T = X_r W (sum(r_b) x d_out, fp32) in the caller's
+// workspace. Code that runs where cudaMalloc is off limits -- a plug-in inside a host process that
+// owns the memory pool, a real-time loop that must not touch the allocator -- has no buffer to
+// hand over and cannot create a context either (atp_create allocates its status word). For those
+// callers the same kernels run here with T placed in a fixed array that is part of the library
+// image: every GPU that loads libatp.so holds ATP_STATIC_SCRATCH_BYTES of it until the process
+// exits, whether or not this entry point is ever called.
+// ------------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_scratch[ATP_STATIC_SCRATCH_BYTES];
+
+#include <mutex>
+static std::mutex g_static_mu;
+static void *g_static_ptr[64];          // device address of g_static_scratch, per device ordinal
+
+// The array's name is only a host-side handle; the device address a kernel can use comes from
+// cudaGetSymbolAddress, asked once per device with that device current.
+static atp_status static_scratch_for_current_device(int *device, void **ptr)
+{
+    if (cudaGetDevice(device) != cudaSuccess) return ATP_ERR_CUDA;
+    if (*device < 0 || *device >= 64) return ATP_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_ptr[*device]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return ATP_ERR_CUDA;
+        g_static_ptr[*device] = p;
+    }
+    *ptr = g_static_ptr[*device];
+    return ATP_OK;
+}
+
+extern "C" atp_status atp_lowrank_linear_static(void *cuda_stream, const atp_mat *U_r, const atp_mat *X_r,
+                                                const atp_mat *W, const atp_seqs *seqs, const atp_linear_opts *opts,
+                                                atp_mat *Y)
+{
+    atp_status st;
+    if ((st = check_mat(U_r)) != ATP_OK || (st = check_mat(X_r)) != ATP_OK || (st = check_mat(W)) != ATP_OK ||
+        (st = check_mat(Y)) != ATP_OK)
+        return st;
+    int act = ATP_ACT_NONE; const float *bias = nullptr;
+    if (opts) {
+        if (opts->struct_size < sizeof(atp_linear_opts)) return ATP_ERR_INVALID_ARG;
+        act = opts->act; bias = opts->bias;
+    }
+    if (act != ATP_ACT_NONE && act != ATP_ACT_GELU) return ATP_ERR_INVALID_ARG;     // no SwiGLU here: it needs L x d_out more
+    if (U_r->dtype != X_r->dtype || W->dtype != X_r->dtype || Y->dtype != U_r->dtype) return ATP_ERR_UNSUPPORTED_DTYPE;
+    std::vector<SeqDims> sd;
+    if ((st = check_seqs(seqs, sd, U_r->rows)) != ATP_OK) return st;
+    int64_t tr = 0; int maxr = 0;
+    for (auto &s : sd) { tr += s.r; if (s.r > maxr) maxr = s.r; }
+    if (X_r->rows != tr || X_r->cols != W->rows || U_r->cols < maxr || Y->rows != U_r->rows || Y->cols != W->cols)
+        return ATP_ERR_INVALID_ARG;
+    if (U_r->rows == 0) return ATP_OK;
+    // T is the only scratch; it is written in full before it is read, so nothing has to be cleared.
+    if ((uint64_t)tr * (uint64_t)W->cols * sizeof(float) > ATP_STATIC_SCRATCH_BYTES) return ATP_ERR_STATIC_SCRATCH_LIMIT;
+    atp_ctx local;                      // host-side bookkeeping only; owns nothing on the device
+    void *scratch = nullptr;
+    if ((st = static_scratch_for_current_device(&local.device, &scratch)) != ATP_OK) return st;
+    local.stream = (cudaStream_t)cuda_stream;
+    local.workspace = scratch;
+    local.workspace_bytes = ATP_STATIC_SCRATCH_BYTES;
+    if (U_r->dtype == ATP_F32) return linear_impl<float>(&local, U_r, X_r, W, sd, act, bias, nullptr, Y);
+    return linear_impl<__nv_bfloat16>(&local, U_r, X_r, W, sd, act, bias, nullptr, Y);
+}
