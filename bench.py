@@ -138,6 +138,9 @@ def main():
     ap.add_argument("--seed", type=int, default=2000)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--power-iters", type=int, default=-1)
+    ap.add_argument("--jacobi-block", type=int, default=0)
+    ap.add_argument("--jacobi-inner", type=int, default=0)
+    ap.add_argument("--max-sweeps", type=int, default=0)
     args = ap.parse_args()
     if args.impl == "reference":
         if args.steps == 20 and args.warmup == 3:
@@ -180,7 +183,9 @@ def main():
 
     ctx = atp.Context(local)
     layer = AtpLayer(ctx, weights, lengths, ranks, w.heads, ffn=w.ffn, input_norm=w.input_norm,
-                     post_norm=POST_NORM[w.ffn], power_iters=args.power_iters)
+                     post_norm=POST_NORM[w.ffn], power_iters=args.power_iters,
+                     basis_kwargs=dict(jacobi_block=args.jacobi_block, jacobi_inner=args.jacobi_inner,
+                                       max_sweeps=args.max_sweeps))
     out_rows, out_cols = None, None
 
     def step(i):

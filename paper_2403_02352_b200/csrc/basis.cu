@@ -8,11 +8,12 @@
 //      rotated rows are sigma_i v_i^T and the accumulated rotations turn Y into singular vectors;
 //   4. sort by sigma, fix signs, write U_r = Y W and X_r.
 #include "gemm_simt.cuh"
+#include "jacobi2.cuh"
 #include <math.h>
 #include <algorithm>
 
 constexpr int PB = 64;            // orthonormalisation panel width
-constexpr int GRAM_ROWS = 512;    // rows per CTA of the panel Gram kernel
+constexpr int GRAM_ROWS = 128;    // rows per CTA of the panel Gram kernel
 constexpr int BJ = 32;            // Jacobi block height (pairs are 64 rows)
 constexpr int BMAX = 32;          // sequences per launch
 
@@ -98,20 +99,22 @@ __global__ void __launch_bounds__(256) panel_chol_kernel(const __grid_constant__
         G[i][j] = den > 0.0 ? G[i][j] / den : 0.0;
     }
     __syncthreads();
-    for (int j = 0; j < n; ++j) {
-        double piv = G[j][j];
-        bool bad = !(piv > 1e-10);
-        double ljj = bad ? 1.0 : sqrt(piv);
-        __syncthreads();
-        if (tid == 0) { G[j][j] = ljj; if (bad) dep[j] = 1; }
-        for (int i = j + 1 + tid; i < n; i += 256) G[i][j] = bad ? 0.0 : G[i][j] / ljj;
-        __syncthreads();
-        // trailing update of the lower triangle
-        int m = n - j - 1;
-        for (int e = tid; e < m * m; e += 256) {
-            int a = e / m, b = e - a * m;
-            if (b <= a) G[j + 1 + a][j + 1 + b] -= G[j + 1 + a][j] * G[j + 1 + b][j];
+    __shared__ double sh_ljj;
+    __shared__ int sh_bad;
+    for (int j = 0; j < n; ++j) {       // left-looking: column j from the finished columns < j
+        double sacc = 0.0;
+        if (tid >= j && tid < n) {
+            sacc = G[tid][j];
+            for (int k = 0; k < j; ++k) sacc -= G[tid][k] * G[j][k];
         }
+        if (tid == j) {
+            int bad = !(sacc > 1e-10);
+            sh_bad = bad;
+            sh_ljj = bad ? 1.0 : sqrt(sacc);
+            if (bad) dep[j] = 1;
+        }
+        __syncthreads();
+        if (tid >= j && tid < n) G[tid][j] = (tid == j) ? sh_ljj : (sh_bad ? 0.0 : sacc / sh_ljj);
         __syncthreads();
     }
     // Li = inverse of the lower-triangular factor, one column per thread
@@ -520,10 +523,122 @@ __global__ void __launch_bounds__(256) select_kernel(const __grid_constant__ Fin
     if (tid == 0 && sq.sigma_out) sq.sigma_out[a] = sq.sig[a];
 }
 
+// ---- finalisation of the two-sided path ----------------------------------------------------------
+struct Fin2Seq {
+    const float *G; const float *Wt; const float *Y; float *sig; int *ord; float *tsum; float *Wsel; int *needfix;
+    void *Xr; void *U; float *sigma_out; int rt, r, d, L, ldy, ldxr, ldu;
+};
+struct Fin2Batch { Fin2Seq s[BMAX]; int count; };
+
+// sigma_i = sqrt(G_ii) and their descending order. One CTA per sequence.
+__global__ void __launch_bounds__(1024) sigma_sort2_kernel(const __grid_constant__ Fin2Batch batch)
+{
+    const Fin2Seq &sq = batch.s[blockIdx.x];
+    extern __shared__ float sh[];
+    int npow = 1;
+    while (npow < sq.rt) npow <<= 1;
+    float *key = sh;
+    int *idx = (int *)(sh + npow);
+    const int tid = threadIdx.x;
+    for (int i = tid; i < npow; i += 1024) {
+        key[i] = (i < sq.rt) ? sqrtf(fmaxf(sq.G[(size_t)i * sq.rt + i], 0.f)) : -1.f;
+        idx[i] = i;
+    }
+    __syncthreads();
+    for (int k = 2; k <= npow; k <<= 1)
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int i = tid; i < npow; i += 1024) {
+                int l = i ^ j;
+                if (l > i) {
+                    bool desc = ((i & k) == 0);
+                    float ki = key[i], kl = key[l];
+                    int ii = idx[i], il = idx[l];
+                    bool i_first = (ki > kl) || (ki == kl && ii < il);
+                    if (desc ? !i_first : i_first) { key[i] = kl; key[l] = ki; idx[i] = il; idx[l] = ii; }
+                }
+            }
+            __syncthreads();
+        }
+    for (int i = tid; i < sq.rt; i += 1024) { sq.sig[i] = key[i]; sq.ord[i] = idx[i]; }
+}
+
+__global__ void colsum2_kernel(const __grid_constant__ Fin2Batch batch)
+{
+    const Fin2Seq &sq = batch.s[blockIdx.y];
+    int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= sq.rt) return;
+    float s = 0.f;
+    for (int l = 0; l < sq.L; ++l) s += sq.Y[(size_t)l * sq.ldy + k];
+    sq.tsum[k] = s;
+}
+
+// One CTA per kept component: sign from the column sum of U (= tsum . w), Wsel column, sigma.
+__global__ void __launch_bounds__(128) select2_kernel(const __grid_constant__ Fin2Batch batch)
+{
+    const Fin2Seq &sq = batch.s[blockIdx.y];
+    const int a = blockIdx.x;
+    if (a >= sq.r) return;
+    const int i = sq.ord[a];
+    const float *w = sq.Wt + (size_t)i * sq.rt;
+    __shared__ float redf[4];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    float s = 0.f;
+    for (int k = tid; k < sq.rt; k += 128) s = fmaf(sq.tsum[k], w[k], s);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) redf[warp] = s;
+    __syncthreads();
+    float colsum = redf[0] + redf[1] + redf[2] + redf[3];
+    float sgn = colsum < 0.f ? -1.f : 1.f;
+    for (int k = tid; k < sq.rt; k += 128) sq.Wsel[(size_t)k * sq.r + a] = sgn * w[k];
+    if (tid == 0) {
+        sq.needfix[a] = fabsf(colsum) < 1e-6f * sqrtf((float)sq.L);
+        if (sq.sigma_out) sq.sigma_out[a] = sq.sig[a];
+    }
+}
+
+// Components whose column sum is ~0 take their sign from the largest-magnitude entry of the X_r row.
+template <typename T>
+__global__ void __launch_bounds__(256) signfix_kernel(const __grid_constant__ Fin2Batch batch)
+{
+    const Fin2Seq &sq = batch.s[blockIdx.y];
+    const int a = blockIdx.x;
+    if (a >= sq.r || !sq.needfix[a]) return;
+    T *row = (T *)sq.Xr + (size_t)a * sq.ldxr;
+    __shared__ float redf[8];
+    __shared__ int redi[8];
+    __shared__ int flip;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    float best = -1.f; int bi = 0x7fffffff;
+    for (int c = tid; c < sq.d; c += 256) {
+        float v = fabsf(to_f32(row[c]));
+        if (v > best) { best = v; bi = c; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        float ob = __shfl_xor_sync(0xffffffffu, best, o);
+        int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (ob > best || (ob == best && oi < bi)) { best = ob; bi = oi; }
+    }
+    if (lane == 0) { redf[warp] = best; redi[warp] = bi; }
+    __syncthreads();
+    if (tid == 0) {
+        float b = redf[0]; int b2 = redi[0];
+        for (int w = 1; w < 8; ++w)
+            if (redf[w] > b || (redf[w] == b && redi[w] < b2)) { b = redf[w]; b2 = redi[w]; }
+        flip = (b2 < sq.d && to_f32(row[b2]) < 0.f);
+    }
+    __syncthreads();
+    if (!flip) return;
+    for (int c = tid; c < sq.d; c += 256) row[c] = from_f32<T>(-to_f32(row[c]));
+    T *u = (T *)sq.U + a;
+    for (int l = tid; l < sq.L; l += 256) u[(size_t)l * sq.ldu] = from_f32<T>(-to_f32(u[(size_t)l * sq.ldu]));
+}
+
 // ------------------------------------------------------------------------------------------------
 struct SeqPlan {
     SeqDims dims; int rt, npanel_L, npanel_d;
-    float *Y, *Z, *BW, *Wsel, *tsum, *sig, *Cc, *rinv; double *gpart; int *ord, *flags, *conv; unsigned *maxoff;
+    float *Y, *Z, *BW, *Wsel, *tsum, *sig, *Cc, *rinv, *G, *Wt, *Vbuf; double *gpart; int *ord, *flags, *conv, *vflag, *needfix; unsigned *maxoff;
 };
 struct BasisPlan {
     std::vector<SeqPlan> seqs; float *omega; float *part; size_t part_stride; int rtmax; int splits;
@@ -561,6 +676,11 @@ static void plan_basis(Arena &ar, const std::vector<SeqDims> &sd, int d, int ove
         p.rinv = ar.take<float>(PB * PB);
         p.flags = ar.take<int>(PB);
         p.gpart = ar.take<double>((size_t)ceil_div(std::max(std::max(L, d), 1), GRAM_ROWS) * PB * PB);
+        p.G = ar.take<float>((size_t)rt * rt);
+        p.Wt = ar.take<float>((size_t)rt * rt);
+        p.Vbuf = ar.take<float>((size_t)(rt / 64 + 2) * 4096 + (size_t)(rt / 32 + 2) * 1024);
+        p.vflag = ar.take<int>(rt / 32 + 4);
+        p.needfix = ar.take<int>(std::max(p.dims.r, 1));
         p.maxoff = ar.take<unsigned>(1);
         p.conv = ar.take<int>(1);
         maxpart = std::max(maxpart, (size_t)rt * PB);
@@ -626,7 +746,7 @@ static atp_status orthonormalise(atp_ctx *ctx, BasisPlan &bp, size_t i0, size_t 
 
 template <typename T>
 static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<SeqDims> &sd, int oversample,
-                             int power_iters, int max_sweeps, uint64_t seed, atp_mat *U_r, atp_mat *X_r, float *sigma)
+                             int power_iters, int max_sweeps, uint64_t seed, int jbj, int jinner, atp_mat *U_r, atp_mat *X_r, float *sigma)
 {
     const int d = (int)X->cols;
     Arena ar(ctx->workspace, ctx->workspace_bytes);
@@ -642,6 +762,7 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
     }
     const float tol_conv = (X->dtype == ATP_F32) ? 1e-6f : 3e-5f;
     const float tol_rot = tol_conv * 0.25f;
+    const bool two_sided = (X->dtype == ATP_BF16);    // fp32 inputs keep the one-sided rotation of B itself
     GemmEpi store{EPI_STORE, nullptr};
 
     for (size_t i0 = 0; i0 < bp.seqs.size(); i0 += BMAX) {
@@ -657,13 +778,14 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
         if ((st = launch_gemm_simt<T, float, float, false>(ctx, g, store)) != ATP_OK) return st;
         if ((st = orthonormalise(ctx, bp, i0, i1, false, d, seed)) != ATP_OK) return st;
         for (int it = 0; it < power_iters; ++it) {
-            // Z = X^T Y ; orth ; Y = X Z ; orth
+            // Z = X^T Y ; Y = X Z ; orth(Y).  Z is not orthonormalised: Y has orthonormal, QR-ordered
+            // columns, so cond(Z) ~ sigma_1 / sigma_r~ and cond(X Z) is its square, which the fp64
+            // panel factorisation of orth(Y) handles.
             for (size_t i = i0; i < i1; ++i) {
                 SeqPlan &p = bp.seqs[i];
                 g.p[i - i0] = GemmProblem{Xb(p), p.Y, p.Z, nullptr, p.rt > 0 ? d : 0, p.rt, p.dims.L, (int)X->ld, p.rt, p.rt, 0};
             }
             if ((st = launch_gemm_simt<T, float, float, true>(ctx, g, store)) != ATP_OK) return st;
-            if ((st = orthonormalise(ctx, bp, i0, i1, true, d, seed + 1000003ull * (it + 1))) != ATP_OK) return st;
             for (size_t i = i0; i < i1; ++i) {
                 SeqPlan &p = bp.seqs[i];
                 g.p[i - i0] = GemmProblem{Xb(p), p.Z, p.Y, nullptr, p.dims.L, p.rt, d, (int)X->ld, p.rt, p.rt, 0};
@@ -671,54 +793,124 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
             if ((st = launch_gemm_simt<T, float, float, false>(ctx, g, store)) != ATP_OK) return st;
             if ((st = orthonormalise(ctx, bp, i0, i1, false, d, seed + 2000003ull * (it + 1))) != ATP_OK) return st;
         }
-        // B = Y^T X into BW[:, :d]; Wt = I
-        JacBatch jb; jb.count = cnt; FinBatch fb; fb.count = cnt;
-        int maxnb = 2, maxrt = 0, maxr = 0;
-        for (size_t i = i0; i < i1; ++i) {
-            SeqPlan &p = bp.seqs[i];
-            int k = (int)(i - i0);
-            g.p[k] = GemmProblem{p.Y, Xb(p), p.BW, nullptr, p.rt, p.rt > 0 ? d : 0, p.dims.L, p.rt, (int)X->ld, d + p.rt, 0};
-            int nb = ceil_div(std::max(p.rt, 1), BJ); nb += nb & 1;
-            jb.s[k] = JacSeq{p.BW, p.rt, d, d + p.rt, nb, p.maxoff, p.conv};
-            fb.s[k] = FinSeq{p.BW, p.Y, p.sig, p.ord, p.tsum, p.Wsel,
-                             (T *)X_r->data + (size_t)p.dims.rank0 * X_r->ld, sigma ? sigma + p.dims.rank0 : nullptr,
-                             p.rt, p.dims.r, d, d + p.rt, p.dims.L, p.rt, (int)X_r->ld};
-            maxnb = std::max(maxnb, nb); maxrt = std::max(maxrt, p.rt); maxr = std::max(maxr, p.dims.r);
-        }
-        if (maxrt == 0) continue;
-        if ((st = launch_gemm_simt<float, T, float, true>(ctx, g, store)) != ATP_OK) return st;
-        ATP_KERNEL(ctx, "init_w", 0, 0);
-        init_w_kernel<<<dim3(64, cnt), 256, 0, ctx->stream>>>(jb);
-        ATP_LAUNCHED(ctx);
-        for (int sw = 0; sw < max_sweeps; ++sw) {
-            for (int step = 0; step < maxnb - 1; ++step) {
-                ATP_KERNEL(ctx, "jacobi_pair", 0, 0);
-                jacobi_pair_kernel<<<dim3(maxnb / 2, cnt), 256, 0, ctx->stream>>>(jb, step, tol_rot, tol_rot);
+        if (!two_sided) {
+            // B = Y^T X into BW[:, :d]; Wt = I
+            JacBatch jb; jb.count = cnt; FinBatch fb; fb.count = cnt;
+            int maxnb = 2, maxrt = 0, maxr = 0;
+            for (size_t i = i0; i < i1; ++i) {
+                SeqPlan &p = bp.seqs[i];
+                int k = (int)(i - i0);
+                g.p[k] = GemmProblem{p.Y, Xb(p), p.BW, nullptr, p.rt, p.rt > 0 ? d : 0, p.dims.L, p.rt, (int)X->ld, d + p.rt, 0};
+                int nb = ceil_div(std::max(p.rt, 1), BJ); nb += nb & 1;
+                jb.s[k] = JacSeq{p.BW, p.rt, d, d + p.rt, nb, p.maxoff, p.conv};
+                fb.s[k] = FinSeq{p.BW, p.Y, p.sig, p.ord, p.tsum, p.Wsel,
+                                 (T *)X_r->data + (size_t)p.dims.rank0 * X_r->ld, sigma ? sigma + p.dims.rank0 : nullptr,
+                                 p.rt, p.dims.r, d, d + p.rt, p.dims.L, p.rt, (int)X_r->ld};
+                maxnb = std::max(maxnb, nb); maxrt = std::max(maxrt, p.rt); maxr = std::max(maxr, p.dims.r);
+            }
+            if (maxrt == 0) continue;
+            if ((st = launch_gemm_simt<float, T, float, true>(ctx, g, store)) != ATP_OK) return st;
+            ATP_KERNEL(ctx, "init_w", 0, 0);
+            init_w_kernel<<<dim3(64, cnt), 256, 0, ctx->stream>>>(jb);
+            ATP_LAUNCHED(ctx);
+            for (int sw = 0; sw < max_sweeps; ++sw) {
+                for (int step = 0; step < maxnb - 1; ++step) {
+                    ATP_KERNEL(ctx, "jacobi_pair", 0, 0);
+                    jacobi_pair_kernel<<<dim3(maxnb / 2, cnt), 256, 0, ctx->stream>>>(jb, step, tol_rot, tol_rot);
+                    ATP_LAUNCHED(ctx);
+                }
+                ATP_KERNEL(ctx, "jacobi_sweep_end", 0, 0);
+                jacobi_sweep_end_kernel<<<1, BMAX, 0, ctx->stream>>>(jb, tol_conv, sw == max_sweeps - 1, ctx->dev_status);
                 ATP_LAUNCHED(ctx);
             }
-            ATP_KERNEL(ctx, "jacobi_sweep_end", 0, 0);
-            jacobi_sweep_end_kernel<<<1, BMAX, 0, ctx->stream>>>(jb, tol_conv, sw == max_sweeps - 1, ctx->dev_status);
+            int npow = 1; while (npow < maxrt) npow <<= 1;
+            size_t sm = (size_t)npow * 8;
+            if (sm > 48 * 1024) ATP_CUDA_OK(ctx, cudaFuncSetAttribute(sigma_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm));
+            ATP_KERNEL(ctx, "sigma_sort", 0, 0);
+            sigma_sort_kernel<<<cnt, 1024, sm, ctx->stream>>>(fb);
+            ATP_LAUNCHED(ctx);
+            ATP_KERNEL(ctx, "colsum", 0, 0);
+            colsum_kernel<<<dim3(ceil_div(maxrt, 128), cnt), 128, 0, ctx->stream>>>(fb);
+            ATP_LAUNCHED(ctx);
+            ATP_KERNEL(ctx, "select", 0, 0);
+            select_kernel<T><<<dim3(maxr, cnt), 256, 0, ctx->stream>>>(fb);
+            ATP_LAUNCHED(ctx);
+            // U_r = Y Wsel
+            for (size_t i = i0; i < i1; ++i) {
+                SeqPlan &p = bp.seqs[i];
+                g.p[i - i0] = GemmProblem{p.Y, p.Wsel, (T *)U_r->data + (size_t)p.dims.row0 * U_r->ld, nullptr,
+                                          p.dims.L, p.dims.r, p.rt, p.rt, p.dims.r, (int)U_r->ld, 0};
+            }
+            if ((st = launch_gemm_simt<float, float, T, false>(ctx, g, store)) != ATP_OK) return st;
+    
+        } else {
+            // B = Y^T X (r~ x d), G = B B^T, two-sided block Jacobi on G, then X_r = Wsel^T B, U_r = Y Wsel
+            Jac2Batch jb; jb.count = cnt; Fin2Batch fb; fb.count = cnt;
+            GemmBatch gg; gg.count = cnt;
+            int maxnb = 2, maxrt = 0, maxr = 0;
+            for (size_t i = i0; i < i1; ++i) {
+                SeqPlan &p = bp.seqs[i];
+                int k = (int)(i - i0);
+                g.p[k] = GemmProblem{p.Y, Xb(p), p.BW, nullptr, p.rt, p.rt > 0 ? d : 0, p.dims.L, p.rt, (int)X->ld, d, 0};
+                gg.p[k] = GemmProblem{p.BW, p.BW, p.G, nullptr, p.rt, p.rt, p.rt > 0 ? d : 0, d, d, p.rt, 0};
+                int nb = ceil_div(std::max(p.rt, 1), jbj); nb += nb & 1;
+                jb.s[k] = Jac2Seq{p.G, p.Wt, p.Vbuf, p.vflag, p.rt, nb, p.maxoff, p.conv};
+                fb.s[k] = Fin2Seq{p.G, p.Wt, p.Y, p.sig, p.ord, p.tsum, p.Wsel, p.needfix,
+                                  (T *)X_r->data + (size_t)p.dims.rank0 * X_r->ld, (T *)U_r->data + (size_t)p.dims.row0 * U_r->ld,
+                                  sigma ? sigma + p.dims.rank0 : nullptr, p.rt, p.dims.r, d, p.dims.L, p.rt, (int)X_r->ld, (int)U_r->ld};
+                maxnb = std::max(maxnb, nb); maxrt = std::max(maxrt, p.rt); maxr = std::max(maxr, p.dims.r);
+            }
+            if (maxrt == 0) continue;
+            if ((st = launch_gemm_simt<float, T, float, true>(ctx, g, store)) != ATP_OK) return st;
+            if ((st = launch_gemm_simt<float, float, float, false, true>(ctx, gg, store)) != ATP_OK) return st;
+            ATP_KERNEL(ctx, "jac2_init", 0, 0);
+            jac2_init_kernel<<<dim3(64, cnt), 256, 0, ctx->stream>>>(jb);
+            ATP_LAUNCHED(ctx);
+            const int npairs = maxnb / 2;
+            const int blk = 2 * jbj;
+            const size_t ash = (size_t)3 * blk * (blk + 1) * sizeof(float);
+            if (jbj == 32) ATP_CUDA_OK(ctx, cudaFuncSetAttribute(jac2_apply_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ash));
+            for (int sw = 0; sw < max_sweeps; ++sw) {
+                for (int step = 0; step < maxnb - 1; ++step) {
+                    ATP_KERNEL(ctx, "jac2_local", 0, 0);
+                    if (jbj == 32) jac2_local_kernel<32><<<dim3(npairs, cnt), 256, 0, ctx->stream>>>(jb, step, tol_rot, jinner);
+                    else jac2_local_kernel<16><<<dim3(npairs, cnt), 128, 0, ctx->stream>>>(jb, step, tol_rot, jinner);
+                    ATP_LAUNCHED(ctx);
+                    ATP_KERNEL(ctx, "jac2_apply", 0, 0);
+                    dim3 ag(npairs + ceil_div(maxrt, blk), npairs, cnt);
+                    if (jbj == 32) jac2_apply_kernel<32><<<ag, 256, ash, ctx->stream>>>(jb, step);
+                    else jac2_apply_kernel<16><<<ag, 128, ash, ctx->stream>>>(jb, step);
+                    ATP_LAUNCHED(ctx);
+                }
+                ATP_KERNEL(ctx, "jac2_sweep_end", 0, 0);
+                jac2_sweep_end_kernel<<<1, J2MAX, 0, ctx->stream>>>(jb, tol_conv, sw == max_sweeps - 1, ctx->dev_status);
+                ATP_LAUNCHED(ctx);
+            }
+            int npow = 1; while (npow < maxrt) npow <<= 1;
+            ATP_KERNEL(ctx, "sigma_sort", 0, 0);
+            sigma_sort2_kernel<<<cnt, 1024, (size_t)npow * 8, ctx->stream>>>(fb);
+            ATP_LAUNCHED(ctx);
+            ATP_KERNEL(ctx, "colsum", 0, 0);
+            colsum2_kernel<<<dim3(ceil_div(maxrt, 128), cnt), 128, 0, ctx->stream>>>(fb);
+            ATP_LAUNCHED(ctx);
+            ATP_KERNEL(ctx, "select", 0, 0);
+            select2_kernel<<<dim3(maxr, cnt), 128, 0, ctx->stream>>>(fb);
+            ATP_LAUNCHED(ctx);
+            for (size_t i = i0; i < i1; ++i) {
+                SeqPlan &p = bp.seqs[i];
+                int k = (int)(i - i0);
+                // X_r = Wsel^T B  and  U_r = Y Wsel
+                g.p[k] = GemmProblem{p.Wsel, p.BW, (T *)X_r->data + (size_t)p.dims.rank0 * X_r->ld, nullptr,
+                                     p.dims.r, p.rt > 0 ? d : 0, p.rt, p.dims.r, d, (int)X_r->ld, 0};
+                gg.p[k] = GemmProblem{p.Y, p.Wsel, (T *)U_r->data + (size_t)p.dims.row0 * U_r->ld, nullptr,
+                                      p.dims.L, p.dims.r, p.rt, p.rt, p.dims.r, (int)U_r->ld, 0};
+            }
+            if ((st = launch_gemm_simt<float, float, T, true>(ctx, g, store)) != ATP_OK) return st;
+            if ((st = launch_gemm_simt<float, float, T, false>(ctx, gg, store)) != ATP_OK) return st;
+            ATP_KERNEL(ctx, "signfix", 0, 0);
+            signfix_kernel<T><<<dim3(maxr, cnt), 256, 0, ctx->stream>>>(fb);
             ATP_LAUNCHED(ctx);
         }
-        int npow = 1; while (npow < maxrt) npow <<= 1;
-        size_t sm = (size_t)npow * 8;
-        if (sm > 48 * 1024) ATP_CUDA_OK(ctx, cudaFuncSetAttribute(sigma_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm));
-        ATP_KERNEL(ctx, "sigma_sort", 0, 0);
-        sigma_sort_kernel<<<cnt, 1024, sm, ctx->stream>>>(fb);
-        ATP_LAUNCHED(ctx);
-        ATP_KERNEL(ctx, "colsum", 0, 0);
-        colsum_kernel<<<dim3(ceil_div(maxrt, 128), cnt), 128, 0, ctx->stream>>>(fb);
-        ATP_LAUNCHED(ctx);
-        ATP_KERNEL(ctx, "select", 0, 0);
-        select_kernel<T><<<dim3(maxr, cnt), 256, 0, ctx->stream>>>(fb);
-        ATP_LAUNCHED(ctx);
-        // U_r = Y Wsel
-        for (size_t i = i0; i < i1; ++i) {
-            SeqPlan &p = bp.seqs[i];
-            g.p[i - i0] = GemmProblem{p.Y, p.Wsel, (T *)U_r->data + (size_t)p.dims.row0 * U_r->ld, nullptr,
-                                      p.dims.L, p.dims.r, p.rt, p.rt, p.dims.r, (int)U_r->ld, 0};
-        }
-        if ((st = launch_gemm_simt<float, float, T, false>(ctx, g, store)) != ATP_OK) return st;
     }
     return ATP_OK;
 }
@@ -729,13 +921,16 @@ extern "C" atp_status atp_principal_basis(atp_ctx *ctx, const atp_mat *X, const 
     if (!ctx) return ATP_ERR_INVALID_ARG;
     atp_status st;
     if ((st = check_mat(X)) != ATP_OK || (st = check_mat(U_r)) != ATP_OK || (st = check_mat(X_r)) != ATP_OK) return st;
-    int oversample = 64, power_iters = 2, max_sweeps = 16; uint64_t seed = 0x243F6A8885A308D3ull;
+    int oversample = 64, power_iters = 2, max_sweeps = 16, jbj = 16, jinner = 1; uint64_t seed = 0x243F6A8885A308D3ull;
     if (opts) {
         if (opts->struct_size < sizeof(atp_basis_opts)) return ATP_ERR_INVALID_ARG;
         if (opts->oversample >= 0) oversample = opts->oversample;
         if (opts->power_iters >= 0) power_iters = opts->power_iters;
         if (opts->max_sweeps > 0) max_sweeps = opts->max_sweeps;
         seed ^= opts->seed * 0x9E3779B97F4A7C15ull;
+        if (opts->jacobi_block == 16 || opts->jacobi_block == 32) jbj = opts->jacobi_block;
+        else if (opts->jacobi_block != 0) return ATP_ERR_INVALID_ARG;
+        if (opts->jacobi_inner > 0) jinner = opts->jacobi_inner;
     }
     if (oversample > 4096 || power_iters > 64 || max_sweeps > 200) return ATP_ERR_INVALID_ARG;
     if (U_r->dtype != X->dtype || X_r->dtype != X->dtype) return ATP_ERR_UNSUPPORTED_DTYPE;
@@ -750,8 +945,8 @@ extern "C" atp_status atp_principal_basis(atp_ctx *ctx, const atp_mat *X, const 
     if (U_r->rows != X->rows || U_r->cols < maxr || X_r->rows != tr || X_r->cols != X->cols) return ATP_ERR_INVALID_ARG;
     if (X->rows == 0) return ATP_OK;
     ATP_CUDA_OK(ctx, cudaSetDevice(ctx->device));
-    if (X->dtype == ATP_F32) return basis_impl<float>(ctx, X, sd, oversample, power_iters, max_sweeps, seed, U_r, X_r, sigma);
-    return basis_impl<__nv_bfloat16>(ctx, X, sd, oversample, power_iters, max_sweeps, seed, U_r, X_r, sigma);
+    if (X->dtype == ATP_F32) return basis_impl<float>(ctx, X, sd, oversample, power_iters, max_sweeps, seed, jbj, jinner, U_r, X_r, sigma);
+    return basis_impl<__nv_bfloat16>(ctx, X, sd, oversample, power_iters, max_sweeps, seed, jbj, jinner, U_r, X_r, sigma);
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -1,6 +1,7 @@
 // Batched SIMT GEMM with fp32 accumulation: C = epilogue(op(A) * B).
 //   A: M x K row-major (TRANS_A = false) or K x M row-major (TRANS_A = true)
-//   B: K x N row-major,  C: M x N row-major,  D (optional addend / gate): M x N fp32
+//   B: K x N row-major (TRANS_B = false) or N x K row-major (TRANS_B = true)
+//   C: M x N row-major,  D (optional addend / gate): M x N fp32
 // Used by the fp32 path everywhere and by the small projections of the bf16 path.
 #pragma once
 #include "common.cuh"
@@ -31,7 +32,7 @@ struct GemmEpi {
 __device__ __forceinline__ float gelu_erf_f(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752f)); }
 __device__ __forceinline__ float silu_f(float x) { return x / (1.0f + __expf(-x)); }
 
-template <typename TA, typename TB, typename TC, bool TRANS_A>
+template <typename TA, typename TB, typename TC, bool TRANS_A, bool TRANS_B>
 __global__ void __launch_bounds__(256)
 gemm_simt_kernel(const __grid_constant__ GemmBatch batch, GemmEpi epi, int splits, float *part, size_t part_stride)
 {
@@ -71,10 +72,15 @@ gemm_simt_kernel(const __grid_constant__ GemmBatch batch, GemmEpi epi, int split
                 if (m0 + m < pr.M && k0 + k < ke) v = to_f32(A[(size_t)(k0 + k) * pr.lda + m0 + m]);
                 As[k][m] = v;
             }
-            {
+            if (!TRANS_B) {
                 int k = e >> 6, n = e & 63;
                 float v = 0.f;
                 if (n0 + n < pr.N && k0 + k < ke) v = to_f32(B[(size_t)(k0 + k) * pr.ldb + n0 + n]);
+                Bs[k][n] = v;
+            } else {
+                int n = e >> 4, k = e & 15;
+                float v = 0.f;
+                if (n0 + n < pr.N && k0 + k < ke) v = to_f32(B[(size_t)(n0 + n) * pr.ldb + k0 + k]);
                 Bs[k][n] = v;
             }
         }
@@ -146,7 +152,7 @@ gemm_splitk_reduce_kernel(const __grid_constant__ GemmBatch batch, int splits, c
 }
 
 // Host launcher. `part` is scratch for split-K (splits * count * part_stride floats) or nullptr.
-template <typename TA, typename TB, typename TC, bool TRANS_A>
+template <typename TA, typename TB, typename TC, bool TRANS_A, bool TRANS_B = false>
 static atp_status launch_gemm_simt(atp_ctx *ctx, const GemmBatch &batch, GemmEpi epi, int splits = 1,
                                    float *part = nullptr, size_t part_stride = 0)
 {
@@ -165,7 +171,7 @@ static atp_status launch_gemm_simt(atp_ctx *ctx, const GemmBatch &batch, GemmEpi
     }
     dim3 grid(ceil_div(maxN, 64), ceil_div(maxM, 64), batch.count * splits);
     ATP_KERNEL(ctx, "gemm_simt", flops, bytes);
-    gemm_simt_kernel<TA, TB, TC, TRANS_A><<<grid, 256, 0, ctx->stream>>>(batch, epi, splits, part, part_stride);
+    gemm_simt_kernel<TA, TB, TC, TRANS_A, TRANS_B><<<grid, 256, 0, ctx->stream>>>(batch, epi, splits, part, part_stride);
     ATP_LAUNCHED(ctx);
     if (splits > 1) {
         int blocks = ceil_div(maxM * maxN, 256);

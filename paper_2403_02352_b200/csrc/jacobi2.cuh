@@ -1,0 +1,228 @@
+// Two-sided block Jacobi eigensolver for the small Gram matrix G = B B^T (r~ x r~, fp32, resident in
+// L2): the rotation that diagonalises G turns the orthonormal range basis into singular vectors
+// (Rayleigh-Ritz step of the basis extraction, Sec. 4.2: X' = [sigma_i v_i]).
+// Blocks of 16 rows; a step handles r~/32 disjoint pairs (round-robin order) with two launches:
+//   jac2_local : per pair, the 32x32 diagonal block is diagonalised on chip (cyclic Jacobi), the
+//                accumulated row operations Vt are published;
+//   jac2_apply : every 32x32 block (p, q) becomes Vt_p G_pq Vt_q^T, rows of Wt become Vt_p Wt.
+// G entries carry errors relative to the norms of the rows of B they come from (B is graded by the
+// QR-ordered range basis), which is what Jacobi needs to resolve small eigenvalues next to large ones.
+#pragma once
+#include "common.cuh"
+
+constexpr int J2MAX = 32;         // sequences per launch
+
+struct Jac2Seq { float *G; float *Wt; float *Vbuf; int *vflag; int rt, nb; unsigned *maxoff; int *conv; };
+struct Jac2Batch { Jac2Seq s[J2MAX]; int count; };
+
+__device__ __forceinline__ void rr_pair2(int nb, int step, int t, int &I, int &J)
+{
+    int m = nb - 1;
+    if (t == 0) { I = m; J = step % m; }
+    else { I = (step + t) % m; J = (step - t + m) % m; }
+    if (I > J) { int x = I; I = J; J = x; }
+}
+template <int BJ2>
+__device__ __forceinline__ int jac2_row(int I, int J, int i, int rt)
+{
+    int g = (i < BJ2) ? I * BJ2 + i : J * BJ2 + (i - BJ2);
+    return g < rt ? g : -1;
+}
+
+__global__ void jac2_init_kernel(const __grid_constant__ Jac2Batch batch)
+{
+    const Jac2Seq &sq = batch.s[blockIdx.y];
+    size_t n = (size_t)sq.rt * sq.rt;
+    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
+        int i = (int)(e / sq.rt), k = (int)(e - (size_t)i * sq.rt);
+        sq.Wt[e] = (i == k) ? 1.f : 0.f;
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) { *sq.maxoff = 0u; *sq.conv = 0; }
+}
+
+// BJ2: block height (16 or 32); the local problem is BLK x BLK with BLK = 2 BJ2, solved by 4 BLK threads.
+template <int BJ2>
+__global__ void __launch_bounds__(BJ2 * 8)
+jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_rot, int max_inner)
+{
+    constexpr int BLK = 2 * BJ2, NT = BLK * 4, HP = BLK / 2;
+    const Jac2Seq &sq = batch.s[blockIdx.y];
+    if (*sq.conv) return;
+    const int npairs = sq.nb / 2;
+    const int pair = blockIdx.x;
+    if (pair >= npairs) return;
+    int I, J;
+    rr_pair2(sq.nb, step % (sq.nb - 1), pair, I, J);
+    __shared__ float A[BLK][BLK + 1];
+    __shared__ float V[BLK][BLK + 1];
+    __shared__ float cs[HP], sn[HP];
+    __shared__ int pp[HP], qq[HP];
+    __shared__ float red[NT / 32];
+    __shared__ int rotated;
+    const int tid = threadIdx.x;
+    for (int e = tid; e < BLK * BLK; e += NT) {
+        int i = e / BLK, j = e % BLK;
+        int gi = jac2_row<BJ2>(I, J, i, sq.rt), gj = jac2_row<BJ2>(I, J, j, sq.rt);
+        A[i][j] = (gi >= 0 && gj >= 0) ? sq.G[(size_t)gi * sq.rt + gj] : 0.f;
+        V[i][j] = (i == j) ? 1.f : 0.f;
+    }
+    __syncthreads();
+    float mo = 0.f;
+    for (int e = tid; e < BLK * BLK; e += NT) {
+        int i = e / BLK, j = e % BLK;
+        if (i != j) {
+            float den = sqrtf(fmaxf(A[i][i], 0.f) * fmaxf(A[j][j], 0.f));
+            if (den > 0.f) mo = fmaxf(mo, fabsf(A[i][j]) / den);
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mo = fmaxf(mo, __shfl_xor_sync(0xffffffffu, mo, o));
+    if ((tid & 31) == 0) red[tid >> 5] = mo;
+    __syncthreads();
+    mo = red[0];
+#pragma unroll
+    for (int w = 1; w < NT / 32; ++w) mo = fmaxf(mo, red[w]);
+    if (tid == 0) atomicMax(sq.maxoff, __float_as_uint(mo));
+    if (mo <= tol_rot) {
+        if (tid == 0) sq.vflag[pair] = 0;
+        return;
+    }
+    for (int sweep = 0; sweep < max_inner; ++sweep) {
+        if (tid == 0) rotated = 0;
+        __syncthreads();
+        for (int st = 0; st < BLK - 1; ++st) {
+            if (tid < HP) {
+                int p, q;
+                rr_pair2(BLK, st, tid, p, q);
+                float gpp = A[p][p], gqq = A[q][q], gpq = A[p][q];
+                float c = 1.f, s = 0.f;
+                if (gpq != 0.f && fabsf(gpq) > tol_rot * sqrtf(fmaxf(gpp, 0.f) * fmaxf(gqq, 0.f))) {
+                    float zeta = (gqq - gpp) / (2.f * gpq);
+                    float t = copysignf(1.f, zeta) / (fabsf(zeta) + sqrtf(1.f + zeta * zeta));
+                    c = 1.f / sqrtf(1.f + t * t);
+                    s = c * t;
+                    rotated = 1;
+                }
+                cs[tid] = c; sn[tid] = s; pp[tid] = p; qq[tid] = q;
+            }
+            __syncthreads();
+#pragma unroll
+            for (int it = 0; it < HP * HP / NT; ++it) {
+                int idx = tid + it * NT;
+                int a = idx / HP, b = idx % HP;
+                int pa = pp[a], qa = qq[a], pb = pp[b], qb = qq[b];
+                float ca = cs[a], sa = sn[a], cb = cs[b], sb = sn[b];
+                float g00 = A[pa][pb], g01 = A[pa][qb], g10 = A[qa][pb], g11 = A[qa][qb];
+                float r00 = ca * g00 - sa * g10, r01 = ca * g01 - sa * g11;
+                float r10 = sa * g00 + ca * g10, r11 = sa * g01 + ca * g11;
+                A[pa][pb] = cb * r00 - sb * r01; A[pa][qb] = sb * r00 + cb * r01;
+                A[qa][pb] = cb * r10 - sb * r11; A[qa][qb] = sb * r10 + cb * r11;
+            }
+#pragma unroll
+            for (int it = 0; it < HP * BLK / NT; ++it) {
+                int idx = tid + it * NT;
+                int a = idx / BLK, col = idx % BLK;
+                int pa = pp[a], qa = qq[a];
+                float ca = cs[a], sa = sn[a];
+                float x = V[pa][col], y = V[qa][col];
+                V[pa][col] = ca * x - sa * y;
+                V[qa][col] = sa * x + ca * y;
+            }
+            __syncthreads();
+        }
+        if (!rotated) break;
+        __syncthreads();
+    }
+    float *dst = sq.Vbuf + (size_t)pair * BLK * BLK;
+    for (int e = tid; e < BLK * BLK; e += NT) dst[e] = V[e / BLK][e % BLK];
+    if (tid == 0) sq.vflag[pair] = 1;
+}
+
+// grid: (npairs + ceil(rt/BLK), npairs, batch); dynamic shared memory: 3 * BLK * (BLK + 1) floats
+template <int BJ2>
+__global__ void __launch_bounds__(BJ2 * 8)
+jac2_apply_kernel(const __grid_constant__ Jac2Batch batch, int step)
+{
+    constexpr int BLK = 2 * BJ2, NT = BLK * 4, CPT = BLK / 4, LD = BLK + 1;
+    const Jac2Seq &sq = batch.s[blockIdx.z];
+    if (*sq.conv) return;
+    const int npairs = sq.nb / 2;
+    const int p = blockIdx.y;
+    if (p >= npairs) return;
+    const int tid = threadIdx.x;
+    extern __shared__ float j2sm[];
+    float *Vp = j2sm, *Vq = j2sm + BLK * LD, *Bk = j2sm + 2 * BLK * LD;
+    int Ip, Jp;
+    rr_pair2(sq.nb, step % (sq.nb - 1), p, Ip, Jp);
+    const int fp = sq.vflag[p];
+    const int row = tid >> 2, c0 = (tid & 3) * CPT;
+    float t[CPT];
+#pragma unroll
+    for (int j = 0; j < CPT; ++j) t[j] = 0.f;
+    if ((int)blockIdx.x < npairs) {
+        const int q = blockIdx.x;
+        const int fq = sq.vflag[q];
+        if (!fp && !fq) return;
+        int Iq, Jq;
+        rr_pair2(sq.nb, step % (sq.nb - 1), q, Iq, Jq);
+        for (int e = tid; e < BLK * BLK; e += NT) {
+            int i = e / BLK, j = e % BLK;
+            Vp[i * LD + j] = fp ? sq.Vbuf[(size_t)p * BLK * BLK + e] : (i == j ? 1.f : 0.f);
+            Vq[i * LD + j] = fq ? sq.Vbuf[(size_t)q * BLK * BLK + e] : (i == j ? 1.f : 0.f);
+            int gi = jac2_row<BJ2>(Ip, Jp, i, sq.rt), gj = jac2_row<BJ2>(Iq, Jq, j, sq.rt);
+            Bk[i * LD + j] = (gi >= 0 && gj >= 0) ? sq.G[(size_t)gi * sq.rt + gj] : 0.f;
+        }
+        __syncthreads();
+        for (int k = 0; k < BLK; ++k) {
+            float a = Vp[row * LD + k];
+#pragma unroll
+            for (int j = 0; j < CPT; ++j) t[j] = fmaf(a, Bk[k * LD + c0 + j], t[j]);
+        }
+        __syncthreads();                       // everyone is done reading Bk: reuse it for T = Vp Bk
+#pragma unroll
+        for (int j = 0; j < CPT; ++j) Bk[row * LD + c0 + j] = t[j];
+        __syncthreads();
+        const int gi = jac2_row<BJ2>(Ip, Jp, row, sq.rt);
+#pragma unroll
+        for (int j = 0; j < CPT; ++j) {
+            float o = 0.f;
+            for (int k = 0; k < BLK; ++k) o = fmaf(Bk[row * LD + k], Vq[(c0 + j) * LD + k], o);     // (T Vq^T)[row][c0+j]
+            int gj = jac2_row<BJ2>(Iq, Jq, c0 + j, sq.rt);
+            if (gi >= 0 && gj >= 0) sq.G[(size_t)gi * sq.rt + gj] = o;
+        }
+    } else {
+        if (!fp) return;
+        const int cb = ((int)blockIdx.x - npairs) * BLK;
+        if (cb >= sq.rt) return;
+        for (int e = tid; e < BLK * BLK; e += NT) {
+            int i = e / BLK, j = e % BLK;
+            Vp[i * LD + j] = sq.Vbuf[(size_t)p * BLK * BLK + e];
+            int gi = jac2_row<BJ2>(Ip, Jp, i, sq.rt);
+            Bk[i * LD + j] = (gi >= 0 && cb + j < sq.rt) ? sq.Wt[(size_t)gi * sq.rt + cb + j] : 0.f;
+        }
+        __syncthreads();
+        for (int k = 0; k < BLK; ++k) {
+            float a = Vp[row * LD + k];
+#pragma unroll
+            for (int j = 0; j < CPT; ++j) t[j] = fmaf(a, Bk[k * LD + c0 + j], t[j]);
+        }
+        const int gi = jac2_row<BJ2>(Ip, Jp, row, sq.rt);
+        if (gi >= 0)
+#pragma unroll
+            for (int j = 0; j < CPT; ++j)
+                if (cb + c0 + j < sq.rt) sq.Wt[(size_t)gi * sq.rt + cb + c0 + j] = t[j];
+    }
+}
+
+__global__ void jac2_sweep_end_kernel(const __grid_constant__ Jac2Batch batch, float tol_conv, int last, int *dev_status)
+{
+    int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= batch.count) return;
+    const Jac2Seq &sq = batch.s[b];
+    if (!*sq.conv) {
+        float mo = __uint_as_float(*sq.maxoff);
+        if (mo <= tol_conv) *sq.conv = 1;
+        else if (last) raise_status(dev_status, ATP_ERR_NOT_CONVERGED);
+    }
+    *sq.maxoff = 0u;
+}

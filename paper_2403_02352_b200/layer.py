@@ -17,11 +17,12 @@ from . import binding as B
 class AtpLayer:
     def __init__(self, ctx: B.Context, weights: Dict[str, torch.Tensor], lengths: Sequence[int], ranks: Sequence[int],
                  heads: int, ffn: Optional[str] = None, input_norm: Optional[str] = None, post_norm: str = "layer",
-                 blocks: str = "auto", power_iters: int = -1, oversample: int = -1, seed: int = 0):
+                 power_iters: int = -1, oversample: int = -1, seed: int = 0, basis_kwargs: Optional[dict] = None):
         self.ctx, self.w = ctx, weights
         self.lengths, self.ranks = [int(x) for x in lengths], [int(x) for x in ranks]
         self.heads, self.ffn, self.input_norm, self.post_norm = heads, ffn, input_norm, post_norm
         self.power_iters, self.oversample, self.seed = power_iters, oversample, seed
+        self.basis_kwargs = dict(basis_kwargs or {})
         self.has_wo = "W_O" in weights
         self.dtype = weights["W_Q"].dtype
         self.device = weights["W_Q"].device
@@ -64,7 +65,8 @@ class AtpLayer:
 
     def _basis(self, X, out):
         return B.atp_principal_basis(self.ctx, X, self.lengths, self.ranks, oversample=self.oversample,
-                                     power_iters=self.power_iters, seed=self.seed, out=out, auto_workspace=False)
+                                     power_iters=self.power_iters, seed=self.seed, out=out, auto_workspace=False,
+                                     **self.basis_kwargs)
 
     def _linear(self, basis, W, out, act=None, W_gate=None):
         return B.atp_lowrank_linear(self.ctx, basis[0], basis[1], W, self.lengths, self.ranks, act=act, W_gate=W_gate,

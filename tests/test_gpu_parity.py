@@ -211,7 +211,7 @@ def test_ragged_batch_end_to_end_stage_parity(ctx, dtype):
 def test_end_to_end_on_gap_input_fp32(ctx):
     """T3: exact-rank input with distinct sigma and r = rank: GPU basis -> GPU attention against
     oracle basis -> oracle attention. The bar is looser than T2's because the logits amplify the
-    fp32 rounding of the basis (documented in the design doc)."""
+    fp32 rounding of the basis before the exponential."""
     atp = _atp()
     L, d, k, heads = 192, 128, 12, 2
     X, s = ai.exact_rank(L, d, k, dtype="f32", decay=0.7, seed=9)
