@@ -1,17 +1,24 @@
 // atp_lowrank_linear: Y = act(U_r (X_r W) + bias)  (Sec. 4.3: linear layers on the r-row representation).
 #include "gemm_simt.cuh"
+#include "gemm_tc.cuh"
+#include <type_traits>
 
 struct LinearPlan {
     float *T = nullptr, *Tg = nullptr, *Yg = nullptr;
+    __nv_bfloat16 *Tb = nullptr, *Tgb = nullptr;     // tensor-core path: T and T_gate in bf16
 };
 
-static size_t plan_linear(Arena &ar, int64_t total_rank, int64_t total_rows, int64_t d_out, bool swiglu, LinearPlan &p)
+static size_t plan_linear(Arena &ar, int64_t total_rank, int64_t total_rows, int64_t d_out, bool swiglu, bool bf16, LinearPlan &p)
 {
-    p.T = ar.take<float>((size_t)total_rank * d_out);
-    if (swiglu) {
-        p.Tg = ar.take<float>((size_t)total_rank * d_out);
-        p.Yg = ar.take<float>((size_t)total_rows * d_out);
+    if (bf16) {
+        const size_t ldt = align_up((size_t)d_out, 8);
+        p.Tb = ar.take<__nv_bfloat16>((size_t)total_rank * ldt);
+        if (swiglu) p.Tgb = ar.take<__nv_bfloat16>((size_t)total_rank * ldt);
+    } else {
+        p.T = ar.take<float>((size_t)total_rank * d_out);
+        if (swiglu) p.Tg = ar.take<float>((size_t)total_rank * d_out);
     }
+    if (swiglu) p.Yg = ar.take<float>((size_t)total_rows * d_out);
     return ar.off;
 }
 
@@ -21,7 +28,7 @@ size_t linear_workspace_bytes(const std::vector<SeqDims> &seqs, int64_t d_out)
     for (auto &s : seqs) { tr += s.r; tl += s.L; }
     Arena ar(nullptr, (size_t)-1);
     LinearPlan p;
-    return plan_linear(ar, tr, tl, d_out, true, p);      // sized for the SwiGLU case (the larger one)
+    return plan_linear(ar, tr, tl, d_out, true, false, p);      // sized for the fp32 SwiGLU case (the largest one)
 }
 
 template <typename T>
@@ -35,10 +42,36 @@ static atp_status linear_impl(atp_ctx *ctx, const atp_mat *U_r, const atp_mat *X
     const bool swiglu = act == ATP_ACT_SWIGLU;
     Arena ar(ctx->workspace, ctx->workspace_bytes);
     LinearPlan pl;
-    plan_linear(ar, tr, tl, d_out, swiglu, pl);
+    plan_linear(ar, tr, tl, d_out, swiglu, std::is_same<T, __nv_bfloat16>::value, pl);
     if (ar.overflow || (!ctx->workspace && ar.off > 0)) return ATP_ERR_WORKSPACE_TOO_SMALL;
 
     atp_status st;
+    if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+        // bf16: both GEMMs on the tensor cores; T is rounded to bf16 once (fp32 accumulation)
+        const int ldt = (int)align_up((size_t)d_out, 8);
+        std::vector<tc::HostProblem> p1;
+        p1.push_back(tc::HostProblem{X_r->data, W->data, nullptr, pl.Tb, nullptr, nullptr, (int)tr, d_out, d_in,
+                                     (int)X_r->ld, (int)W->ld, ldt, 0});
+        if (swiglu)
+            p1.push_back(tc::HostProblem{X_r->data, Wg->data, nullptr, pl.Tgb, nullptr, nullptr, (int)tr, d_out, d_in,
+                                         (int)X_r->ld, (int)Wg->ld, ldt, 0});
+        if ((st = tc::launch<false, false, tc::OUT_BF16>(ctx, p1, GemmEpi{EPI_STORE, nullptr})) != ATP_OK) return st;
+        std::vector<tc::HostProblem> pg, pm;
+        for (auto &s : seqs) {
+            if (s.L == 0) continue;
+            const T *u = (const T *)U_r->data + (size_t)s.row0 * U_r->ld;
+            T *y = (T *)Y->data + (size_t)s.row0 * Y->ld;
+            float *yg = swiglu ? pl.Yg + (size_t)s.row0 * d_out : nullptr;
+            if (swiglu)
+                pg.push_back(tc::HostProblem{u, pl.Tgb + (size_t)s.rank0 * ldt, nullptr, yg, nullptr, nullptr, s.L, d_out, s.r,
+                                             (int)U_r->ld, ldt, d_out, 0});
+            pm.push_back(tc::HostProblem{u, pl.Tb + (size_t)s.rank0 * ldt, nullptr, y, nullptr, yg, s.L, d_out, s.r,
+                                         (int)U_r->ld, ldt, (int)Y->ld, d_out});
+        }
+        if (swiglu && (st = tc::launch<false, false, tc::OUT_F32>(ctx, pg, GemmEpi{EPI_STORE, nullptr})) != ATP_OK) return st;
+        GemmEpi epi{swiglu ? EPI_SILU_D_MUL : (act == ATP_ACT_GELU ? EPI_BIAS_GELU : EPI_BIAS), bias};
+        return tc::launch<false, false, tc::OUT_BF16>(ctx, pm, epi);
+    }
     // T = X_r W for all sequences at once (rows of X_r are packed)
     {
         GemmBatch b; b.count = 1;
