@@ -1,6 +1,8 @@
 // atp_attention: Eq. 6 projections of the r-row representation, then attention of every query
 // on the r principal keys/values (the procedure of Eq. 1 with K', V' in place of K, V).
 #include "gemm_simt.cuh"
+#include "gemm_tc.cuh"
+#include <type_traits>
 #include <math.h>
 
 constexpr int ATT_MAX_BATCH = 32;
@@ -120,13 +122,15 @@ attn_simt_kernel(const __grid_constant__ AttnBatch batch, int dh, int ldq, int l
     }
 }
 
-struct AttnPlan { float *Qp, *Kp, *Vp, *Q; };
+struct AttnPlan { float *Qp, *Kp, *Vp, *Q; __nv_bfloat16 *Qph, *Qpl; };
 static void plan_attn(Arena &ar, int64_t tr, int64_t tl, int64_t dp, AttnPlan &p)
 {
     p.Qp = ar.take<float>((size_t)tr * dp);
     p.Kp = ar.take<float>((size_t)tr * dp);
     p.Vp = ar.take<float>((size_t)tr * dp);
     p.Q = ar.take<float>((size_t)tl * dp);
+    p.Qph = ar.take<__nv_bfloat16>((size_t)tr * align_up((size_t)dp, 8));     // Q' as a bf16 hi/lo pair (tensor-core path)
+    p.Qpl = ar.take<__nv_bfloat16>((size_t)tr * align_up((size_t)dp, 8));
 }
 size_t attention_workspace_bytes(const std::vector<SeqDims> &seqs, int64_t dp)
 {
@@ -152,6 +156,30 @@ static atp_status attention_impl(atp_ctx *ctx, const atp_mat *X, const atp_mat *
     if (ar.overflow || !ctx->workspace) return ATP_ERR_WORKSPACE_TOO_SMALL;
     atp_status st;
     GemmEpi store{EPI_STORE, nullptr};
+    if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+        // bf16: projections on the tensor cores with fp32 results. Q' is kept as a bf16 hi/lo pair so
+        // that the expansion Q = U_r Q' loses nothing against fp32 (the logits reach magnitudes of
+        // 10^2, where a bf16-rounded query would move the softmax).
+        const int ldq = (int)align_up((size_t)dp, 8);
+        std::vector<tc::HostProblem> kv;
+        kv.push_back(tc::HostProblem{X_r->data, WK->data, nullptr, pl.Kp, nullptr, nullptr, (int)tr, dp, d, (int)X_r->ld, (int)WK->ld, dp, 0});
+        kv.push_back(tc::HostProblem{X_r->data, WV->data, nullptr, pl.Vp, nullptr, nullptr, (int)tr, dp, d, (int)X_r->ld, (int)WV->ld, dp, 0});
+        if (q_mode == ATP_Q_FULL)
+            kv.push_back(tc::HostProblem{X->data, WQ->data, nullptr, pl.Q, nullptr, nullptr, (int)tl, dp, d, (int)X->ld, (int)WQ->ld, dp, 0});
+        if ((st = tc::launch<false, false, tc::OUT_F32>(ctx, kv, store)) != ATP_OK) return st;
+        if (q_mode == ATP_Q_LOWRANK) {
+            std::vector<tc::HostProblem> qp;
+            qp.push_back(tc::HostProblem{X_r->data, WQ->data, nullptr, pl.Qph, pl.Qpl, nullptr, (int)tr, dp, d, (int)X_r->ld, (int)WQ->ld, ldq, 0});
+            if ((st = tc::launch<false, false, tc::OUT_BF16_SPLIT>(ctx, qp, store)) != ATP_OK) return st;
+            std::vector<tc::HostProblem> qe;
+            for (auto &s : seqs)
+                if (s.L > 0)
+                    qe.push_back(tc::HostProblem{(const T *)U_r->data + (size_t)s.row0 * U_r->ld, pl.Qph + (size_t)s.rank0 * ldq,
+                                                 pl.Qpl + (size_t)s.rank0 * ldq, pl.Q + (size_t)s.row0 * dp, nullptr, nullptr,
+                                                 s.L, dp, s.r, (int)U_r->ld, ldq, dp, 0});
+            if ((st = tc::launch<false, true, tc::OUT_F32>(ctx, qe, store)) != ATP_OK) return st;
+        }
+    } else {
     {   // Q', K', V' = X_r W (Eq. 6), all sequences at once
         GemmBatch b; b.count = (q_mode == ATP_Q_LOWRANK) ? 3 : 2;
         const atp_mat *Ws[3] = {WK, WV, WQ};
@@ -172,6 +200,7 @@ static atp_status attention_impl(atp_ctx *ctx, const atp_mat *X, const atp_mat *
         GemmBatch b; b.count = 1;
         b.p[0] = GemmProblem{X->data, WQ->data, pl.Q, nullptr, (int)tl, dp, d, (int)X->ld, (int)WQ->ld, dp, 0};
         if ((st = launch_gemm_simt<T, T, float, false>(ctx, b, store)) != ATP_OK) return st;
+    }
     }
     size_t smem = ((size_t)dh * 68 * 2 + (size_t)64 * dh + 64 * 65) * sizeof(float);
     ATP_CUDA_OK(ctx, cudaFuncSetAttribute(attn_simt_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));

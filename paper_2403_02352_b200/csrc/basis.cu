@@ -8,7 +8,9 @@
 //      rotated rows are sigma_i v_i^T and the accumulated rotations turn Y into singular vectors;
 //   4. sort by sigma, fix signs, write U_r = Y W and X_r.
 #include "gemm_simt.cuh"
+#include "gemm_tc.cuh"
 #include "jacobi2.cuh"
+#include <type_traits>
 #include <math.h>
 #include <algorithm>
 
@@ -18,6 +20,15 @@ constexpr int BJ = 32;            // Jacobi block height (pairs are 64 rows)
 constexpr int BMAX = 32;          // sequences per launch
 
 // ------------------------------------------------------------------------------------------------
+__global__ void fill_omega_bf16_kernel(__nv_bfloat16 *om, int rows, int cols, int ld, uint64_t seed)
+{
+    size_t n = (size_t)rows * cols;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        int r = (int)(i / cols), c = (int)(i - (size_t)r * cols);
+        om[(size_t)r * ld + c] = __float2bfloat16_rn((mix64(seed, i) & 1) ? 1.f : -1.f);
+    }
+}
+
 __global__ void fill_omega_kernel(float *om, size_t n, uint64_t seed)
 {
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
@@ -638,10 +649,10 @@ __global__ void __launch_bounds__(256) signfix_kernel(const __grid_constant__ Fi
 // ------------------------------------------------------------------------------------------------
 struct SeqPlan {
     SeqDims dims; int rt, npanel_L, npanel_d;
-    float *Y, *Z, *BW, *Wsel, *tsum, *sig, *Cc, *rinv, *G, *Wt, *Vbuf; double *gpart; int *ord, *flags, *conv, *vflag, *needfix; unsigned *maxoff;
+    __nv_bfloat16 *Yb, *Zb; float *Y, *Z, *BW, *Wsel, *tsum, *sig, *Cc, *rinv, *G, *Wt, *Vbuf; double *gpart; int *ord, *flags, *conv, *vflag, *needfix; unsigned *maxoff;
 };
 struct BasisPlan {
-    std::vector<SeqPlan> seqs; float *omega; float *part; size_t part_stride; int rtmax; int splits;
+    std::vector<SeqPlan> seqs; float *omega; __nv_bfloat16 *omega_b; float *part; size_t part_stride; int rtmax; int splits;
 };
 
 constexpr size_t CHOL_SMEM = 2 * PB * (PB + 1) * sizeof(double);
@@ -662,11 +673,14 @@ static void plan_basis(Arena &ar, const std::vector<SeqDims> &sd, int d, int ove
         bp.seqs.push_back(p);
     }
     bp.omega = ar.take<float>((size_t)d * bp.rtmax);
+    bp.omega_b = ar.take<__nv_bfloat16>((size_t)d * align_up((size_t)bp.rtmax, 8));
     bp.splits = pick_splits(maxdim);
     for (auto &p : bp.seqs) {
         int L = p.dims.L, rt = p.rt;
         p.Y = ar.take<float>((size_t)L * rt);
         p.Z = ar.take<float>((size_t)d * rt);
+        p.Yb = ar.take<__nv_bfloat16>((size_t)L * align_up((size_t)rt, 8));
+        p.Zb = ar.take<__nv_bfloat16>((size_t)d * align_up((size_t)rt, 8));
         p.BW = ar.take<float>((size_t)rt * (d + rt));
         p.Wsel = ar.take<float>((size_t)rt * p.dims.r);
         p.tsum = ar.take<float>(rt);
@@ -770,28 +784,75 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
         const int cnt = (int)(i1 - i0);
         auto Xb = [&](const SeqPlan &p) { return (const T *)X->data + (size_t)p.dims.row0 * X->ld; };
         GemmBatch g; g.count = cnt;
-        // Y = X Omega
-        for (size_t i = i0; i < i1; ++i) {
-            SeqPlan &p = bp.seqs[i];
-            g.p[i - i0] = GemmProblem{Xb(p), bp.omega, p.Y, nullptr, p.dims.L, p.rt, d, (int)X->ld, bp.rtmax, p.rt, 0};
-        }
-        if ((st = launch_gemm_simt<T, float, float, false>(ctx, g, store)) != ATP_OK) return st;
-        if ((st = orthonormalise(ctx, bp, i0, i1, false, d, seed)) != ATP_OK) return st;
-        for (int it = 0; it < power_iters; ++it) {
-            // Z = X^T Y ; Y = X Z ; orth(Y).  Z is not orthonormalised: Y has orthonormal, QR-ordered
-            // columns, so cond(Z) ~ sigma_1 / sigma_r~ and cond(X Z) is its square, which the fp64
-            // panel factorisation of orth(Y) handles.
+        if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+            // bf16: every pass over X is a tensor-core GEMM with fp32 results; the iterates are
+            // orthonormalised in fp32 and handed to the next pass as bf16 copies.
+            const int ldo = (int)align_up((size_t)bp.rtmax, 8);
+            ATP_KERNEL(ctx, "fill_omega", 0, 0);
+            fill_omega_bf16_kernel<<<1024, 256, 0, ctx->stream>>>(bp.omega_b, d, bp.rtmax, ldo, seed);
+            ATP_LAUNCHED(ctx);
+            auto to_bf16 = [&](bool zside) -> atp_status {
+                for (size_t i = i0; i < i1; ++i) {
+                    SeqPlan &p = bp.seqs[i];
+                    int rows = zside ? d : p.dims.L;
+                    if (rows == 0 || p.rt == 0) continue;
+                    ATP_KERNEL(ctx, "f32_to_bf16", 0, (double)rows * p.rt * 6);
+                    tc::f32_to_bf16_kernel<<<std::min(1024, ceil_div(rows * p.rt, 256)), 256, 0, ctx->stream>>>(
+                        zside ? p.Z : p.Y, p.rt, zside ? p.Zb : p.Yb, (int)align_up((size_t)p.rt, 8), rows, p.rt);
+                    ATP_LAUNCHED(ctx);
+                }
+                return ATP_OK;
+            };
+            std::vector<tc::HostProblem> hp;
             for (size_t i = i0; i < i1; ++i) {
                 SeqPlan &p = bp.seqs[i];
-                g.p[i - i0] = GemmProblem{Xb(p), p.Y, p.Z, nullptr, p.rt > 0 ? d : 0, p.rt, p.dims.L, (int)X->ld, p.rt, p.rt, 0};
+                hp.push_back(tc::HostProblem{Xb(p), bp.omega_b, nullptr, p.Y, nullptr, nullptr, p.dims.L, p.rt, d, (int)X->ld, ldo, p.rt, 0});
             }
-            if ((st = launch_gemm_simt<T, float, float, true>(ctx, g, store)) != ATP_OK) return st;
+            if ((st = tc::launch<false, false, tc::OUT_F32>(ctx, hp, store)) != ATP_OK) return st;
+            if ((st = orthonormalise(ctx, bp, i0, i1, false, d, seed)) != ATP_OK) return st;
+            if ((st = to_bf16(false)) != ATP_OK) return st;
+            for (int it = 0; it < power_iters; ++it) {
+                hp.clear();
+                for (size_t i = i0; i < i1; ++i) {      // Z = X^T Y (bf16 result: only the next pass reads it)
+                    SeqPlan &p = bp.seqs[i];
+                    int ldb = (int)align_up((size_t)p.rt, 8);
+                    hp.push_back(tc::HostProblem{Xb(p), p.Yb, nullptr, p.Zb, nullptr, nullptr, d, p.rt, p.dims.L, (int)X->ld, ldb, ldb, 0});
+                }
+                if ((st = tc::launch<true, false, tc::OUT_BF16>(ctx, hp, store)) != ATP_OK) return st;
+                hp.clear();
+                for (size_t i = i0; i < i1; ++i) {      // Y = X Z
+                    SeqPlan &p = bp.seqs[i];
+                    int ldb = (int)align_up((size_t)p.rt, 8);
+                    hp.push_back(tc::HostProblem{Xb(p), p.Zb, nullptr, p.Y, nullptr, nullptr, p.dims.L, p.rt, d, (int)X->ld, ldb, p.rt, 0});
+                }
+                if ((st = tc::launch<false, false, tc::OUT_F32>(ctx, hp, store)) != ATP_OK) return st;
+                if ((st = orthonormalise(ctx, bp, i0, i1, false, d, seed + 2000003ull * (it + 1))) != ATP_OK) return st;
+                if ((st = to_bf16(false)) != ATP_OK) return st;
+            }
+        } else {
+            // Y = X Omega
             for (size_t i = i0; i < i1; ++i) {
                 SeqPlan &p = bp.seqs[i];
-                g.p[i - i0] = GemmProblem{Xb(p), p.Z, p.Y, nullptr, p.dims.L, p.rt, d, (int)X->ld, p.rt, p.rt, 0};
+                g.p[i - i0] = GemmProblem{Xb(p), bp.omega, p.Y, nullptr, p.dims.L, p.rt, d, (int)X->ld, bp.rtmax, p.rt, 0};
             }
             if ((st = launch_gemm_simt<T, float, float, false>(ctx, g, store)) != ATP_OK) return st;
-            if ((st = orthonormalise(ctx, bp, i0, i1, false, d, seed + 2000003ull * (it + 1))) != ATP_OK) return st;
+            if ((st = orthonormalise(ctx, bp, i0, i1, false, d, seed)) != ATP_OK) return st;
+            for (int it = 0; it < power_iters; ++it) {
+                // Z = X^T Y ; Y = X Z ; orth(Y).  Z is not orthonormalised: Y has orthonormal, QR-ordered
+                // columns, so cond(Z) ~ sigma_1 / sigma_r~ and cond(X Z) is its square, which the fp64
+                // panel factorisation of orth(Y) handles.
+                for (size_t i = i0; i < i1; ++i) {
+                    SeqPlan &p = bp.seqs[i];
+                    g.p[i - i0] = GemmProblem{Xb(p), p.Y, p.Z, nullptr, p.rt > 0 ? d : 0, p.rt, p.dims.L, (int)X->ld, p.rt, p.rt, 0};
+                }
+                if ((st = launch_gemm_simt<T, float, float, true>(ctx, g, store)) != ATP_OK) return st;
+                for (size_t i = i0; i < i1; ++i) {
+                    SeqPlan &p = bp.seqs[i];
+                    g.p[i - i0] = GemmProblem{Xb(p), p.Z, p.Y, nullptr, p.dims.L, p.rt, d, (int)X->ld, p.rt, p.rt, 0};
+                }
+                if ((st = launch_gemm_simt<T, float, float, false>(ctx, g, store)) != ATP_OK) return st;
+                if ((st = orthonormalise(ctx, bp, i0, i1, false, d, seed + 2000003ull * (it + 1))) != ATP_OK) return st;
+            }
         }
         if (!two_sided) {
             // B = Y^T X into BW[:, :d]; Wt = I
@@ -861,7 +922,17 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
                 maxnb = std::max(maxnb, nb); maxrt = std::max(maxrt, p.rt); maxr = std::max(maxr, p.dims.r);
             }
             if (maxrt == 0) continue;
-            if ((st = launch_gemm_simt<float, T, float, true>(ctx, g, store)) != ATP_OK) return st;
+            if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+                std::vector<tc::HostProblem> hp;
+                for (size_t i = i0; i < i1; ++i) {      // B = Yb^T X
+                    SeqPlan &p = bp.seqs[i];
+                    hp.push_back(tc::HostProblem{p.Yb, Xb(p), nullptr, p.BW, nullptr, nullptr, p.rt, d, p.dims.L,
+                                                 (int)align_up((size_t)p.rt, 8), (int)X->ld, d, 0});
+                }
+                if ((st = tc::launch<true, false, tc::OUT_F32>(ctx, hp, store)) != ATP_OK) return st;
+            } else {
+                if ((st = launch_gemm_simt<float, T, float, true>(ctx, g, store)) != ATP_OK) return st;
+            }
             if ((st = launch_gemm_simt<float, float, float, false, true>(ctx, gg, store)) != ATP_OK) return st;
             ATP_KERNEL(ctx, "jac2_init", 0, 0);
             jac2_init_kernel<<<dim3(64, cnt), 256, 0, ctx->stream>>>(jb);

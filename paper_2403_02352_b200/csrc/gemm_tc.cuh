@@ -348,7 +348,7 @@ static atp_status launch(atp_ctx *ctx, const std::vector<HostProblem> &probs, Ge
 }
 
 // fp32 -> bf16 copy (rows x cols), destination leading dimension ldd (multiple of 8 for TMA).
-__global__ void f32_to_bf16_kernel(const float *src, int lds, __nv_bfloat16 *dst, int ldd, int rows, int cols)
+static __global__ void f32_to_bf16_kernel(const float *src, int lds, __nv_bfloat16 *dst, int ldd, int rows, int cols)
 {
     size_t n = (size_t)rows * cols;
     for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
