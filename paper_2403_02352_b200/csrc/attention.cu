@@ -2,6 +2,7 @@
 // on the r principal keys/values (the procedure of Eq. 1 with K', V' in place of K, V).
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
+#include "attention_tc.cuh"
 #include <type_traits>
 #include <math.h>
 
@@ -122,7 +123,7 @@ attn_simt_kernel(const __grid_constant__ AttnBatch batch, int dh, int ldq, int l
     }
 }
 
-struct AttnPlan { float *Qp, *Kp, *Vp, *Q; __nv_bfloat16 *Qph, *Qpl; };
+struct AttnPlan { float *Qp, *Kp, *Vp, *Q; __nv_bfloat16 *Qph, *Qpl, *Kh, *Kl, *Vb, *Qh, *Ql; };
 static void plan_attn(Arena &ar, int64_t tr, int64_t tl, int64_t dp, AttnPlan &p)
 {
     p.Qp = ar.take<float>((size_t)tr * dp);
@@ -131,6 +132,11 @@ static void plan_attn(Arena &ar, int64_t tr, int64_t tl, int64_t dp, AttnPlan &p
     p.Q = ar.take<float>((size_t)tl * dp);
     p.Qph = ar.take<__nv_bfloat16>((size_t)tr * align_up((size_t)dp, 8));     // Q' as a bf16 hi/lo pair (tensor-core path)
     p.Qpl = ar.take<__nv_bfloat16>((size_t)tr * align_up((size_t)dp, 8));
+    p.Kh = ar.take<__nv_bfloat16>((size_t)tr * align_up((size_t)dp, 8));      // fused tensor-core attention operands
+    p.Kl = ar.take<__nv_bfloat16>((size_t)tr * align_up((size_t)dp, 8));
+    p.Vb = ar.take<__nv_bfloat16>((size_t)tr * align_up((size_t)dp, 8));
+    p.Qh = ar.take<__nv_bfloat16>((size_t)tl * align_up((size_t)dp, 8));
+    p.Ql = ar.take<__nv_bfloat16>((size_t)tl * align_up((size_t)dp, 8));
 }
 size_t attention_workspace_bytes(const std::vector<SeqDims> &seqs, int64_t dp)
 {
@@ -157,7 +163,37 @@ static atp_status attention_impl(atp_ctx *ctx, const atp_mat *X, const atp_mat *
     atp_status st;
     GemmEpi store{EPI_STORE, nullptr};
     if constexpr (std::is_same<T, __nv_bfloat16>::value) {
-        // bf16: projections on the tensor cores with fp32 results. Q' is kept as a bf16 hi/lo pair so
+        if (dh == 64 || dh == 128) {
+            // bf16, head width 64 or 128: everything on the tensor cores. K' and Q are produced as
+            // bf16 hi/lo pairs by the GEMM epilogues, V' as bf16; the fused kernel does the rest.
+            const int ldq = (int)align_up((size_t)dp, 8);
+            std::vector<tc::HostProblem> g1, g2;
+            g1.push_back(tc::HostProblem{X_r->data, WK->data, nullptr, pl.Kh, pl.Kl, nullptr, (int)tr, dp, d, (int)X_r->ld, (int)WK->ld, ldq, 0});
+            if (q_mode == ATP_Q_LOWRANK)
+                g1.push_back(tc::HostProblem{X_r->data, WQ->data, nullptr, pl.Qph, pl.Qpl, nullptr, (int)tr, dp, d, (int)X_r->ld, (int)WQ->ld, ldq, 0});
+            else
+                g1.push_back(tc::HostProblem{X->data, WQ->data, nullptr, pl.Qh, pl.Ql, nullptr, (int)tl, dp, d, (int)X->ld, (int)WQ->ld, ldq, 0});
+            if ((st = tc::launch<false, false, tc::OUT_BF16_SPLIT>(ctx, g1, store)) != ATP_OK) return st;
+            g2.push_back(tc::HostProblem{X_r->data, WV->data, nullptr, pl.Vb, nullptr, nullptr, (int)tr, dp, d, (int)X_r->ld, (int)WV->ld, ldq, 0});
+            if ((st = tc::launch<false, false, tc::OUT_BF16>(ctx, g2, store)) != ATP_OK) return st;
+            if (q_mode == ATP_Q_LOWRANK) {
+                std::vector<tc::HostProblem> qe;
+                for (auto &s : seqs)
+                    if (s.L > 0)
+                        qe.push_back(tc::HostProblem{(const T *)U_r->data + (size_t)s.row0 * U_r->ld, pl.Qph + (size_t)s.rank0 * ldq,
+                                                     pl.Qpl + (size_t)s.rank0 * ldq, pl.Qh + (size_t)s.row0 * ldq, pl.Ql + (size_t)s.row0 * ldq,
+                                                     nullptr, s.L, dp, s.r, (int)U_r->ld, ldq, ldq, 0});
+                if ((st = tc::launch<false, true, tc::OUT_BF16_SPLIT>(ctx, qe, store)) != ATP_OK) return st;
+            }
+            std::vector<atc::HostSeq> hs;
+            for (auto &s : seqs)
+                if (s.L > 0)
+                    hs.push_back(atc::HostSeq{pl.Qh + (size_t)s.row0 * ldq, pl.Ql + (size_t)s.row0 * ldq, pl.Kh + (size_t)s.rank0 * ldq,
+                                              pl.Kl + (size_t)s.rank0 * ldq, pl.Vb + (size_t)s.rank0 * ldq,
+                                              (T *)O->data + (size_t)s.row0 * O->ld, s.L, s.r, ldq, ldq, (int)O->ld, dp});
+            return dh == 64 ? atc::launch<64>(ctx, hs, heads, scale) : atc::launch<128>(ctx, hs, heads, scale);
+        }
+        // bf16, other head widths: projections on the tensor cores with fp32 results. Q' is kept as a bf16 hi/lo pair so
         // that the expansion Q = U_r Q' loses nothing against fp32 (the logits reach magnitudes of
         // 10^2, where a bf16-rounded query would move the softmax).
         const int ldq = (int)align_up((size_t)dp, 8);

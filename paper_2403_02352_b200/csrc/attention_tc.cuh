@@ -1,0 +1,331 @@
+// Fused attention of 128 queries of one head on the r principal keys/values of their sequence
+// (score GEMM, row softmax, value GEMM in one kernel; Sec. 4.1 closing paragraph, Eq. 1 on r keys).
+//
+//   S = Q_h K'_h^T          tcgen05.mma, accumulator in TMEM (two 128 x 128 fp32 buffers)
+//   P = exp2(S * c - m)     one thread per query row (TMEM lane = row), online maximum
+//   O += P V'_h             tcgen05.mma, accumulator 128 x d_h fp32 in TMEM
+//
+// Q and K' arrive as bf16 hi/lo pairs and the scores are accumulated from three products
+// (Qh Kh + Qh Kl + Ql Kh): with logits of magnitude 10^2 a single bf16 rounding of Q or K' moves
+// the softmax by more than the accuracy bar, the split keeps ~16 mantissa bits. P and V' are bf16.
+// Operands are staged by TMA (128-byte swizzle): Q once, then per 128-key block K'_hi, K'_lo, V'
+// through a ring of tile slots. Warp 4 issues TMA, warp 5 issues the MMAs, warps 0-3 run softmax,
+// the O rescale (only when a row maximum grows by more than 2^8) and the final normalisation.
+// Every mbarrier wait is bounded; on expiry the kernel records ATP_ERR_TIMEOUT and winds down.
+#pragma once
+#include "gemm_tc.cuh"
+
+namespace atc {
+using namespace tc;
+
+constexpr int MAX_SEQ = 16;
+struct Seq {
+    CUtensorMap qh, ql, kh, kl, v;      // Q hi/lo: L x d' ; K' hi/lo, V': r x d'
+    void *O; int L, r, ldo, tile0;
+};
+struct Batch { Seq s[MAX_SEQ]; int count, total_tiles; };
+
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32])
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+                 "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+                 "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+                   "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+                   "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+                   "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+                 : "memory");
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ float fast_exp2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+template <int DH> struct Cfg {
+    static constexpr int TILE = 128 * DH * 2;                   // one 128-row operand tile (bf16)
+    static constexpr int NSLOT = (DH == 128) ? 3 : 6;           // K'_hi / K'_lo / V' tile slots
+    static constexpr int P_BYTES = 128 * 128 * 2;               // one P buffer
+    static constexpr int OFF_Q = 0;                             // Q hi, Q lo
+    static constexpr int OFF_SLOT = 2 * TILE;
+    static constexpr int OFF_P = OFF_SLOT + NSLOT * TILE;       // single P buffer (reused once its MMAs finished)
+    static constexpr int OFF_BAR = OFF_P + P_BYTES;
+    static constexpr int NBAR = 1 + 2 * NSLOT + 2 + 2 + 1 + 1 + 1;   // q, slot full/empty, s_full[2], s_free[2], p_full, p_free, o_done
+    static constexpr int SMEM = OFF_BAR + 8 * NBAR + 16 + 1024;
+};
+
+template <int DH>
+__global__ void __launch_bounds__(192)
+attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e, int *dev_status)
+{
+    using C_ = Cfg<DH>;
+    constexpr int NS = C_::NSLOT;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t *gbase = smem_raw + (base - raw);
+    const uint32_t bar0 = base + C_::OFF_BAR;
+    const uint32_t b_q = bar0, b_full = bar0 + 8, b_empty = b_full + 8 * NS, b_sfull = b_empty + 8 * NS, b_sfree = b_sfull + 16,
+                   b_pfull = b_sfree + 16, b_pfree = b_pfull + 8, b_odone = b_pfree + 8;
+    uint32_t *tmem_slot = (uint32_t *)(gbase + C_::OFF_BAR + 8 * C_::NBAR);
+    __shared__ int abort_flag;
+
+    // work item: (sequence, query tile) from blockIdx.x, head from blockIdx.y
+    int si = 0;
+#pragma unroll 1
+    for (int i = 1; i < batch.count; ++i) if ((int)blockIdx.x >= batch.s[i].tile0) si = i;
+    const Seq &sq = batch.s[si];
+    const int q0 = ((int)blockIdx.x - sq.tile0) * 128;
+    const int head = blockIdx.y;
+    const int col0 = head * DH;
+    const int nblk = (sq.r + 127) / 128;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(b_q, 1);
+        for (int s = 0; s < NS; ++s) { mbar_init(b_full + 8 * s, 1); mbar_init(b_empty + 8 * s, 1); }
+        mbar_init(b_sfull, 1); mbar_init(b_sfull + 8, 1);
+        mbar_init(b_sfree, 4); mbar_init(b_sfree + 8, 4);
+        mbar_init(b_pfull, 4); mbar_init(b_pfree, 1); mbar_init(b_odone, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 5) tmem_alloc(smem_u32(tmem_slot), 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t t_s0 = tmem_base, t_o = tmem_base + 256;
+
+    if (warp == 4) {
+        if (lane == 0) {
+            mbar_expect_tx(b_q, 2 * C_::TILE);
+#pragma unroll
+            for (int c = 0; c < DH / 64; ++c) {
+                tma_load_2d(base + C_::OFF_Q + c * 16384, &sq.qh, col0 + 64 * c, q0, b_q);
+                tma_load_2d(base + C_::OFF_Q + C_::TILE + c * 16384, &sq.ql, col0 + 64 * c, q0, b_q);
+            }
+            int li = 0;                                   // running load index: K'_hi, K'_lo, V' per block
+            for (int j = 0; j < nblk; ++j) {
+                for (int which = 0; which < 3; ++which, ++li) {
+                    const int s = li % NS, n = li / NS;
+                    if (n >= 1 && !mbar_wait(b_empty + 8 * s, (n - 1) & 1, &abort_flag)) { j = nblk; break; }
+                    const uint32_t dst = base + C_::OFF_SLOT + s * C_::TILE;
+                    const CUtensorMap *m = which == 0 ? &sq.kh : (which == 1 ? &sq.kl : &sq.v);
+                    mbar_expect_tx(b_full + 8 * s, C_::TILE);
+#pragma unroll
+                    for (int c = 0; c < DH / 64; ++c) tma_load_2d(dst + c * 16384, m, col0 + 64 * c, j * 128, b_full + 8 * s);
+                }
+            }
+        }
+    } else if (warp == 5) {
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = instr_desc(128, 128, false, false);
+            constexpr uint32_t idesc_o = instr_desc(128, DH, false, true);
+            const uint32_t q_hi = base + C_::OFF_Q, q_lo = q_hi + C_::TILE;
+            bool ok = mbar_wait(b_q, 0, &abort_flag);
+            tc_fence_after();
+            // S_j for block j into buffer j & 1: Qh Kh^T + Qh Kl^T + Ql Kh^T
+            auto issue_s = [&](int j) -> bool {
+                const int lk = 3 * j, sh = lk % NS, sl = (lk + 1) % NS;
+                if (j >= 2 && !mbar_wait(b_sfree + 8 * (j & 1), ((j >> 1) - 1) & 1, &abort_flag)) return false;
+                if (!mbar_wait(b_full + 8 * sh, (lk / NS) & 1, &abort_flag)) return false;
+                if (!mbar_wait(b_full + 8 * sl, ((lk + 1) / NS) & 1, &abort_flag)) return false;
+                tc_fence_after();
+                const uint32_t kh = base + C_::OFF_SLOT + sh * C_::TILE, kl = base + C_::OFF_SLOT + sl * C_::TILE;
+                const uint32_t d = t_s0 + 128 * (j & 1);
+#pragma unroll
+                for (int kk = 0; kk < DH / 16; ++kk) {
+                    const uint32_t off = (kk >> 2) * 16384 + (kk & 3) * 32;
+                    const uint64_t aqh = smem_desc(q_hi + off, 16, 1024), aql = smem_desc(q_lo + off, 16, 1024);
+                    const uint64_t bkh = smem_desc(kh + off, 16, 1024), bkl = smem_desc(kl + off, 16, 1024);
+                    umma_bf16(d, aqh, bkh, idesc_s, kk > 0 ? 1u : 0u);
+                    umma_bf16(d, aqh, bkl, idesc_s, 1u);
+                    umma_bf16(d, aql, bkh, idesc_s, 1u);
+                }
+                umma_commit(b_empty + 8 * sh);
+                umma_commit(b_empty + 8 * sl);
+                umma_commit(b_sfull + 8 * (j & 1));
+                return true;
+            };
+            if (ok) ok = issue_s(0);
+            for (int j = 0; j < nblk && ok; ++j) {
+                if (j + 1 < nblk) { ok = issue_s(j + 1); if (!ok) break; }
+                // O += P_j V_j
+                const int lv = 3 * j + 2, sv = lv % NS;
+                if (!mbar_wait(b_full + 8 * sv, (lv / NS) & 1, &abort_flag)) { ok = false; break; }
+                if (!mbar_wait(b_pfull, j & 1, &abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t pv = base + C_::OFF_P, vv = base + C_::OFF_SLOT + sv * C_::TILE;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint64_t ap = smem_desc(pv + (kk >> 2) * 16384 + (kk & 3) * 32, 16, 1024);
+                    const uint64_t bv = smem_desc(vv + kk * 2048, 16384, 1024);
+                    umma_bf16(t_o, ap, bv, idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
+                }
+                umma_commit(b_empty + 8 * sv);
+                umma_commit(b_pfree);
+                umma_commit(b_odone);
+            }
+        }
+    } else {
+        // softmax / correction / epilogue: thread = query row, TMEM lane = warp * 32 + lane
+        const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+        const int row = warp * 32 + lane;
+        float m_used = -INFINITY, l_sum = 0.f;
+        bool ok = true;
+        for (int j = 0; j < nblk; ++j) {
+            int ok_i = 0;
+            if (lane == 0) ok_i = mbar_wait(b_sfull + 8 * (j & 1), (j >> 1) & 1, &abort_flag) ? 1 : 0;
+            ok = __shfl_sync(0xffffffffu, ok_i, 0) != 0;
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t t_s = t_s0 + 128 * (j & 1) + lane_addr;
+            const int kvalid = sq.r - j * 128;                 // keys of this block that exist
+            // pass A: block maximum of the scaled scores
+            float mx = -INFINITY;
+#pragma unroll 1
+            for (int c = 0; c < 128; c += 32) {
+                uint32_t rr[32];
+                tmem_ld32(t_s + c, rr);
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    if (c + i < kvalid) mx = fmaxf(mx, __uint_as_float(rr[i]) * scale_log2e);
+            }
+            // the exponent offset only moves when the maximum grew by more than 8 (factor 256)
+            float alpha = 1.f;
+            bool grow = (mx > m_used + 8.f) || (j == 0);
+            if (grow) { alpha = (j == 0) ? 0.f : fast_exp2(m_used - mx); m_used = mx; }
+            if (j > 0 && __any_sync(0xffffffffu, grow)) {
+                // O must be quiescent: P V of block j-1 done (block j's waits for the P written below)
+                if (lane == 0) ok_i = mbar_wait(b_odone, (j - 1) & 1, &abort_flag) ? 1 : 0;
+                ok = __shfl_sync(0xffffffffu, ok_i, 0) != 0;
+                if (!ok) break;
+                tc_fence_after();
+#pragma unroll 1
+                for (int c = 0; c < DH; c += 32) {
+                    uint32_t rr[32];
+                    tmem_ld32(t_o + lane_addr + c, rr);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) rr[i] = __float_as_uint(__uint_as_float(rr[i]) * alpha);
+                    tmem_st32(t_o + lane_addr + c, rr);
+                }
+                tc_fence_before();
+            }
+            l_sum *= alpha;
+            // the single P buffer is free once the value MMAs of block j-1 have read it
+            if (j > 0) {
+                if (lane == 0) ok_i = mbar_wait(b_pfree, (j - 1) & 1, &abort_flag) ? 1 : 0;
+                ok = __shfl_sync(0xffffffffu, ok_i, 0) != 0;
+                if (!ok) break;
+            }
+            // pass B: P = exp2(s - m) as bf16 into the swizzled K-major A tile, row sums in fp32
+            uint8_t *prow = gbase + C_::OFF_P + row * 128;
+#pragma unroll 1
+            for (int c = 0; c < 128; c += 32) {
+                uint32_t rr[32];
+                tmem_ld32(t_s + c, rr);
+                uint32_t packed[16];
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) {
+                    float p0 = (c + i < kvalid) ? fast_exp2(__uint_as_float(rr[i]) * scale_log2e - m_used) : 0.f;
+                    float p1 = (c + i + 1 < kvalid) ? fast_exp2(__uint_as_float(rr[i + 1]) * scale_log2e - m_used) : 0.f;
+                    __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+                    l_sum += __low2float(h) + __high2float(h);          // sum what the value GEMM will see
+                    packed[i >> 1] = *(uint32_t *)&h;
+                }
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {                           // four 16-byte chunks of 8 keys
+                    const int chunk16 = (c >> 3) + q;                   // 0..15 along the 128 keys
+                    const int region = chunk16 >> 3, within = chunk16 & 7;
+                    uint4 val = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+                    *(uint4 *)(prow + region * 16384 + ((within ^ (row & 7)) << 4)) = val;
+                }
+            }
+            tc_fence_before();
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA
+            __syncwarp();
+            if (lane == 0) { mbar_arrive(b_sfree + 8 * (j & 1)); mbar_arrive(b_pfull); }
+        }
+        // epilogue: O / l
+        int ok_i = 0;
+        if (ok && lane == 0) ok_i = mbar_wait(b_odone, (nblk - 1) & 1, &abort_flag) ? 1 : 0;
+        ok = ok && (__shfl_sync(0xffffffffu, ok_i, 0) != 0);
+        tc_fence_after();
+        if (ok) {
+            const float inv = 1.f / l_sum;
+            const int grow_ = q0 + row;
+            __nv_bfloat16 *dst = (__nv_bfloat16 *)sq.O + (size_t)grow_ * sq.ldo + col0;
+#pragma unroll 1
+            for (int c = 0; c < DH; c += 32) {
+                uint32_t rr[32];
+                tmem_ld32(t_o + lane_addr + c, rr);
+                if (grow_ < sq.L) {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 8) {
+                        __nv_bfloat162 h[4];
+#pragma unroll
+                        for (int t = 0; t < 4; ++t)
+                            h[t] = __floats2bfloat162_rn(__uint_as_float(rr[i + 2 * t]) * inv, __uint_as_float(rr[i + 2 * t + 1]) * inv);
+                        *(uint4 *)(dst + c + i) = *(uint4 *)h;
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && abort_flag && dev_status) raise_status(dev_status, ATP_ERR_TIMEOUT);
+    if (warp == 5) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+struct HostSeq {
+    const void *Qh, *Ql, *Kh, *Kl, *V; void *O;
+    int L, r, ldq, ldk, ldo, dp;
+};
+
+template <int DH>
+static atp_status launch(atp_ctx *ctx, const std::vector<HostSeq> &seqs, int heads, float scale)
+{
+    using C_ = Cfg<DH>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        ATP_CUDA_OK(ctx, cudaFuncSetAttribute(attn_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::SMEM));
+        attr_set = true;
+    }
+    size_t i = 0;
+    while (i < seqs.size()) {
+        Batch b; b.count = 0; b.total_tiles = 0;
+        double flops = 0, bytes = 0;
+        for (; i < seqs.size() && b.count < MAX_SEQ; ++i) {
+            const HostSeq &h = seqs[i];
+            if (h.L <= 0) continue;
+            Seq &s = b.s[b.count];
+            bool ok = make_map(&s.qh, h.Qh, h.L, h.dp, h.ldq, 128) && make_map(&s.ql, h.Ql, h.L, h.dp, h.ldq, 128) &&
+                      make_map(&s.kh, h.Kh, h.r, h.dp, h.ldk, 128) && make_map(&s.kl, h.Kl, h.r, h.dp, h.ldk, 128) &&
+                      make_map(&s.v, h.V, h.r, h.dp, h.ldk, 128);
+            if (!ok) return ATP_ERR_INVALID_ARG;
+            s.O = h.O; s.L = h.L; s.r = h.r; s.ldo = h.ldo; s.tile0 = b.total_tiles;
+            b.total_tiles += ceil_div(h.L, 128);
+            b.count++;
+            flops += 4.0 * h.L * h.r * h.dp;                                   // algorithmic: one score and one value product
+            bytes += 2.0 * (2.0 * h.L * h.dp + 3.0 * h.r * h.dp) + 2.0 * h.L * h.dp;
+        }
+        if (b.count == 0) continue;
+        ATP_KERNEL(ctx, "attn_tc", flops, bytes);
+        attn_tc_kernel<DH><<<dim3(b.total_tiles, heads), 192, C_::SMEM, ctx->stream>>>(b, heads, scale * 1.4426950408889634f, ctx->dev_status);
+        ATP_LAUNCHED(ctx);
+    }
+    return ATP_OK;
+}
+
+}  // namespace atc

@@ -79,21 +79,22 @@ __global__ void __launch_bounds__(256) panel_gram_kernel(const __grid_constant__
         for (int j = 0; j < 4; ++j) dst[(ty * 4 + i) * PB + tx * 4 + j] = acc[i][j];
 }
 
-// Sums the partial Gram matrices in order, scales to unit diagonal, Cholesky-factors in fp64 and
-// writes Rinv (pb x pb, fp32) such that P * Rinv has orthonormal columns. A column whose scaled
-// pivot falls below 1e-10 (its part outside the span of the earlier columns is below 1e-5 of its
-// norm) is flagged as dependent: its Rinv column is zero and the apply kernel replaces it by a
-// pseudo-random vector, which the second Gram-Schmidt pass orthonormalises.
+// Sums the partial Gram matrices in order, scales to unit diagonal and Cholesky-factors in fp64:
+// D^-1 G D^-1 = L L^T. Writes L (fp32, row-major pb x PB) followed by 1/D, so that
+// P D^-1 L^-T has orthonormal columns. A column whose scaled pivot falls below 1e-10 (its part
+// outside the span of the earlier columns is below 1e-5 of its norm) is flagged as dependent: the
+// apply kernel replaces it by a pseudo-random vector, which the second Gram-Schmidt pass
+// orthonormalises. Four threads share a row of the factor (partial dot products + shuffles).
 __global__ void __launch_bounds__(256) panel_chol_kernel(const __grid_constant__ PanelBatch batch)
 {
     const PanelSeq &sq = batch.s[blockIdx.x];
     const int n = sq.pb;
     if (n <= 0) return;
-    extern __shared__ double chol_sm[];
-    double (*G)[PB + 1] = (double (*)[PB + 1])chol_sm;
-    double (*Li)[PB + 1] = (double (*)[PB + 1])(chol_sm + PB * (PB + 1));
+    __shared__ double G[PB][PB + 1];
     __shared__ double dsc[PB];
     __shared__ int dep[PB];
+    __shared__ double sh_ljj;
+    __shared__ int sh_bad;
     const int tid = threadIdx.x;
     const int nchunks = (sq.n + GRAM_ROWS - 1) / GRAM_ROWS;
     for (int e = tid; e < PB * PB; e += 256) {
@@ -110,93 +111,73 @@ __global__ void __launch_bounds__(256) panel_chol_kernel(const __grid_constant__
         G[i][j] = den > 0.0 ? G[i][j] / den : 0.0;
     }
     __syncthreads();
-    __shared__ double sh_ljj;
-    __shared__ int sh_bad;
+    const int row = tid >> 2, part = tid & 3;
     for (int j = 0; j < n; ++j) {       // left-looking: column j from the finished columns < j
         double sacc = 0.0;
-        if (tid >= j && tid < n) {
-            sacc = G[tid][j];
-            for (int k = 0; k < j; ++k) sacc -= G[tid][k] * G[j][k];
-        }
-        if (tid == j) {
+        if (row >= j && row < n)
+            for (int k = part; k < j; k += 4) sacc -= G[row][k] * G[j][k];
+        sacc += __shfl_xor_sync(0xffffffffu, sacc, 1);
+        sacc += __shfl_xor_sync(0xffffffffu, sacc, 2);
+        if (row >= j && row < n) sacc += G[row][j];
+        if (row == j && part == 0) {
             int bad = !(sacc > 1e-10);
             sh_bad = bad;
             sh_ljj = bad ? 1.0 : sqrt(sacc);
             if (bad) dep[j] = 1;
         }
         __syncthreads();
-        if (tid >= j && tid < n) G[tid][j] = (tid == j) ? sh_ljj : (sh_bad ? 0.0 : sacc / sh_ljj);
+        if (part == 0 && row >= j && row < n) G[row][j] = (row == j) ? sh_ljj : (sh_bad ? 0.0 : sacc / sh_ljj);
         __syncthreads();
     }
-    // Li = inverse of the lower-triangular factor, one column per thread
-    if (tid < n) {
-        int c = tid;
-        for (int i = 0; i < n; ++i) {
-            double x = 0.0;
-            if (i >= c) {
-                x = (i == c) ? 1.0 : 0.0;
-                for (int k = c; k < i; ++k) x -= G[i][k] * Li[k][c];
-                x /= G[i][i];
-            }
-            Li[i][c] = x;
-        }
-    }
-    __syncthreads();
     for (int e = tid; e < PB * PB; e += 256) {
-        int k = e >> 6, c = e & 63;      // Rinv[k][c] = Li[c][k] / dsc[k]
-        double v = 0.0;
-        if (k < n && c < n && !dep[c] && !dep[k] && dsc[k] > 0.0) v = Li[c][k] / dsc[k];
-        sq.rinv[e] = (float)v;
+        int i = e >> 6, k = e & 63;
+        sq.rinv[e] = (i < n && k <= i) ? (float)G[i][k] : (i == k ? 1.f : 0.f);
     }
-    if (tid < PB) sq.flags[tid] = (tid < n) ? dep[tid] : 0;
+    if (tid < PB) {
+        sq.rinv[PB * PB + tid] = (tid < n && dsc[tid] > 0.0) ? (float)(1.0 / dsc[tid]) : 0.f;
+        sq.flags[tid] = (tid < n) ? (dep[tid] || !(dsc[tid] > 0.0)) : 0;
+    }
 }
 
-// P <- P * Rinv in place (each CTA owns 64 rows); flagged columns are refilled with hash noise.
-__global__ void __launch_bounds__(256) panel_apply_kernel(const __grid_constant__ PanelBatch batch, uint64_t seed)
+// P <- P D^-1 L^-T in place: every thread solves the triangular system of one row (forward
+// substitution, fully unrolled, L broadcast from shared memory); rows are staged through shared
+// memory so that global accesses stay coalesced. Flagged columns are refilled with hash noise.
+__global__ void __launch_bounds__(64) panel_apply_kernel(const __grid_constant__ PanelBatch batch, uint64_t seed)
 {
     const PanelSeq &sq = batch.s[blockIdx.y];
     const int r0 = blockIdx.x * 64;
     if (sq.pb <= 0 || r0 >= sq.n) return;
-    __shared__ __align__(16) float Rs[PB][PB + 4];
+    __shared__ float Ls[PB][PB + 1];
     __shared__ float Ts[64][PB + 1];
+    __shared__ float dinv[PB];
     __shared__ int fl[PB];
-    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-    for (int e = tid; e < PB * PB; e += 256) Rs[e >> 6][e & 63] = sq.rinv[e];
-    if (tid < PB) fl[tid] = sq.flags[tid];
-    for (int e = tid; e < 64 * PB; e += 256) {
+    const int tid = threadIdx.x;
+    for (int e = tid; e < PB * PB; e += 64) Ls[e >> 6][e & 63] = sq.rinv[e];
+    dinv[tid] = sq.rinv[PB * PB + tid];
+    fl[tid] = sq.flags[tid];
+    for (int e = tid; e < 64 * PB; e += 64) {
         int row = e >> 6, c = e & 63;
         float v = 0.f;
         if (r0 + row < sq.n && c < sq.pb) v = sq.P[(size_t)(r0 + row) * sq.ld + c];
         Ts[row][c] = v;
     }
     __syncthreads();
-    float acc[4][4];
+    float x[PB];
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
+    for (int c = 0; c < PB; ++c) {
+        float acc = Ts[tid][c] * dinv[c];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
-    for (int k = 0; k < PB; ++k) {
-        float4 b = *(const float4 *)&Rs[k][tx * 4];
-        float bv[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            float a = Ts[ty * 4 + i][k];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a, bv[j], acc[i][j]);
-        }
+        for (int k = 0; k < c; ++k) acc = fmaf(-x[k], Ls[c][k], acc);
+        x[c] = acc / Ls[c][c];
     }
+    const int grow = r0 + tid;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        int row = r0 + ty * 4 + i;
-        if (row >= sq.n) continue;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            int c = tx * 4 + j;
-            if (c >= sq.pb) continue;
-            float v = acc[i][j];
-            if (fl[c]) v = hash_uniform(seed, ((uint64_t)blockIdx.y << 40) ^ ((uint64_t)row << 8) ^ (uint64_t)c);
-            sq.P[(size_t)row * sq.ld + c] = v;
-        }
+    for (int c = 0; c < PB; ++c)
+        Ts[tid][c] = fl[c] ? hash_uniform(seed, ((uint64_t)blockIdx.y << 40) ^ ((uint64_t)grow << 8) ^ (uint64_t)c) : x[c];
+    __syncthreads();
+    for (int e = tid; e < 64 * PB; e += 64) {
+        int row = e >> 6, c = e & 63;
+        if (r0 + row < sq.n && c < sq.pb) sq.P[(size_t)(r0 + row) * sq.ld + c] = Ts[row][c];
     }
 }
 
@@ -655,8 +636,6 @@ struct BasisPlan {
     std::vector<SeqPlan> seqs; float *omega; __nv_bfloat16 *omega_b; float *part; size_t part_stride; int rtmax; int splits;
 };
 
-constexpr size_t CHOL_SMEM = 2 * PB * (PB + 1) * sizeof(double);
-
 static int pick_splits(int K) { int s = K / 1024; return s < 1 ? 1 : (s > 16 ? 16 : s); }
 
 static void plan_basis(Arena &ar, const std::vector<SeqDims> &sd, int d, int oversample, BasisPlan &bp)
@@ -687,7 +666,7 @@ static void plan_basis(Arena &ar, const std::vector<SeqDims> &sd, int d, int ove
         p.sig = ar.take<float>(rt);
         p.ord = ar.take<int>(rt);
         p.Cc = ar.take<float>((size_t)rt * PB);
-        p.rinv = ar.take<float>(PB * PB);
+        p.rinv = ar.take<float>(PB * PB + PB);
         p.flags = ar.take<int>(PB);
         p.gpart = ar.take<double>((size_t)ceil_div(std::max(std::max(L, d), 1), GRAM_ROWS) * PB * PB);
         p.G = ar.take<float>((size_t)rt * rt);
@@ -720,7 +699,6 @@ static atp_status orthonormalise(atp_ctx *ctx, BasisPlan &bp, size_t i0, size_t 
         maxn = std::max(maxn, z_side ? d : bp.seqs[i].dims.L);
     }
     atp_status st;
-    ATP_CUDA_OK(ctx, cudaFuncSetAttribute(panel_chol_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHOL_SMEM));
     for (int pj = 0; pj < maxpan; ++pj) {
         const int j0 = pj * PB;
         for (int rep = 0; rep < 2; ++rep) {
@@ -747,10 +725,10 @@ static atp_status orthonormalise(atp_ctx *ctx, BasisPlan &bp, size_t i0, size_t 
             panel_gram_kernel<<<dim3(ceil_div(maxn, GRAM_ROWS), pb.count), 256, 0, ctx->stream>>>(pb);
             ATP_LAUNCHED(ctx);
             ATP_KERNEL(ctx, "panel_chol", 0, 0);
-            panel_chol_kernel<<<pb.count, 256, CHOL_SMEM, ctx->stream>>>(pb);
+            panel_chol_kernel<<<pb.count, 256, 0, ctx->stream>>>(pb);
             ATP_LAUNCHED(ctx);
             ATP_KERNEL(ctx, "panel_apply", 0, 0);
-            panel_apply_kernel<<<dim3(ceil_div(maxn, 64), pb.count), 256, 0, ctx->stream>>>(
+            panel_apply_kernel<<<dim3(ceil_div(maxn, 64), pb.count), 64, 0, ctx->stream>>>(
                 pb, seed + 7919ull * (uint64_t)(pj * 2 + rep) + (z_side ? 104729ull : 0ull));
             ATP_LAUNCHED(ctx);
         }
