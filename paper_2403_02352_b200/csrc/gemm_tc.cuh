@@ -288,15 +288,33 @@ gemm_tc_kernel(const __grid_constant__ Batch batch, GemmEpi epi, int *dev_status
 
 // ---- host side ---------------------------------------------------------------------------------
 // Tensor map over a row-major bf16 matrix (rows x cols, ld elements): box {64 cols, box_rows rows}, 128-byte swizzle.
+// The driver entry point is looked up at run time (the library does not link against libcuda, so it
+// still loads on machines without a driver, where only the symbol table is inspected).
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static inline EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
 static inline bool make_map(CUtensorMap *m, const void *ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows)
 {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return false;
     cuuint64_t dims[2] = {cols, rows};
     cuuint64_t strides[1] = {ld * 2};
     cuuint32_t box[2] = {64, box_rows};
     cuuint32_t estr[2] = {1, 1};
-    return cuTensorMapEncodeTiled(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
-                                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 struct HostProblem {
@@ -354,6 +372,19 @@ static __global__ void f32_to_bf16_kernel(const float *src, int lds, __nv_bfloat
     for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
         int r = (int)(e / cols), c = (int)(e - (size_t)r * cols);
         dst[(size_t)r * ldd + c] = __float2bfloat16_rn(src[(size_t)r * lds + c]);
+    }
+}
+
+// fp32 -> bf16 hi/lo pair: hi = bf16(x), lo = bf16(x - hi).
+static __global__ void f32_to_bf16_split_kernel(const float *src, int lds, __nv_bfloat16 *hi, __nv_bfloat16 *lo, int ldd, int rows, int cols)
+{
+    size_t n = (size_t)rows * cols;
+    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
+        int r = (int)(e / cols), c = (int)(e - (size_t)r * cols);
+        float x = src[(size_t)r * lds + c];
+        __nv_bfloat16 h = __float2bfloat16_rn(x);
+        hi[(size_t)r * ldd + c] = h;
+        lo[(size_t)r * ldd + c] = __float2bfloat16_rn(x - __bfloat162float(h));
     }
 }
 
