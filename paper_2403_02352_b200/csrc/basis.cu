@@ -630,7 +630,7 @@ __global__ void __launch_bounds__(256) signfix_kernel(const __grid_constant__ Fi
 // ------------------------------------------------------------------------------------------------
 struct SeqPlan {
     SeqDims dims; int rt, npanel_L, npanel_d;
-    __nv_bfloat16 *Yb, *Zb; float *Y, *Z, *BW, *Wsel, *tsum, *sig, *Cc, *rinv, *G, *Wt, *Vbuf; double *gpart; int *ord, *flags, *conv, *vflag, *needfix; unsigned *maxoff;
+    __nv_bfloat16 *Yb, *Yl, *Zb, *Zl; float *Y2; float *Y, *Z, *BW, *Wsel, *tsum, *sig, *Cc, *rinv, *G, *Wt, *Vbuf; double *gpart; int *ord, *flags, *conv, *vflag, *needfix; unsigned *maxoff;
 };
 struct BasisPlan {
     std::vector<SeqPlan> seqs; float *omega; __nv_bfloat16 *omega_b; float *part; size_t part_stride; int rtmax; int splits;
@@ -659,7 +659,10 @@ static void plan_basis(Arena &ar, const std::vector<SeqDims> &sd, int d, int ove
         p.Y = ar.take<float>((size_t)L * rt);
         p.Z = ar.take<float>((size_t)d * rt);
         p.Yb = ar.take<__nv_bfloat16>((size_t)L * align_up((size_t)rt, 8));
+        p.Yl = ar.take<__nv_bfloat16>((size_t)L * align_up((size_t)rt, 8));
         p.Zb = ar.take<__nv_bfloat16>((size_t)d * align_up((size_t)rt, 8));
+        p.Zl = ar.take<__nv_bfloat16>((size_t)d * align_up((size_t)rt, 8));
+        p.Y2 = ar.take<float>((size_t)L * rt);
         p.BW = ar.take<float>((size_t)rt * (d + rt));
         p.Wsel = ar.take<float>((size_t)rt * p.dims.r);
         p.tsum = ar.take<float>(rt);
@@ -769,14 +772,17 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
             ATP_KERNEL(ctx, "fill_omega", 0, 0);
             fill_omega_bf16_kernel<<<1024, 256, 0, ctx->stream>>>(bp.omega_b, d, bp.rtmax, ldo, seed);
             ATP_LAUNCHED(ctx);
-            auto to_bf16 = [&](bool zside) -> atp_status {
+            // The orthonormal iterate goes to the next pass as a bf16 hi/lo pair (about 16 mantissa
+            // bits): a single bf16 rounding of Y would leak sigma_1 * 2^-9 / sqrt(L) of the leading
+            // direction into every column and bury directions that are 10^3..10^4 times weaker.
+            auto to_bf16 = [&]() -> atp_status {
                 for (size_t i = i0; i < i1; ++i) {
                     SeqPlan &p = bp.seqs[i];
-                    int rows = zside ? d : p.dims.L;
+                    int rows = p.dims.L;
                     if (rows == 0 || p.rt == 0) continue;
-                    ATP_KERNEL(ctx, "f32_to_bf16", 0, (double)rows * p.rt * 6);
-                    tc::f32_to_bf16_kernel<<<std::min(1024, ceil_div(rows * p.rt, 256)), 256, 0, ctx->stream>>>(
-                        zside ? p.Z : p.Y, p.rt, zside ? p.Zb : p.Yb, (int)align_up((size_t)p.rt, 8), rows, p.rt);
+                    ATP_KERNEL(ctx, "f32_to_bf16", 0, (double)rows * p.rt * 8);
+                    tc::f32_to_bf16_split_kernel<<<std::min(1024, ceil_div(rows * p.rt, 256)), 256, 0, ctx->stream>>>(
+                        p.Y, p.rt, p.Yb, p.Yl, (int)align_up((size_t)p.rt, 8), rows, p.rt);
                     ATP_LAUNCHED(ctx);
                 }
                 return ATP_OK;
@@ -788,24 +794,24 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
             }
             if ((st = tc::launch<false, false, tc::OUT_F32>(ctx, hp, store)) != ATP_OK) return st;
             if ((st = orthonormalise(ctx, bp, i0, i1, false, d, seed)) != ATP_OK) return st;
-            if ((st = to_bf16(false)) != ATP_OK) return st;
+            if ((st = to_bf16()) != ATP_OK) return st;
             for (int it = 0; it < power_iters; ++it) {
                 hp.clear();
-                for (size_t i = i0; i < i1; ++i) {      // Z = X^T Y (bf16 result: only the next pass reads it)
+                for (size_t i = i0; i < i1; ++i) {      // Z = X^T Y, kept as a bf16 hi/lo pair (only the next pass reads it)
                     SeqPlan &p = bp.seqs[i];
                     int ldb = (int)align_up((size_t)p.rt, 8);
-                    hp.push_back(tc::HostProblem{Xb(p), p.Yb, nullptr, p.Zb, nullptr, nullptr, d, p.rt, p.dims.L, (int)X->ld, ldb, ldb, 0});
+                    hp.push_back(tc::HostProblem{Xb(p), p.Yb, p.Yl, p.Zb, p.Zl, nullptr, d, p.rt, p.dims.L, (int)X->ld, ldb, ldb, 0});
                 }
-                if ((st = tc::launch<true, false, tc::OUT_BF16>(ctx, hp, store)) != ATP_OK) return st;
+                if ((st = tc::launch<true, true, tc::OUT_BF16_SPLIT>(ctx, hp, store)) != ATP_OK) return st;
                 hp.clear();
                 for (size_t i = i0; i < i1; ++i) {      // Y = X Z
                     SeqPlan &p = bp.seqs[i];
                     int ldb = (int)align_up((size_t)p.rt, 8);
-                    hp.push_back(tc::HostProblem{Xb(p), p.Zb, nullptr, p.Y, nullptr, nullptr, p.dims.L, p.rt, d, (int)X->ld, ldb, p.rt, 0});
+                    hp.push_back(tc::HostProblem{Xb(p), p.Zb, p.Zl, p.Y, nullptr, nullptr, p.dims.L, p.rt, d, (int)X->ld, ldb, p.rt, 0});
                 }
-                if ((st = tc::launch<false, false, tc::OUT_F32>(ctx, hp, store)) != ATP_OK) return st;
+                if ((st = tc::launch<false, true, tc::OUT_F32>(ctx, hp, store)) != ATP_OK) return st;
                 if ((st = orthonormalise(ctx, bp, i0, i1, false, d, seed + 2000003ull * (it + 1))) != ATP_OK) return st;
-                if ((st = to_bf16(false)) != ATP_OK) return st;
+                if ((st = to_bf16()) != ATP_OK) return st;
             }
         } else {
             // Y = X Omega
@@ -883,15 +889,16 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
             if ((st = launch_gemm_simt<float, float, T, false>(ctx, g, store)) != ATP_OK) return st;
     
         } else {
-            // B = Y^T X (r~ x d), G = B B^T, two-sided block Jacobi on G, then X_r = Wsel^T B, U_r = Y Wsel
+            // Bt = X^T Y (d x r~, i.e. B^T), G = Bt^T Bt, two-sided block Jacobi on G, then
+            // X_r = Wsel^T Bt^T and U_r = Y Wsel
             Jac2Batch jb; jb.count = cnt; Fin2Batch fb; fb.count = cnt;
             GemmBatch gg; gg.count = cnt;
             int maxnb = 2, maxrt = 0, maxr = 0;
             for (size_t i = i0; i < i1; ++i) {
                 SeqPlan &p = bp.seqs[i];
                 int k = (int)(i - i0);
-                g.p[k] = GemmProblem{p.Y, Xb(p), p.BW, nullptr, p.rt, p.rt > 0 ? d : 0, p.dims.L, p.rt, (int)X->ld, d, 0};
-                gg.p[k] = GemmProblem{p.BW, p.BW, p.G, nullptr, p.rt, p.rt, p.rt > 0 ? d : 0, d, d, p.rt, 0};
+                g.p[k] = GemmProblem{Xb(p), p.Y, p.BW, nullptr, p.rt > 0 ? d : 0, p.rt, p.dims.L, (int)X->ld, p.rt, p.rt, 0};
+                gg.p[k] = GemmProblem{p.BW, p.BW, p.G, nullptr, p.rt, p.rt, p.rt > 0 ? d : 0, p.rt, p.rt, p.rt, 0};
                 int nb = ceil_div(std::max(p.rt, 1), jbj); nb += nb & 1;
                 jb.s[k] = Jac2Seq{p.G, p.Wt, p.Vbuf, p.vflag, p.rt, nb, p.maxoff, p.conv};
                 fb.s[k] = Fin2Seq{p.G, p.Wt, p.Y, p.sig, p.ord, p.tsum, p.Wsel, p.needfix,
@@ -902,38 +909,60 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
             if (maxrt == 0) continue;
             if constexpr (std::is_same<T, __nv_bfloat16>::value) {
                 std::vector<tc::HostProblem> hp;
-                for (size_t i = i0; i < i1; ++i) {      // B = Yb^T X
+                for (size_t i = i0; i < i1; ++i) {      // Bt = X^T (Yb + Yl)
                     SeqPlan &p = bp.seqs[i];
-                    hp.push_back(tc::HostProblem{p.Yb, Xb(p), nullptr, p.BW, nullptr, nullptr, p.rt, d, p.dims.L,
-                                                 (int)align_up((size_t)p.rt, 8), (int)X->ld, d, 0});
+                    int ldb = (int)align_up((size_t)p.rt, 8);
+                    hp.push_back(tc::HostProblem{Xb(p), p.Yb, p.Yl, p.BW, nullptr, nullptr, d, p.rt, p.dims.L, (int)X->ld, ldb, p.rt, 0});
                 }
-                if ((st = tc::launch<true, false, tc::OUT_F32>(ctx, hp, store)) != ATP_OK) return st;
+                if ((st = tc::launch<true, true, tc::OUT_F32>(ctx, hp, store)) != ATP_OK) return st;
             } else {
-                if ((st = launch_gemm_simt<float, T, float, true>(ctx, g, store)) != ATP_OK) return st;
+                if ((st = launch_gemm_simt<T, float, float, true>(ctx, g, store)) != ATP_OK) return st;
             }
-            if ((st = launch_gemm_simt<float, float, float, false, true>(ctx, gg, store)) != ATP_OK) return st;
-            ATP_KERNEL(ctx, "jac2_init", 0, 0);
-            jac2_init_kernel<<<dim3(64, cnt), 256, 0, ctx->stream>>>(jb);
-            ATP_LAUNCHED(ctx);
+            // Two passes. G squares the condition number of B, so when sigma_1 / sigma_r~ exceeds ~10^3
+            // the first diagonalisation resolves the weak components only roughly. Its rotation W1 is
+            // orthogonal all the same, so (Bt, Y) <- (Bt W1, Y W1) loses nothing; the rotated rows are
+            // graded and nearly orthogonal, their Gram matrix carries errors relative to the row norms,
+            // and a short second pass on it finishes the job (a one-sided Jacobi in two strokes).
             const int npairs = maxnb / 2;
             const int blk = 2 * jbj;
             const size_t ash = (size_t)3 * blk * (blk + 1) * sizeof(float);
             if (jbj == 32) ATP_CUDA_OK(ctx, cudaFuncSetAttribute(jac2_apply_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ash));
-            for (int sw = 0; sw < max_sweeps; ++sw) {
-                for (int step = 0; step < maxnb - 1; ++step) {
-                    ATP_KERNEL(ctx, "jac2_local", 0, 0);
-                    if (jbj == 32) jac2_local_kernel<32><<<dim3(npairs, cnt), 256, 0, ctx->stream>>>(jb, step, tol_rot, jinner);
-                    else jac2_local_kernel<16><<<dim3(npairs, cnt), 128, 0, ctx->stream>>>(jb, step, tol_rot, jinner);
-                    ATP_LAUNCHED(ctx);
-                    ATP_KERNEL(ctx, "jac2_apply", 0, 0);
-                    dim3 ag(npairs + ceil_div(maxrt, blk), npairs, cnt);
-                    if (jbj == 32) jac2_apply_kernel<32><<<ag, 256, ash, ctx->stream>>>(jb, step);
-                    else jac2_apply_kernel<16><<<ag, 128, ash, ctx->stream>>>(jb, step);
+            for (int pass = 0; pass < 2; ++pass) {
+                if ((st = launch_gemm_simt<float, float, float, true, false>(ctx, gg, store)) != ATP_OK) return st;
+                ATP_KERNEL(ctx, "jac2_init", 0, 0);
+                jac2_init_kernel<<<dim3(64, cnt), 256, 0, ctx->stream>>>(jb);
+                ATP_LAUNCHED(ctx);
+                const int nsw = pass == 0 ? max_sweeps : std::min(max_sweeps, 6);
+                for (int sw = 0; sw < nsw; ++sw) {
+                    for (int step = 0; step < maxnb - 1; ++step) {
+                        ATP_KERNEL(ctx, "jac2_local", 0, 0);
+                        if (jbj == 32) jac2_local_kernel<32><<<dim3(npairs, cnt), 256, 0, ctx->stream>>>(jb, step, tol_rot, jinner);
+                        else jac2_local_kernel<16><<<dim3(npairs, cnt), 128, 0, ctx->stream>>>(jb, step, tol_rot, jinner);
+                        ATP_LAUNCHED(ctx);
+                        ATP_KERNEL(ctx, "jac2_apply", 0, 0);
+                        dim3 ag(npairs + ceil_div(maxrt, blk), npairs, cnt);
+                        if (jbj == 32) jac2_apply_kernel<32><<<ag, 256, ash, ctx->stream>>>(jb, step);
+                        else jac2_apply_kernel<16><<<ag, 128, ash, ctx->stream>>>(jb, step);
+                        ATP_LAUNCHED(ctx);
+                    }
+                    ATP_KERNEL(ctx, "jac2_sweep_end", 0, 0);
+                    jac2_sweep_end_kernel<<<1, J2MAX, 0, ctx->stream>>>(jb, tol_conv, pass == 1 && sw == nsw - 1, ctx->dev_status);
                     ATP_LAUNCHED(ctx);
                 }
-                ATP_KERNEL(ctx, "jac2_sweep_end", 0, 0);
-                jac2_sweep_end_kernel<<<1, J2MAX, 0, ctx->stream>>>(jb, tol_conv, sw == max_sweeps - 1, ctx->dev_status);
-                ATP_LAUNCHED(ctx);
+                if (pass == 0) {
+                    GemmBatch r1, r2; r1.count = r2.count = cnt;
+                    for (size_t i = i0; i < i1; ++i) {
+                        SeqPlan &p = bp.seqs[i];
+                        int k = (int)(i - i0);
+                        // Bt2 = Bt Wt^T (d x r~),  Y2 = Y Wt^T (L x r~);  Wt rows are the eigenvectors
+                        r1.p[k] = GemmProblem{p.BW, p.Wt, p.Z, nullptr, p.rt > 0 ? d : 0, p.rt, p.rt, p.rt, p.rt, p.rt, 0};
+                        r2.p[k] = GemmProblem{p.Y, p.Wt, p.Y2, nullptr, p.dims.L, p.rt, p.rt, p.rt, p.rt, p.rt, 0};
+                        gg.p[k].A = p.Z; gg.p[k].B = p.Z;
+                        fb.s[k].Y = p.Y2;
+                    }
+                    if ((st = launch_gemm_simt<float, float, float, false, true>(ctx, r1, store)) != ATP_OK) return st;
+                    if ((st = launch_gemm_simt<float, float, float, false, true>(ctx, r2, store)) != ATP_OK) return st;
+                }
             }
             int npow = 1; while (npow < maxrt) npow <<= 1;
             ATP_KERNEL(ctx, "sigma_sort", 0, 0);
@@ -948,13 +977,13 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
             for (size_t i = i0; i < i1; ++i) {
                 SeqPlan &p = bp.seqs[i];
                 int k = (int)(i - i0);
-                // X_r = Wsel^T B  and  U_r = Y Wsel
-                g.p[k] = GemmProblem{p.Wsel, p.BW, (T *)X_r->data + (size_t)p.dims.rank0 * X_r->ld, nullptr,
-                                     p.dims.r, p.rt > 0 ? d : 0, p.rt, p.dims.r, d, (int)X_r->ld, 0};
-                gg.p[k] = GemmProblem{p.Y, p.Wsel, (T *)U_r->data + (size_t)p.dims.row0 * U_r->ld, nullptr,
+                // X_r = Wsel^T Bt2^T  and  U_r = Y2 Wsel  (Bt2, Y2: rotated by the first pass)
+                g.p[k] = GemmProblem{p.Wsel, p.Z, (T *)X_r->data + (size_t)p.dims.rank0 * X_r->ld, nullptr,
+                                     p.dims.r, p.rt > 0 ? d : 0, p.rt, p.dims.r, p.rt, (int)X_r->ld, 0};
+                gg.p[k] = GemmProblem{p.Y2, p.Wsel, (T *)U_r->data + (size_t)p.dims.row0 * U_r->ld, nullptr,
                                       p.dims.L, p.dims.r, p.rt, p.rt, p.dims.r, (int)U_r->ld, 0};
             }
-            if ((st = launch_gemm_simt<float, float, T, true>(ctx, g, store)) != ATP_OK) return st;
+            if ((st = launch_gemm_simt<float, float, T, true, true>(ctx, g, store)) != ATP_OK) return st;
             if ((st = launch_gemm_simt<float, float, T, false>(ctx, gg, store)) != ATP_OK) return st;
             ATP_KERNEL(ctx, "signfix", 0, 0);
             signfix_kernel<T><<<dim3(maxr, cnt), 256, 0, ctx->stream>>>(fb);
