@@ -757,7 +757,7 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
     }
     const float tol_conv = (X->dtype == ATP_F32) ? 1e-6f : 3e-5f;
     const float tol_rot = tol_conv * 0.25f;
-    const bool two_sided = (X->dtype == ATP_BF16);    // fp32 inputs keep the one-sided rotation of B itself
+    const bool two_sided = (X->dtype == ATP_BF16) && jbj != 1;    // fp32 inputs keep the one-sided rotation of B itself
     GemmEpi store{EPI_STORE, nullptr};
 
     for (size_t i0 = 0; i0 < bp.seqs.size(); i0 += BMAX) {
@@ -1006,7 +1006,7 @@ extern "C" atp_status atp_principal_basis(atp_ctx *ctx, const atp_mat *X, const 
         if (opts->power_iters >= 0) power_iters = opts->power_iters;
         if (opts->max_sweeps > 0) max_sweeps = opts->max_sweeps;
         seed ^= opts->seed * 0x9E3779B97F4A7C15ull;
-        if (opts->jacobi_block == 16 || opts->jacobi_block == 32) jbj = opts->jacobi_block;
+        if (opts->jacobi_block == 16 || opts->jacobi_block == 32 || opts->jacobi_block == 1) jbj = opts->jacobi_block;
         else if (opts->jacobi_block != 0) return ATP_ERR_INVALID_ARG;
         if (opts->jacobi_inner > 0) jinner = opts->jacobi_inner;
     }

@@ -44,6 +44,7 @@ def basis_invariants(X, U, Xr, sig):
     out["opt"] = opt
     out["res_sub"] = res_sub
     out["res_ratio"] = res_sub / opt if opt > 1e-12 * s_true[0] else 1.0 + res_sub / s_true[0]
+    out["normX"] = float(np.linalg.norm(X))
     out["res_pair"] = float(np.linalg.norm(X - U @ Xr))
     G = Xr @ Xr.T
     dg = np.sqrt(np.maximum(np.diag(G), 0))
@@ -58,3 +59,11 @@ def basis_invariants(X, U, Xr, sig):
     out["sigma_rel"] = np.abs(sig - s_true[:r]) / s_true[0]
     out["s_true"] = s_true
     return out
+
+
+def residual_ok(res_sub, opt, norm_x, dtype, tol):
+    """Subspace residual against the Eckart-Young optimum. The range finder reaches (1 + tol) * opt;
+    a basis stored in bf16 additionally tilts every direction by its entry rounding (relative
+    2^-9), which costs up to (2^-9 |X|_F)^2 of captured energy whatever the algorithm."""
+    eps = 2.0 ** -9 if dtype == "bf16" else 2.0 ** -22
+    return res_sub ** 2 <= ((1.0 + tol) * opt) ** 2 + (eps * norm_x) ** 2
