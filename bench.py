@@ -92,6 +92,16 @@ class ClockSampler:
         return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def workload_config(w, world):
+    ranks = w.ranks
+    return {"workload": w.name, "batch": len(w.lengths), "tokens_per_step_per_gpu": w.tokens, "d": w.d,
+            "heads": w.heads, "rank": ranks[0] if len(set(ranks)) == 1 else "L_b/4",
+            "ffn": w.ffn, "d_ff": w.d_ff, "input_norm": w.input_norm,
+            "layer": "basis+attention" + ("+W_O" if "W_O" in w.weights else "") + ("+FFN" if w.ffn else ""),
+            "l2": "flushed between steps (256 MiB memset), rotating input copies",
+            "parallelism": f"dp{world} (independent sequences per rank)"}
+
+
 def oracle_step(w, seq_index):
     import oracle
     s = w.seqs[seq_index]
@@ -120,7 +130,7 @@ def run_reference(args):
     line = {"impl": "reference", "metric": "ATP layer prefill tokens/sec", "value": val, "unit": "tokens/s",
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": w.name, "sequences_per_step": 1, "heads": w.heads, "d": w.d, "rank": w.ranks[0]},
+            "config": dict(workload_config(w, args.gpus), sample="one sequence of the batch per step"),
             "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -261,22 +271,23 @@ def main():
     prof = ctx.profile_stop()
     total_ms = sum(v["ms"] for v in prof.values()) or 1.0
     dom_name, dom = max(prof.items(), key=lambda kv: kv[1]["ms"])
-    per_launch_s = dom["ms"] / 1e3 / max(dom["launches"], 1)
-    ridge = pk["bf16_tflops"] * 1e12 / (pk["hbm_gbs"] * 1e9)
-    if dom_name.endswith("_simt") or dom_name.startswith("jacobi"):
-        bound, peak, unit = "alu", FP32_ALU_TFLOPS, "TFLOP/s"
-        achieved = dom["flops"] / max(dom["launches"], 1) / per_launch_s / 1e12
-    elif dom["flops"] > 0 and dom["flops"] / max(dom["bytes"], 1.0) > ridge:
-        bound, peak, unit = "tensor", pk["bf16_tflops"], "TFLOP/s"
-        achieved = dom["flops"] / max(dom["launches"], 1) / per_launch_s / 1e12
-    else:
-        bound, peak, unit = "hbm", pk["hbm_gbs"], "GB/s"
-        achieved = dom["bytes"] / max(dom["launches"], 1) / per_launch_s / 1e9
+    def rate(name, rec):
+        per_launch_s = rec["ms"] / 1e3 / max(rec["launches"], 1)
+        fl, by = rec["flops"] / max(rec["launches"], 1), rec["bytes"] / max(rec["launches"], 1)
+        if name.endswith("_tc") or name.endswith("_tc_split"):
+            return "tensor", fl / per_launch_s / 1e12, pk["bf16_tflops"], "TFLOP/s"
+        if fl > 0:
+            return "alu", fl / per_launch_s / 1e12, FP32_ALU_TFLOPS, "TFLOP/s"
+        return "hbm", by / per_launch_s / 1e9, pk["hbm_gbs"], "GB/s"
+
+    bound, achieved, peak, unit = rate(dom_name, dom)
     roofline = {"kernel": dom_name, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
                 "frac": achieved / peak, "traffic": None, "peak_source": pk["source"],
                 "share_of_step": dom["ms"] / total_ms,
                 "kernels": {k: {"launches": v["launches"] // nprof, "ms_per_step": v["ms"] / nprof,
-                                "share": v["ms"] / total_ms} for k, v in sorted(prof.items(), key=lambda kv: -kv[1]["ms"])}}
+                                "share": v["ms"] / total_ms, "bound": rate(k, v)[0], "achieved": rate(k, v)[1],
+                                "frac": rate(k, v)[1] / rate(k, v)[2], "unit": rate(k, v)[3]}
+                            for k, v in sorted(prof.items(), key=lambda kv: -kv[1]["ms"])}}
 
     # ---- CPU baseline: the oracle on a bounded sample of the same workload
     cpu = None
@@ -296,12 +307,7 @@ def main():
     line = {"metric": "ATP layer prefill tokens/sec", "value": value, "unit": "tokens/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
-            "config": {"workload": w.name, "batch": len(lengths), "tokens_per_step_per_gpu": tokens, "d": w.d,
-                       "heads": w.heads, "rank": ranks[0] if len(set(ranks)) == 1 else "L_b/4",
-                       "ffn": w.ffn, "d_ff": w.d_ff, "input_norm": w.input_norm,
-                       "layer": "basis+attention" + ("+W_O" if "W_O" in w.weights else "") + ("+FFN" if w.ffn else ""),
-                       "l2": "flushed between steps (256 MiB memset), %d rotating input copies" % nsets,
-                       "parallelism": f"dp{world} (independent sequences per rank)"},
+            "config": workload_config(w, world),
             "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)
     if world > 1:

@@ -935,11 +935,14 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
                 const int nsw = pass == 0 ? max_sweeps : std::min(max_sweeps, 6);
                 for (int sw = 0; sw < nsw; ++sw) {
                     for (int step = 0; step < maxnb - 1; ++step) {
-                        ATP_KERNEL(ctx, "jac2_local", 0, 0);
+                        // algorithmic work of a step when every pair rotates (converged pairs skip it)
+                        const double nseq = cnt, bl = blk;
+                        ATP_KERNEL(ctx, "jac2_local", nseq * npairs * jinner * (bl - 1) * (bl * bl * 6.0 + bl * bl * 3.0), 0);
                         if (jbj == 32) jac2_local_kernel<32><<<dim3(npairs, cnt), 256, 0, ctx->stream>>>(jb, step, tol_rot, jinner);
                         else jac2_local_kernel<16><<<dim3(npairs, cnt), 128, 0, ctx->stream>>>(jb, step, tol_rot, jinner);
                         ATP_LAUNCHED(ctx);
-                        ATP_KERNEL(ctx, "jac2_apply", 0, 0);
+                        ATP_KERNEL(ctx, "jac2_apply", nseq * npairs * (npairs * 4.0 + ceil_div(maxrt, blk) * 2.0) * bl * bl * bl,
+                                   nseq * npairs * (npairs * 2.0 + ceil_div(maxrt, blk) * 2.0) * bl * bl * 4.0);
                         dim3 ag(npairs + ceil_div(maxrt, blk), npairs, cnt);
                         if (jbj == 32) jac2_apply_kernel<32><<<ag, 256, ash, ctx->stream>>>(jb, step);
                         else jac2_apply_kernel<16><<<ag, 128, ash, ctx->stream>>>(jb, step);
