@@ -92,7 +92,7 @@ typedef struct {
     uint32_t struct_size;
     int32_t oversample;    /* extra columns of the range finder; < 0: default 64              */
     int32_t power_iters;   /* subspace (power) iterations;        < 0: default 2              */
-    int32_t max_sweeps;    /* Jacobi sweep limit;                 <= 0: default 16            */
+    int32_t max_sweeps;    /* Jacobi sweep limit;                 <= 0: default 12            */
     uint64_t seed;         /* seed of the +-1 test matrix                                      */
     int32_t jacobi_block;  /* tuning: rows per Jacobi block, 16 or 32; 0: default 16 (bf16 path only)  */
     int32_t jacobi_inner;  /* tuning: on-chip sweeps per block visit;   <= 0: default 1                */

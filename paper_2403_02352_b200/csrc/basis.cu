@@ -925,14 +925,14 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
             // and a short second pass on it finishes the job (a one-sided Jacobi in two strokes).
             const int npairs = maxnb / 2;
             const int blk = 2 * jbj;
-            const size_t ash = (size_t)3 * blk * (blk + 1) * sizeof(float);
+            const size_t ash = jbj == 32 ? JAC2_APPLY_SMEM(64) : JAC2_APPLY_SMEM(32);
             if (jbj == 32) ATP_CUDA_OK(ctx, cudaFuncSetAttribute(jac2_apply_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ash));
             for (int pass = 0; pass < 2; ++pass) {
                 if ((st = launch_gemm_simt<float, float, float, true, false>(ctx, gg, store)) != ATP_OK) return st;
                 ATP_KERNEL(ctx, "jac2_init", 0, 0);
                 jac2_init_kernel<<<dim3(64, cnt), 256, 0, ctx->stream>>>(jb);
                 ATP_LAUNCHED(ctx);
-                const int nsw = pass == 0 ? max_sweeps : std::min(max_sweeps, 6);
+                const int nsw = pass == 0 ? max_sweeps : std::min(max_sweeps, 4);
                 for (int sw = 0; sw < nsw; ++sw) {
                     for (int step = 0; step < maxnb - 1; ++step) {
                         // algorithmic work of a step when every pair rotates (converged pairs skip it)
@@ -1002,7 +1002,7 @@ extern "C" atp_status atp_principal_basis(atp_ctx *ctx, const atp_mat *X, const 
     if (!ctx) return ATP_ERR_INVALID_ARG;
     atp_status st;
     if ((st = check_mat(X)) != ATP_OK || (st = check_mat(U_r)) != ATP_OK || (st = check_mat(X_r)) != ATP_OK) return st;
-    int oversample = 64, power_iters = 2, max_sweeps = 16, jbj = 16, jinner = 1; uint64_t seed = 0x243F6A8885A308D3ull;
+    int oversample = 64, power_iters = 2, max_sweeps = 12, jbj = 16, jinner = 1; uint64_t seed = 0x243F6A8885A308D3ull;
     if (opts) {
         if (opts->struct_size < sizeof(atp_basis_opts)) return ATP_ERR_INVALID_ARG;
         if (opts->oversample >= 0) oversample = opts->oversample;

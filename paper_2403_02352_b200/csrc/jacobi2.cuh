@@ -59,7 +59,13 @@ jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_r
     __shared__ int pp[HP], qq[HP];
     __shared__ float red[NT / 32];
     __shared__ int rotated;
+    __shared__ unsigned char sp[BLK - 1][HP], sqq[BLK - 1][HP];      // round-robin schedule of the local sweep
     const int tid = threadIdx.x;
+    for (int e = tid; e < (BLK - 1) * HP; e += NT) {
+        int p_, q_;
+        rr_pair2(BLK, e / HP, e % HP, p_, q_);
+        sp[e / HP][e % HP] = (unsigned char)p_; sqq[e / HP][e % HP] = (unsigned char)q_;
+    }
     for (int e = tid; e < BLK * BLK; e += NT) {
         int i = e / BLK, j = e % BLK;
         int gi = jac2_row<BJ2>(I, J, i, sq.rt), gj = jac2_row<BJ2>(I, J, j, sq.rt);
@@ -92,8 +98,7 @@ jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_r
         __syncthreads();
         for (int st = 0; st < BLK - 1; ++st) {
             if (tid < HP) {
-                int p, q;
-                rr_pair2(BLK, st, tid, p, q);
+                const int p = sp[st][tid], q = sqq[st][tid];
                 float gpp = A[p][p], gqq = A[q][q], gpq = A[p][q];
                 float c = 1.f, s = 0.f;
                 if (gpq != 0.f && fabsf(gpq) > tol_rot * sqrtf(fmaxf(gpp, 0.f) * fmaxf(gqq, 0.f))) {
@@ -138,79 +143,107 @@ jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_r
     if (tid == 0) sq.vflag[pair] = 1;
 }
 
-// grid: (npairs + ceil(rt/BLK), npairs, batch); dynamic shared memory: 3 * BLK * (BLK + 1) floats
+// grid: (npairs + ceil(rt/BLK), npairs, batch); dynamic shared memory: JAC2_APPLY_SMEM(BLK) bytes.
+// G is symmetric: only blocks (p, q) with q >= p are computed, the mirror block is written from the
+// transposed result. Each thread owns an MR x 4 register tile of the BLK x BLK block.
+#define JAC2_APPLY_SMEM(BLK) ((size_t)(2 * (BLK) * ((BLK) + 1) + 2 * (BLK) * ((BLK) + 4)) * sizeof(float))
 template <int BJ2>
 __global__ void __launch_bounds__(BJ2 * 8)
 jac2_apply_kernel(const __grid_constant__ Jac2Batch batch, int step)
 {
-    constexpr int BLK = 2 * BJ2, NT = BLK * 4, CPT = BLK / 4, LD = BLK + 1;
+    constexpr int BLK = 2 * BJ2, NT = BLK * 4, MR = BLK / 16, LD = BLK + 1, LD4 = BLK + 4;
     const Jac2Seq &sq = batch.s[blockIdx.z];
     if (*sq.conv) return;
     const int npairs = sq.nb / 2;
     const int p = blockIdx.y;
     if (p >= npairs) return;
-    const int tid = threadIdx.x;
-    extern __shared__ float j2sm[];
-    float *Vp = j2sm, *Vq = j2sm + BLK * LD, *Bk = j2sm + 2 * BLK * LD;
-    int Ip, Jp;
-    rr_pair2(sq.nb, step % (sq.nb - 1), p, Ip, Jp);
+    const bool gblock = (int)blockIdx.x < npairs;
+    const int q = blockIdx.x;
+    if (gblock && q < p) return;
     const int fp = sq.vflag[p];
-    const int row = tid >> 2, c0 = (tid & 3) * CPT;
-    float t[CPT];
-#pragma unroll
-    for (int j = 0; j < CPT; ++j) t[j] = 0.f;
-    if ((int)blockIdx.x < npairs) {
-        const int q = blockIdx.x;
-        const int fq = sq.vflag[q];
-        if (!fp && !fq) return;
-        int Iq, Jq;
-        rr_pair2(sq.nb, step % (sq.nb - 1), q, Iq, Jq);
-        for (int e = tid; e < BLK * BLK; e += NT) {
-            int i = e / BLK, j = e % BLK;
-            Vp[i * LD + j] = fp ? sq.Vbuf[(size_t)p * BLK * BLK + e] : (i == j ? 1.f : 0.f);
-            Vq[i * LD + j] = fq ? sq.Vbuf[(size_t)q * BLK * BLK + e] : (i == j ? 1.f : 0.f);
-            int gi = jac2_row<BJ2>(Ip, Jp, i, sq.rt), gj = jac2_row<BJ2>(Iq, Jq, j, sq.rt);
-            Bk[i * LD + j] = (gi >= 0 && gj >= 0) ? sq.G[(size_t)gi * sq.rt + gj] : 0.f;
+    const int fq = gblock ? sq.vflag[q] : 0;
+    if (gblock ? (!fp && !fq) : !fp) return;
+    const int tid = threadIdx.x;
+    extern __shared__ __align__(16) float j2sm[];
+    float *Vp = j2sm;                       // [BLK][LD]   Vp[r][k]
+    float *Tm = Vp + BLK * LD;              // [BLK][LD]   T[r][k]
+    float *Bk = Tm + BLK * LD;              // [BLK][LD4]  B[k][c]
+    float *VqT = Bk + BLK * LD4;            // [BLK][LD4]  Vq^T[k][c] = Vq[c][k]
+    int Ip, Jp, Iq = 0, Jq = 0;
+    rr_pair2(sq.nb, step % (sq.nb - 1), p, Ip, Jp);
+    const int r0 = (tid / (BLK / 4)) * MR, c0 = (tid % (BLK / 4)) * 4;
+    const int cb = gblock ? 0 : ((int)blockIdx.x - npairs) * BLK;
+    if (!gblock && cb >= sq.rt) return;
+    if (gblock) rr_pair2(sq.nb, step % (sq.nb - 1), q, Iq, Jq);
+    for (int e = tid; e < BLK * BLK; e += NT) {
+        int i = e / BLK, j = e % BLK;
+        Vp[i * LD + j] = fp ? sq.Vbuf[(size_t)p * BLK * BLK + e] : (i == j ? 1.f : 0.f);
+        int gi = jac2_row<BJ2>(Ip, Jp, i, sq.rt);
+        if (gblock) {
+            VqT[j * LD4 + i] = fq ? sq.Vbuf[(size_t)q * BLK * BLK + e] : (i == j ? 1.f : 0.f);
+            int gj = jac2_row<BJ2>(Iq, Jq, j, sq.rt);
+            Bk[i * LD4 + j] = (gi >= 0 && gj >= 0) ? sq.G[(size_t)gi * sq.rt + gj] : 0.f;
+        } else {
+            Bk[i * LD4 + j] = (gi >= 0 && cb + j < sq.rt) ? sq.Wt[(size_t)gi * sq.rt + cb + j] : 0.f;
         }
-        __syncthreads();
-        for (int k = 0; k < BLK; ++k) {
-            float a = Vp[row * LD + k];
+    }
+    __syncthreads();
+    float acc[MR][4];
 #pragma unroll
-            for (int j = 0; j < CPT; ++j) t[j] = fmaf(a, Bk[k * LD + c0 + j], t[j]);
+    for (int i = 0; i < MR; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+#pragma unroll 8
+    for (int k = 0; k < BLK; ++k) {
+        const float4 b = *(const float4 *)&Bk[k * LD4 + c0];
+#pragma unroll
+        for (int i = 0; i < MR; ++i) {
+            const float a = Vp[(r0 + i) * LD + k];
+            acc[i][0] = fmaf(a, b.x, acc[i][0]); acc[i][1] = fmaf(a, b.y, acc[i][1]);
+            acc[i][2] = fmaf(a, b.z, acc[i][2]); acc[i][3] = fmaf(a, b.w, acc[i][3]);
         }
-        __syncthreads();                       // everyone is done reading Bk: reuse it for T = Vp Bk
+    }
+    if (!gblock) {                          // rows of Wt: Vt_p * Wt
 #pragma unroll
-        for (int j = 0; j < CPT; ++j) Bk[row * LD + c0 + j] = t[j];
-        __syncthreads();
-        const int gi = jac2_row<BJ2>(Ip, Jp, row, sq.rt);
+        for (int i = 0; i < MR; ++i) {
+            const int gi = jac2_row<BJ2>(Ip, Jp, r0 + i, sq.rt);
+            if (gi < 0) continue;
 #pragma unroll
-        for (int j = 0; j < CPT; ++j) {
-            float o = 0.f;
-            for (int k = 0; k < BLK; ++k) o = fmaf(Bk[row * LD + k], Vq[(c0 + j) * LD + k], o);     // (T Vq^T)[row][c0+j]
-            int gj = jac2_row<BJ2>(Iq, Jq, c0 + j, sq.rt);
-            if (gi >= 0 && gj >= 0) sq.G[(size_t)gi * sq.rt + gj] = o;
+            for (int j = 0; j < 4; ++j)
+                if (cb + c0 + j < sq.rt) sq.Wt[(size_t)gi * sq.rt + cb + c0 + j] = acc[i][j];
         }
-    } else {
-        if (!fp) return;
-        const int cb = ((int)blockIdx.x - npairs) * BLK;
-        if (cb >= sq.rt) return;
-        for (int e = tid; e < BLK * BLK; e += NT) {
-            int i = e / BLK, j = e % BLK;
-            Vp[i * LD + j] = sq.Vbuf[(size_t)p * BLK * BLK + e];
-            int gi = jac2_row<BJ2>(Ip, Jp, i, sq.rt);
-            Bk[i * LD + j] = (gi >= 0 && cb + j < sq.rt) ? sq.Wt[(size_t)gi * sq.rt + cb + j] : 0.f;
-        }
-        __syncthreads();
-        for (int k = 0; k < BLK; ++k) {
-            float a = Vp[row * LD + k];
+        return;
+    }
 #pragma unroll
-            for (int j = 0; j < CPT; ++j) t[j] = fmaf(a, Bk[k * LD + c0 + j], t[j]);
-        }
-        const int gi = jac2_row<BJ2>(Ip, Jp, row, sq.rt);
-        if (gi >= 0)
+    for (int i = 0; i < MR; ++i)
 #pragma unroll
-            for (int j = 0; j < CPT; ++j)
-                if (cb + c0 + j < sq.rt) sq.Wt[(size_t)gi * sq.rt + cb + c0 + j] = t[j];
+        for (int j = 0; j < 4; ++j) Tm[(r0 + i) * LD + c0 + j] = acc[i][j];
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < MR; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+#pragma unroll 8
+    for (int k = 0; k < BLK; ++k) {         // Out = T * Vq^T
+        const float4 b = *(const float4 *)&VqT[k * LD4 + c0];
+#pragma unroll
+        for (int i = 0; i < MR; ++i) {
+            const float a = Tm[(r0 + i) * LD + k];
+            acc[i][0] = fmaf(a, b.x, acc[i][0]); acc[i][1] = fmaf(a, b.y, acc[i][1]);
+            acc[i][2] = fmaf(a, b.z, acc[i][2]); acc[i][3] = fmaf(a, b.w, acc[i][3]);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < MR; ++i) {
+        const int gi = jac2_row<BJ2>(Ip, Jp, r0 + i, sq.rt);
+        if (gi < 0) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int gj = jac2_row<BJ2>(Iq, Jq, c0 + j, sq.rt);
+            if (gj < 0) continue;
+            sq.G[(size_t)gi * sq.rt + gj] = acc[i][j];
+            if (q != p) sq.G[(size_t)gj * sq.rt + gi] = acc[i][j];
+        }
     }
 }
 
