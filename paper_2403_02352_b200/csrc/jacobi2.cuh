@@ -101,10 +101,13 @@ jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_r
                 const int p = sp[st][tid], q = sqq[st][tid];
                 float gpp = A[p][p], gqq = A[q][q], gpq = A[p][q];
                 float c = 1.f, s = 0.f;
-                if (gpq != 0.f && fabsf(gpq) > tol_rot * sqrtf(fmaxf(gpp, 0.f) * fmaxf(gqq, 0.f))) {
-                    float zeta = (gqq - gpp) / (2.f * gpq);
-                    float t = copysignf(1.f, zeta) / (fabsf(zeta) + sqrtf(1.f + zeta * zeta));
-                    c = 1.f / sqrtf(1.f + t * t);
+                // fast reciprocal / rsqrt: c^2 + s^2 = 1 to ~2 ulp, ample for a basis stored in bf16
+                if (gpq != 0.f && gpq * gpq > tol_rot * tol_rot * fmaxf(gpp, 0.f) * fmaxf(gqq, 0.f)) {
+                    float zeta = __fdividef(gqq - gpp, 2.f * gpq);
+                    float az = fabsf(zeta), t;
+                    if (az > 1e15f) t = __fdividef(0.5f, zeta);
+                    else { float h = 1.f + zeta * zeta; t = __fdividef(copysignf(1.f, zeta), az + h * rsqrtf(h)); }
+                    c = rsqrtf(1.f + t * t);
                     s = c * t;
                     rotated = 1;
                 }
