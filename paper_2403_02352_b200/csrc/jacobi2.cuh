@@ -40,12 +40,15 @@ __global__ void jac2_init_kernel(const __grid_constant__ Jac2Batch batch)
     if (blockIdx.x == 0 && threadIdx.x == 0) { *sq.maxoff = 0u; *sq.conv = 0; }
 }
 
-// BJ2: block height (16 or 32); the local problem is BLK x BLK with BLK = 2 BJ2, solved by 4 BLK threads.
+// BJ2: block height (16 or 32); the local problem is BLK x BLK with BLK = 2 BJ2, solved by 16 BLK threads.
+// The sweep is a chain of BLK - 1 dependent rotation steps, so the time of a step is the length of one
+// thread's instruction chain: every thread updates at most one 2x2 block of A and a few pairs of V.
 template <int BJ2>
-__global__ void __launch_bounds__(BJ2 * 8)
+__global__ void __launch_bounds__(BJ2 * 32)
 jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_rot, int max_inner)
 {
-    constexpr int BLK = 2 * BJ2, NT = BLK * 4, HP = BLK / 2;
+    constexpr int BLK = 2 * BJ2, NT = BLK * 16, HP = BLK / 2;
+    constexpr int VPT = HP * BLK / NT;                 // V pair-elements per thread (1 or 2)
     const Jac2Seq &sq = batch.s[blockIdx.y];
     if (*sq.conv) return;
     const int npairs = sq.nb / 2;
@@ -55,16 +58,16 @@ jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_r
     rr_pair2(sq.nb, step % (sq.nb - 1), pair, I, J);
     __shared__ float A[BLK][BLK + 1];
     __shared__ float V[BLK][BLK + 1];
-    __shared__ float cs[HP], sn[HP];
-    __shared__ int pp[HP], qq[HP];
+    __shared__ float2 cs[HP];
+    __shared__ uchar2 pq[HP];
     __shared__ float red[NT / 32];
     __shared__ int rotated;
-    __shared__ unsigned char sp[BLK - 1][HP], sqq[BLK - 1][HP];      // round-robin schedule of the local sweep
+    __shared__ uchar2 sched[BLK - 1][HP];              // round-robin schedule of the local sweep
     const int tid = threadIdx.x;
     for (int e = tid; e < (BLK - 1) * HP; e += NT) {
         int p_, q_;
         rr_pair2(BLK, e / HP, e % HP, p_, q_);
-        sp[e / HP][e % HP] = (unsigned char)p_; sqq[e / HP][e % HP] = (unsigned char)q_;
+        sched[e / HP][e % HP] = make_uchar2((unsigned char)p_, (unsigned char)q_);
     }
     for (int e = tid; e < BLK * BLK; e += NT) {
         int i = e / BLK, j = e % BLK;
@@ -93,12 +96,15 @@ jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_r
         if (tid == 0) sq.vflag[pair] = 0;
         return;
     }
+    const bool has_block = tid < HP * HP;
+    const int ba = tid / HP, bb = tid % HP;            // 2x2 block (pair ba rows, pair bb columns)
     for (int sweep = 0; sweep < max_inner; ++sweep) {
         if (tid == 0) rotated = 0;
         __syncthreads();
         for (int st = 0; st < BLK - 1; ++st) {
             if (tid < HP) {
-                const int p = sp[st][tid], q = sqq[st][tid];
+                const uchar2 pr_ = sched[st][tid];
+                const int p = pr_.x, q = pr_.y;
                 float gpp = A[p][p], gqq = A[q][q], gpq = A[p][q];
                 float c = 1.f, s = 0.f;
                 // fast reciprocal / rsqrt: c^2 + s^2 = 1 to ~2 ulp, ample for a basis stored in bf16
@@ -111,30 +117,35 @@ jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_r
                     s = c * t;
                     rotated = 1;
                 }
-                cs[tid] = c; sn[tid] = s; pp[tid] = p; qq[tid] = q;
+                cs[tid] = make_float2(c, s);
+                pq[tid] = pr_;
             }
             __syncthreads();
+            // loads of this step first (independent), then the arithmetic, then the stores
+            float g00 = 0.f, g01 = 0.f, g10 = 0.f, g11 = 0.f;
+            uchar2 ra = make_uchar2(0, 0), rb = make_uchar2(0, 0);
+            float2 ca = make_float2(1.f, 0.f), cb = ca;
+            if (has_block) {
+                ra = pq[ba]; rb = pq[bb]; ca = cs[ba]; cb = cs[bb];
+                g00 = A[ra.x][rb.x]; g01 = A[ra.x][rb.y]; g10 = A[ra.y][rb.x]; g11 = A[ra.y][rb.y];
+            }
+            float vx[VPT], vy[VPT]; uchar2 rv[VPT]; float2 cv[VPT]; int vc[VPT];
 #pragma unroll
-            for (int it = 0; it < HP * HP / NT; ++it) {
-                int idx = tid + it * NT;
-                int a = idx / HP, b = idx % HP;
-                int pa = pp[a], qa = qq[a], pb = pp[b], qb = qq[b];
-                float ca = cs[a], sa = sn[a], cb = cs[b], sb = sn[b];
-                float g00 = A[pa][pb], g01 = A[pa][qb], g10 = A[qa][pb], g11 = A[qa][qb];
-                float r00 = ca * g00 - sa * g10, r01 = ca * g01 - sa * g11;
-                float r10 = sa * g00 + ca * g10, r11 = sa * g01 + ca * g11;
-                A[pa][pb] = cb * r00 - sb * r01; A[pa][qb] = sb * r00 + cb * r01;
-                A[qa][pb] = cb * r10 - sb * r11; A[qa][qb] = sb * r10 + cb * r11;
+            for (int it = 0; it < VPT; ++it) {
+                const int idx = tid + it * NT;
+                rv[it] = pq[idx / BLK]; cv[it] = cs[idx / BLK]; vc[it] = idx % BLK;
+                vx[it] = V[rv[it].x][vc[it]]; vy[it] = V[rv[it].y][vc[it]];
+            }
+            if (has_block) {
+                float r00 = ca.x * g00 - ca.y * g10, r01 = ca.x * g01 - ca.y * g11;
+                float r10 = ca.y * g00 + ca.x * g10, r11 = ca.y * g01 + ca.x * g11;
+                A[ra.x][rb.x] = cb.x * r00 - cb.y * r01; A[ra.x][rb.y] = cb.y * r00 + cb.x * r01;
+                A[ra.y][rb.x] = cb.x * r10 - cb.y * r11; A[ra.y][rb.y] = cb.y * r10 + cb.x * r11;
             }
 #pragma unroll
-            for (int it = 0; it < HP * BLK / NT; ++it) {
-                int idx = tid + it * NT;
-                int a = idx / BLK, col = idx % BLK;
-                int pa = pp[a], qa = qq[a];
-                float ca = cs[a], sa = sn[a];
-                float x = V[pa][col], y = V[qa][col];
-                V[pa][col] = ca * x - sa * y;
-                V[qa][col] = sa * x + ca * y;
+            for (int it = 0; it < VPT; ++it) {
+                V[rv[it].x][vc[it]] = cv[it].x * vx[it] - cv[it].y * vy[it];
+                V[rv[it].y][vc[it]] = cv[it].y * vx[it] + cv[it].x * vy[it];
             }
             __syncthreads();
         }
