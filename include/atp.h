@@ -18,8 +18,9 @@
  *     over with atp_set_workspace(); its required size comes from atp_workspace_bytes().
  *     atp_create() allocates one small device status word and a pinned staging page, freed by
  *     atp_destroy().
- *   - Calls only enqueue work on the context's stream (atp_set_stream) and return; they never
- *     synchronise, except atp_poll_device_status().
+ *   - Calls only enqueue work and return; they never synchronise, except atp_poll_device_status().
+ *     Work is ordered on the context's stream (atp_set_stream); atp_principal_basis can fork part of
+ *     a batch onto two internal streams (opts->groups) and joins them back before it returns.
  *   - Errors the host can detect are returned at once and nothing is launched. Conditions only
  *     the device can see (a Jacobi iteration that hit its sweep limit, a bounded wait that ran
  *     out, a value outside the representable range) are recorded in the status word and read
@@ -96,6 +97,8 @@ typedef struct {
     uint64_t seed;         /* seed of the +-1 test matrix                                      */
     int32_t jacobi_block;  /* tuning: rows per Jacobi block, 16 or 32; 0: default 16 (bf16 path only)  */
     int32_t jacobi_inner;  /* tuning: on-chip sweeps per block visit;   <= 0: default 1                */
+    int32_t groups;        /* tuning: 0 / 1 = run the whole batch on the caller's stream; 2 = split the */
+                           /* batch in two groups on internal streams (forked from and joined to it)   */
 } atp_basis_opts;
 
 typedef struct {

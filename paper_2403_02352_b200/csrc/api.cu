@@ -58,6 +58,11 @@ atp_status atp_create(atp_ctx **out, int device)
     ctx->sm_count = prop.multiProcessorCount;
     if (cudaMalloc(&ctx->dev_status, sizeof(int)) != cudaSuccess) { delete ctx; return ATP_ERR_CUDA; }
     if (cudaMemset(ctx->dev_status, 0, sizeof(int)) != cudaSuccess) { cudaFree(ctx->dev_status); delete ctx; return ATP_ERR_CUDA; }
+    bool ok = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; i < 2 && ok; ++i)
+        ok = cudaStreamCreateWithFlags(&ctx->aux[i], cudaStreamNonBlocking) == cudaSuccess &&
+             cudaEventCreateWithFlags(&ctx->ev_join[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) { atp_destroy(ctx); return ATP_ERR_CUDA; }
     *out = ctx;
     return ATP_OK;
 }
@@ -67,6 +72,11 @@ atp_status atp_destroy(atp_ctx *ctx)
     if (!ctx) return ATP_ERR_INVALID_ARG;
     cudaSetDevice(ctx->device);
     if (ctx->dev_status) cudaFree(ctx->dev_status);
+    for (int i = 0; i < 2; ++i) {
+        if (ctx->aux[i]) cudaStreamDestroy(ctx->aux[i]);
+        if (ctx->ev_join[i]) cudaEventDestroy(ctx->ev_join[i]);
+    }
+    if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
     delete ctx;
     return ATP_OK;
 }

@@ -633,7 +633,7 @@ struct SeqPlan {
     __nv_bfloat16 *Yb, *Yl, *Zb, *Zl; float *Y2; float *Y, *Z, *BW, *Wsel, *tsum, *sig, *Cc, *rinv, *G, *Wt, *Vbuf; double *gpart; int *ord, *flags, *conv, *vflag, *needfix; unsigned *maxoff;
 };
 struct BasisPlan {
-    std::vector<SeqPlan> seqs; float *omega; __nv_bfloat16 *omega_b; float *part; size_t part_stride; int rtmax; int splits;
+    std::vector<SeqPlan> seqs; float *omega; __nv_bfloat16 *omega_b; float *part; size_t part_stride, part_group; int group = 0; int rtmax; int splits;
 };
 
 static int pick_splits(int K) { int s = K / 1024; return s < 1 ? 1 : (s > 16 ? 16 : s); }
@@ -682,7 +682,8 @@ static void plan_basis(Arena &ar, const std::vector<SeqDims> &sd, int d, int ove
         maxpart = std::max(maxpart, (size_t)rt * PB);
     }
     bp.part_stride = maxpart;
-    bp.part = ar.take<float>((size_t)bp.splits * std::min<size_t>(bp.seqs.size(), BMAX) * maxpart);
+    bp.part_group = (size_t)bp.splits * std::min<size_t>(bp.seqs.size(), BMAX) * maxpart;
+    bp.part = ar.take<float>(2 * bp.part_group);        // one region per concurrent group
 }
 
 size_t basis_workspace_bytes(const std::vector<SeqDims> &sd, int d, int oversample)
@@ -720,8 +721,8 @@ static atp_status orthonormalise(atp_ctx *ctx, BasisPlan &bp, size_t i0, size_t 
                 pb.s[k] = PanelSeq{M + j0, n, w, p.rt, p.gpart, p.rinv, p.flags};
             }
             if (j0 > 0) {
-                if ((st = launch_gemm_simt<float, float, float, true>(ctx, proj, GemmEpi{EPI_STORE, nullptr}, bp.splits, bp.part,
-                                                                      bp.part_stride)) != ATP_OK) return st;
+                if ((st = launch_gemm_simt<float, float, float, true>(ctx, proj, GemmEpi{EPI_STORE, nullptr}, bp.splits,
+                                                                      bp.part + bp.group * bp.part_group, bp.part_stride)) != ATP_OK) return st;
                 if ((st = launch_gemm_simt<float, float, float, false>(ctx, upd, GemmEpi{EPI_D_MINUS, nullptr})) != ATP_OK) return st;
             }
             ATP_KERNEL(ctx, "panel_gram", 0, 0);
@@ -741,7 +742,7 @@ static atp_status orthonormalise(atp_ctx *ctx, BasisPlan &bp, size_t i0, size_t 
 
 template <typename T>
 static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<SeqDims> &sd, int oversample,
-                             int power_iters, int max_sweeps, uint64_t seed, int jbj, int jinner, atp_mat *U_r, atp_mat *X_r, float *sigma)
+                             int power_iters, int max_sweeps, uint64_t seed, int jbj, int jinner, int groups, atp_mat *U_r, atp_mat *X_r, float *sigma)
 {
     const int d = (int)X->cols;
     Arena ar(ctx->workspace, ctx->workspace_bytes);
@@ -749,7 +750,11 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
     plan_basis(ar, sd, d, oversample, bp);
     if (ar.overflow || !ctx->workspace) return ATP_ERR_WORKSPACE_TOO_SMALL;
     atp_status st;
-    {
+    if (X->dtype == ATP_BF16) {
+        ATP_KERNEL(ctx, "fill_omega", 0, 0);
+        fill_omega_bf16_kernel<<<1024, 256, 0, ctx->stream>>>(bp.omega_b, d, bp.rtmax, (int)align_up((size_t)bp.rtmax, 8), seed);
+        ATP_LAUNCHED(ctx);
+    } else {
         size_t n = (size_t)d * bp.rtmax;
         ATP_KERNEL(ctx, "fill_omega", 0, 0);
         fill_omega_kernel<<<(unsigned)std::min<size_t>((n + 255) / 256, 4096), 256, 0, ctx->stream>>>(bp.omega, n, seed);
@@ -760,18 +765,33 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
     const bool two_sided = (X->dtype == ATP_BF16) && jbj != 1;    // fp32 inputs keep the one-sided rotation of B itself
     GemmEpi store{EPI_STORE, nullptr};
 
-    for (size_t i0 = 0; i0 < bp.seqs.size(); i0 += BMAX) {
-        const size_t i1 = std::min(bp.seqs.size(), i0 + BMAX);
+    // The chains below are many small dependent launches (latency-bound). On request (groups = 2) the
+    // batch is cut in two groups that run on the context's two auxiliary streams, forked from and
+    // joined back into the caller's stream. Measured: no gain at batch 16 (the chain length, not the
+    // occupancy, sets the time, and the launch count doubles), so it is off by default.
+    const size_t nseq = bp.seqs.size();
+    const bool forked = groups == 2 && nseq >= 2 && ctx->aux[0] && ctx->aux[1] && !ctx->profiling;
+    const size_t gsz = forked ? std::min<size_t>(BMAX, (nseq + 1) / 2) : BMAX;
+    struct StreamGuard {
+        atp_ctx *c; cudaStream_t saved;
+        ~StreamGuard() { c->stream = saved; }
+    } guard{ctx, ctx->stream};
+    const cudaStream_t main_stream = ctx->stream;
+    if (forked) {
+        ATP_CUDA_OK(ctx, cudaEventRecord(ctx->ev_fork, main_stream));
+        for (int gq = 0; gq < 2; ++gq) ATP_CUDA_OK(ctx, cudaStreamWaitEvent(ctx->aux[gq], ctx->ev_fork, 0));
+    }
+    for (size_t i0 = 0; i0 < nseq; i0 += gsz) {
+        const size_t i1 = std::min(nseq, i0 + gsz);
         const int cnt = (int)(i1 - i0);
+        bp.group = forked ? (int)((i0 / gsz) & 1) : 0;
+        if (forked) ctx->stream = ctx->aux[bp.group];
         auto Xb = [&](const SeqPlan &p) { return (const T *)X->data + (size_t)p.dims.row0 * X->ld; };
         GemmBatch g; g.count = cnt;
         if constexpr (std::is_same<T, __nv_bfloat16>::value) {
             // bf16: every pass over X is a tensor-core GEMM with fp32 results; the iterates are
             // orthonormalised in fp32 and handed to the next pass as bf16 copies.
             const int ldo = (int)align_up((size_t)bp.rtmax, 8);
-            ATP_KERNEL(ctx, "fill_omega", 0, 0);
-            fill_omega_bf16_kernel<<<1024, 256, 0, ctx->stream>>>(bp.omega_b, d, bp.rtmax, ldo, seed);
-            ATP_LAUNCHED(ctx);
             // The orthonormal iterate goes to the next pass as a bf16 hi/lo pair (about 16 mantissa
             // bits): a single bf16 rounding of Y would leak sigma_1 * 2^-9 / sqrt(L) of the leading
             // direction into every column and bury directions that are 10^3..10^4 times weaker.
@@ -932,7 +952,8 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
                 ATP_KERNEL(ctx, "jac2_init", 0, 0);
                 jac2_init_kernel<<<dim3(64, cnt), 256, 0, ctx->stream>>>(jb);
                 ATP_LAUNCHED(ctx);
-                const int nsw = pass == 0 ? max_sweeps : std::min(max_sweeps, 4);
+                // the second pass continues the same iteration on the rotated data: split the sweep budget
+                const int nsw = pass == 0 ? (max_sweeps + 1) / 2 : max_sweeps / 2;
                 for (int sw = 0; sw < nsw; ++sw) {
                     for (int step = 0; step < maxnb - 1; ++step) {
                         // algorithmic work of a step when every pair rotates (converged pairs skip it)
@@ -993,6 +1014,12 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
             ATP_LAUNCHED(ctx);
         }
     }
+    if (forked) {
+        for (int gq = 0; gq < 2; ++gq) {
+            ATP_CUDA_OK(ctx, cudaEventRecord(ctx->ev_join[gq], ctx->aux[gq]));
+            ATP_CUDA_OK(ctx, cudaStreamWaitEvent(main_stream, ctx->ev_join[gq], 0));
+        }
+    }
     return ATP_OK;
 }
 
@@ -1002,7 +1029,7 @@ extern "C" atp_status atp_principal_basis(atp_ctx *ctx, const atp_mat *X, const 
     if (!ctx) return ATP_ERR_INVALID_ARG;
     atp_status st;
     if ((st = check_mat(X)) != ATP_OK || (st = check_mat(U_r)) != ATP_OK || (st = check_mat(X_r)) != ATP_OK) return st;
-    int oversample = 64, power_iters = 2, max_sweeps = 12, jbj = 16, jinner = 1; uint64_t seed = 0x243F6A8885A308D3ull;
+    int oversample = 64, power_iters = 2, max_sweeps = 12, jbj = 16, jinner = 1, groups = 0; uint64_t seed = 0x243F6A8885A308D3ull;
     if (opts) {
         if (opts->struct_size < sizeof(atp_basis_opts)) return ATP_ERR_INVALID_ARG;
         if (opts->oversample >= 0) oversample = opts->oversample;
@@ -1012,6 +1039,7 @@ extern "C" atp_status atp_principal_basis(atp_ctx *ctx, const atp_mat *X, const 
         if (opts->jacobi_block == 16 || opts->jacobi_block == 32 || opts->jacobi_block == 1) jbj = opts->jacobi_block;
         else if (opts->jacobi_block != 0) return ATP_ERR_INVALID_ARG;
         if (opts->jacobi_inner > 0) jinner = opts->jacobi_inner;
+        groups = opts->groups;
     }
     if (oversample > 4096 || power_iters > 64 || max_sweeps > 200) return ATP_ERR_INVALID_ARG;
     if (U_r->dtype != X->dtype || X_r->dtype != X->dtype) return ATP_ERR_UNSUPPORTED_DTYPE;
@@ -1026,8 +1054,8 @@ extern "C" atp_status atp_principal_basis(atp_ctx *ctx, const atp_mat *X, const 
     if (U_r->rows != X->rows || U_r->cols < maxr || X_r->rows != tr || X_r->cols != X->cols) return ATP_ERR_INVALID_ARG;
     if (X->rows == 0) return ATP_OK;
     ATP_CUDA_OK(ctx, cudaSetDevice(ctx->device));
-    if (X->dtype == ATP_F32) return basis_impl<float>(ctx, X, sd, oversample, power_iters, max_sweeps, seed, jbj, jinner, U_r, X_r, sigma);
-    return basis_impl<__nv_bfloat16>(ctx, X, sd, oversample, power_iters, max_sweeps, seed, jbj, jinner, U_r, X_r, sigma);
+    if (X->dtype == ATP_F32) return basis_impl<float>(ctx, X, sd, oversample, power_iters, max_sweeps, seed, jbj, jinner, groups, U_r, X_r, sigma);
+    return basis_impl<__nv_bfloat16>(ctx, X, sd, oversample, power_iters, max_sweeps, seed, jbj, jinner, groups, U_r, X_r, sigma);
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -22,6 +22,9 @@ struct atp_ctx {
     int64_t launches = 0;
     cudaError_t last_cuda = cudaSuccess;
     int sm_count = 148;
+    // two auxiliary streams: halves of a batch run their latency-bound kernel chains side by side
+    cudaStream_t aux[2] = {nullptr, nullptr};
+    cudaEvent_t ev_fork = nullptr, ev_join[2] = {nullptr, nullptr};
 };
 
 #define ATP_CUDA_OK(ctx, expr)                                   \
