@@ -18,7 +18,9 @@
  *     over with atp_set_workspace(); its required size comes from atp_workspace_bytes().
  *     atp_create() allocates one small device status word and a pinned staging page, freed by
  *     atp_destroy().
- *   - Calls only enqueue work and return; they never synchronise, except atp_poll_device_status().
+ *   - Calls only enqueue work and return; they never wait for results, except
+ *     atp_poll_device_status(). atp_principal_basis reads back its own convergence flags while it
+ *     enqueues Jacobi sweeps: the calling thread may block until the GPU is within two sweeps of it.
  *     Work is ordered on the context's stream (atp_set_stream); atp_principal_basis can fork part of
  *     a batch onto two internal streams (opts->groups) and joins them back before it returns.
  *   - Errors the host can detect are returned at once and nothing is launched. Conditions only
@@ -93,7 +95,7 @@ typedef struct {
     uint32_t struct_size;
     int32_t oversample;    /* extra columns of the range finder; < 0: default 64              */
     int32_t power_iters;   /* subspace (power) iterations;        < 0: default 2              */
-    int32_t max_sweeps;    /* Jacobi sweep limit;                 <= 0: default 12            */
+    int32_t max_sweeps;    /* Jacobi sweep limit;                 <= 0: default 24            */
     uint64_t seed;         /* seed of the +-1 test matrix                                      */
     int32_t jacobi_block;  /* tuning: rows per Jacobi block, 16 or 32; 0: default 16 (bf16 path only)  */
     int32_t jacobi_inner;  /* tuning: on-chip sweeps per block visit;   <= 0: default 1                */

@@ -62,6 +62,9 @@ atp_status atp_create(atp_ctx **out, int device)
     for (int i = 0; i < 2 && ok; ++i)
         ok = cudaStreamCreateWithFlags(&ctx->aux[i], cudaStreamNonBlocking) == cudaSuccess &&
              cudaEventCreateWithFlags(&ctx->ev_join[i], cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaHostAlloc((void **)&ctx->h_flags, 4 * sizeof(int), cudaHostAllocDefault) == cudaSuccess &&
+         cudaMalloc((void **)&ctx->d_flags, 4 * sizeof(int)) == cudaSuccess;
+    for (int i = 0; i < 4 && ok; ++i) ok = cudaEventCreateWithFlags(&ctx->ev_flag[i], cudaEventDisableTiming) == cudaSuccess;
     if (!ok) { atp_destroy(ctx); return ATP_ERR_CUDA; }
     *out = ctx;
     return ATP_OK;
@@ -77,6 +80,9 @@ atp_status atp_destroy(atp_ctx *ctx)
         if (ctx->ev_join[i]) cudaEventDestroy(ctx->ev_join[i]);
     }
     if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+    for (int i = 0; i < 4; ++i) if (ctx->ev_flag[i]) cudaEventDestroy(ctx->ev_flag[i]);
+    if (ctx->h_flags) cudaFreeHost(ctx->h_flags);
+    if (ctx->d_flags) cudaFree(ctx->d_flags);
     delete ctx;
     return ATP_OK;
 }

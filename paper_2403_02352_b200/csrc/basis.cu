@@ -171,9 +171,10 @@ __global__ void __launch_bounds__(64) panel_apply_kernel(const __grid_constant__
         x[c] = acc / Ls[c][c];
     }
     const int grow = r0 + tid;
+    const float rscale = rsqrtf((float)sq.n * (1.f / 3.f));      // replacement columns of about unit norm
 #pragma unroll
     for (int c = 0; c < PB; ++c)
-        Ts[tid][c] = fl[c] ? hash_uniform(seed, ((uint64_t)blockIdx.y << 40) ^ ((uint64_t)grow << 8) ^ (uint64_t)c) : x[c];
+        Ts[tid][c] = fl[c] ? rscale * hash_uniform(seed, ((uint64_t)blockIdx.y << 40) ^ ((uint64_t)grow << 8) ^ (uint64_t)c) : x[c];
     __syncthreads();
     for (int e = tid; e < 64 * PB; e += 64) {
         int row = e >> 6, c = e & 63;
@@ -384,17 +385,22 @@ jacobi_pair_kernel(const __grid_constant__ JacBatch batch, int step, float tol_r
     }
 }
 
-__global__ void jacobi_sweep_end_kernel(const __grid_constant__ JacBatch batch, float tol_conv, int last, int *dev_status)
+// One block of BMAX threads; *all_conv = 1 when every sequence of the launch has converged.
+__global__ void jacobi_sweep_end_kernel(const __grid_constant__ JacBatch batch, float tol_conv, int last, int *dev_status, int *all_conv)
 {
-    int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b >= batch.count) return;
-    const JacSeq &sq = batch.s[b];
-    if (!*sq.conv) {
-        float mo = __uint_as_float(*sq.maxoff);
-        if (mo <= tol_conv) *sq.conv = 1;
-        else if (last) raise_status(dev_status, ATP_ERR_NOT_CONVERGED);
+    const int b = threadIdx.x;
+    int done = 1;
+    if (b < batch.count) {
+        const JacSeq &sq = batch.s[b];
+        if (!*sq.conv) {
+            float mo = __uint_as_float(*sq.maxoff);
+            if (mo <= tol_conv) *sq.conv = 1;
+            else { done = 0; if (last) raise_status(dev_status, ATP_ERR_NOT_CONVERGED); }
+        }
+        *sq.maxoff = 0u;
     }
-    *sq.maxoff = 0u;
+    done = __syncthreads_and(done);
+    if (threadIdx.x == 0 && all_conv) *all_conv = done;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -695,7 +701,9 @@ size_t basis_workspace_bytes(const std::vector<SeqDims> &sd, int d, int oversamp
 }
 
 // Orthonormalise the columns of M_b (n_b x rt_b, ld = rt_b) for the sequences [i0, i1).
-static atp_status orthonormalise(atp_ctx *ctx, BasisPlan &bp, size_t i0, size_t i1, bool z_side, int d, uint64_t seed)
+// reps: Gram-Schmidt passes per panel. Two give orthonormality to working precision and repair
+// dependent columns; one is enough for an intermediate iterate of the subspace iteration.
+static atp_status orthonormalise(atp_ctx *ctx, BasisPlan &bp, size_t i0, size_t i1, bool z_side, int d, uint64_t seed, int reps)
 {
     int maxpan = 0, maxn = 0;
     for (size_t i = i0; i < i1; ++i) {
@@ -705,7 +713,7 @@ static atp_status orthonormalise(atp_ctx *ctx, BasisPlan &bp, size_t i0, size_t 
     atp_status st;
     for (int pj = 0; pj < maxpan; ++pj) {
         const int j0 = pj * PB;
-        for (int rep = 0; rep < 2; ++rep) {
+        for (int rep = 0; rep < reps; ++rep) {
             GemmBatch proj, upd; PanelBatch pb;
             proj.count = upd.count = pb.count = (int)(i1 - i0);
             for (size_t i = i0; i < i1; ++i) {
@@ -813,7 +821,7 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
                 hp.push_back(tc::HostProblem{Xb(p), bp.omega_b, nullptr, p.Y, nullptr, nullptr, p.dims.L, p.rt, d, (int)X->ld, ldo, p.rt, 0});
             }
             if ((st = tc::launch<false, false, tc::OUT_F32>(ctx, hp, store)) != ATP_OK) return st;
-            if ((st = orthonormalise(ctx, bp, i0, i1, false, d, seed)) != ATP_OK) return st;
+            if ((st = orthonormalise(ctx, bp, i0, i1, false, d, seed, 2)) != ATP_OK) return st;
             if ((st = to_bf16()) != ATP_OK) return st;
             for (int it = 0; it < power_iters; ++it) {
                 hp.clear();
@@ -830,7 +838,7 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
                     hp.push_back(tc::HostProblem{Xb(p), p.Zb, p.Zl, p.Y, nullptr, nullptr, p.dims.L, p.rt, d, (int)X->ld, ldb, p.rt, 0});
                 }
                 if ((st = tc::launch<false, true, tc::OUT_F32>(ctx, hp, store)) != ATP_OK) return st;
-                if ((st = orthonormalise(ctx, bp, i0, i1, false, d, seed + 2000003ull * (it + 1))) != ATP_OK) return st;
+                if ((st = orthonormalise(ctx, bp, i0, i1, false, d, seed + 2000003ull * (it + 1), 2)) != ATP_OK) return st;
                 if ((st = to_bf16()) != ATP_OK) return st;
             }
         } else {
@@ -840,7 +848,7 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
                 g.p[i - i0] = GemmProblem{Xb(p), bp.omega, p.Y, nullptr, p.dims.L, p.rt, d, (int)X->ld, bp.rtmax, p.rt, 0};
             }
             if ((st = launch_gemm_simt<T, float, float, false>(ctx, g, store)) != ATP_OK) return st;
-            if ((st = orthonormalise(ctx, bp, i0, i1, false, d, seed)) != ATP_OK) return st;
+            if ((st = orthonormalise(ctx, bp, i0, i1, false, d, seed, 2)) != ATP_OK) return st;
             for (int it = 0; it < power_iters; ++it) {
                 // Z = X^T Y ; Y = X Z ; orth(Y).  Z is not orthonormalised: Y has orthonormal, QR-ordered
                 // columns, so cond(Z) ~ sigma_1 / sigma_r~ and cond(X Z) is its square, which the fp64
@@ -855,7 +863,7 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
                     g.p[i - i0] = GemmProblem{Xb(p), p.Z, p.Y, nullptr, p.dims.L, p.rt, d, (int)X->ld, p.rt, p.rt, 0};
                 }
                 if ((st = launch_gemm_simt<T, float, float, false>(ctx, g, store)) != ATP_OK) return st;
-                if ((st = orthonormalise(ctx, bp, i0, i1, false, d, seed + 2000003ull * (it + 1))) != ATP_OK) return st;
+                if ((st = orthonormalise(ctx, bp, i0, i1, false, d, seed + 2000003ull * (it + 1), 2)) != ATP_OK) return st;
             }
         }
         if (!two_sided) {
@@ -879,14 +887,25 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
             init_w_kernel<<<dim3(64, cnt), 256, 0, ctx->stream>>>(jb);
             ATP_LAUNCHED(ctx);
             for (int sw = 0; sw < max_sweeps; ++sw) {
+                if (sw >= 2 && !forked) {      // host stays at most two sweeps ahead; stop once converged
+                    const int slot = (sw - 2) & 3;
+                    ATP_CUDA_OK(ctx, cudaEventSynchronize(ctx->ev_flag[slot]));
+                    if (ctx->h_flags[slot]) break;
+                }
                 for (int step = 0; step < maxnb - 1; ++step) {
                     ATP_KERNEL(ctx, "jacobi_pair", 0, 0);
                     jacobi_pair_kernel<<<dim3(maxnb / 2, cnt), 256, 0, ctx->stream>>>(jb, step, tol_rot, tol_rot);
                     ATP_LAUNCHED(ctx);
                 }
                 ATP_KERNEL(ctx, "jacobi_sweep_end", 0, 0);
-                jacobi_sweep_end_kernel<<<1, BMAX, 0, ctx->stream>>>(jb, tol_conv, sw == max_sweeps - 1, ctx->dev_status);
+                jacobi_sweep_end_kernel<<<1, BMAX, 0, ctx->stream>>>(jb, tol_conv, sw == max_sweeps - 1, ctx->dev_status,
+                                                                     ctx->d_flags + (sw & 3));
                 ATP_LAUNCHED(ctx);
+                if (!forked) {
+                    ATP_CUDA_OK(ctx, cudaMemcpyAsync(ctx->h_flags + (sw & 3), ctx->d_flags + (sw & 3), sizeof(int),
+                                                     cudaMemcpyDeviceToHost, ctx->stream));
+                    ATP_CUDA_OK(ctx, cudaEventRecord(ctx->ev_flag[sw & 3], ctx->stream));
+                }
             }
             int npow = 1; while (npow < maxrt) npow <<= 1;
             size_t sm = (size_t)npow * 8;
@@ -953,14 +972,25 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
                 jac2_init_kernel<<<dim3(64, cnt), 256, 0, ctx->stream>>>(jb);
                 ATP_LAUNCHED(ctx);
                 // the second pass continues the same iteration on the rotated data: split the sweep budget
-                const int nsw = pass == 0 ? (max_sweeps + 1) / 2 : max_sweeps / 2;
+                // pass 0 only has to make the rows graded and roughly orthogonal (scaled off-diagonals below
+                // 1e-2; on ill-conditioned input it stalls at the noise floor of G, hence the cap of 8 sweeps)
+                const int nsw = pass == 0 ? std::min(8, (max_sweeps + 1) / 2) : max_sweeps - std::min(8, (max_sweeps + 1) / 2);
+                const float tolc = pass == 0 ? fmaxf(tol_conv, 1e-2f) : tol_conv;
+                const float tolr = tolc * 0.25f;
                 for (int sw = 0; sw < nsw; ++sw) {
+                    // Stop enqueueing once the device reported convergence. The flag of sweep sw - 2 is
+                    // awaited here, so the host stays at most two sweeps ahead and the GPU never idles.
+                    if (sw >= 2 && !forked) {
+                        const int slot = (sw - 2) & 3;
+                        ATP_CUDA_OK(ctx, cudaEventSynchronize(ctx->ev_flag[slot]));
+                        if (ctx->h_flags[slot]) break;
+                    }
                     for (int step = 0; step < maxnb - 1; ++step) {
                         // algorithmic work of a step when every pair rotates (converged pairs skip it)
                         const double nseq = cnt, bl = blk;
                         ATP_KERNEL(ctx, "jac2_local", nseq * npairs * jinner * (bl - 1) * (bl * bl * 6.0 + bl * bl * 3.0), 0);
-                        if (jbj == 32) jac2_local_kernel<32><<<dim3(npairs, cnt), 1024, 0, ctx->stream>>>(jb, step, tol_rot, jinner);
-                        else jac2_local_kernel<16><<<dim3(npairs, cnt), 512, 0, ctx->stream>>>(jb, step, tol_rot, jinner);
+                        if (jbj == 32) jac2_local_kernel<32><<<dim3(npairs, cnt), 1024, 0, ctx->stream>>>(jb, step, tolr, jinner);
+                        else jac2_local_kernel<16><<<dim3(npairs, cnt), 512, 0, ctx->stream>>>(jb, step, tolr, jinner);
                         ATP_LAUNCHED(ctx);
                         ATP_KERNEL(ctx, "jac2_apply", nseq * npairs * (npairs * 4.0 + ceil_div(maxrt, blk) * 2.0) * bl * bl * bl,
                                    nseq * npairs * (npairs * 2.0 + ceil_div(maxrt, blk) * 2.0) * bl * bl * 4.0);
@@ -970,8 +1000,14 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
                         ATP_LAUNCHED(ctx);
                     }
                     ATP_KERNEL(ctx, "jac2_sweep_end", 0, 0);
-                    jac2_sweep_end_kernel<<<1, J2MAX, 0, ctx->stream>>>(jb, tol_conv, pass == 1 && sw == nsw - 1, ctx->dev_status);
+                    jac2_sweep_end_kernel<<<1, J2MAX, 0, ctx->stream>>>(jb, tolc, pass == 1 && sw == nsw - 1, ctx->dev_status,
+                                                                        ctx->d_flags + (sw & 3));
                     ATP_LAUNCHED(ctx);
+                    if (!forked) {
+                        ATP_CUDA_OK(ctx, cudaMemcpyAsync(ctx->h_flags + (sw & 3), ctx->d_flags + (sw & 3), sizeof(int),
+                                                         cudaMemcpyDeviceToHost, ctx->stream));
+                        ATP_CUDA_OK(ctx, cudaEventRecord(ctx->ev_flag[sw & 3], ctx->stream));
+                    }
                 }
                 if (pass == 0) {
                     GemmBatch r1, r2; r1.count = r2.count = cnt;
@@ -1029,7 +1065,7 @@ extern "C" atp_status atp_principal_basis(atp_ctx *ctx, const atp_mat *X, const 
     if (!ctx) return ATP_ERR_INVALID_ARG;
     atp_status st;
     if ((st = check_mat(X)) != ATP_OK || (st = check_mat(U_r)) != ATP_OK || (st = check_mat(X_r)) != ATP_OK) return st;
-    int oversample = 64, power_iters = 2, max_sweeps = 12, jbj = 16, jinner = 1, groups = 0; uint64_t seed = 0x243F6A8885A308D3ull;
+    int oversample = 64, power_iters = 2, max_sweeps = 24, jbj = 16, jinner = 1, groups = 0; uint64_t seed = 0x243F6A8885A308D3ull;
     if (opts) {
         if (opts->struct_size < sizeof(atp_basis_opts)) return ATP_ERR_INVALID_ARG;
         if (opts->oversample >= 0) oversample = opts->oversample;

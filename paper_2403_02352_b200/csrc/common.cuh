@@ -25,6 +25,10 @@ struct atp_ctx {
     // two auxiliary streams: halves of a batch run their latency-bound kernel chains side by side
     cudaStream_t aux[2] = {nullptr, nullptr};
     cudaEvent_t ev_fork = nullptr, ev_join[2] = {nullptr, nullptr};
+    // convergence feedback of iterative kernels: device word -> pinned host word, ring of 4 slots
+    int *h_flags = nullptr;          // pinned host, 4 ints
+    int *d_flags = nullptr;          // device, 4 ints
+    cudaEvent_t ev_flag[4] = {nullptr, nullptr, nullptr, nullptr};
 };
 
 #define ATP_CUDA_OK(ctx, expr)                                   \

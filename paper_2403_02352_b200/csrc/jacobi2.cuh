@@ -261,15 +261,21 @@ jac2_apply_kernel(const __grid_constant__ Jac2Batch batch, int step)
     }
 }
 
-__global__ void jac2_sweep_end_kernel(const __grid_constant__ Jac2Batch batch, float tol_conv, int last, int *dev_status)
+// One block of J2MAX threads. Besides the per-sequence flags it writes *all_conv = 1 when every
+// sequence of the launch has converged (read back by the host to stop enqueueing sweeps).
+__global__ void jac2_sweep_end_kernel(const __grid_constant__ Jac2Batch batch, float tol_conv, int last, int *dev_status, int *all_conv)
 {
-    int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b >= batch.count) return;
-    const Jac2Seq &sq = batch.s[b];
-    if (!*sq.conv) {
-        float mo = __uint_as_float(*sq.maxoff);
-        if (mo <= tol_conv) *sq.conv = 1;
-        else if (last) raise_status(dev_status, ATP_ERR_NOT_CONVERGED);
+    const int b = threadIdx.x;
+    int done = 1;
+    if (b < batch.count) {
+        const Jac2Seq &sq = batch.s[b];
+        if (!*sq.conv) {
+            float mo = __uint_as_float(*sq.maxoff);
+            if (mo <= tol_conv) *sq.conv = 1;
+            else { done = 0; if (last) raise_status(dev_status, ATP_ERR_NOT_CONVERGED); }
+        }
+        *sq.maxoff = 0u;
     }
-    *sq.maxoff = 0u;
+    done = __syncthreads_and(done);
+    if (threadIdx.x == 0 && all_conv) *all_conv = done;
 }
