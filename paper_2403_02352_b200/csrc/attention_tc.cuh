@@ -188,16 +188,27 @@ attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e
             tc_fence_after();
             const uint32_t t_s = t_s0 + 128 * (j & 1) + lane_addr;
             const int kvalid = sq.r - j * 128;                 // keys of this block that exist
-            // pass A: block maximum of the scaled scores
+            // pass A: block maximum of the raw scores (the scale is positive: applied once at the end)
             float mx = -INFINITY;
+            if (kvalid >= 128) {
 #pragma unroll 1
-            for (int c = 0; c < 128; c += 32) {
-                uint32_t rr[32];
-                tmem_ld32(t_s + c, rr);
+                for (int c = 0; c < 128; c += 32) {
+                    uint32_t rr[32];
+                    tmem_ld32(t_s + c, rr);
 #pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    if (c + i < kvalid) mx = fmaxf(mx, __uint_as_float(rr[i]) * scale_log2e);
+                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(rr[i]));
+                }
+            } else {
+#pragma unroll 1
+                for (int c = 0; c < 128; c += 32) {
+                    uint32_t rr[32];
+                    tmem_ld32(t_s + c, rr);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (c + i < kvalid) mx = fmaxf(mx, __uint_as_float(rr[i]));
+                }
             }
+            mx *= scale_log2e;
             // the exponent offset only moves when the maximum grew by more than 8 (factor 256)
             float alpha = 1.f;
             bool grow = (mx > m_used + 8.f) || (j == 0);
@@ -225,8 +236,11 @@ attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e
                 ok = __shfl_sync(0xffffffffu, ok_i, 0) != 0;
                 if (!ok) break;
             }
-            // pass B: P = exp2(s - m) as bf16 into the swizzled K-major A tile, row sums in fp32
+            // pass B: P = exp2(s * c - m) as bf16 into the swizzled K-major A tile; the row sum is taken
+            // from the unrounded values (the bf16 rounding of P averages out over the r keys)
             uint8_t *prow = gbase + C_::OFF_P + row * 128;
+            const float neg_m = -m_used;
+            const bool full = kvalid >= 128;
 #pragma unroll 1
             for (int c = 0; c < 128; c += 32) {
                 uint32_t rr[32];
@@ -234,10 +248,14 @@ attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e
                 uint32_t packed[16];
 #pragma unroll
                 for (int i = 0; i < 32; i += 2) {
-                    float p0 = (c + i < kvalid) ? fast_exp2(__uint_as_float(rr[i]) * scale_log2e - m_used) : 0.f;
-                    float p1 = (c + i + 1 < kvalid) ? fast_exp2(__uint_as_float(rr[i + 1]) * scale_log2e - m_used) : 0.f;
+                    float p0 = fast_exp2(fmaf(__uint_as_float(rr[i]), scale_log2e, neg_m));
+                    float p1 = fast_exp2(fmaf(__uint_as_float(rr[i + 1]), scale_log2e, neg_m));
+                    if (!full) {
+                        if (c + i >= kvalid) p0 = 0.f;
+                        if (c + i + 1 >= kvalid) p1 = 0.f;
+                    }
+                    l_sum += p0 + p1;
                     __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-                    l_sum += __low2float(h) + __high2float(h);          // sum what the value GEMM will see
                     packed[i >> 1] = *(uint32_t *)&h;
                 }
 #pragma unroll
