@@ -123,8 +123,8 @@ attn_simt_kernel(const __grid_constant__ AttnBatch batch, int dh, int ldq, int l
     }
 }
 
-struct AttnPlan { float *Qp, *Kp, *Vp, *Q; __nv_bfloat16 *Qph, *Qpl, *Kh, *Kl, *Vb, *Qh, *Ql; };
-static void plan_attn(Arena &ar, int64_t tr, int64_t tl, int64_t dp, AttnPlan &p)
+struct AttnPlan { float *Qp, *Kp, *Vp, *Q; __nv_bfloat16 *Qph, *Qpl, *Kh, *Kl, *Vb, *Qh, *Ql; float *nrm; };
+static void plan_attn(Arena &ar, int64_t tr, int64_t tl, int64_t dp, int64_t nseq, AttnPlan &p)
 {
     p.Qp = ar.take<float>((size_t)tr * dp);
     p.Kp = ar.take<float>((size_t)tr * dp);
@@ -137,6 +137,7 @@ static void plan_attn(Arena &ar, int64_t tr, int64_t tl, int64_t dp, AttnPlan &p
     p.Vb = ar.take<__nv_bfloat16>((size_t)tr * align_up((size_t)dp, 8));
     p.Qh = ar.take<__nv_bfloat16>((size_t)tl * align_up((size_t)dp, 8));
     p.Ql = ar.take<__nv_bfloat16>((size_t)tl * align_up((size_t)dp, 8));
+    p.nrm = ar.take<float>((size_t)nseq * dp + (size_t)(tr / 128 + nseq) * dp);    // per head norms: queries, key blocks
 }
 size_t attention_workspace_bytes(const std::vector<SeqDims> &seqs, int64_t dp)
 {
@@ -144,7 +145,7 @@ size_t attention_workspace_bytes(const std::vector<SeqDims> &seqs, int64_t dp)
     for (auto &s : seqs) { tr += s.r; tl += s.L; }
     Arena ar(nullptr, (size_t)-1);
     AttnPlan p;
-    plan_attn(ar, tr, tl, dp, p);
+    plan_attn(ar, tr, tl, dp, (int64_t)seqs.size(), p);
     return ar.off;
 }
 
@@ -158,7 +159,7 @@ static atp_status attention_impl(atp_ctx *ctx, const atp_mat *X, const atp_mat *
     for (auto &s : seqs) { tr += s.r; tl += s.L; }
     Arena ar(ctx->workspace, ctx->workspace_bytes);
     AttnPlan pl;
-    plan_attn(ar, tr, tl, dp, pl);
+    plan_attn(ar, tr, tl, dp, (int64_t)seqs.size(), pl);
     if (ar.overflow || !ctx->workspace) return ATP_ERR_WORKSPACE_TOO_SMALL;
     atp_status st;
     GemmEpi store{EPI_STORE, nullptr};
@@ -186,11 +187,15 @@ static atp_status attention_impl(atp_ctx *ctx, const atp_mat *X, const atp_mat *
                 if ((st = tc::launch<false, true, tc::OUT_BF16_SPLIT>(ctx, qe, store)) != ATP_OK) return st;
             }
             std::vector<atc::HostSeq> hs;
+            float *nrm = pl.nrm;
             for (auto &s : seqs)
-                if (s.L > 0)
+                if (s.L > 0) {
+                    float *qmax = nrm, *kmax = nrm + heads;
+                    nrm += heads + (size_t)heads * ceil_div(s.r, 128);
                     hs.push_back(atc::HostSeq{pl.Qh + (size_t)s.row0 * ldq, pl.Ql + (size_t)s.row0 * ldq, pl.Kh + (size_t)s.rank0 * ldq,
                                               pl.Kl + (size_t)s.rank0 * ldq, pl.Vb + (size_t)s.rank0 * ldq,
-                                              (T *)O->data + (size_t)s.row0 * O->ld, s.L, s.r, ldq, ldq, (int)O->ld, dp});
+                                              (T *)O->data + (size_t)s.row0 * O->ld, s.L, s.r, ldq, ldq, (int)O->ld, dp, qmax, kmax});
+                }
             return dh == 64 ? atc::launch<64>(ctx, hs, heads, scale) : atc::launch<128>(ctx, hs, heads, scale);
         }
         // bf16, other head widths: projections on the tensor cores with fp32 results. Q' is kept as a bf16 hi/lo pair so

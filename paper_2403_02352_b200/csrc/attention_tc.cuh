@@ -22,6 +22,8 @@ constexpr int MAX_SEQ = 16;
 struct Seq {
     CUtensorMap qh, ql, kh, kl, v;      // Q hi/lo: L x d' ; K' hi/lo, V': r x d'
     void *O; int L, r, ldo, tile0;
+    const float *qmax;                  // per head: largest query norm (head slice)
+    const float *kmax;                  // per head and 128-key block: largest key norm
 };
 struct Batch { Seq s[MAX_SEQ]; int count, total_tiles; };
 
@@ -62,7 +64,7 @@ template <int DH> struct Cfg {
 
 template <int DH>
 __global__ void __launch_bounds__(192)
-attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e, int *dev_status)
+attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e, float lo_thresh, int *dev_status)
 {
     using C_ = Cfg<DH>;
     constexpr int NS = C_::NSLOT;
@@ -85,6 +87,10 @@ attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e
     const int head = blockIdx.y;
     const int col0 = head * DH;
     const int nblk = (sq.r + 127) / 128;
+    // The lo terms of a key block matter only while |q| |k| 2^-8 * scale can move a logit: blocks whose
+    // largest key norm is below the threshold get the single product Qh Kh^T.
+    const float qm = sq.qmax[head];
+    const float *km = sq.kmax + (size_t)head * nblk;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
@@ -118,6 +124,7 @@ attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e
                     if (n >= 1 && !mbar_wait(b_empty + 8 * s, (n - 1) & 1, &abort_flag)) { j = nblk; break; }
                     const uint32_t dst = base + C_::OFF_SLOT + s * C_::TILE;
                     const CUtensorMap *m = which == 0 ? &sq.kh : (which == 1 ? &sq.kl : &sq.v);
+                    if (which == 1 && !(qm * km[j] > lo_thresh)) { mbar_arrive(b_full + 8 * s); continue; }   // K'_lo not needed
                     mbar_expect_tx(b_full + 8 * s, C_::TILE);
 #pragma unroll
                     for (int c = 0; c < DH / 64; ++c) tma_load_2d(dst + c * 16384, m, col0 + 64 * c, j * 128, b_full + 8 * s);
@@ -134,6 +141,7 @@ attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e
             // S_j for block j into buffer j & 1: Qh Kh^T + Qh Kl^T + Ql Kh^T
             auto issue_s = [&](int j) -> bool {
                 const int lk = 3 * j, sh = lk % NS, sl = (lk + 1) % NS;
+                const bool need_lo = qm * km[j] > lo_thresh;
                 if (j >= 2 && !mbar_wait(b_sfree + 8 * (j & 1), ((j >> 1) - 1) & 1, &abort_flag)) return false;
                 if (!mbar_wait(b_full + 8 * sh, (lk / NS) & 1, &abort_flag)) return false;
                 if (!mbar_wait(b_full + 8 * sl, ((lk + 1) / NS) & 1, &abort_flag)) return false;
@@ -146,8 +154,10 @@ attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e
                     const uint64_t aqh = smem_desc(q_hi + off, 16, 1024), aql = smem_desc(q_lo + off, 16, 1024);
                     const uint64_t bkh = smem_desc(kh + off, 16, 1024), bkl = smem_desc(kl + off, 16, 1024);
                     umma_bf16(d, aqh, bkh, idesc_s, kk > 0 ? 1u : 0u);
-                    umma_bf16(d, aqh, bkl, idesc_s, 1u);
-                    umma_bf16(d, aql, bkh, idesc_s, 1u);
+                    if (need_lo) {
+                        umma_bf16(d, aqh, bkl, idesc_s, 1u);
+                        umma_bf16(d, aql, bkh, idesc_s, 1u);
+                    }
                 }
                 umma_commit(b_empty + 8 * sh);
                 umma_commit(b_empty + 8 * sl);
@@ -309,7 +319,27 @@ attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e
 struct HostSeq {
     const void *Qh, *Ql, *Kh, *Kl, *V; void *O;
     int L, r, ldq, ldk, ldo, dp;
+    float *qmax, *kmax;                 // device scratch: heads and heads * ceil(r / 128) floats, zeroed by launch()
 };
+
+// Largest row norm of the head slices of M (rows x heads*DH, bf16): out[head * nblk + row / rows_per_blk].
+template <int DH>
+__global__ void __launch_bounds__(256)
+head_norm_max_kernel(const __nv_bfloat16 *M, int rows, int ld, int heads, int rows_per_blk, int nblk, float *out)
+{
+    const int w = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (w >= rows * heads) return;
+    const int row = w / heads, head = w - row * heads;
+    const __nv_bfloat16 *p = M + (size_t)row * ld + head * DH;
+    float s = 0.f;
+    for (int c = lane * 2; c < DH; c += 64) {
+        float2 v = __bfloat1622float2(*(const __nv_bfloat162 *)(p + c));
+        s = fmaf(v.x, v.x, fmaf(v.y, v.y, s));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) atomicMax((unsigned *)(out + (size_t)head * nblk + row / rows_per_blk), __float_as_uint(sqrtf(s)));
+}
 
 template <int DH>
 static atp_status launch(atp_ctx *ctx, const std::vector<HostSeq> &seqs, int heads, float scale)
@@ -333,6 +363,18 @@ static atp_status launch(atp_ctx *ctx, const std::vector<HostSeq> &seqs, int hea
                       make_map(&s.v, h.V, h.r, h.dp, h.ldk, 128);
             if (!ok) return ATP_ERR_INVALID_ARG;
             s.O = h.O; s.L = h.L; s.r = h.r; s.ldo = h.ldo; s.tile0 = b.total_tiles;
+            s.qmax = h.qmax; s.kmax = h.kmax;
+            {
+                const int nblk = ceil_div(h.r, 128);
+                ATP_CUDA_OK(ctx, cudaMemsetAsync(h.qmax, 0, sizeof(float) * heads, ctx->stream));
+                ATP_CUDA_OK(ctx, cudaMemsetAsync(h.kmax, 0, sizeof(float) * heads * nblk, ctx->stream));
+                ATP_KERNEL(ctx, "head_norm_max", 0, 2.0 * (h.L + h.r) * h.dp);
+                head_norm_max_kernel<DH><<<ceil_div(h.L * heads, 8), 256, 0, ctx->stream>>>((const __nv_bfloat16 *)h.Qh, h.L, h.ldq, heads, h.L, 1, h.qmax);
+                ATP_LAUNCHED(ctx);
+                ATP_KERNEL(ctx, "head_norm_max", 0, 0);
+                head_norm_max_kernel<DH><<<ceil_div(h.r * heads, 8), 256, 0, ctx->stream>>>((const __nv_bfloat16 *)h.Kh, h.r, h.ldk, heads, 128, nblk, h.kmax);
+                ATP_LAUNCHED(ctx);
+            }
             b.total_tiles += ceil_div(h.L, 128);
             b.count++;
             flops += 4.0 * h.L * h.r * h.dp;                                   // algorithmic: one score and one value product
@@ -340,7 +382,9 @@ static atp_status launch(atp_ctx *ctx, const std::vector<HostSeq> &seqs, int hea
         }
         if (b.count == 0) continue;
         ATP_KERNEL(ctx, "attn_tc", flops, bytes);
-        attn_tc_kernel<DH><<<dim3(b.total_tiles, heads), 192, C_::SMEM, ctx->stream>>>(b, heads, scale * 1.4426950408889634f, ctx->dev_status);
+        // drop the lo products of a key block when scale * |q|max * |k|max * 2^-8 <= 2^-10 (logit error bound)
+        const float lo_thresh = 0.25f / scale;
+        attn_tc_kernel<DH><<<dim3(b.total_tiles, heads), 192, C_::SMEM, ctx->stream>>>(b, heads, scale * 1.4426950408889634f, lo_thresh, ctx->dev_status);
         ATP_LAUNCHED(ctx);
     }
     return ATP_OK;
