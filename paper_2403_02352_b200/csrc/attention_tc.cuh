@@ -9,8 +9,9 @@
 // (Qh Kh + Qh Kl + Ql Kh): with logits of magnitude 10^2 a single bf16 rounding of Q or K' moves
 // the softmax by more than the accuracy bar, the split keeps ~16 mantissa bits. P and V' are bf16.
 // Operands are staged by TMA (128-byte swizzle): Q once, then per 128-key block K'_hi, K'_lo, V'
-// through a ring of tile slots. Warp 4 issues TMA, warp 5 issues the MMAs, warps 0-3 run softmax,
-// the O rescale (only when a row maximum grows by more than 2^8) and the final normalisation.
+// through a ring of tile slots. Warp 8 issues TMA, warp 9 issues the MMAs, warps 0-7 run softmax (two
+// threads per query row, each on 64 of the 128 keys of a block), the O rescale (only when a row maximum
+// grows by more than 2^8) and the final normalisation.
 // Every mbarrier wait is bounded; on expiry the kernel records ATP_ERR_TIMEOUT and winds down.
 #pragma once
 #include "gemm_tc.cuh"
@@ -53,29 +54,35 @@ __device__ __forceinline__ float fast_exp2(float x)
 template <int DH> struct Cfg {
     static constexpr int TILE = 128 * DH * 2;                   // one 128-row operand tile (bf16)
     static constexpr int NSLOT = (DH == 128) ? 3 : 6;           // K'_hi / K'_lo / V' tile slots
+    static constexpr int NPBUF = (DH == 128) ? 1 : 2;           // P buffers (shared memory allows two at d_h = 64)
     static constexpr int P_BYTES = 128 * 128 * 2;               // one P buffer
     static constexpr int OFF_Q = 0;                             // Q hi, Q lo
     static constexpr int OFF_SLOT = 2 * TILE;
-    static constexpr int OFF_P = OFF_SLOT + NSLOT * TILE;       // single P buffer (reused once its MMAs finished)
-    static constexpr int OFF_BAR = OFF_P + P_BYTES;
-    static constexpr int NBAR = 1 + 2 * NSLOT + 2 + 2 + 1 + 1 + 1;   // q, slot full/empty, s_full[2], s_free[2], p_full, p_free, o_done
-    static constexpr int SMEM = OFF_BAR + 8 * NBAR + 16 + 1024;
+    static constexpr int OFF_P = OFF_SLOT + NSLOT * TILE;
+    static constexpr int OFF_BAR = OFF_P + NPBUF * P_BYTES;
+    // q, slot full/empty, s_full[2], s_free[2], p_full[2], p_free[2], o_done, xchg
+    static constexpr int NBAR = 1 + 2 * NSLOT + 2 + 2 + 2 + 2 + 1 + 1;
+    static constexpr int OFF_XCH = OFF_BAR + 8 * NBAR + 16;     // float[2 parity][2 halves][128 rows]
+    static constexpr int SMEM = OFF_XCH + 2 * 2 * 128 * 4 + 1024;
 };
 
+// Warps 0-7: softmax (warp w and w + 4 share the TMEM lanes 32 (w & 3) .. and split the 128 keys of a
+// block in halves), warp 8: TMA, warp 9: MMA.
 template <int DH>
-__global__ void __launch_bounds__(192)
+__global__ void __launch_bounds__(320)
 attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e, float lo_thresh, int *dev_status)
 {
     using C_ = Cfg<DH>;
-    constexpr int NS = C_::NSLOT;
+    constexpr int NS = C_::NSLOT, NP = C_::NPBUF;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t *gbase = smem_raw + (base - raw);
     const uint32_t bar0 = base + C_::OFF_BAR;
     const uint32_t b_q = bar0, b_full = bar0 + 8, b_empty = b_full + 8 * NS, b_sfull = b_empty + 8 * NS, b_sfree = b_sfull + 16,
-                   b_pfull = b_sfree + 16, b_pfree = b_pfull + 8, b_odone = b_pfree + 8;
+                   b_pfull = b_sfree + 16, b_pfree = b_pfull + 16, b_odone = b_pfree + 16, b_xchg = b_odone + 8;
     uint32_t *tmem_slot = (uint32_t *)(gbase + C_::OFF_BAR + 8 * C_::NBAR);
+    float *xch = (float *)(gbase + C_::OFF_XCH);
     __shared__ int abort_flag;
 
     // work item: (sequence, query tile) from blockIdx.x, head from blockIdx.y
@@ -98,18 +105,20 @@ attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e
         mbar_init(b_q, 1);
         for (int s = 0; s < NS; ++s) { mbar_init(b_full + 8 * s, 1); mbar_init(b_empty + 8 * s, 1); }
         mbar_init(b_sfull, 1); mbar_init(b_sfull + 8, 1);
-        mbar_init(b_sfree, 4); mbar_init(b_sfree + 8, 4);
-        mbar_init(b_pfull, 4); mbar_init(b_pfree, 1); mbar_init(b_odone, 1);
+        mbar_init(b_sfree, 8); mbar_init(b_sfree + 8, 8);
+        mbar_init(b_pfull, 8); mbar_init(b_pfull + 8, 8);
+        mbar_init(b_pfree, 1); mbar_init(b_pfree + 8, 1);
+        mbar_init(b_odone, 1); mbar_init(b_xchg, 8);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 5) tmem_alloc(smem_u32(tmem_slot), 512);
+    if (warp == 9) tmem_alloc(smem_u32(tmem_slot), 512);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     const uint32_t t_s0 = tmem_base, t_o = tmem_base + 256;
 
-    if (warp == 4) {
+    if (warp == 8) {
         if (lane == 0) {
             mbar_expect_tx(b_q, 2 * C_::TILE);
 #pragma unroll
@@ -131,14 +140,14 @@ attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e
                 }
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == 9) {
         if (lane == 0) {
             constexpr uint32_t idesc_s = instr_desc(128, 128, false, false);
             constexpr uint32_t idesc_o = instr_desc(128, DH, false, true);
             const uint32_t q_hi = base + C_::OFF_Q, q_lo = q_hi + C_::TILE;
             bool ok = mbar_wait(b_q, 0, &abort_flag);
             tc_fence_after();
-            // S_j for block j into buffer j & 1: Qh Kh^T + Qh Kl^T + Ql Kh^T
+            // S_j for block j into buffer j & 1: Qh Kh^T (+ Qh Kl^T + Ql Kh^T)
             auto issue_s = [&](int j) -> bool {
                 const int lk = 3 * j, sh = lk % NS, sl = (lk + 1) % NS;
                 const bool need_lo = qm * km[j] > lo_thresh;
@@ -168,11 +177,11 @@ attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e
             for (int j = 0; j < nblk && ok; ++j) {
                 if (j + 1 < nblk) { ok = issue_s(j + 1); if (!ok) break; }
                 // O += P_j V_j
-                const int lv = 3 * j + 2, sv = lv % NS;
+                const int lv = 3 * j + 2, sv = lv % NS, pb = j % NP, pu = j / NP;
                 if (!mbar_wait(b_full + 8 * sv, (lv / NS) & 1, &abort_flag)) { ok = false; break; }
-                if (!mbar_wait(b_pfull, j & 1, &abort_flag)) { ok = false; break; }
+                if (!mbar_wait(b_pfull + 8 * pb, pu & 1, &abort_flag)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t pv = base + C_::OFF_P, vv = base + C_::OFF_SLOT + sv * C_::TILE;
+                const uint32_t pv = base + C_::OFF_P + pb * C_::P_BYTES, vv = base + C_::OFF_SLOT + sv * C_::TILE;
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk) {
                     const uint64_t ap = smem_desc(pv + (kk >> 2) * 16384 + (kk & 3) * 32, 16, 1024);
@@ -180,79 +189,84 @@ attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e
                     umma_bf16(t_o, ap, bv, idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
                 }
                 umma_commit(b_empty + 8 * sv);
-                umma_commit(b_pfree);
+                umma_commit(b_pfree + 8 * pb);
                 umma_commit(b_odone);
             }
         }
     } else {
-        // softmax / correction / epilogue: thread = query row, TMEM lane = warp * 32 + lane
-        const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
-        const int row = warp * 32 + lane;
+        // softmax / correction / epilogue: thread = (query row, half of the keys of a block)
+        const int quad = warp & 3, half = warp >> 2;
+        const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+        const int row = quad * 32 + lane;
+        constexpr int OC = DH / 2;                                   // O columns owned by this thread
         float m_used = -INFINITY, l_sum = 0.f;
         bool ok = true;
+        int ok_i = 0;
+        auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {   // lane 0 polls, the warp follows
+            if (lane == 0) ok_i = mbar_wait(bar, parity, &abort_flag) ? 1 : 0;
+            return __shfl_sync(0xffffffffu, ok_i, 0) != 0;
+        };
         for (int j = 0; j < nblk; ++j) {
-            int ok_i = 0;
-            if (lane == 0) ok_i = mbar_wait(b_sfull + 8 * (j & 1), (j >> 1) & 1, &abort_flag) ? 1 : 0;
-            ok = __shfl_sync(0xffffffffu, ok_i, 0) != 0;
+            ok = wait_all(b_sfull + 8 * (j & 1), (j >> 1) & 1);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t t_s = t_s0 + 128 * (j & 1) + lane_addr;
-            const int kvalid = sq.r - j * 128;                 // keys of this block that exist
-            // pass A: block maximum of the raw scores (the scale is positive: applied once at the end)
+            const uint32_t t_s = t_s0 + 128 * (j & 1) + lane_addr + half * 64;
+            const int kvalid = sq.r - j * 128 - half * 64;            // keys of this half-block that exist
+            // pass A: maximum of the raw scores of this half (the scale is positive: applied once)
             float mx = -INFINITY;
-            if (kvalid >= 128) {
-#pragma unroll 1
-                for (int c = 0; c < 128; c += 32) {
-                    uint32_t rr[32];
-                    tmem_ld32(t_s + c, rr);
+#pragma unroll
+            for (int c = 0; c < 64; c += 32) {
+                uint32_t rr[32];
+                tmem_ld32(t_s + c, rr);
+                if (kvalid >= 64) {
 #pragma unroll
                     for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(rr[i]));
-                }
-            } else {
-#pragma unroll 1
-                for (int c = 0; c < 128; c += 32) {
-                    uint32_t rr[32];
-                    tmem_ld32(t_s + c, rr);
+                } else {
 #pragma unroll
                     for (int i = 0; i < 32; ++i)
                         if (c + i < kvalid) mx = fmaxf(mx, __uint_as_float(rr[i]));
                 }
             }
-            mx *= scale_log2e;
+            // exchange with the thread that holds the other half of the row
+            float *xb = xch + (j & 1) * 256;
+            xb[half * 128 + row] = mx;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(b_xchg);
+            ok = wait_all(b_xchg, j & 1);
+            if (!ok) break;
+            mx = fmaxf(mx, xb[(half ^ 1) * 128 + row]) * scale_log2e;
             // the exponent offset only moves when the maximum grew by more than 8 (factor 256)
             float alpha = 1.f;
             bool grow = (mx > m_used + 8.f) || (j == 0);
             if (grow) { alpha = (j == 0) ? 0.f : fast_exp2(m_used - mx); m_used = mx; }
             if (j > 0 && __any_sync(0xffffffffu, grow)) {
                 // O must be quiescent: P V of block j-1 done (block j's waits for the P written below)
-                if (lane == 0) ok_i = mbar_wait(b_odone, (j - 1) & 1, &abort_flag) ? 1 : 0;
-                ok = __shfl_sync(0xffffffffu, ok_i, 0) != 0;
+                ok = wait_all(b_odone, (j - 1) & 1);
                 if (!ok) break;
                 tc_fence_after();
-#pragma unroll 1
-                for (int c = 0; c < DH; c += 32) {
+#pragma unroll
+                for (int c = 0; c < OC; c += 32) {
                     uint32_t rr[32];
-                    tmem_ld32(t_o + lane_addr + c, rr);
+                    tmem_ld32(t_o + lane_addr + half * OC + c, rr);
 #pragma unroll
                     for (int i = 0; i < 32; ++i) rr[i] = __float_as_uint(__uint_as_float(rr[i]) * alpha);
-                    tmem_st32(t_o + lane_addr + c, rr);
+                    tmem_st32(t_o + lane_addr + half * OC + c, rr);
                 }
                 tc_fence_before();
             }
             l_sum *= alpha;
-            // the single P buffer is free once the value MMAs of block j-1 have read it
-            if (j > 0) {
-                if (lane == 0) ok_i = mbar_wait(b_pfree, (j - 1) & 1, &abort_flag) ? 1 : 0;
-                ok = __shfl_sync(0xffffffffu, ok_i, 0) != 0;
+            // the P buffer is free once the value MMAs that read it (block j - NP) have finished
+            const int pb = j % NP, pu = j / NP;
+            if (pu > 0) {
+                ok = wait_all(b_pfree + 8 * pb, (pu - 1) & 1);
                 if (!ok) break;
             }
-            // pass B: P = exp2(s * c - m) as bf16 into the swizzled K-major A tile; the row sum is taken
-            // from the unrounded values (the bf16 rounding of P averages out over the r keys)
-            uint8_t *prow = gbase + C_::OFF_P + row * 128;
+            // pass B: P = exp2(s * c - m) as bf16 into the swizzled K-major A tile (this half = one 64-key
+            // region); the row sum is taken from the unrounded values
+            uint8_t *prow = gbase + C_::OFF_P + pb * C_::P_BYTES + half * 16384 + row * 128;
             const float neg_m = -m_used;
-            const bool full = kvalid >= 128;
-#pragma unroll 1
-            for (int c = 0; c < 128; c += 32) {
+#pragma unroll
+            for (int c = 0; c < 64; c += 32) {
                 uint32_t rr[32];
                 tmem_ld32(t_s + c, rr);
                 uint32_t packed[16];
@@ -260,7 +274,7 @@ attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e
                 for (int i = 0; i < 32; i += 2) {
                     float p0 = fast_exp2(fmaf(__uint_as_float(rr[i]), scale_log2e, neg_m));
                     float p1 = fast_exp2(fmaf(__uint_as_float(rr[i + 1]), scale_log2e, neg_m));
-                    if (!full) {
+                    if (kvalid < 64) {
                         if (c + i >= kvalid) p0 = 0.f;
                         if (c + i + 1 >= kvalid) p1 = 0.f;
                     }
@@ -270,30 +284,35 @@ attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e
                 }
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {                           // four 16-byte chunks of 8 keys
-                    const int chunk16 = (c >> 3) + q;                   // 0..15 along the 128 keys
-                    const int region = chunk16 >> 3, within = chunk16 & 7;
+                    const int within = (c >> 3) + q;                    // 0..7 inside the 64-key region
                     uint4 val = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
-                    *(uint4 *)(prow + region * 16384 + ((within ^ (row & 7)) << 4)) = val;
+                    *(uint4 *)(prow + ((within ^ (row & 7)) << 4)) = val;
                 }
             }
             tc_fence_before();
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA
             __syncwarp();
-            if (lane == 0) { mbar_arrive(b_sfree + 8 * (j & 1)); mbar_arrive(b_pfull); }
+            if (lane == 0) { mbar_arrive(b_sfree + 8 * (j & 1)); mbar_arrive(b_pfull + 8 * pb); }
         }
-        // epilogue: O / l
-        int ok_i = 0;
-        if (ok && lane == 0) ok_i = mbar_wait(b_odone, (nblk - 1) & 1, &abort_flag) ? 1 : 0;
-        ok = ok && (__shfl_sync(0xffffffffu, ok_i, 0) != 0);
+        // epilogue: O / l, with l summed over the two halves of the row
+        if (ok) {
+            float *xb = xch + (nblk & 1) * 256;
+            xb[half * 128 + row] = l_sum;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(b_xchg);
+            ok = wait_all(b_xchg, nblk & 1);
+            if (ok) l_sum += xb[(half ^ 1) * 128 + row];
+        }
+        if (ok) ok = wait_all(b_odone, (nblk - 1) & 1);
         tc_fence_after();
         if (ok) {
             const float inv = 1.f / l_sum;
             const int grow_ = q0 + row;
-            __nv_bfloat16 *dst = (__nv_bfloat16 *)sq.O + (size_t)grow_ * sq.ldo + col0;
-#pragma unroll 1
-            for (int c = 0; c < DH; c += 32) {
+            __nv_bfloat16 *dst = (__nv_bfloat16 *)sq.O + (size_t)grow_ * sq.ldo + col0 + half * OC;
+#pragma unroll
+            for (int c = 0; c < OC; c += 32) {
                 uint32_t rr[32];
-                tmem_ld32(t_o + lane_addr + c, rr);
+                tmem_ld32(t_o + lane_addr + half * OC + c, rr);
                 if (grow_ < sq.L) {
 #pragma unroll
                     for (int i = 0; i < 32; i += 8) {
@@ -310,7 +329,7 @@ attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e
     tc_fence_before();
     __syncthreads();
     if (threadIdx.x == 0 && abort_flag && dev_status) raise_status(dev_status, ATP_ERR_TIMEOUT);
-    if (warp == 5) {
+    if (warp == 9) {
         tc_fence_after();
         tmem_dealloc(tmem_base, 512);
     }
@@ -384,7 +403,7 @@ static atp_status launch(atp_ctx *ctx, const std::vector<HostSeq> &seqs, int hea
         ATP_KERNEL(ctx, "attn_tc", flops, bytes);
         // drop the lo products of a key block when scale * |q|max * |k|max * 2^-8 <= 2^-10 (logit error bound)
         const float lo_thresh = 0.25f / scale;
-        attn_tc_kernel<DH><<<dim3(b.total_tiles, heads), 192, C_::SMEM, ctx->stream>>>(b, heads, scale * 1.4426950408889634f, lo_thresh, ctx->dev_status);
+        attn_tc_kernel<DH><<<dim3(b.total_tiles, heads), 320, C_::SMEM, ctx->stream>>>(b, heads, scale * 1.4426950408889634f, lo_thresh, ctx->dev_status);
         ATP_LAUNCHED(ctx);
     }
     return ATP_OK;
