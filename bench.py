@@ -158,20 +158,17 @@ def main():
         return run_reference(args)
 
     import torch
-    import torch.distributed as dist
     import paper_2403_02352_b200 as atp          # raises if libatp.so is missing: no fallback
     from paper_2403_02352_b200.layer import AtpLayer
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2403_02352_b200 import dist as pdist
+    world, rank, local = pdist.env_ranks()
     torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     dev = torch.device("cuda", local)
+    pdist.init("nccl", dev)
     args.warmup = max(args.warmup, 3)
 
-    w = WORKLOADS[args.workload]["build"](args.rank, args.seed + 17 * rank)   # every rank: its own sequences
+    w = WORKLOADS[args.workload]["build"](args.rank, pdist.rank_seed(args.seed, rank))   # every rank: its own sequences
     tdt = torch.float32 if w.dtype == "f32" else torch.bfloat16
 
     def dev_mat(a, pin=False):
@@ -209,8 +206,7 @@ def main():
 
     def barrier():
         torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
+        pdist.barrier()
         torch.cuda.synchronize()
 
     # ---- device-timed region: K steps, CUDA events per step, L2 flushed between steps
@@ -229,12 +225,8 @@ def main():
     clocks = sampler.stop() if sampler else None
     launches = (ctx.launches - launches0)
     ctx.poll()
-    ms = sum(a.elapsed_time(b) for a, b in evs)
-    if world > 1:
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    value = world * tokens * args.steps / (ms / 1e3)
+    ms = pdist.max_over_ranks(sum(a.elapsed_time(b) for a, b in evs), dev)
+    value = pdist.aggregate_tokens_per_s(tokens, args.steps, ms, world)
 
     # ---- end to end: pinned host input -> device, layer, result -> host, every step
     xd = torch.empty_like(Xsets[0])
@@ -248,17 +240,12 @@ def main():
         Yhost.copy_(yy, non_blocking=True)
         e2e_ev[i][1].record()
     barrier()
-    ms_e2e = sum(a.elapsed_time(b) for a, b in e2e_ev)
-    if world > 1:
-        t = torch.tensor([ms_e2e], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
-    e2e = {"value": world * tokens * args.steps / (ms_e2e / 1e3), "unit": "tokens/s",
+    ms_e2e = pdist.max_over_ranks(sum(a.elapsed_time(b) for a, b in e2e_ev), dev)
+    e2e = {"value": pdist.aggregate_tokens_per_s(tokens, args.steps, ms_e2e, world), "unit": "tokens/s",
            "h2d_bytes_per_step": int(x_bytes), "d2h_bytes_per_step": int(Yhost.numel() * Yhost.element_size())}
 
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
+        pdist.finish()
         return
 
     # ---- per-kernel times (event pair around every launch; separate pass, not the timed one)
@@ -310,8 +297,7 @@ def main():
             "config": workload_config(w, world),
             "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+    pdist.finish()
 
 
 if __name__ == "__main__":
