@@ -965,7 +965,9 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
             const int npairs = maxnb / 2;
             const int blk = 2 * jbj;
             const size_t ash = jbj == 32 ? JAC2_APPLY_SMEM(64) : JAC2_APPLY_SMEM(32);
+            const size_t lsh = jbj == 32 ? JAC2_LOCAL_SMEM(64) : JAC2_LOCAL_SMEM(32);
             if (jbj == 32) ATP_CUDA_OK(ctx, cudaFuncSetAttribute(jac2_apply_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ash));
+            if (jbj == 32) ATP_CUDA_OK(ctx, cudaFuncSetAttribute(jac2_local_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lsh));
             for (int pass = 0; pass < 2; ++pass) {
                 if ((st = launch_gemm_simt<float, float, float, true, false>(ctx, gg, store)) != ATP_OK) return st;
                 ATP_KERNEL(ctx, "jac2_init", 0, 0);
@@ -989,8 +991,8 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
                         // algorithmic work of a step when every pair rotates (converged pairs skip it)
                         const double nseq = cnt, bl = blk;
                         ATP_KERNEL(ctx, "jac2_local", nseq * npairs * jinner * (bl - 1) * (bl * bl * 6.0 + bl * bl * 3.0), 0);
-                        if (jbj == 32) jac2_local_kernel<32><<<dim3(npairs, cnt), 1024, 0, ctx->stream>>>(jb, step, tolr, jinner);
-                        else jac2_local_kernel<16><<<dim3(npairs, cnt), 512, 0, ctx->stream>>>(jb, step, tolr, jinner);
+                        if (jbj == 32) jac2_local_kernel<32><<<dim3(npairs, cnt), 1024, lsh, ctx->stream>>>(jb, step, tolr, jinner);
+                        else jac2_local_kernel<16><<<dim3(npairs, cnt), 256, lsh, ctx->stream>>>(jb, step, tolr, jinner);
                         ATP_LAUNCHED(ctx);
                         ATP_KERNEL(ctx, "jac2_apply", nseq * npairs * (npairs * 4.0 + ceil_div(maxrt, blk) * 2.0) * bl * bl * bl,
                                    nseq * npairs * (npairs * 2.0 + ceil_div(maxrt, blk) * 2.0) * bl * bl * 4.0);

@@ -40,15 +40,37 @@ __global__ void jac2_init_kernel(const __grid_constant__ Jac2Batch batch)
     if (blockIdx.x == 0 && threadIdx.x == 0) { *sq.maxoff = 0u; *sq.conv = 0; }
 }
 
-// BJ2: block height (16 or 32); the local problem is BLK x BLK with BLK = 2 BJ2, solved by 16 BLK threads.
-// The sweep is a chain of BLK - 1 dependent rotation steps, so the time of a step is the length of one
-// thread's instruction chain: every thread updates at most one 2x2 block of A and a few pairs of V.
+// Rotation (c, s) that annihilates the (p, q) entry of a symmetric matrix; identity when the entry is
+// already small against its diagonal. Fast reciprocal / rsqrt: c^2 + s^2 = 1 to ~2 ulp, ample for a
+// basis stored in bf16.
+__device__ __forceinline__ float2 jac2_rotation(float gpp, float gqq, float gpq, float tol_rot, bool &did)
+{
+    float c = 1.f, s = 0.f;
+    if (gpq != 0.f && gpq * gpq > tol_rot * tol_rot * fmaxf(gpp, 0.f) * fmaxf(gqq, 0.f)) {
+        float zeta = __fdividef(gqq - gpp, 2.f * gpq);
+        float az = fabsf(zeta), t;
+        if (az > 1e15f) t = __fdividef(0.5f, zeta);
+        else { float h = 1.f + zeta * zeta; t = __fdividef(copysignf(1.f, zeta), az + h * rsqrtf(h)); }
+        c = rsqrtf(1.f + t * t);
+        s = c * t;
+        did = true;
+    }
+    return make_float2(c, s);
+}
+
+// BJ2: block height (16 or 32); the local problem is BLK x BLK with BLK = 2 BJ2, solved by (BLK/2)^2
+// threads. The sweep is a chain of BLK - 1 dependent rotation steps, so the time of a step is the
+// length of one thread's instruction chain plus ONE block barrier: thread (a, b) owns, in every step,
+// the 2x2 block (rows of pair a, columns of pair b) of A and the two column pairs {2b, 2b+1} of the rows
+// of pair a of V. It derives the two rotations it needs (pair a, pair b) itself from the previous step's
+// A (all threads that need a rotation compute the same values from the same inputs), reads A from one
+// buffer and writes the other.
+#define JAC2_LOCAL_SMEM(BLK) ((size_t)(3 * (BLK) * ((BLK) + 1)) * sizeof(float))
 template <int BJ2>
-__global__ void __launch_bounds__(BJ2 * 32)
+__global__ void __launch_bounds__(BJ2 * BJ2)
 jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_rot, int max_inner)
 {
-    constexpr int BLK = 2 * BJ2, NT = BLK * 16, HP = BLK / 2;
-    constexpr int VPT = HP * BLK / NT;                 // V pair-elements per thread (1 or 2)
+    constexpr int BLK = 2 * BJ2, HP = BLK / 2, NT = HP * HP;
     const Jac2Seq &sq = batch.s[blockIdx.y];
     if (*sq.conv) return;
     const int npairs = sq.nb / 2;
@@ -56,10 +78,9 @@ jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_r
     if (pair >= npairs) return;
     int I, J;
     rr_pair2(sq.nb, step % (sq.nb - 1), pair, I, J);
-    __shared__ float A[BLK][BLK + 1];
-    __shared__ float V[BLK][BLK + 1];
-    __shared__ float2 cs[HP];
-    __shared__ uchar2 pq[HP];
+    extern __shared__ __align__(16) float j2l[];       // JAC2_LOCAL_SMEM(BLK) bytes
+    float (*Ab)[BLK][BLK + 1] = (float (*)[BLK][BLK + 1])j2l;                     // two copies of A
+    float (*V)[BLK + 1] = (float (*)[BLK + 1])(j2l + 2 * BLK * (BLK + 1));
     __shared__ float red[NT / 32];
     __shared__ int rotated;
     __shared__ uchar2 sched[BLK - 1][HP];              // round-robin schedule of the local sweep
@@ -72,16 +93,17 @@ jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_r
     for (int e = tid; e < BLK * BLK; e += NT) {
         int i = e / BLK, j = e % BLK;
         int gi = jac2_row<BJ2>(I, J, i, sq.rt), gj = jac2_row<BJ2>(I, J, j, sq.rt);
-        A[i][j] = (gi >= 0 && gj >= 0) ? sq.G[(size_t)gi * sq.rt + gj] : 0.f;
+        Ab[0][i][j] = (gi >= 0 && gj >= 0) ? sq.G[(size_t)gi * sq.rt + gj] : 0.f;
         V[i][j] = (i == j) ? 1.f : 0.f;
     }
+    if (tid == 0) rotated = 0;
     __syncthreads();
     float mo = 0.f;
     for (int e = tid; e < BLK * BLK; e += NT) {
         int i = e / BLK, j = e % BLK;
         if (i != j) {
-            float den = sqrtf(fmaxf(A[i][i], 0.f) * fmaxf(A[j][j], 0.f));
-            if (den > 0.f) mo = fmaxf(mo, fabsf(A[i][j]) / den);
+            float den = sqrtf(fmaxf(Ab[0][i][i], 0.f) * fmaxf(Ab[0][j][j], 0.f));
+            if (den > 0.f) mo = fmaxf(mo, fabsf(Ab[0][i][j]) / den);
         }
     }
 #pragma unroll
@@ -96,61 +118,39 @@ jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_r
         if (tid == 0) sq.vflag[pair] = 0;
         return;
     }
-    const bool has_block = tid < HP * HP;
     const int ba = tid / HP, bb = tid % HP;            // 2x2 block (pair ba rows, pair bb columns)
+    int cur = 0;
     for (int sweep = 0; sweep < max_inner; ++sweep) {
-        if (tid == 0) rotated = 0;
-        __syncthreads();
         for (int st = 0; st < BLK - 1; ++st) {
-            if (tid < HP) {
-                const uchar2 pr_ = sched[st][tid];
-                const int p = pr_.x, q = pr_.y;
-                float gpp = A[p][p], gqq = A[q][q], gpq = A[p][q];
-                float c = 1.f, s = 0.f;
-                // fast reciprocal / rsqrt: c^2 + s^2 = 1 to ~2 ulp, ample for a basis stored in bf16
-                if (gpq != 0.f && gpq * gpq > tol_rot * tol_rot * fmaxf(gpp, 0.f) * fmaxf(gqq, 0.f)) {
-                    float zeta = __fdividef(gqq - gpp, 2.f * gpq);
-                    float az = fabsf(zeta), t;
-                    if (az > 1e15f) t = __fdividef(0.5f, zeta);
-                    else { float h = 1.f + zeta * zeta; t = __fdividef(copysignf(1.f, zeta), az + h * rsqrtf(h)); }
-                    c = rsqrtf(1.f + t * t);
-                    s = c * t;
-                    rotated = 1;
-                }
-                cs[tid] = make_float2(c, s);
-                pq[tid] = pr_;
-            }
-            __syncthreads();
+            const float (*Ao)[BLK + 1] = Ab[cur];
+            float (*An)[BLK + 1] = Ab[cur ^ 1];
+            const uchar2 ra = sched[st][ba], rb = sched[st][bb];
             // loads of this step first (independent), then the arithmetic, then the stores
-            float g00 = 0.f, g01 = 0.f, g10 = 0.f, g11 = 0.f;
-            uchar2 ra = make_uchar2(0, 0), rb = make_uchar2(0, 0);
-            float2 ca = make_float2(1.f, 0.f), cb = ca;
-            if (has_block) {
-                ra = pq[ba]; rb = pq[bb]; ca = cs[ba]; cb = cs[bb];
-                g00 = A[ra.x][rb.x]; g01 = A[ra.x][rb.y]; g10 = A[ra.y][rb.x]; g11 = A[ra.y][rb.y];
-            }
-            float vx[VPT], vy[VPT]; uchar2 rv[VPT]; float2 cv[VPT]; int vc[VPT];
-#pragma unroll
-            for (int it = 0; it < VPT; ++it) {
-                const int idx = tid + it * NT;
-                rv[it] = pq[idx / BLK]; cv[it] = cs[idx / BLK]; vc[it] = idx % BLK;
-                vx[it] = V[rv[it].x][vc[it]]; vy[it] = V[rv[it].y][vc[it]];
-            }
-            if (has_block) {
-                float r00 = ca.x * g00 - ca.y * g10, r01 = ca.x * g01 - ca.y * g11;
-                float r10 = ca.y * g00 + ca.x * g10, r11 = ca.y * g01 + ca.x * g11;
-                A[ra.x][rb.x] = cb.x * r00 - cb.y * r01; A[ra.x][rb.y] = cb.y * r00 + cb.x * r01;
-                A[ra.y][rb.x] = cb.x * r10 - cb.y * r11; A[ra.y][rb.y] = cb.y * r10 + cb.x * r11;
-            }
-#pragma unroll
-            for (int it = 0; it < VPT; ++it) {
-                V[rv[it].x][vc[it]] = cv[it].x * vx[it] - cv[it].y * vy[it];
-                V[rv[it].y][vc[it]] = cv[it].y * vx[it] + cv[it].x * vy[it];
-            }
+            const float app = Ao[ra.x][ra.x], aqq = Ao[ra.y][ra.y], apq = Ao[ra.x][ra.y];
+            const float bpp = Ao[rb.x][rb.x], bqq = Ao[rb.y][rb.y], bpq = Ao[rb.x][rb.y];
+            const float g00 = Ao[ra.x][rb.x], g01 = Ao[ra.x][rb.y], g10 = Ao[ra.y][rb.x], g11 = Ao[ra.y][rb.y];
+            const int vc = 2 * bb;
+            const float v00 = V[ra.x][vc], v01 = V[ra.x][vc + 1], v10 = V[ra.y][vc], v11 = V[ra.y][vc + 1];
+            bool did = false;
+            const float2 ca = jac2_rotation(app, aqq, apq, tol_rot, did);
+            const float2 cb = jac2_rotation(bpp, bqq, bpq, tol_rot, did);
+            const float r00 = ca.x * g00 - ca.y * g10, r01 = ca.x * g01 - ca.y * g11;
+            const float r10 = ca.y * g00 + ca.x * g10, r11 = ca.y * g01 + ca.x * g11;
+            An[ra.x][rb.x] = cb.x * r00 - cb.y * r01; An[ra.x][rb.y] = cb.y * r00 + cb.x * r01;
+            An[ra.y][rb.x] = cb.x * r10 - cb.y * r11; An[ra.y][rb.y] = cb.y * r10 + cb.x * r11;
+            V[ra.x][vc] = ca.x * v00 - ca.y * v10; V[ra.x][vc + 1] = ca.x * v01 - ca.y * v11;
+            V[ra.y][vc] = ca.y * v00 + ca.x * v10; V[ra.y][vc + 1] = ca.y * v01 + ca.x * v11;
+            if (did && max_inner > 1) rotated = 1;
+            cur ^= 1;
             __syncthreads();
         }
-        if (!rotated) break;
-        __syncthreads();
+        if (max_inner > 1) {
+            const int any = rotated;
+            __syncthreads();
+            if (!any) break;
+            if (tid == 0) rotated = 0;
+            __syncthreads();
+        }
     }
     float *dst = sq.Vbuf + (size_t)pair * BLK * BLK;
     for (int e = tid; e < BLK * BLK; e += NT) dst[e] = V[e / BLK][e % BLK];
