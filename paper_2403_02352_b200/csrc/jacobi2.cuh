@@ -3,7 +3,7 @@
 // (Rayleigh-Ritz step of the basis extraction, Sec. 4.2: X' = [sigma_i v_i]).
 // Blocks of 16 rows; a step handles r~/32 disjoint pairs (round-robin order) with two launches:
 //   jac2_local : per pair, the 32x32 diagonal block is diagonalised on chip (cyclic Jacobi), the
-//                accumulated row operations Vt are published;
+//                accumulated row operations Vt are published (stored transposed);
 //   jac2_apply : every 32x32 block (p, q) becomes Vt_p G_pq Vt_q^T, rows of Wt become Vt_p Wt.
 // G entries carry errors relative to the norms of the rows of B they come from (B is graded by the
 // QR-ordered range basis), which is what Jacobi needs to resolve small eigenvalues next to large ones.
@@ -102,8 +102,8 @@ jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_r
     for (int e = tid; e < BLK * BLK; e += NT) {
         int i = e / BLK, j = e % BLK;
         if (i != j) {
-            float den = sqrtf(fmaxf(Ab[0][i][i], 0.f) * fmaxf(Ab[0][j][j], 0.f));
-            if (den > 0.f) mo = fmaxf(mo, fabsf(Ab[0][i][j]) / den);
+            const float dd = fmaxf(Ab[0][i][i], 0.f) * fmaxf(Ab[0][j][j], 0.f);
+            if (dd > 0.f) mo = fmaxf(mo, fabsf(Ab[0][i][j]) * rsqrtf(dd));
         }
     }
 #pragma unroll
@@ -126,14 +126,16 @@ jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_r
             float (*An)[BLK + 1] = Ab[cur ^ 1];
             const uchar2 ra = sched[st][ba], rb = sched[st][bb];
             // loads of this step first (independent), then the arithmetic, then the stores
-            const float app = Ao[ra.x][ra.x], aqq = Ao[ra.y][ra.y], apq = Ao[ra.x][ra.y];
             const float bpp = Ao[rb.x][rb.x], bqq = Ao[rb.y][rb.y], bpq = Ao[rb.x][rb.y];
             const float g00 = Ao[ra.x][rb.x], g01 = Ao[ra.x][rb.y], g10 = Ao[ra.y][rb.x], g11 = Ao[ra.y][rb.y];
             const int vc = 2 * bb;
             const float v00 = V[ra.x][vc], v01 = V[ra.x][vc + 1], v10 = V[ra.y][vc], v11 = V[ra.y][vc + 1];
             bool did = false;
-            const float2 ca = jac2_rotation(app, aqq, apq, tol_rot, did);
+            // lane l derives the rotation of pair l mod HP (its column pair); the row pair's comes by shuffle
             const float2 cb = jac2_rotation(bpp, bqq, bpq, tol_rot, did);
+            float2 ca;
+            ca.x = __shfl_sync(0xffffffffu, cb.x, ba & 31);
+            ca.y = __shfl_sync(0xffffffffu, cb.y, ba & 31);
             const float r00 = ca.x * g00 - ca.y * g10, r01 = ca.x * g01 - ca.y * g11;
             const float r10 = ca.y * g00 + ca.x * g10, r11 = ca.y * g01 + ca.x * g11;
             An[ra.x][rb.x] = cb.x * r00 - cb.y * r01; An[ra.x][rb.y] = cb.y * r00 + cb.x * r01;
@@ -153,19 +155,21 @@ jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_r
         }
     }
     float *dst = sq.Vbuf + (size_t)pair * BLK * BLK;
-    for (int e = tid; e < BLK * BLK; e += NT) dst[e] = V[e / BLK][e % BLK];
+    for (int e = tid; e < BLK * BLK; e += NT) dst[e] = V[e % BLK][e / BLK];   // transposed: what jac2_apply reads
     if (tid == 0) sq.vflag[pair] = 1;
 }
 
 // grid: (npairs + ceil(rt/BLK), npairs, batch); dynamic shared memory: JAC2_APPLY_SMEM(BLK) bytes.
 // G is symmetric: only blocks (p, q) with q >= p are computed, the mirror block is written from the
-// transposed result. Each thread owns an MR x 4 register tile of the BLK x BLK block.
-#define JAC2_APPLY_SMEM(BLK) ((size_t)(2 * (BLK) * ((BLK) + 1) + 2 * (BLK) * ((BLK) + 4)) * sizeof(float))
+// transposed register tile. Each thread owns a 4 x 4 tile of the BLK x BLK block; every shared-memory
+// operand is read as one 16-byte vector per 16 multiply-adds, and when the row length of G is a multiple
+// of four the global traffic is 16-byte vectors too (the 16 or 32 columns of a block are contiguous).
+#define JAC2_APPLY_SMEM(BLK) ((size_t)(4 * (BLK) * ((BLK) + 4)) * sizeof(float))
 template <int BJ2>
-__global__ void __launch_bounds__(BJ2 * 8)
+__global__ void __launch_bounds__(BJ2 * BJ2 / 4)
 jac2_apply_kernel(const __grid_constant__ Jac2Batch batch, int step)
 {
-    constexpr int BLK = 2 * BJ2, NT = BLK * 4, MR = BLK / 16, LD = BLK + 1, LD4 = BLK + 4;
+    constexpr int BLK = 2 * BJ2, NT = BLK * BLK / 16, LD4 = BLK + 4, Q = BLK / 4;   // Q: 4-vectors per row
     const Jac2Seq &sq = batch.s[blockIdx.z];
     if (*sq.conv) return;
     const int npairs = sq.nb / 2;
@@ -178,85 +182,121 @@ jac2_apply_kernel(const __grid_constant__ Jac2Batch batch, int step)
     const int fq = gblock ? sq.vflag[q] : 0;
     if (gblock ? (!fp && !fq) : !fp) return;
     const int tid = threadIdx.x;
+    const int rt = sq.rt;
+    const bool vec = (rt & 3) == 0;
     extern __shared__ __align__(16) float j2sm[];
-    float *Vp = j2sm;                       // [BLK][LD]   Vp[r][k]
-    float *Tm = Vp + BLK * LD;              // [BLK][LD]   T[r][k]
-    float *Bk = Tm + BLK * LD;              // [BLK][LD4]  B[k][c]
-    float *VqT = Bk + BLK * LD4;            // [BLK][LD4]  Vq^T[k][c] = Vq[c][k]
+    float *VpT = j2sm;                      // [BLK][LD4]  VpT[k][r] = Vt_p[r][k]
+    float *TmT = VpT + BLK * LD4;           // [BLK][LD4]  TmT[k][r] = T[r][k]
+    float *Bk = TmT + BLK * LD4;            // [BLK][LD4]  B[k][c]
+    float *VqT = Bk + BLK * LD4;            // [BLK][LD4]  VqT[k][c] = Vt_q[c][k]
     int Ip, Jp, Iq = 0, Jq = 0;
     rr_pair2(sq.nb, step % (sq.nb - 1), p, Ip, Jp);
-    const int r0 = (tid / (BLK / 4)) * MR, c0 = (tid % (BLK / 4)) * 4;
     const int cb = gblock ? 0 : ((int)blockIdx.x - npairs) * BLK;
-    if (!gblock && cb >= sq.rt) return;
+    if (!gblock && cb >= rt) return;
     if (gblock) rr_pair2(sq.nb, step % (sq.nb - 1), q, Iq, Jq);
-    for (int e = tid; e < BLK * BLK; e += NT) {
-        int i = e / BLK, j = e % BLK;
-        Vp[i * LD + j] = fp ? sq.Vbuf[(size_t)p * BLK * BLK + e] : (i == j ? 1.f : 0.f);
-        int gi = jac2_row<BJ2>(Ip, Jp, i, sq.rt);
+    // global column of local column c (a multiple of 4): the 4-vector starting there is contiguous
+    auto gcol = [&](int c) -> int { return gblock ? ((c < BJ2) ? Iq * BJ2 + c : Jq * BJ2 + (c - BJ2)) : cb + c; };
+    auto grow = [&](int r) -> int { return (r < BJ2) ? Ip * BJ2 + r : Jp * BJ2 + (r - BJ2); };
+    const float *src_b = gblock ? sq.G : sq.Wt;
+    const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int f = tid; f < BLK * Q; f += NT) {
+        const int i = f / Q, c = (f % Q) * 4;
+        // the published rotations are stored transposed: element (k, r) of the copy is Vt[r][k]
+        float4 vp = fp ? *(const float4 *)(sq.Vbuf + (size_t)p * BLK * BLK + i * BLK + c)
+                       : make_float4(i == c ? 1.f : 0.f, i == c + 1 ? 1.f : 0.f, i == c + 2 ? 1.f : 0.f, i == c + 3 ? 1.f : 0.f);
+        *(float4 *)&VpT[i * LD4 + c] = vp;
         if (gblock) {
-            VqT[j * LD4 + i] = fq ? sq.Vbuf[(size_t)q * BLK * BLK + e] : (i == j ? 1.f : 0.f);
-            int gj = jac2_row<BJ2>(Iq, Jq, j, sq.rt);
-            Bk[i * LD4 + j] = (gi >= 0 && gj >= 0) ? sq.G[(size_t)gi * sq.rt + gj] : 0.f;
-        } else {
-            Bk[i * LD4 + j] = (gi >= 0 && cb + j < sq.rt) ? sq.Wt[(size_t)gi * sq.rt + cb + j] : 0.f;
+            float4 vq = fq ? *(const float4 *)(sq.Vbuf + (size_t)q * BLK * BLK + i * BLK + c)
+                           : make_float4(i == c ? 1.f : 0.f, i == c + 1 ? 1.f : 0.f, i == c + 2 ? 1.f : 0.f, i == c + 3 ? 1.f : 0.f);
+            *(float4 *)&VqT[i * LD4 + c] = vq;
         }
+        const int gi = grow(i), gc = gcol(c);
+        float4 bv = zero4;
+        if (gi < rt) {
+            const float *src = src_b + (size_t)gi * rt + gc;
+            if (vec) { if (gc < rt) bv = *(const float4 *)src; }
+            else {
+                if (gc < rt) bv.x = src[0];
+                if (gc + 1 < rt) bv.y = src[1];
+                if (gc + 2 < rt) bv.z = src[2];
+                if (gc + 3 < rt) bv.w = src[3];
+            }
+        }
+        *(float4 *)&Bk[i * LD4 + c] = bv;
     }
     __syncthreads();
-    float acc[MR][4];
+    const int r0 = (tid / Q) * 4, c0 = (tid % Q) * 4;
+    float acc[4][4];
 #pragma unroll
-    for (int i = 0; i < MR; ++i)
+    for (int i = 0; i < 4; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
 #pragma unroll 8
-    for (int k = 0; k < BLK; ++k) {
+    for (int k = 0; k < BLK; ++k) {         // T = Vt_p * B
+        const float4 a = *(const float4 *)&VpT[k * LD4 + r0];
         const float4 b = *(const float4 *)&Bk[k * LD4 + c0];
+        const float av[4] = {a.x, a.y, a.z, a.w};
 #pragma unroll
-        for (int i = 0; i < MR; ++i) {
-            const float a = Vp[(r0 + i) * LD + k];
-            acc[i][0] = fmaf(a, b.x, acc[i][0]); acc[i][1] = fmaf(a, b.y, acc[i][1]);
-            acc[i][2] = fmaf(a, b.z, acc[i][2]); acc[i][3] = fmaf(a, b.w, acc[i][3]);
+        for (int i = 0; i < 4; ++i) {
+            acc[i][0] = fmaf(av[i], b.x, acc[i][0]); acc[i][1] = fmaf(av[i], b.y, acc[i][1]);
+            acc[i][2] = fmaf(av[i], b.z, acc[i][2]); acc[i][3] = fmaf(av[i], b.w, acc[i][3]);
         }
     }
     if (!gblock) {                          // rows of Wt: Vt_p * Wt
+        const int gc = cb + c0;
 #pragma unroll
-        for (int i = 0; i < MR; ++i) {
-            const int gi = jac2_row<BJ2>(Ip, Jp, r0 + i, sq.rt);
-            if (gi < 0) continue;
+        for (int i = 0; i < 4; ++i) {
+            const int gi = grow(r0 + i);
+            if (gi >= rt || gc >= rt) continue;
+            float *dst = sq.Wt + (size_t)gi * rt + gc;
+            if (vec) *(float4 *)dst = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+            else {
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (cb + c0 + j < sq.rt) sq.Wt[(size_t)gi * sq.rt + cb + c0 + j] = acc[i][j];
+                for (int j = 0; j < 4; ++j) if (gc + j < rt) dst[j] = acc[i][j];
+            }
         }
         return;
     }
 #pragma unroll
-    for (int i = 0; i < MR; ++i)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) Tm[(r0 + i) * LD + c0 + j] = acc[i][j];
+    for (int j = 0; j < 4; ++j)
+        *(float4 *)&TmT[(c0 + j) * LD4 + r0] = make_float4(acc[0][j], acc[1][j], acc[2][j], acc[3][j]);
     __syncthreads();
 #pragma unroll
-    for (int i = 0; i < MR; ++i)
+    for (int i = 0; i < 4; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
 #pragma unroll 8
-    for (int k = 0; k < BLK; ++k) {         // Out = T * Vq^T
+    for (int k = 0; k < BLK; ++k) {         // Out = T * Vt_q^T
+        const float4 a = *(const float4 *)&TmT[k * LD4 + r0];
         const float4 b = *(const float4 *)&VqT[k * LD4 + c0];
+        const float av[4] = {a.x, a.y, a.z, a.w};
 #pragma unroll
-        for (int i = 0; i < MR; ++i) {
-            const float a = Tm[(r0 + i) * LD + k];
-            acc[i][0] = fmaf(a, b.x, acc[i][0]); acc[i][1] = fmaf(a, b.y, acc[i][1]);
-            acc[i][2] = fmaf(a, b.z, acc[i][2]); acc[i][3] = fmaf(a, b.w, acc[i][3]);
+        for (int i = 0; i < 4; ++i) {
+            acc[i][0] = fmaf(av[i], b.x, acc[i][0]); acc[i][1] = fmaf(av[i], b.y, acc[i][1]);
+            acc[i][2] = fmaf(av[i], b.z, acc[i][2]); acc[i][3] = fmaf(av[i], b.w, acc[i][3]);
         }
     }
+    const int gi0 = grow(r0), gj0 = gcol(c0);   // rows gi0..gi0+3 and columns gj0..gj0+3 are contiguous
 #pragma unroll
-    for (int i = 0; i < MR; ++i) {
-        const int gi = jac2_row<BJ2>(Ip, Jp, r0 + i, sq.rt);
-        if (gi < 0) continue;
+    for (int i = 0; i < 4; ++i) {
+        if (gi0 + i >= rt || gj0 >= rt) continue;
+        float *dst = sq.G + (size_t)(gi0 + i) * rt + gj0;
+        if (vec) *(float4 *)dst = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+        else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) if (gj0 + j < rt) dst[j] = acc[i][j];
+        }
+    }
+    if (q != p) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const int gj = jac2_row<BJ2>(Iq, Jq, c0 + j, sq.rt);
-            if (gj < 0) continue;
-            sq.G[(size_t)gi * sq.rt + gj] = acc[i][j];
-            if (q != p) sq.G[(size_t)gj * sq.rt + gi] = acc[i][j];
+            if (gj0 + j >= rt || gi0 >= rt) continue;
+            float *dst = sq.G + (size_t)(gj0 + j) * rt + gi0;
+            if (vec) *(float4 *)dst = make_float4(acc[0][j], acc[1][j], acc[2][j], acc[3][j]);
+            else {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) if (gi0 + i < rt) dst[i] = acc[i][j];
+            }
         }
     }
 }
