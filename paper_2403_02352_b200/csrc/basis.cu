@@ -79,22 +79,24 @@ __global__ void __launch_bounds__(256) panel_gram_kernel(const __grid_constant__
         for (int j = 0; j < 4; ++j) dst[(ty * 4 + i) * PB + tx * 4 + j] = acc[i][j];
 }
 
-// Sums the partial Gram matrices in order, scales to unit diagonal and Cholesky-factors in fp64:
-// D^-1 G D^-1 = L L^T. Writes L (fp32, row-major pb x PB) followed by 1/D, so that
-// P D^-1 L^-T has orthonormal columns. A column whose scaled pivot falls below 1e-10 (its part
-// outside the span of the earlier columns is below 1e-5 of its norm) is flagged as dependent: the
-// apply kernel replaces it by a pseudo-random vector, which the second Gram-Schmidt pass
-// orthonormalises. Four threads share a row of the factor (partial dot products + shuffles).
+// Sums the partial Gram matrices in order, scales to unit diagonal, Cholesky-factors in fp64,
+// D^-1 G D^-1 = L L^T, and inverts the factor: writes W = D^-1 L^-T (upper triangular, fp32, PB x PB
+// row-major), so that P W has orthonormal columns. A column whose scaled pivot falls below 1e-10 (its
+// part outside the span of the earlier columns is below 1e-5 of its norm) is flagged as dependent:
+// the apply kernel replaces it by a pseudo-random vector, which the second Gram-Schmidt pass
+// orthonormalises.
+// Four threads share a row. Factorisation, left-looking: every group forms the dot product of its own
+// row and, redundantly, the pivot's, so a column costs one block barrier. Inversion: group c solves
+// L x = e_c by forward substitution into the unused upper triangle (row c), no block barrier at all.
 __global__ void __launch_bounds__(256) panel_chol_kernel(const __grid_constant__ PanelBatch batch)
 {
     const PanelSeq &sq = batch.s[blockIdx.x];
     const int n = sq.pb;
     if (n <= 0) return;
     __shared__ double G[PB][PB + 1];
-    __shared__ double dsc[PB];
+    __shared__ double rs[PB];          // 1 / sqrt(diagonal of the Gram matrix)
+    __shared__ double invd[PB];        // 1 / L_jj
     __shared__ int dep[PB];
-    __shared__ double sh_ljj;
-    __shared__ int sh_bad;
     const int tid = threadIdx.x;
     const int nchunks = (sq.n + GRAM_ROWS - 1) / GRAM_ROWS;
     for (int e = tid; e < PB * PB; e += 256) {
@@ -103,82 +105,129 @@ __global__ void __launch_bounds__(256) panel_chol_kernel(const __grid_constant__
         G[e >> 6][e & 63] = s;
     }
     __syncthreads();
-    if (tid < PB) { dsc[tid] = (tid < n && G[tid][tid] > 0.0) ? sqrt(G[tid][tid]) : 0.0; dep[tid] = 0; }
+    if (tid < PB) {
+        const double g = G[tid][tid];
+        rs[tid] = (tid < n && g > 0.0) ? rsqrt(g) : 0.0;
+        dep[tid] = 0; invd[tid] = 1.0;
+    }
     __syncthreads();
     for (int e = tid; e < PB * PB; e += 256) {
-        int i = e >> 6, j = e & 63;
-        double den = dsc[i] * dsc[j];
-        G[i][j] = den > 0.0 ? G[i][j] / den : 0.0;
+        const int i = e >> 6, j = e & 63;
+        G[i][j] = (i == j) ? (rs[i] > 0.0 ? 1.0 : 0.0) : G[i][j] * rs[i] * rs[j];
     }
     __syncthreads();
     const int row = tid >> 2, part = tid & 3;
-    for (int j = 0; j < n; ++j) {       // left-looking: column j from the finished columns < j
-        double sacc = 0.0;
-        if (row >= j && row < n)
-            for (int k = part; k < j; k += 4) sacc -= G[row][k] * G[j][k];
-        sacc += __shfl_xor_sync(0xffffffffu, sacc, 1);
-        sacc += __shfl_xor_sync(0xffffffffu, sacc, 2);
-        if (row >= j && row < n) sacc += G[row][j];
-        if (row == j && part == 0) {
-            int bad = !(sacc > 1e-10);
-            sh_bad = bad;
-            sh_ljj = bad ? 1.0 : sqrt(sacc);
-            if (bad) dep[j] = 1;
+    for (int j = 0; j < n; ++j) {
+        double s1 = 0.0, s2 = 0.0;
+        for (int k = part; k < j; k += 4) {
+            const double a = G[j][k];
+            s1 = fma(-G[row][k], a, s1);
+            s2 = fma(-a, a, s2);
+        }
+        s1 += __shfl_xor_sync(0xffffffffu, s1, 1); s2 += __shfl_xor_sync(0xffffffffu, s2, 1);
+        s1 += __shfl_xor_sync(0xffffffffu, s1, 2); s2 += __shfl_xor_sync(0xffffffffu, s2, 2);
+        const double piv = G[j][j] + s2;
+        const bool bad = !(piv > 1e-10);
+        const double rinv = bad ? 0.0 : rsqrt(piv);
+        const double mine = G[row][j] + s1;
+        // column j below the diagonal is written here and first read in step j + 1; the diagonal entry of
+        // G itself stays untouched (every group reads it in this step), 1 / L_jj lives in invd
+        if (part == 0 && row < n) {
+            if (row > j) G[row][j] = mine * rinv;      // a dependent column leaves zeros below a unit pivot
+            else if (row == j) { invd[j] = bad ? 1.0 : rinv; dep[j] = bad ? 1 : 0; }
         }
         __syncthreads();
-        if (part == 0 && row >= j && row < n) G[row][j] = (row == j) ? sh_ljj : (sh_bad ? 0.0 : sacc / sh_ljj);
-        __syncthreads();
     }
+    // inverse of L, column c by group c, stored in row c of the upper triangle: G[c][i] = (L^-1)[i][c]
+    {
+        const int c = row;
+        const int i_first = ((tid >> 5) << 3) + 1;     // the first column of this warp, plus one
+        const double xc = invd[c];
+        for (int i = i_first; i < n; ++i) {
+            double s = 0.0;
+            if (i > c) {
+                for (int k = c + part; k < i; k += 4) s = fma(G[i][k], (k == c) ? xc : G[c][k], s);
+            }
+            s += __shfl_xor_sync(0xffffffffu, s, 1);
+            s += __shfl_xor_sync(0xffffffffu, s, 2);
+            if (part == 0 && i > c && c < n) G[c][i] = -s * invd[i];
+            __syncwarp();
+        }
+    }
+    __syncthreads();
     for (int e = tid; e < PB * PB; e += 256) {
-        int i = e >> 6, k = e & 63;
-        sq.rinv[e] = (i < n && k <= i) ? (float)G[i][k] : (i == k ? 1.f : 0.f);
+        const int k = e >> 6, c = e & 63;
+        float w = 0.f;
+        if (k < n && c < n) {
+            if (k < c) w = (float)(rs[k] * G[k][c]);
+            else if (k == c) w = (float)(rs[k] * invd[k]);
+        }
+        sq.rinv[e] = w;
     }
-    if (tid < PB) {
-        sq.rinv[PB * PB + tid] = (tid < n && dsc[tid] > 0.0) ? (float)(1.0 / dsc[tid]) : 0.f;
-        sq.flags[tid] = (tid < n) ? (dep[tid] || !(dsc[tid] > 0.0)) : 0;
-    }
+    if (tid < PB) sq.flags[tid] = (tid < n) ? (dep[tid] || !(rs[tid] > 0.0)) : 0;
 }
 
-// P <- P D^-1 L^-T in place: every thread solves the triangular system of one row (forward
-// substitution, fully unrolled, L broadcast from shared memory); rows are staged through shared
-// memory so that global accesses stay coalesced. Flagged columns are refilled with hash noise.
-__global__ void __launch_bounds__(64) panel_apply_kernel(const __grid_constant__ PanelBatch batch, uint64_t seed)
+// P <- P W in place (W = D^-1 L^-T from panel_chol_kernel): a 64 x 64 x 64 product per CTA, 4 x 4
+// register tiles. Flagged columns are refilled with hash noise.
+__global__ void __launch_bounds__(256) panel_apply_kernel(const __grid_constant__ PanelBatch batch, uint64_t seed)
 {
     const PanelSeq &sq = batch.s[blockIdx.y];
     const int r0 = blockIdx.x * 64;
     if (sq.pb <= 0 || r0 >= sq.n) return;
-    __shared__ float Ls[PB][PB + 1];
-    __shared__ float Ts[64][PB + 1];
-    __shared__ float dinv[PB];
+    __shared__ __align__(16) float Ws[PB][PB + 4];
+    __shared__ float Ps[64][PB + 1];
     __shared__ int fl[PB];
     const int tid = threadIdx.x;
-    for (int e = tid; e < PB * PB; e += 64) Ls[e >> 6][e & 63] = sq.rinv[e];
-    dinv[tid] = sq.rinv[PB * PB + tid];
-    fl[tid] = sq.flags[tid];
-    for (int e = tid; e < 64 * PB; e += 64) {
-        int row = e >> 6, c = e & 63;
-        float v = 0.f;
-        if (r0 + row < sq.n && c < sq.pb) v = sq.P[(size_t)(r0 + row) * sq.ld + c];
-        Ts[row][c] = v;
+    const bool vec = (sq.ld & 3) == 0 && ((size_t)sq.P & 15) == 0;
+    for (int f = tid; f < 64 * (PB / 4); f += 256) {
+        const int row = f >> 4, c = (f & 15) * 4;
+        *(float4 *)&Ws[row][c] = *(const float4 *)(sq.rinv + row * PB + c);
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (r0 + row < sq.n) {
+            const float *src = sq.P + (size_t)(r0 + row) * sq.ld + c;
+            if (vec && c + 3 < sq.pb) v = *(const float4 *)src;
+            else {
+                if (c < sq.pb) v.x = src[0];
+                if (c + 1 < sq.pb) v.y = src[1];
+                if (c + 2 < sq.pb) v.z = src[2];
+                if (c + 3 < sq.pb) v.w = src[3];
+            }
+        }
+        Ps[row][c] = v.x; Ps[row][c + 1] = v.y; Ps[row][c + 2] = v.z; Ps[row][c + 3] = v.w;
     }
+    if (tid < PB) fl[tid] = sq.flags[tid];
     __syncthreads();
-    float x[PB];
+    const int rr = (tid >> 4) * 4, c0 = (tid & 15) * 4;
+    float acc[4][4];
 #pragma unroll
-    for (int c = 0; c < PB; ++c) {
-        float acc = Ts[tid][c] * dinv[c];
+    for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int k = 0; k < c; ++k) acc = fmaf(-x[k], Ls[c][k], acc);
-        x[c] = acc / Ls[c][c];
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+#pragma unroll 8
+    for (int k = 0; k < PB; ++k) {
+        const float4 b = *(const float4 *)&Ws[k][c0];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float a = Ps[rr + i][k];
+            acc[i][0] = fmaf(a, b.x, acc[i][0]); acc[i][1] = fmaf(a, b.y, acc[i][1]);
+            acc[i][2] = fmaf(a, b.z, acc[i][2]); acc[i][3] = fmaf(a, b.w, acc[i][3]);
+        }
     }
-    const int grow = r0 + tid;
     const float rscale = rsqrtf((float)sq.n * (1.f / 3.f));      // replacement columns of about unit norm
 #pragma unroll
-    for (int c = 0; c < PB; ++c)
-        Ts[tid][c] = fl[c] ? rscale * hash_uniform(seed, ((uint64_t)blockIdx.y << 40) ^ ((uint64_t)grow << 8) ^ (uint64_t)c) : x[c];
-    __syncthreads();
-    for (int e = tid; e < 64 * PB; e += 64) {
-        int row = e >> 6, c = e & 63;
-        if (r0 + row < sq.n && c < sq.pb) sq.P[(size_t)(r0 + row) * sq.ld + c] = Ts[row][c];
+    for (int i = 0; i < 4; ++i) {
+        const int grow = r0 + rr + i;
+        if (grow >= sq.n) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (fl[c0 + j])
+                acc[i][j] = rscale * hash_uniform(seed, ((uint64_t)blockIdx.y << 40) ^ ((uint64_t)grow << 8) ^ (uint64_t)(c0 + j));
+        float *dst = sq.P + (size_t)grow * sq.ld + c0;
+        if (vec && c0 + 3 < sq.pb) *(float4 *)dst = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+        else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) if (c0 + j < sq.pb) dst[j] = acc[i][j];
+        }
     }
 }
 
@@ -642,7 +691,14 @@ struct BasisPlan {
     std::vector<SeqPlan> seqs; float *omega; __nv_bfloat16 *omega_b; float *part; size_t part_stride, part_group; int group = 0; int rtmax; int splits;
 };
 
-static int pick_splits(int K) { int s = K / 1024; return s < 1 ? 1 : (s > 16 ? 16 : s); }
+// Split-K factor of the thin projections C = Q^T P (few output tiles, long K): enough slices to put
+// about two CTAs on every SM, each at least 64 deep.
+static int pick_splits(int K, int nseq)
+{
+    int want = (296 + std::max(nseq, 1) - 1) / std::max(nseq, 1);
+    int s = std::min(std::min(want, K / 64), 16);
+    return s < 1 ? 1 : s;
+}
 
 static void plan_basis(Arena &ar, const std::vector<SeqDims> &sd, int d, int oversample, BasisPlan &bp)
 {
@@ -659,7 +715,7 @@ static void plan_basis(Arena &ar, const std::vector<SeqDims> &sd, int d, int ove
     }
     bp.omega = ar.take<float>((size_t)d * bp.rtmax);
     bp.omega_b = ar.take<__nv_bfloat16>((size_t)d * align_up((size_t)bp.rtmax, 8));
-    bp.splits = pick_splits(maxdim);
+    bp.splits = pick_splits(maxdim, (int)std::min<size_t>(sd.size(), BMAX));
     for (auto &p : bp.seqs) {
         int L = p.dims.L, rt = p.rt;
         p.Y = ar.take<float>((size_t)L * rt);
@@ -740,7 +796,7 @@ static atp_status orthonormalise(atp_ctx *ctx, BasisPlan &bp, size_t i0, size_t 
             panel_chol_kernel<<<pb.count, 256, 0, ctx->stream>>>(pb);
             ATP_LAUNCHED(ctx);
             ATP_KERNEL(ctx, "panel_apply", 0, 0);
-            panel_apply_kernel<<<dim3(ceil_div(maxn, 64), pb.count), 64, 0, ctx->stream>>>(
+            panel_apply_kernel<<<dim3(ceil_div(maxn, 64), pb.count), 256, 0, ctx->stream>>>(
                 pb, seed + 7919ull * (uint64_t)(pj * 2 + rep) + (z_side ? 104729ull : 0ull));
             ATP_LAUNCHED(ctx);
         }

@@ -1,4 +1,5 @@
-// Batched SIMT GEMM with fp32 accumulation: C = epilogue(op(A) * B).
+// Batched SIMT GEMM with fp32 accumulation: C = epilogue(op(A) * B). 64 x 64 x 32 tiles, the next
+// tile prefetched into registers during the multiply.
 //   A: M x K row-major (TRANS_A = false) or K x M row-major (TRANS_A = true)
 //   B: K x N row-major (TRANS_B = false) or N x K row-major (TRANS_B = true)
 //   C: M x N row-major,  D (optional addend / gate): M x N fp32
@@ -42,12 +43,13 @@ gemm_simt_kernel(const __grid_constant__ GemmBatch batch, GemmEpi epi, int split
     const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
     if (m0 >= pr.M || n0 >= pr.N) return;
     int kchunk = (pr.K + splits - 1) / splits;
-    kchunk = (kchunk + 15) / 16 * 16;
+    kchunk = (kchunk + 31) / 32 * 32;
     const int kb = split * kchunk;
     const int ke = min(pr.K, kb + kchunk);
 
-    __shared__ __align__(16) float As[16][68];
-    __shared__ __align__(16) float Bs[16][68];
+    constexpr int BK = 32;                              // K tile; 8 elements of A and of B per thread
+    __shared__ __align__(16) float As[BK][68];
+    __shared__ __align__(16) float Bs[BK][68];
     const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
     const TA *A = (const TA *)pr.A;
     const TB *B = (const TB *)pr.B;
@@ -57,36 +59,42 @@ gemm_simt_kernel(const __grid_constant__ GemmBatch batch, GemmEpi epi, int split
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
 
-    for (int k0 = kb; k0 < ke; k0 += 16) {
+    // the next tile travels from global memory into registers while the current one is multiplied
+    float ra[8], rb[8];
+    auto fetch = [&](int k0) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            int e = tid + i * 256;
+        for (int i = 0; i < 8; ++i) {
+            const int e = tid + i * 256;
+            float va = 0.f, vb = 0.f;
             if (!TRANS_A) {
-                int m = e >> 4, k = e & 15;
-                float v = 0.f;
-                if (m0 + m < pr.M && k0 + k < ke) v = to_f32(A[(size_t)(m0 + m) * pr.lda + k0 + k]);
-                As[k][m] = v;
+                const int m = e >> 5, k = e & 31;
+                if (m0 + m < pr.M && k0 + k < ke) va = to_f32(A[(size_t)(m0 + m) * pr.lda + k0 + k]);
             } else {
-                int k = e >> 6, m = e & 63;
-                float v = 0.f;
-                if (m0 + m < pr.M && k0 + k < ke) v = to_f32(A[(size_t)(k0 + k) * pr.lda + m0 + m]);
-                As[k][m] = v;
+                const int k = e >> 6, m = e & 63;
+                if (m0 + m < pr.M && k0 + k < ke) va = to_f32(A[(size_t)(k0 + k) * pr.lda + m0 + m]);
             }
             if (!TRANS_B) {
-                int k = e >> 6, n = e & 63;
-                float v = 0.f;
-                if (n0 + n < pr.N && k0 + k < ke) v = to_f32(B[(size_t)(k0 + k) * pr.ldb + n0 + n]);
-                Bs[k][n] = v;
+                const int k = e >> 6, n = e & 63;
+                if (n0 + n < pr.N && k0 + k < ke) vb = to_f32(B[(size_t)(k0 + k) * pr.ldb + n0 + n]);
             } else {
-                int n = e >> 4, k = e & 15;
-                float v = 0.f;
-                if (n0 + n < pr.N && k0 + k < ke) v = to_f32(B[(size_t)(n0 + n) * pr.ldb + k0 + k]);
-                Bs[k][n] = v;
+                const int n = e >> 5, k = e & 31;
+                if (n0 + n < pr.N && k0 + k < ke) vb = to_f32(B[(size_t)(n0 + n) * pr.ldb + k0 + k]);
             }
+            ra[i] = va; rb[i] = vb;
+        }
+    };
+    if (kb < ke) fetch(kb);
+    for (int k0 = kb; k0 < ke; k0 += BK) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int e = tid + i * 256;
+            if (!TRANS_A) As[e & 31][e >> 5] = ra[i]; else As[e >> 6][e & 63] = ra[i];
+            if (!TRANS_B) Bs[e >> 6][e & 63] = rb[i]; else Bs[e & 31][e >> 5] = rb[i];
         }
         __syncthreads();
+        if (k0 + BK < ke) fetch(k0 + BK);
 #pragma unroll
-        for (int k = 0; k < 16; ++k) {
+        for (int k = 0; k < BK; ++k) {
             float4 a = *(const float4 *)&As[k][ty * 4];
             float4 b = *(const float4 *)&Bs[k][tx * 4];
             float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
