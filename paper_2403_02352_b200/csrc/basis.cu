@@ -85,85 +85,104 @@ __global__ void __launch_bounds__(256) panel_gram_kernel(const __grid_constant__
 // part outside the span of the earlier columns is below 1e-5 of its norm) is flagged as dependent:
 // the apply kernel replaces it by a pseudo-random vector, which the second Gram-Schmidt pass
 // orthonormalises.
-// Four threads share a row. Factorisation, left-looking: every group forms the dot product of its own
-// row and, redundantly, the pivot's, so a column costs one block barrier. Inversion: group c solves
-// L x = e_c by forward substitution into the unused upper triangle (row c), no block barrier at all.
+// Right-looking, in registers: thread (br, bc) owns the 4 x 4 blocks of G and of X (X starts as the
+// identity and ends as L^-1) at rows 4 br, columns 4 bc. Step j: the owner of the pivot publishes
+// 1 / L_jj; the owners of column j publish l = G[:, j] / L_jj and the owners of row j of X scale and
+// publish it; everybody subtracts l l^T from G and l x_j from X. Two short barriers per column, the
+// arithmetic between them is 32 independent multiply-adds per thread.
 __global__ void __launch_bounds__(256) panel_chol_kernel(const __grid_constant__ PanelBatch batch)
 {
     const PanelSeq &sq = batch.s[blockIdx.x];
     const int n = sq.pb;
     if (n <= 0) return;
-    __shared__ double G[PB][PB + 1];
     __shared__ double rs[PB];          // 1 / sqrt(diagonal of the Gram matrix)
-    __shared__ double invd[PB];        // 1 / L_jj
+    __shared__ double lcol[PB];        // column j of L below the diagonal (zero at and above it)
+    __shared__ double xrow[PB];        // row j of L^-1
+    __shared__ double sh_rinv;
     __shared__ int dep[PB];
     const int tid = threadIdx.x;
+    const int br = tid >> 4, bc = tid & 15;
     const int nchunks = (sq.n + GRAM_ROWS - 1) / GRAM_ROWS;
-    for (int e = tid; e < PB * PB; e += 256) {
-        double s = 0.0;
-        for (int c = 0; c < nchunks; ++c) s += sq.gpart[(size_t)c * PB * PB + e];
-        G[e >> 6][e & 63] = s;
-    }
-    __syncthreads();
-    if (tid < PB) {
-        const double g = G[tid][tid];
-        rs[tid] = (tid < n && g > 0.0) ? rsqrt(g) : 0.0;
-        dep[tid] = 0; invd[tid] = 1.0;
-    }
-    __syncthreads();
-    for (int e = tid; e < PB * PB; e += 256) {
-        const int i = e >> 6, j = e & 63;
-        G[i][j] = (i == j) ? (rs[i] > 0.0 ? 1.0 : 0.0) : G[i][j] * rs[i] * rs[j];
-    }
-    __syncthreads();
-    const int row = tid >> 2, part = tid & 3;
-    for (int j = 0; j < n; ++j) {
-        double s1 = 0.0, s2 = 0.0;
-        for (int k = part; k < j; k += 4) {
-            const double a = G[j][k];
-            s1 = fma(-G[row][k], a, s1);
-            s2 = fma(-a, a, s2);
+    double g[4][4], x[4][4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            double s = 0.0;
+            const int e = (4 * br + a) * PB + 4 * bc + b;
+            for (int c = 0; c < nchunks; ++c) s += sq.gpart[(size_t)c * PB * PB + e];
+            g[a][b] = s;
+            x[a][b] = (br == bc && a == b) ? 1.0 : 0.0;
         }
-        s1 += __shfl_xor_sync(0xffffffffu, s1, 1); s2 += __shfl_xor_sync(0xffffffffu, s2, 1);
-        s1 += __shfl_xor_sync(0xffffffffu, s1, 2); s2 += __shfl_xor_sync(0xffffffffu, s2, 2);
-        const double piv = G[j][j] + s2;
-        const bool bad = !(piv > 1e-10);
-        const double rinv = bad ? 0.0 : rsqrt(piv);
-        const double mine = G[row][j] + s1;
-        // column j below the diagonal is written here and first read in step j + 1; the diagonal entry of
-        // G itself stays untouched (every group reads it in this step), 1 / L_jj lives in invd
-        if (part == 0 && row < n) {
-            if (row > j) G[row][j] = mine * rinv;      // a dependent column leaves zeros below a unit pivot
-            else if (row == j) { invd[j] = bad ? 1.0 : rinv; dep[j] = bad ? 1 : 0; }
+    if (br == bc) {
+#pragma unroll
+        for (int a = 0; a < 4; ++a) {
+            const int i = 4 * br + a;
+            rs[i] = (i < n && g[a][a] > 0.0) ? rsqrt(g[a][a]) : 0.0;
+            dep[i] = 0;
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const double ra = rs[4 * br + a], rb = rs[4 * bc + b];
+            g[a][b] = (br == bc && a == b) ? (ra > 0.0 ? 1.0 : 0.0) : g[a][b] * ra * rb;
+        }
+    for (int j = 0; j < n; ++j) {
+        const int jb = j >> 2, jj = j & 3;
+        if (br == jb && bc == jb) {
+            double piv = 0.0;
+#pragma unroll
+            for (int a = 0; a < 4; ++a) if (a == jj) piv = g[a][a];
+            const bool bad = !(piv > 1e-10);
+            sh_rinv = bad ? 0.0 : rsqrt(piv);          // a dependent column: unit pivot, zeros below
+            if (bad) dep[j] = 1;
         }
         __syncthreads();
-    }
-    // inverse of L, column c by group c, stored in row c of the upper triangle: G[c][i] = (L^-1)[i][c]
-    {
-        const int c = row;
-        const int i_first = ((tid >> 5) << 3) + 1;     // the first column of this warp, plus one
-        const double xc = invd[c];
-        for (int i = i_first; i < n; ++i) {
-            double s = 0.0;
-            if (i > c) {
-                for (int k = c + part; k < i; k += 4) s = fma(G[i][k], (k == c) ? xc : G[c][k], s);
+        const double rinv = sh_rinv;
+        if (bc == jb) {                                 // owners of column j of G
+#pragma unroll
+            for (int a = 0; a < 4; ++a) {
+                double v = 0.0;
+#pragma unroll
+                for (int b = 0; b < 4; ++b) if (b == jj) v = g[a][b];
+                const int i = 4 * br + a;
+                lcol[i] = (i > j) ? v * rinv : 0.0;
             }
-            s += __shfl_xor_sync(0xffffffffu, s, 1);
-            s += __shfl_xor_sync(0xffffffffu, s, 2);
-            if (part == 0 && i > c && c < n) G[c][i] = -s * invd[i];
-            __syncwarp();
         }
+        if (br == jb) {                                 // owners of row j of X: x_j <- x_j / L_jj
+            const double sc = (rinv > 0.0) ? rinv : 1.0;
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+                if (a == jj) {
+#pragma unroll
+                    for (int b = 0; b < 4; ++b) { x[a][b] *= sc; xrow[4 * bc + b] = x[a][b]; }
+                }
+        }
+        __syncthreads();
+        double la[4], lb[4], xb[4];
+#pragma unroll
+        for (int a = 0; a < 4; ++a) { la[a] = lcol[4 * br + a]; lb[a] = lcol[4 * bc + a]; xb[a] = xrow[4 * bc + a]; }
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                g[a][b] = fma(-la[a], lb[b], g[a][b]);
+                x[a][b] = fma(-la[a], xb[b], x[a][b]);
+            }
+    }
+    // W[k][c] = (L^-1)[c][k] / D_k ; this thread holds (L^-1)[4 br + a][4 bc + b]
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+        const int k = 4 * bc + b;
+        const double rk = rs[k];
+        float4 w;
+        w.x = (float)(rk * x[0][b]); w.y = (float)(rk * x[1][b]); w.z = (float)(rk * x[2][b]); w.w = (float)(rk * x[3][b]);
+        *(float4 *)(sq.rinv + k * PB + 4 * br) = w;
     }
     __syncthreads();
-    for (int e = tid; e < PB * PB; e += 256) {
-        const int k = e >> 6, c = e & 63;
-        float w = 0.f;
-        if (k < n && c < n) {
-            if (k < c) w = (float)(rs[k] * G[k][c]);
-            else if (k == c) w = (float)(rs[k] * invd[k]);
-        }
-        sq.rinv[e] = w;
-    }
     if (tid < PB) sq.flags[tid] = (tid < n) ? (dep[tid] || !(rs[tid] > 0.0)) : 0;
 }
 
