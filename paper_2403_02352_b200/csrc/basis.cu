@@ -1071,7 +1071,7 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
                         ATP_LAUNCHED(ctx);
                         ATP_KERNEL(ctx, "jac2_apply", nseq * npairs * (npairs * 4.0 + ceil_div(maxrt, blk) * 2.0) * bl * bl * bl,
                                    nseq * npairs * (npairs * 2.0 + ceil_div(maxrt, blk) * 2.0) * bl * bl * 4.0);
-                        dim3 ag(npairs + ceil_div(maxrt, blk), npairs, cnt);
+                        dim3 ag(npairs * (npairs + 1) / 2 + npairs * ceil_div(maxrt, blk), 1, cnt);
                         if (jbj == 32) jac2_apply_kernel<32><<<ag, 256, ash, ctx->stream>>>(jb, step);
                         else jac2_apply_kernel<16><<<ag, 64, ash, ctx->stream>>>(jb, step);
                         ATP_LAUNCHED(ctx);

@@ -41,18 +41,24 @@ __global__ void jac2_init_kernel(const __grid_constant__ Jac2Batch batch)
 }
 
 // Rotation (c, s) that annihilates the (p, q) entry of a symmetric matrix; identity when the entry is
-// already small against its diagonal. Fast reciprocal / rsqrt: c^2 + s^2 = 1 to ~2 ulp, ample for a
-// basis stored in bf16.
+// already small against its diagonal. With a = g_qq - g_pp, b = 2 g_pq, r = sqrt(a^2 + b^2):
+//   cos 2t = |a| / r,  c = sqrt((1 + cos 2t) / 2),  s = sign(a) b / (2 r c)      (|t| <= pi/4),
+// two reciprocal square roots in a row instead of two divisions and two roots; c^2 + s^2 = 1 to a few
+// ulp, ample for a basis stored in bf16. a and b are rescaled when their squares would leave the
+// fp32 range.
 __device__ __forceinline__ float2 jac2_rotation(float gpp, float gqq, float gpq, float tol_rot, bool &did)
 {
     float c = 1.f, s = 0.f;
     if (gpq != 0.f && gpq * gpq > tol_rot * tol_rot * fmaxf(gpp, 0.f) * fmaxf(gqq, 0.f)) {
-        float zeta = __fdividef(gqq - gpp, 2.f * gpq);
-        float az = fabsf(zeta), t;
-        if (az > 1e15f) t = __fdividef(0.5f, zeta);
-        else { float h = 1.f + zeta * zeta; t = __fdividef(copysignf(1.f, zeta), az + h * rsqrtf(h)); }
-        c = rsqrtf(1.f + t * t);
-        s = c * t;
+        float a = gqq - gpp, b = 2.f * gpq;
+        const float m = fmaxf(fabsf(a), fabsf(b));
+        const float sc = m < 1e-18f ? 0x1p60f : (m > 1e18f ? 0x1p-60f : 1.f);
+        a *= sc; b *= sc;
+        const float rh = rsqrtf(fmaf(a, a, b * b));
+        const float c2 = fmaf(0.5f * fabsf(a), rh, 0.5f);
+        const float rc = rsqrtf(c2);
+        c = c2 * rc;
+        s = copysignf(0.5f, a) * b * rh * rc;
         did = true;
     }
     return make_float2(c, s);
@@ -159,7 +165,7 @@ jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_r
     if (tid == 0) sq.vflag[pair] = 1;
 }
 
-// grid: (npairs + ceil(rt/BLK), npairs, batch); dynamic shared memory: JAC2_APPLY_SMEM(BLK) bytes.
+// grid: (npairs (npairs + 1) / 2 + npairs ceil(rt/BLK), 1, batch); dynamic shared memory: JAC2_APPLY_SMEM(BLK) bytes.
 // G is symmetric: only blocks (p, q) with q >= p are computed, the mirror block is written from the
 // transposed register tile. Each thread owns a 4 x 4 tile of the BLK x BLK block; every shared-memory
 // operand is read as one 16-byte vector per 16 multiply-adds, and when the row length of G is a multiple
@@ -171,15 +177,26 @@ jac2_apply_kernel(const __grid_constant__ Jac2Batch batch, int step)
 {
     constexpr int BLK = 2 * BJ2, NT = BLK * BLK / 16, LD4 = BLK + 4, Q = BLK / 4;   // Q: 4-vectors per row
     const Jac2Seq &sq = batch.s[blockIdx.z];
-    if (*sq.conv) return;
     const int npairs = sq.nb / 2;
-    const int p = blockIdx.y;
-    if (p >= npairs) return;
-    const bool gblock = (int)blockIdx.x < npairs;
-    const int q = blockIdx.x;
-    if (gblock && q < p) return;
+    // blockIdx.x enumerates the blocks (p, q >= p) of the upper triangle row by row, then the
+    // (pair, column chunk) blocks of Wt
+    const int ntri = npairs * (npairs + 1) / 2, nw = (sq.rt + BLK - 1) / BLK;
+    int idx = blockIdx.x;
+    if (idx >= ntri + npairs * nw) return;
+    const bool gblock = idx < ntri;
+    int p = 0, q = 0, wchunk = 0;
+    if (gblock) {
+        while (idx >= npairs - p) { idx -= npairs - p; ++p; }
+        q = p + idx;
+    } else {
+        idx -= ntri;
+        p = idx / nw; wchunk = idx - p * nw;
+    }
+    // the three flags travel together (one memory latency), then the decision
+    const int conv = *sq.conv;
     const int fp = sq.vflag[p];
     const int fq = gblock ? sq.vflag[q] : 0;
+    if (conv) return;
     if (gblock ? (!fp && !fq) : !fp) return;
     const int tid = threadIdx.x;
     const int rt = sq.rt;
@@ -191,8 +208,7 @@ jac2_apply_kernel(const __grid_constant__ Jac2Batch batch, int step)
     float *VqT = Bk + BLK * LD4;            // [BLK][LD4]  VqT[k][c] = Vt_q[c][k]
     int Ip, Jp, Iq = 0, Jq = 0;
     rr_pair2(sq.nb, step % (sq.nb - 1), p, Ip, Jp);
-    const int cb = gblock ? 0 : ((int)blockIdx.x - npairs) * BLK;
-    if (!gblock && cb >= rt) return;
+    const int cb = wchunk * BLK;
     if (gblock) rr_pair2(sq.nb, step % (sq.nb - 1), q, Iq, Jq);
     // global column of local column c (a multiple of 4): the 4-vector starting there is contiguous
     auto gcol = [&](int c) -> int { return gblock ? ((c < BJ2) ? Iq * BJ2 + c : Jq * BJ2 + (c - BJ2)) : cb + c; };
