@@ -1066,8 +1066,8 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
                         // algorithmic work of a step when every pair rotates (converged pairs skip it)
                         const double nseq = cnt, bl = blk;
                         ATP_KERNEL(ctx, "jac2_local", nseq * npairs * jinner * (bl - 1) * (bl * bl * 6.0 + bl * bl * 3.0), 0);
-                        if (jbj == 32) jac2_local_kernel<32><<<dim3(npairs, cnt), 1024, lsh, ctx->stream>>>(jb, step, tolr, jinner);
-                        else jac2_local_kernel<16><<<dim3(npairs, cnt), 256, lsh, ctx->stream>>>(jb, step, tolr, jinner);
+                        if (jbj == 32) jac2_local_kernel<32><<<dim3(npairs, cnt), 1024, lsh, ctx->stream>>>(jb, step, tolr, jinner, step > 0);
+                        else jac2_local_kernel<16><<<dim3(npairs, cnt), 256, lsh, ctx->stream>>>(jb, step, tolr, jinner, step > 0);
                         ATP_LAUNCHED(ctx);
                         ATP_KERNEL(ctx, "jac2_apply", nseq * npairs * (npairs * 4.0 + ceil_div(maxrt, blk) * 2.0) * bl * bl * bl,
                                    nseq * npairs * (npairs * 2.0 + ceil_div(maxrt, blk) * 2.0) * bl * bl * 4.0);

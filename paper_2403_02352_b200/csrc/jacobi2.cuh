@@ -2,8 +2,11 @@
 // L2): the rotation that diagonalises G turns the orthonormal range basis into singular vectors
 // (Rayleigh-Ritz step of the basis extraction, Sec. 4.2: X' = [sigma_i v_i]).
 // Blocks of 16 rows; a step handles r~/32 disjoint pairs (round-robin order) with two launches:
-//   jac2_local : per pair, the 32x32 diagonal block is diagonalised on chip (cyclic Jacobi), the
-//                accumulated row operations Vt are published (stored transposed);
+//   jac2_local : per pair, the 32x32 diagonal block is swept on chip (cyclic Jacobi: all its pairs in
+//                the first step of a sweep, when every block meets exactly one partner, and only the
+//                pairs that couple the two blocks in the other steps, so that a sweep rotates every
+//                pair of rows exactly once), the accumulated row operations Vt are published
+//                (stored transposed);
 //   jac2_apply : every 32x32 block (p, q) becomes Vt_p G_pq Vt_q^T, rows of Wt become Vt_p Wt.
 // G entries carry errors relative to the norms of the rows of B they come from (B is graded by the
 // QR-ordered range basis), which is what Jacobi needs to resolve small eigenvalues next to large ones.
@@ -74,7 +77,7 @@ __device__ __forceinline__ float2 jac2_rotation(float gpp, float gqq, float gpq,
 #define JAC2_LOCAL_SMEM(BLK) ((size_t)(3 * (BLK) * ((BLK) + 1)) * sizeof(float))
 template <int BJ2>
 __global__ void __launch_bounds__(BJ2 * BJ2)
-jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_rot, int max_inner)
+jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_rot, int max_inner, int cross_only)
 {
     constexpr int BLK = 2 * BJ2, HP = BLK / 2, NT = HP * HP;
     const Jac2Seq &sq = batch.s[blockIdx.y];
@@ -91,9 +94,13 @@ jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_r
     __shared__ int rotated;
     __shared__ uchar2 sched[BLK - 1][HP];              // round-robin schedule of the local sweep
     const int tid = threadIdx.x;
-    for (int e = tid; e < (BLK - 1) * HP; e += NT) {
+    // cross_only: the BJ2 steps that pair every row of block I with every row of block J once; otherwise
+    // the full round-robin over all BLK rows (which also rotates the pairs inside I and inside J)
+    const int nsteps = cross_only ? BJ2 : BLK - 1;
+    for (int e = tid; e < nsteps * HP; e += NT) {
         int p_, q_;
-        rr_pair2(BLK, e / HP, e % HP, p_, q_);
+        if (cross_only) { p_ = e % HP; q_ = BJ2 + (e % HP + e / HP) % BJ2; }
+        else rr_pair2(BLK, e / HP, e % HP, p_, q_);
         sched[e / HP][e % HP] = make_uchar2((unsigned char)p_, (unsigned char)q_);
     }
     for (int e = tid; e < BLK * BLK; e += NT) {
@@ -127,7 +134,7 @@ jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_r
     const int ba = tid / HP, bb = tid % HP;            // 2x2 block (pair ba rows, pair bb columns)
     int cur = 0;
     for (int sweep = 0; sweep < max_inner; ++sweep) {
-        for (int st = 0; st < BLK - 1; ++st) {
+        for (int st = 0; st < nsteps; ++st) {
             const float (*Ao)[BLK + 1] = Ab[cur];
             float (*An)[BLK + 1] = Ab[cur ^ 1];
             const uchar2 ra = sched[st][ba], rb = sched[st][bb];
