@@ -41,6 +41,8 @@ struct PanelBatch { PanelSeq s[BMAX]; int count; };
 // Partial Gram matrices of a panel: G_chunk = P_chunk^T P_chunk, fp64 accumulation.
 __global__ void __launch_bounds__(256) panel_gram_kernel(const __grid_constant__ PanelBatch batch)
 {
+    pdl_trigger();
+    pdl_wait();
     const PanelSeq &sq = batch.s[blockIdx.y];
     const int r0 = blockIdx.x * GRAM_ROWS;
     if (sq.pb <= 0 || r0 >= sq.n) return;
@@ -92,6 +94,8 @@ __global__ void __launch_bounds__(256) panel_gram_kernel(const __grid_constant__
 // arithmetic between them is 32 independent multiply-adds per thread.
 __global__ void __launch_bounds__(256) panel_chol_kernel(const __grid_constant__ PanelBatch batch)
 {
+    pdl_trigger();
+    pdl_wait();
     const PanelSeq &sq = batch.s[blockIdx.x];
     const int n = sq.pb;
     if (n <= 0) return;
@@ -190,6 +194,8 @@ __global__ void __launch_bounds__(256) panel_chol_kernel(const __grid_constant__
 // register tiles. Flagged columns are refilled with hash noise.
 __global__ void __launch_bounds__(256) panel_apply_kernel(const __grid_constant__ PanelBatch batch, uint64_t seed)
 {
+    pdl_trigger();
+    pdl_wait();
     const PanelSeq &sq = batch.s[blockIdx.y];
     const int r0 = blockIdx.x * 64;
     if (sq.pb <= 0 || r0 >= sq.n) return;
@@ -809,14 +815,14 @@ static atp_status orthonormalise(atp_ctx *ctx, BasisPlan &bp, size_t i0, size_t 
                 if ((st = launch_gemm_simt<float, float, float, false>(ctx, upd, GemmEpi{EPI_D_MINUS, nullptr})) != ATP_OK) return st;
             }
             ATP_KERNEL(ctx, "panel_gram", 0, 0);
-            panel_gram_kernel<<<dim3(ceil_div(maxn, GRAM_ROWS), pb.count), 256, 0, ctx->stream>>>(pb);
+            launch_pdl(panel_gram_kernel, dim3(ceil_div(maxn, GRAM_ROWS), pb.count), dim3(256), 0, ctx->stream, pb);
             ATP_LAUNCHED(ctx);
             ATP_KERNEL(ctx, "panel_chol", 0, 0);
-            panel_chol_kernel<<<pb.count, 256, 0, ctx->stream>>>(pb);
+            launch_pdl(panel_chol_kernel, dim3(pb.count), dim3(256), 0, ctx->stream, pb);
             ATP_LAUNCHED(ctx);
             ATP_KERNEL(ctx, "panel_apply", 0, 0);
-            panel_apply_kernel<<<dim3(ceil_div(maxn, 64), pb.count), 256, 0, ctx->stream>>>(
-                pb, seed + 7919ull * (uint64_t)(pj * 2 + rep) + (z_side ? 104729ull : 0ull));
+            launch_pdl(panel_apply_kernel, dim3(ceil_div(maxn, 64), pb.count), dim3(256), 0, ctx->stream, pb,
+                       (uint64_t)(seed + 7919ull * (uint64_t)(pj * 2 + rep) + (z_side ? 104729ull : 0ull)));
             ATP_LAUNCHED(ctx);
         }
     }
@@ -1041,7 +1047,7 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
             const int blk = 2 * jbj;
             const size_t ash = jbj == 32 ? JAC2_APPLY_SMEM(64) : JAC2_APPLY_SMEM(32);
             const size_t lsh = jbj == 32 ? JAC2_LOCAL_SMEM(64) : JAC2_LOCAL_SMEM(32);
-            if (jbj == 32) ATP_CUDA_OK(ctx, cudaFuncSetAttribute(jac2_apply_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ash));
+            if (jbj == 32) ATP_CUDA_OK(ctx, cudaFuncSetAttribute(jac2_apply_kernel<32, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ash));
             if (jbj == 32) ATP_CUDA_OK(ctx, cudaFuncSetAttribute(jac2_local_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lsh));
             for (int pass = 0; pass < 2; ++pass) {
                 if ((st = launch_gemm_simt<float, float, float, true, false>(ctx, gg, store)) != ATP_OK) return st;
@@ -1066,14 +1072,14 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
                         // algorithmic work of a step when every pair rotates (converged pairs skip it)
                         const double nseq = cnt, bl = blk;
                         ATP_KERNEL(ctx, "jac2_local", nseq * npairs * jinner * (bl - 1) * (bl * bl * 6.0 + bl * bl * 3.0), 0);
-                        if (jbj == 32) jac2_local_kernel<32><<<dim3(npairs, cnt), 1024, lsh, ctx->stream>>>(jb, step, tolr, jinner, step > 0);
-                        else jac2_local_kernel<16><<<dim3(npairs, cnt), 256, lsh, ctx->stream>>>(jb, step, tolr, jinner, step > 0);
+                        if (jbj == 32) launch_pdl(jac2_local_kernel<32>, dim3(npairs, cnt), dim3(1024), lsh, ctx->stream, jb, step, tolr, jinner, (int)(step > 0));
+                        else launch_pdl(jac2_local_kernel<16>, dim3(npairs, cnt), dim3(256), lsh, ctx->stream, jb, step, tolr, jinner, (int)(step > 0));
                         ATP_LAUNCHED(ctx);
                         ATP_KERNEL(ctx, "jac2_apply", nseq * npairs * (npairs * 4.0 + ceil_div(maxrt, blk) * 2.0) * bl * bl * bl,
                                    nseq * npairs * (npairs * 2.0 + ceil_div(maxrt, blk) * 2.0) * bl * bl * 4.0);
                         dim3 ag(npairs * (npairs + 1) / 2 + npairs * ceil_div(maxrt, blk), 1, cnt);
-                        if (jbj == 32) jac2_apply_kernel<32><<<ag, 256, ash, ctx->stream>>>(jb, step);
-                        else jac2_apply_kernel<16><<<ag, 64, ash, ctx->stream>>>(jb, step);
+                        if (jbj == 32) launch_pdl(jac2_apply_kernel<32, 4>, ag, dim3(256), ash, ctx->stream, jb, step);
+                        else launch_pdl(jac2_apply_kernel<16, 2>, ag, dim3(128), ash, ctx->stream, jb, step);
                         ATP_LAUNCHED(ctx);
                     }
                     ATP_KERNEL(ctx, "jac2_sweep_end", 0, 0);

@@ -62,6 +62,26 @@ static inline void prof_end(atp_ctx *ctx)
         if (e__ != cudaSuccess) { (ctx)->last_cuda = e__; return ATP_ERR_CUDA; } \
     } while (0)
 
+// Programmatic dependent launch: a kernel launched through launch_pdl may begin (run its prologue, which
+// must touch no global data) while its predecessor in the stream is still draining; pdl_wait() then
+// blocks until the predecessor has completed and its writes are visible. Every thread of such a kernel
+// calls pdl_wait() before its first global access and before any exit, so "this kernel has completed"
+// keeps implying "everything before it has completed". pdl_trigger() lets the successor start launching.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 

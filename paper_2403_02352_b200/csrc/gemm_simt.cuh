@@ -37,6 +37,8 @@ template <typename TA, typename TB, typename TC, bool TRANS_A, bool TRANS_B>
 __global__ void __launch_bounds__(256)
 gemm_simt_kernel(const __grid_constant__ GemmBatch batch, GemmEpi epi, int splits, float *part, size_t part_stride)
 {
+    pdl_trigger();
+    pdl_wait();
     const int z = blockIdx.z;
     const int pidx = z / splits, split = z - pidx * splits;
     const GemmProblem &pr = batch.p[pidx];
@@ -147,6 +149,8 @@ template <typename TC>
 __global__ void __launch_bounds__(256)
 gemm_splitk_reduce_kernel(const __grid_constant__ GemmBatch batch, int splits, const float *part, size_t part_stride)
 {
+    pdl_trigger();
+    pdl_wait();
     const int pidx = blockIdx.y;
     const GemmProblem &pr = batch.p[pidx];
     size_t total = (size_t)pr.M * pr.N;
@@ -179,13 +183,13 @@ static atp_status launch_gemm_simt(atp_ctx *ctx, const GemmBatch &batch, GemmEpi
     }
     dim3 grid(ceil_div(maxN, 64), ceil_div(maxM, 64), batch.count * splits);
     ATP_KERNEL(ctx, "gemm_simt", flops, bytes);
-    gemm_simt_kernel<TA, TB, TC, TRANS_A, TRANS_B><<<grid, 256, 0, ctx->stream>>>(batch, epi, splits, part, part_stride);
+    launch_pdl(gemm_simt_kernel<TA, TB, TC, TRANS_A, TRANS_B>, grid, dim3(256), 0, ctx->stream, batch, epi, splits, part, part_stride);
     ATP_LAUNCHED(ctx);
     if (splits > 1) {
         int blocks = ceil_div(maxM * maxN, 256);
         if (blocks > 1024) blocks = 1024;
         ATP_KERNEL(ctx, "gemm_splitk_reduce", 0, 0);
-        gemm_splitk_reduce_kernel<TC><<<dim3(blocks, batch.count), 256, 0, ctx->stream>>>(batch, splits, part, part_stride);
+        launch_pdl(gemm_splitk_reduce_kernel<TC>, dim3(blocks, batch.count), dim3(256), 0, ctx->stream, batch, splits, (const float *)part, part_stride);
         ATP_LAUNCHED(ctx);
     }
     return ATP_OK;

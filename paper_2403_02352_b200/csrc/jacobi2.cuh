@@ -80,13 +80,12 @@ __global__ void __launch_bounds__(BJ2 * BJ2)
 jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_rot, int max_inner, int cross_only)
 {
     constexpr int BLK = 2 * BJ2, HP = BLK / 2, NT = HP * HP;
+    pdl_trigger();
     const Jac2Seq &sq = batch.s[blockIdx.y];
-    if (*sq.conv) return;
     const int npairs = sq.nb / 2;
     const int pair = blockIdx.x;
-    if (pair >= npairs) return;
     int I, J;
-    rr_pair2(sq.nb, step % (sq.nb - 1), pair, I, J);
+    rr_pair2(sq.nb, step % (sq.nb - 1), pair < npairs ? pair : 0, I, J);
     extern __shared__ __align__(16) float j2l[];       // JAC2_LOCAL_SMEM(BLK) bytes
     float (*Ab)[BLK][BLK + 1] = (float (*)[BLK][BLK + 1])j2l;                     // two copies of A
     float (*V)[BLK + 1] = (float (*)[BLK + 1])(j2l + 2 * BLK * (BLK + 1));
@@ -103,6 +102,8 @@ jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_r
         else rr_pair2(BLK, e / HP, e % HP, p_, q_);
         sched[e / HP][e % HP] = make_uchar2((unsigned char)p_, (unsigned char)q_);
     }
+    pdl_wait();                                        // nothing above touches global memory
+    if (pair >= npairs || *sq.conv) return;
     for (int e = tid; e < BLK * BLK; e += NT) {
         int i = e / BLK, j = e % BLK;
         int gi = jac2_row<BJ2>(I, J, i, sq.rt), gj = jac2_row<BJ2>(I, J, j, sq.rt);
@@ -174,22 +175,24 @@ jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_r
 
 // grid: (npairs (npairs + 1) / 2 + npairs ceil(rt/BLK), 1, batch); dynamic shared memory: JAC2_APPLY_SMEM(BLK) bytes.
 // G is symmetric: only blocks (p, q) with q >= p are computed, the mirror block is written from the
-// transposed register tile. Each thread owns a 4 x 4 tile of the BLK x BLK block; every shared-memory
+// transposed register tile. Each thread owns an MR x 4 tile (MR = 2 or 4) of the BLK x BLK block; every shared-memory
 // operand is read as one 16-byte vector per 16 multiply-adds, and when the row length of G is a multiple
 // of four the global traffic is 16-byte vectors too (the 16 or 32 columns of a block are contiguous).
 #define JAC2_APPLY_SMEM(BLK) ((size_t)(4 * (BLK) * ((BLK) + 4)) * sizeof(float))
-template <int BJ2>
-__global__ void __launch_bounds__(BJ2 * BJ2 / 4)
+template <int BJ2, int MR>
+__global__ void __launch_bounds__(BJ2 * BJ2 / MR)
 jac2_apply_kernel(const __grid_constant__ Jac2Batch batch, int step)
 {
-    constexpr int BLK = 2 * BJ2, NT = BLK * BLK / 16, LD4 = BLK + 4, Q = BLK / 4;   // Q: 4-vectors per row
+    constexpr int BLK = 2 * BJ2, NT = BLK * BLK / (4 * MR), LD4 = BLK + 4, Q = BLK / 4;   // Q: 4-vectors per row
+    pdl_trigger();
     const Jac2Seq &sq = batch.s[blockIdx.z];
     const int npairs = sq.nb / 2;
     // blockIdx.x enumerates the blocks (p, q >= p) of the upper triangle row by row, then the
     // (pair, column chunk) blocks of Wt
     const int ntri = npairs * (npairs + 1) / 2, nw = (sq.rt + BLK - 1) / BLK;
     int idx = blockIdx.x;
-    if (idx >= ntri + npairs * nw) return;
+    const bool in_range = idx < ntri + npairs * nw;
+    if (!in_range) idx = 0;
     const bool gblock = idx < ntri;
     int p = 0, q = 0, wchunk = 0;
     if (gblock) {
@@ -199,6 +202,8 @@ jac2_apply_kernel(const __grid_constant__ Jac2Batch batch, int step)
         idx -= ntri;
         p = idx / nw; wchunk = idx - p * nw;
     }
+    pdl_wait();                             // nothing above touches global memory
+    if (!in_range) return;
     // the three flags travel together (one memory latency), then the decision
     const int conv = *sq.conv;
     const int fp = sq.vflag[p];
@@ -248,27 +253,32 @@ jac2_apply_kernel(const __grid_constant__ Jac2Batch batch, int step)
         *(float4 *)&Bk[i * LD4 + c] = bv;
     }
     __syncthreads();
-    const int r0 = (tid / Q) * 4, c0 = (tid % Q) * 4;
-    float acc[4][4];
+    const int r0 = (tid / Q) * MR, c0 = (tid % Q) * 4;
+    float acc[MR][4];
+    // acc = (rows r0.. of the operand stored transposed in At) * Bm
+    auto product = [&](const float *At, const float *Bm) {
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
+        for (int i = 0; i < MR; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
-#pragma unroll 8
-    for (int k = 0; k < BLK; ++k) {         // T = Vt_p * B
-        const float4 a = *(const float4 *)&VpT[k * LD4 + r0];
-        const float4 b = *(const float4 *)&Bk[k * LD4 + c0];
-        const float av[4] = {a.x, a.y, a.z, a.w};
+            for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            acc[i][0] = fmaf(av[i], b.x, acc[i][0]); acc[i][1] = fmaf(av[i], b.y, acc[i][1]);
-            acc[i][2] = fmaf(av[i], b.z, acc[i][2]); acc[i][3] = fmaf(av[i], b.w, acc[i][3]);
+        for (int k = 0; k < BLK; ++k) {
+            float av[MR];
+            if (MR == 4) { const float4 a = *(const float4 *)&At[k * LD4 + r0]; av[0] = a.x; av[1] = a.y; av[MR - 2] = a.z; av[MR - 1] = a.w; }
+            else { const float2 a = *(const float2 *)&At[k * LD4 + r0]; av[0] = a.x; av[1] = a.y; }
+            const float4 b = *(const float4 *)&Bm[k * LD4 + c0];
+#pragma unroll
+            for (int i = 0; i < MR; ++i) {
+                acc[i][0] = fmaf(av[i], b.x, acc[i][0]); acc[i][1] = fmaf(av[i], b.y, acc[i][1]);
+                acc[i][2] = fmaf(av[i], b.z, acc[i][2]); acc[i][3] = fmaf(av[i], b.w, acc[i][3]);
+            }
         }
-    }
+    };
+    product(VpT, Bk);                       // T = Vt_p * B
     if (!gblock) {                          // rows of Wt: Vt_p * Wt
         const int gc = cb + c0;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < MR; ++i) {
             const int gi = grow(r0 + i);
             if (gi >= rt || gc >= rt) continue;
             float *dst = sq.Wt + (size_t)gi * rt + gc;
@@ -281,27 +291,15 @@ jac2_apply_kernel(const __grid_constant__ Jac2Batch batch, int step)
         return;
     }
 #pragma unroll
-    for (int j = 0; j < 4; ++j)
-        *(float4 *)&TmT[(c0 + j) * LD4 + r0] = make_float4(acc[0][j], acc[1][j], acc[2][j], acc[3][j]);
-    __syncthreads();
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
-#pragma unroll 8
-    for (int k = 0; k < BLK; ++k) {         // Out = T * Vt_q^T
-        const float4 a = *(const float4 *)&TmT[k * LD4 + r0];
-        const float4 b = *(const float4 *)&VqT[k * LD4 + c0];
-        const float av[4] = {a.x, a.y, a.z, a.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            acc[i][0] = fmaf(av[i], b.x, acc[i][0]); acc[i][1] = fmaf(av[i], b.y, acc[i][1]);
-            acc[i][2] = fmaf(av[i], b.z, acc[i][2]); acc[i][3] = fmaf(av[i], b.w, acc[i][3]);
-        }
+    for (int j = 0; j < 4; ++j) {
+        if (MR == 4) *(float4 *)&TmT[(c0 + j) * LD4 + r0] = make_float4(acc[0][j], acc[1][j], acc[MR - 2][j], acc[MR - 1][j]);
+        else *(float2 *)&TmT[(c0 + j) * LD4 + r0] = make_float2(acc[0][j], acc[1][j]);
     }
-    const int gi0 = grow(r0), gj0 = gcol(c0);   // rows gi0..gi0+3 and columns gj0..gj0+3 are contiguous
+    __syncthreads();
+    product(TmT, VqT);                      // Out = T * Vt_q^T
+    const int gi0 = grow(r0), gj0 = gcol(c0);   // rows gi0.. and columns gj0..gj0+3 are contiguous
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < MR; ++i) {
         if (gi0 + i >= rt || gj0 >= rt) continue;
         float *dst = sq.G + (size_t)(gi0 + i) * rt + gj0;
         if (vec) *(float4 *)dst = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
@@ -315,10 +313,11 @@ jac2_apply_kernel(const __grid_constant__ Jac2Batch batch, int step)
         for (int j = 0; j < 4; ++j) {
             if (gj0 + j >= rt || gi0 >= rt) continue;
             float *dst = sq.G + (size_t)(gj0 + j) * rt + gi0;
-            if (vec) *(float4 *)dst = make_float4(acc[0][j], acc[1][j], acc[2][j], acc[3][j]);
+            if (vec && MR == 4) *(float4 *)dst = make_float4(acc[0][j], acc[1][j], acc[MR - 2][j], acc[MR - 1][j]);
+            else if (vec) *(float2 *)dst = make_float2(acc[0][j], acc[1][j]);
             else {
 #pragma unroll
-                for (int i = 0; i < 4; ++i) if (gi0 + i < rt) dst[i] = acc[i][j];
+                for (int i = 0; i < MR; ++i) if (gi0 + i < rt) dst[i] = acc[i][j];
             }
         }
     }
@@ -330,6 +329,8 @@ __global__ void jac2_sweep_end_kernel(const __grid_constant__ Jac2Batch batch, f
 {
     const int b = threadIdx.x;
     int done = 1;
+    pdl_trigger();
+    pdl_wait();
     if (b < batch.count) {
         const Jac2Seq &sq = batch.s[b];
         if (!*sq.conv) {
