@@ -15,7 +15,7 @@
 #include <algorithm>
 
 constexpr int PB = 64;            // orthonormalisation panel width
-constexpr int GRAM_ROWS = 128;    // rows per CTA of the panel Gram kernel
+constexpr int GRAM_ROWS = 64;     // rows per CTA of the panel Gram kernel
 constexpr int BJ = 32;            // Jacobi block height (pairs are 64 rows)
 constexpr int BMAX = 32;          // sequences per launch
 
@@ -87,11 +87,14 @@ __global__ void __launch_bounds__(256) panel_gram_kernel(const __grid_constant__
 // part outside the span of the earlier columns is below 1e-5 of its norm) is flagged as dependent:
 // the apply kernel replaces it by a pseudo-random vector, which the second Gram-Schmidt pass
 // orthonormalises.
-// Right-looking, in registers: thread (br, bc) owns the 4 x 4 blocks of G and of X (X starts as the
-// identity and ends as L^-1) at rows 4 br, columns 4 bc. Step j: the owner of the pivot publishes
-// 1 / L_jj; the owners of column j publish l = G[:, j] / L_jj and the owners of row j of X scale and
-// publish it; everybody subtracts l l^T from G and l x_j from X. Two short barriers per column, the
-// arithmetic between them is 32 independent multiply-adds per thread.
+// Right-looking by blocks of four columns, in registers: thread (br, bc) owns the 4 x 4 blocks of G
+// and of X (X starts as the identity and ends as L^-1) at rows 4 br, columns 4 bc. Block step jb:
+//   1. the owner of the diagonal block factors it (four pivots) and publishes L_bb and 1 / L_jj;
+//   2. the owners of the block column below it solve for their rows of L, the owners of block row jb of
+//      X apply L_bb^-1 to it; both publish;
+//   3. everybody below subtracts L_i L_k^T from G (columns right of jb) or L_i X_b from X (columns up
+//      to jb): 64 independent multiply-adds per thread.
+// Two block barriers per four columns.
 __global__ void __launch_bounds__(256) panel_chol_kernel(const __grid_constant__ PanelBatch batch)
 {
     pdl_trigger();
@@ -100,9 +103,10 @@ __global__ void __launch_bounds__(256) panel_chol_kernel(const __grid_constant__
     const int n = sq.pb;
     if (n <= 0) return;
     __shared__ double rs[PB];          // 1 / sqrt(diagonal of the Gram matrix)
-    __shared__ double lcol[PB];        // column j of L below the diagonal (zero at and above it)
-    __shared__ double xrow[PB];        // row j of L^-1
-    __shared__ double sh_rinv;
+    __shared__ double lcol4[PB][4];    // block column jb of L (rows below the diagonal block)
+    __shared__ double xrow4[4][PB];    // block row jb of L^-1
+    __shared__ double Lbb[4][4];       // the factored diagonal block (strictly lower part)
+    __shared__ double rinv4[4];        // 1 / L_jj, 0 for a dependent column
     __shared__ int dep[PB];
     const int tid = threadIdx.x;
     const int br = tid >> 4, bc = tid & 15;
@@ -111,13 +115,20 @@ __global__ void __launch_bounds__(256) panel_chol_kernel(const __grid_constant__
 #pragma unroll
     for (int a = 0; a < 4; ++a)
 #pragma unroll
-        for (int b = 0; b < 4; ++b) {
-            double s = 0.0;
-            const int e = (4 * br + a) * PB + 4 * bc + b;
-            for (int c = 0; c < nchunks; ++c) s += sq.gpart[(size_t)c * PB * PB + e];
-            g[a][b] = s;
-            x[a][b] = (br == bc && a == b) ? 1.0 : 0.0;
+        for (int b = 0; b < 4; ++b) { g[a][b] = 0.0; x[a][b] = (br == bc && a == b) ? 1.0 : 0.0; }
+    // chunk by chunk (a fixed order), the eight 16-byte loads of a chunk in flight together
+    const double2 *gp = (const double2 *)(sq.gpart + (size_t)(4 * br) * PB + 4 * bc);
+#pragma unroll 2
+    for (int c = 0; c < nchunks; ++c) {
+        double2 v[4][2];
+#pragma unroll
+        for (int a = 0; a < 4; ++a) {
+            v[a][0] = gp[((size_t)c * PB * PB + (size_t)a * PB) / 2];
+            v[a][1] = gp[((size_t)c * PB * PB + (size_t)a * PB) / 2 + 1];
         }
+#pragma unroll
+        for (int a = 0; a < 4; ++a) { g[a][0] += v[a][0].x; g[a][1] += v[a][0].y; g[a][2] += v[a][1].x; g[a][3] += v[a][1].y; }
+    }
     if (br == bc) {
 #pragma unroll
         for (int a = 0; a < 4; ++a) {
@@ -134,48 +145,101 @@ __global__ void __launch_bounds__(256) panel_chol_kernel(const __grid_constant__
             const double ra = rs[4 * br + a], rb = rs[4 * bc + b];
             g[a][b] = (br == bc && a == b) ? (ra > 0.0 ? 1.0 : 0.0) : g[a][b] * ra * rb;
         }
-    for (int j = 0; j < n; ++j) {
-        const int jb = j >> 2, jj = j & 3;
+    const int nblk = (n + 3) >> 2;
+    for (int jb = 0; jb < nblk; ++jb) {
         if (br == jb && bc == jb) {
-            double piv = 0.0;
+            // 1. the diagonal block, column by column; a dependent column gets a unit pivot and zeros below
+            double ri[4];
 #pragma unroll
-            for (int a = 0; a < 4; ++a) if (a == jj) piv = g[a][a];
-            const bool bad = !(piv > 1e-10);
-            sh_rinv = bad ? 0.0 : rsqrt(piv);          // a dependent column: unit pivot, zeros below
-            if (bad) dep[j] = 1;
+            for (int c = 0; c < 4; ++c) {
+                double piv = g[c][c];
+#pragma unroll
+                for (int k = 0; k < c; ++k) piv = fma(-g[c][k], g[c][k], piv);
+                const bool bad = !(piv > 1e-10);
+                // 1/sqrt in fp64 from the fp32 approximation and two Newton steps (piv is in (1e-10, ~1])
+                double y = (double)rsqrtf((float)piv);
+                y = y * (1.5 - 0.5 * piv * y * y);
+                y = y * (1.5 - 0.5 * piv * y * y);
+                ri[c] = bad ? 0.0 : y;
+                if (bad && 4 * jb + c < n) dep[4 * jb + c] = 1;
+#pragma unroll
+                for (int r = c + 1; r < 4; ++r) {
+                    double v = g[r][c];
+#pragma unroll
+                    for (int k = 0; k < c; ++k) v = fma(-g[r][k], g[c][k], v);
+                    g[r][c] = v * ri[c];
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                rinv4[r] = ri[r];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) Lbb[r][c] = (c < r) ? g[r][c] : 0.0;
+            }
         }
         __syncthreads();
-        const double rinv = sh_rinv;
-        if (bc == jb) {                                 // owners of column j of G
+        if (bc == jb && br > jb) {
+            // 2a. rows of L below the diagonal block: l_c = (g_c - sum_{k<c} l_k L_bb[c][k]) / L_cc
 #pragma unroll
             for (int a = 0; a < 4; ++a) {
-                double v = 0.0;
+                double l[4];
 #pragma unroll
-                for (int b = 0; b < 4; ++b) if (b == jj) v = g[a][b];
-                const int i = 4 * br + a;
-                lcol[i] = (i > j) ? v * rinv : 0.0;
+                for (int c = 0; c < 4; ++c) {
+                    double v = g[a][c];
+#pragma unroll
+                    for (int k = 0; k < c; ++k) v = fma(-l[k], Lbb[c][k], v);
+                    l[c] = v * rinv4[c];
+                    lcol4[4 * br + a][c] = l[c];
+                }
             }
         }
-        if (br == jb) {                                 // owners of row j of X: x_j <- x_j / L_jj
-            const double sc = (rinv > 0.0) ? rinv : 1.0;
+        if (br == jb && bc <= jb) {
+            // 2b. block row jb of X: forward substitution with L_bb (a dependent column keeps its scale)
 #pragma unroll
-            for (int a = 0; a < 4; ++a)
-                if (a == jj) {
+            for (int c = 0; c < 4; ++c) {
+                const double sc = rinv4[c] > 0.0 ? rinv4[c] : 1.0;
 #pragma unroll
-                    for (int b = 0; b < 4; ++b) { x[a][b] *= sc; xrow[4 * bc + b] = x[a][b]; }
+                for (int b = 0; b < 4; ++b) {
+                    double v = x[c][b];
+#pragma unroll
+                    for (int k = 0; k < c; ++k) v = fma(-Lbb[c][k], x[k][b], v);
+                    x[c][b] = v * sc;
+                    xrow4[c][4 * bc + b] = x[c][b];
                 }
+            }
         }
         __syncthreads();
-        double la[4], lb[4], xb[4];
+        if (br > jb && bc <= br) {
+            // 3. trailing update
+            double la[4][4];
 #pragma unroll
-        for (int a = 0; a < 4; ++a) { la[a] = lcol[4 * br + a]; lb[a] = lcol[4 * bc + a]; xb[a] = xrow[4 * bc + a]; }
+            for (int a = 0; a < 4; ++a)
 #pragma unroll
-        for (int a = 0; a < 4; ++a)
+                for (int c = 0; c < 4; ++c) la[a][c] = lcol4[4 * br + a][c];
+            if (bc > jb) {
 #pragma unroll
-            for (int b = 0; b < 4; ++b) {
-                g[a][b] = fma(-la[a], lb[b], g[a][b]);
-                x[a][b] = fma(-la[a], xb[b], x[a][b]);
+                for (int b = 0; b < 4; ++b) {
+                    double lb[4];
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) lb[c] = lcol4[4 * bc + b][c];
+#pragma unroll
+                    for (int a = 0; a < 4; ++a)
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) g[a][b] = fma(-la[a][c], lb[c], g[a][b]);
+                }
+            } else {
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                    double xb[4];
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) xb[c] = xrow4[c][4 * bc + b];
+#pragma unroll
+                    for (int a = 0; a < 4; ++a)
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) x[a][b] = fma(-la[a][c], xb[c], x[a][b]);
+                }
             }
+        }
     }
     // W[k][c] = (L^-1)[c][k] / D_k ; this thread holds (L^-1)[4 br + a][4 bc + b]
 #pragma unroll
