@@ -320,6 +320,24 @@ __global__ void __launch_bounds__(256) panel_apply_kernel(const __grid_constant_
     }
 }
 
+// fp32 -> bf16 hi/lo pair (hi = bf16(x), lo = bf16(x - hi)) for every sequence of a batch.
+struct SplitSeq { const float *src; __nv_bfloat16 *hi, *lo; int lds, ldd, rows, cols; };
+struct SplitBatch { SplitSeq s[BMAX]; int count; };
+__global__ void __launch_bounds__(256) split_bf16_batch_kernel(const __grid_constant__ SplitBatch batch)
+{
+    pdl_trigger();
+    pdl_wait();
+    const SplitSeq &q = batch.s[blockIdx.y];
+    const size_t n = (size_t)q.rows * q.cols;
+    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
+        const int r = (int)(e / q.cols), c = (int)(e - (size_t)r * q.cols);
+        const float x = q.src[(size_t)r * q.lds + c];
+        const __nv_bfloat16 h = __float2bfloat16_rn(x);
+        q.hi[(size_t)r * q.ldd + c] = h;
+        q.lo[(size_t)r * q.ldd + c] = __float2bfloat16_rn(x - __bfloat162float(h));
+    }
+}
+
 // ------------------------------------------------------------------------------------------------
 // One-sided block Jacobi on the rows of BW = [B | Wt] (r~ x (d + r~)); only the first d columns
 // enter the inner products, all d + r~ columns are rotated.
@@ -949,15 +967,18 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
             // bits): a single bf16 rounding of Y would leak sigma_1 * 2^-9 / sqrt(L) of the leading
             // direction into every column and bury directions that are 10^3..10^4 times weaker.
             auto to_bf16 = [&]() -> atp_status {
+                SplitBatch sb; sb.count = (int)(i1 - i0);
+                double bytes = 0; int maxel = 0;
                 for (size_t i = i0; i < i1; ++i) {
                     SeqPlan &p = bp.seqs[i];
-                    int rows = p.dims.L;
-                    if (rows == 0 || p.rt == 0) continue;
-                    ATP_KERNEL(ctx, "f32_to_bf16", 0, (double)rows * p.rt * 8);
-                    tc::f32_to_bf16_split_kernel<<<std::min(1024, ceil_div(rows * p.rt, 256)), 256, 0, ctx->stream>>>(
-                        p.Y, p.rt, p.Yb, p.Yl, (int)align_up((size_t)p.rt, 8), rows, p.rt);
-                    ATP_LAUNCHED(ctx);
+                    sb.s[i - i0] = SplitSeq{p.Y, p.Yb, p.Yl, p.rt, (int)align_up((size_t)p.rt, 8), p.dims.L, p.rt};
+                    bytes += (double)p.dims.L * p.rt * 8;
+                    maxel = std::max(maxel, p.dims.L * p.rt);
                 }
+                if (maxel == 0) return ATP_OK;
+                ATP_KERNEL(ctx, "f32_to_bf16", 0, bytes);
+                launch_pdl(split_bf16_batch_kernel, dim3(std::min(64, ceil_div(maxel, 1024)), sb.count), dim3(256), 0, ctx->stream, sb);
+                ATP_LAUNCHED(ctx);
                 return ATP_OK;
             };
             std::vector<tc::HostProblem> hp;

@@ -180,7 +180,7 @@ jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_r
 // of four the global traffic is 16-byte vectors too (the 16 or 32 columns of a block are contiguous).
 #define JAC2_APPLY_SMEM(BLK) ((size_t)(4 * (BLK) * ((BLK) + 4)) * sizeof(float))
 template <int BJ2, int MR>
-__global__ void __launch_bounds__(BJ2 * BJ2 / MR)
+__global__ void __launch_bounds__(BJ2 * BJ2 / MR, BJ2 == 16 ? 12 : 1)      // 12 CTAs per SM: one wave at batch 16, r~ = 320
 jac2_apply_kernel(const __grid_constant__ Jac2Batch batch, int step)
 {
     constexpr int BLK = 2 * BJ2, NT = BLK * BLK / (4 * MR), LD4 = BLK + 4, Q = BLK / 4;   // Q: 4-vectors per row
