@@ -893,8 +893,8 @@ static atp_status orthonormalise(atp_ctx *ctx, BasisPlan &bp, size_t i0, size_t 
             }
             if (j0 > 0) {
                 if ((st = launch_gemm_simt<float, float, float, true>(ctx, proj, GemmEpi{EPI_STORE, nullptr}, bp.splits,
-                                                                      bp.part + bp.group * bp.part_group, bp.part_stride)) != ATP_OK) return st;
-                if ((st = launch_gemm_simt<float, float, float, false>(ctx, upd, GemmEpi{EPI_D_MINUS, nullptr})) != ATP_OK) return st;
+                                                                      bp.part + bp.group * bp.part_group, bp.part_stride, "gemm_simt_proj")) != ATP_OK) return st;
+                if ((st = launch_gemm_simt<float, float, float, false>(ctx, upd, GemmEpi{EPI_D_MINUS, nullptr}, 1, nullptr, 0, "gemm_simt_upd")) != ATP_OK) return st;
             }
             ATP_KERNEL(ctx, "panel_gram", 0, 0);
             launch_pdl(panel_gram_kernel, dim3(ceil_div(maxn, GRAM_ROWS), pb.count), dim3(256), 0, ctx->stream, pb);
@@ -1135,7 +1135,7 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
             if (jbj == 32) ATP_CUDA_OK(ctx, cudaFuncSetAttribute(jac2_apply_kernel<32, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ash));
             if (jbj == 32) ATP_CUDA_OK(ctx, cudaFuncSetAttribute(jac2_local_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lsh));
             for (int pass = 0; pass < 2; ++pass) {
-                if ((st = launch_gemm_simt<float, float, float, true, false>(ctx, gg, store)) != ATP_OK) return st;
+                if ((st = launch_gemm_simt<float, float, float, true, false>(ctx, gg, store, 1, nullptr, 0, "gemm_simt_gram")) != ATP_OK) return st;
                 ATP_KERNEL(ctx, "jac2_init", 0, 0);
                 jac2_init_kernel<<<dim3(64, cnt), 256, 0, ctx->stream>>>(jb);
                 ATP_LAUNCHED(ctx);
@@ -1188,8 +1188,8 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
                         gg.p[k].A = p.Z; gg.p[k].B = p.Z;
                         fb.s[k].Y = p.Y2;
                     }
-                    if ((st = launch_gemm_simt<float, float, float, false, true>(ctx, r1, store)) != ATP_OK) return st;
-                    if ((st = launch_gemm_simt<float, float, float, false, true>(ctx, r2, store)) != ATP_OK) return st;
+                    if ((st = launch_gemm_simt<float, float, float, false, true>(ctx, r1, store, 1, nullptr, 0, "gemm_simt_rot")) != ATP_OK) return st;
+                    if ((st = launch_gemm_simt<float, float, float, false, true>(ctx, r2, store, 1, nullptr, 0, "gemm_simt_rot")) != ATP_OK) return st;
                 }
             }
             int npow = 1; while (npow < maxrt) npow <<= 1;
@@ -1211,8 +1211,8 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
                 gg.p[k] = GemmProblem{p.Y2, p.Wsel, (T *)U_r->data + (size_t)p.dims.row0 * U_r->ld, nullptr,
                                       p.dims.L, p.dims.r, p.rt, p.rt, p.dims.r, (int)U_r->ld, 0};
             }
-            if ((st = launch_gemm_simt<float, float, T, true, true>(ctx, g, store)) != ATP_OK) return st;
-            if ((st = launch_gemm_simt<float, float, T, false>(ctx, gg, store)) != ATP_OK) return st;
+            if ((st = launch_gemm_simt<float, float, T, true, true>(ctx, g, store, 1, nullptr, 0, "gemm_simt_out")) != ATP_OK) return st;
+            if ((st = launch_gemm_simt<float, float, T, false>(ctx, gg, store, 1, nullptr, 0, "gemm_simt_out")) != ATP_OK) return st;
             ATP_KERNEL(ctx, "signfix", 0, 0);
             signfix_kernel<T><<<dim3(maxr, cnt), 256, 0, ctx->stream>>>(fb);
             ATP_LAUNCHED(ctx);

@@ -166,7 +166,7 @@ gemm_splitk_reduce_kernel(const __grid_constant__ GemmBatch batch, int splits, c
 // Host launcher. `part` is scratch for split-K (splits * count * part_stride floats) or nullptr.
 template <typename TA, typename TB, typename TC, bool TRANS_A, bool TRANS_B = false>
 static atp_status launch_gemm_simt(atp_ctx *ctx, const GemmBatch &batch, GemmEpi epi, int splits = 1,
-                                   float *part = nullptr, size_t part_stride = 0)
+                                   float *part = nullptr, size_t part_stride = 0, const char *name = "gemm_simt")
 {
     int maxM = 0, maxN = 0;
     for (int i = 0; i < batch.count; ++i) {
@@ -182,7 +182,7 @@ static atp_status launch_gemm_simt(atp_ctx *ctx, const GemmBatch &batch, GemmEpi
         bytes += (double)q.M * q.K * sizeof(TA) + (double)q.K * q.N * sizeof(TB) + (double)q.M * q.N * sizeof(TC);
     }
     dim3 grid(ceil_div(maxN, 64), ceil_div(maxM, 64), batch.count * splits);
-    ATP_KERNEL(ctx, "gemm_simt", flops, bytes);
+    ATP_KERNEL(ctx, name, flops, bytes);
     launch_pdl(gemm_simt_kernel<TA, TB, TC, TRANS_A, TRANS_B>, grid, dim3(256), 0, ctx->stream, batch, epi, splits, part, part_stride);
     ATP_LAUNCHED(ctx);
     if (splits > 1) {
