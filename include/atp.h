@@ -9,6 +9,8 @@
  *   atp_lowrank_linear(U_r, X_r, W)               -> Y            Sec. 4.3 (linear layers on the
  *                                                                 r-row representation)
  *   atp_input_norm(X [, residual])                -> X_n          the "Norm" box of Fig. 3
+ *   atp_alternating_basis(X, V0, inner)           -> (U, X')      Algorithm 1 (appendix B)
+ *   atp_svd_entropy(sigma)                        -> (mu, rank)   Eq. 4
  *
  * General conventions
  *   - Plain C ABI. Every matrix is row-major with a leading dimension `ld` in elements.
@@ -84,7 +86,7 @@ typedef struct {
     const int32_t *rank_off;  /* batch + 1 entries: rows of X_r per sequence               */
 } atp_seqs;
 
-typedef enum { ATP_OP_BASIS = 0, ATP_OP_ATTENTION = 1, ATP_OP_LINEAR = 2, ATP_OP_NORM = 3 } atp_op;
+typedef enum { ATP_OP_BASIS = 0, ATP_OP_ATTENTION = 1, ATP_OP_LINEAR = 2, ATP_OP_NORM = 3, ATP_OP_ALTERNATING = 4 } atp_op;
 typedef enum { ATP_Q_LOWRANK = 0, ATP_Q_FULL = 1 } atp_q_mode;
 typedef enum { ATP_ACT_NONE = 0, ATP_ACT_GELU = 1, ATP_ACT_SWIGLU = 2 } atp_act;
 typedef enum { ATP_NORM_RMS = 0, ATP_NORM_LAYER = 1 } atp_norm_kind;
@@ -218,6 +220,41 @@ ATP_API atp_status atp_profile_stop(atp_ctx *ctx, char *buf, size_t cap, size_t 
 ATP_API atp_status atp_lowrank_linear_static(void *cuda_stream, const atp_mat *U_r, const atp_mat *X_r,
                                              const atp_mat *W, const atp_seqs *seqs, const atp_linear_opts *opts,
                                              atp_mat *Y);
+
+/*
+ * Algorithm 1 (appendix B; described in Sec. 4.2): the paper's own approximate extraction by
+ * alternating rank-1 fits with deflation. For every sequence b and component i < r_b, starting from
+ * v = row (rank_off[b] + i) of V0:  `inner` rounds of  u = R v / |v|^2,  v = R^T u / |u|^2  on the
+ * deflated matrix R (R = X for i = 0), then R <- R - u v^T. Outputs, as Sec. 4.2 puts the scale into
+ * v:  U_r[:, i] = u / |u|  and  X_r[i, :] = v |u|.  The columns of U_r are NOT orthonormalised and not
+ * sorted; no sign rule is applied (the result is fixed by V0). The paper runs inner = 2.
+ *   X      in   sum(L_b) x d                      (f32 or bf16)
+ *   V0     in   sum(r_b) x d, f32                 the start vectors (the method's random draw is an
+ *                                                 input, so that two implementations can be compared)
+ *   inner  in   1..64
+ *   U_r    out  sum(L_b) x max_b(r_b), same dtype as X
+ *   X_r    out  sum(r_b) x d, same dtype as X
+ * Arithmetic: R, u, v are held in fp32, every dot product accumulates in fp64.
+ * Workspace: atp_workspace_bytes(ATP_OP_ALTERNATING, seqs, d, 0, dtype). r_b <= min(L_b, d).
+ * Errors: as atp_principal_basis (no convergence status: the iteration count is fixed).
+ */
+ATP_API atp_status atp_alternating_basis(atp_ctx *ctx, const atp_mat *X, const atp_seqs *seqs, const atp_mat *V0,
+                                         int inner, atp_mat *U_r, atp_mat *X_r);
+
+/*
+ * SVD entropy (Eq. 4) and the rank it suggests (Sec. 3): for each of `batch` groups of singular
+ * values, mu = -log2(sum_i sbar_i^2) with sbar_i = sigma_i / sum_j sigma_j, and rank = ceil(2^mu).
+ *   sigma    in   device, f32, packed groups
+ *   offsets  in   HOST, batch + 1 ints: group b is sigma[offsets[b] .. offsets[b+1]); offsets[0] = 0
+ *   mu       out  device, f32, batch values
+ *   rank     out  device, int32, batch values; may be NULL
+ * Sums, the logarithm and the ceiling are taken in fp64 (an exact power of two such as 8 equal values
+ * gives rank 8, not 9: 1e-9 is subtracted before the ceiling). An empty or all-zero group gives mu = 0,
+ * rank = 0. The entropy describes the WHOLE spectrum: feed it the sigma of a full-rank call
+ * (r_b = min(L_b, d)) of atp_principal_basis.
+ */
+ATP_API atp_status atp_svd_entropy(atp_ctx *ctx, const float *sigma, const int32_t *offsets, int32_t batch, float *mu,
+                                   int32_t *rank);
 
 #ifdef __cplusplus
 }

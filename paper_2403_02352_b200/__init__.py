@@ -6,5 +6,5 @@ importing the binding without a built libatp.so raises.
 """
 from .binding import (  # noqa: F401
     Context, AtpError, atp_principal_basis, atp_attention, atp_lowrank_linear, atp_input_norm,
-    library_path, exported_symbols, atp_lowrank_linear_static,
+    library_path, exported_symbols, atp_lowrank_linear_static, atp_alternating_basis, atp_svd_entropy,
 )

@@ -15,7 +15,7 @@ OK, ERR_INVALID_ARG, ERR_INVALID_RANK, ERR_UNSUPPORTED_DTYPE, ERR_WORKSPACE_TOO_
     ERR_NOT_CONVERGED, ERR_TIMEOUT, ERR_RANGE, ERR_STATIC_SCRATCH_LIMIT = range(10)
 STATIC_SCRATCH_BYTES = 8 << 20
 F32, BF16 = 0, 1
-OP_BASIS, OP_ATTENTION, OP_LINEAR, OP_NORM = 0, 1, 2, 3
+OP_BASIS, OP_ATTENTION, OP_LINEAR, OP_NORM, OP_ALTERNATING = 0, 1, 2, 3, 4
 Q_LOWRANK, Q_FULL = 0, 1
 ACT = {None: 0, "none": 0, "gelu": 1, "swiglu": 2}
 NORM = {"rms": 0, "layer": 1}
@@ -24,7 +24,7 @@ exported_symbols = (
     "atp_create", "atp_destroy", "atp_set_stream", "atp_workspace_bytes", "atp_set_workspace",
     "atp_input_norm", "atp_principal_basis", "atp_attention", "atp_lowrank_linear",
     "atp_poll_device_status", "atp_launch_count", "atp_status_string", "atp_profile_start", "atp_profile_stop",
-    "atp_lowrank_linear_static",
+    "atp_lowrank_linear_static", "atp_alternating_basis", "atp_svd_entropy",
 )
 
 
@@ -78,6 +78,9 @@ def _load():
     lib.atp_profile_start.argtypes = [C.c_void_p]
     lib.atp_profile_stop.argtypes = [C.c_void_p, C.c_char_p, C.c_size_t, C.POINTER(C.c_size_t)]
     lib.atp_input_norm.argtypes = [C.c_void_p, C.POINTER(Mat), C.POINTER(Mat), C.c_int, C.c_float, C.POINTER(Mat)]
+    lib.atp_alternating_basis.argtypes = [C.c_void_p, C.POINTER(Mat), C.POINTER(Seqs), C.POINTER(Mat), C.c_int,
+                                          C.POINTER(Mat), C.POINTER(Mat)]
+    lib.atp_svd_entropy.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int32), C.c_int32, C.c_void_p, C.c_void_p]
     lib.atp_principal_basis.argtypes = [C.c_void_p, C.POINTER(Mat), C.POINTER(Seqs), C.POINTER(BasisOpts),
                                         C.POINTER(Mat), C.POINTER(Mat), C.c_void_p]
     lib.atp_attention.argtypes = [C.c_void_p, C.POINTER(Mat), C.POINTER(Mat), C.POINTER(Mat), C.POINTER(Mat),
@@ -300,3 +303,32 @@ def atp_lowrank_linear_static(U_r, X_r, W, lengths, ranks, out, bias=None, act=N
         _check(lib.atp_lowrank_linear_static(C.c_void_p(s), C.byref(ms[0]), C.byref(ms[1]), C.byref(ms[2]),
                                              C.byref(sd.c), C.byref(opts), C.byref(ms[3])), "atp_lowrank_linear_static")
     return out
+
+
+def atp_alternating_basis(ctx: Context, X, V0, lengths, ranks, inner=2, out=None, auto_workspace=True):
+    """Algorithm 1: (U, X') from alternating rank-1 fits with deflation; see include/atp.h."""
+    sd = SeqDesc(lengths, ranks)
+    d = X.shape[1]
+    maxr = max(sd.ranks) if sd.ranks else 0
+    if out is None:
+        U = torch.zeros((sd.total_rows, (maxr + 7) // 8 * 8), dtype=X.dtype, device=X.device)[:, :maxr]
+        Xr = torch.empty((sd.total_rank, (d + 7) // 8 * 8), dtype=X.dtype, device=X.device)[:, :d]
+    else:
+        U, Xr = out
+    if auto_workspace:
+        ctx.ensure_workspace(ctx.workspace_bytes(OP_ALTERNATING, sd, d, 0, _dt(X)))
+    mx, mv, mu, mxr = mat(X), mat(V0), mat(U), mat(Xr)
+    _check(lib.atp_alternating_basis(ctx._h, C.byref(mx), C.byref(sd.c), C.byref(mv), int(inner), C.byref(mu), C.byref(mxr)),
+           "atp_alternating_basis")
+    return U, Xr
+
+
+def atp_svd_entropy(ctx: Context, sigma: torch.Tensor, counts: Sequence[int]):
+    """(mu, rank) per group of singular values (Eq. 4, rank = ceil(2^mu)); `counts` = group sizes."""
+    off = np.zeros(len(counts) + 1, dtype=np.int32)
+    off[1:] = np.cumsum(np.asarray(counts, dtype=np.int64))
+    mu = torch.empty(len(counts), dtype=torch.float32, device=sigma.device)
+    rk = torch.empty(len(counts), dtype=torch.int32, device=sigma.device)
+    _check(lib.atp_svd_entropy(ctx._h, C.c_void_p(sigma.data_ptr()), off.ctypes.data_as(C.POINTER(C.c_int32)), len(counts),
+                               C.c_void_p(mu.data_ptr()), C.c_void_p(rk.data_ptr())), "atp_svd_entropy")
+    return mu, rk

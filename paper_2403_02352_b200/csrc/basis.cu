@@ -1281,6 +1281,7 @@ extern "C" atp_status atp_workspace_bytes(atp_ctx *ctx, int op, const atp_seqs *
         case ATP_OP_BASIS: *bytes = basis_workspace_bytes(sd, (int)d, 64) + 256; return ATP_OK;
         case ATP_OP_ATTENTION: if (d_out < 1) return ATP_ERR_INVALID_ARG; *bytes = attention_workspace_bytes(sd, d_out) + 256; return ATP_OK;
         case ATP_OP_LINEAR: if (d_out < 1) return ATP_ERR_INVALID_ARG; *bytes = linear_workspace_bytes(sd, d_out) + 256; return ATP_OK;
+        case ATP_OP_ALTERNATING: *bytes = alternating_workspace_bytes(sd, (int)d) + 256; return ATP_OK;
         default: return ATP_ERR_INVALID_ARG;
     }
 }

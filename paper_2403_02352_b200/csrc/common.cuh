@@ -124,3 +124,4 @@ static inline size_t dtype_size(atp_dtype t) { return t == ATP_BF16 ? 2 : 4; }
 struct SeqDims { int row0, L, r, rank0; };
 atp_status check_seqs(const atp_seqs *s, std::vector<SeqDims> &out, int64_t total_rows_expected);
 atp_status check_mat(const atp_mat *m, bool need_data = true);
+size_t alternating_workspace_bytes(const std::vector<SeqDims> &sd, int d);
