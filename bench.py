@@ -92,19 +92,35 @@ class ClockSampler:
         return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def workload_config(w, world):
+ALT_INNER = 2        # rounds per component of Algorithm 1, as the paper runs it
+
+
+def alt_start_vectors(w, seed):
+    """The Gaussian start vectors of Algorithm 1 (one row per component), part of the seeded input."""
+    rng = np.random.default_rng(seed + 7)
+    return [rng.standard_normal((s.r, w.d)).astype(np.float32) for s in w.seqs]
+
+
+def workload_config(w, world, extraction="randomized"):
     ranks = w.ranks
-    return {"workload": w.name, "batch": len(w.lengths), "tokens_per_step_per_gpu": w.tokens, "d": w.d,
+    layer = "basis+attention" + ("+W_O" if "W_O" in w.weights else "") + ("+FFN" if w.ffn else "")
+    if extraction == "alternating":
+        layer = f"attention block: Algorithm 1 extraction (inner {ALT_INNER}) + attention"
+    return {"workload": w.name + ("_alg1" if extraction == "alternating" else ""), "batch": len(w.lengths),
+            "tokens_per_step_per_gpu": w.tokens, "d": w.d,
             "heads": w.heads, "rank": ranks[0] if len(set(ranks)) == 1 else "L_b/4",
-            "ffn": w.ffn, "d_ff": w.d_ff, "input_norm": w.input_norm,
-            "layer": "basis+attention" + ("+W_O" if "W_O" in w.weights else "") + ("+FFN" if w.ffn else ""),
+            "ffn": w.ffn, "d_ff": w.d_ff, "input_norm": w.input_norm, "extraction": extraction,
+            "layer": layer,
             "l2": "flushed between steps (256 MiB memset), rotating input copies",
             "parallelism": f"dp{world} (independent sequences per rank)"}
 
 
-def oracle_step(w, seq_index):
+def oracle_step(w, seq_index, extraction="randomized", v0=None):
     import oracle
     s = w.seqs[seq_index]
+    if extraction == "alternating":
+        U, Xp = oracle.alternating_svd(s.X, s.r, v0[seq_index].astype(np.float64), inner=ALT_INNER)
+        return oracle.attention(s.X, U, Xp, w.weights["W_Q"], w.weights["W_K"], w.weights["W_V"], w.heads)
     return oracle.layer_forward(s.X, w.weights, s.r, w.heads, ffn=w.ffn, input_norm=w.input_norm,
                                 post_norm=POST_NORM[w.ffn])
 
@@ -117,20 +133,22 @@ def run_reference(args):
     import oracle
     w = WORKLOADS[args.workload]["build"](args.rank, args.seed)
     nseq = len(w.seqs)
+    v0 = alt_start_vectors(w, args.seed) if args.extraction == "alternating" else None
     for i in range(args.warmup):
-        oracle_step(w, i % nseq)
+        oracle_step(w, i % nseq, args.extraction, v0)
     t0 = time.perf_counter()
     toks = 0
     for i in range(args.steps):
-        oracle_step(w, i % nseq)
+        oracle_step(w, i % nseq, args.extraction, v0)
         toks += w.seqs[i % nseq].X.shape[0]
     dt = time.perf_counter() - t0
     val = toks / dt
-    sample = f"one sequence of the batch per step ({w.seqs[0].X.shape[0]} tokens), full layer"
+    what = "full layer" if args.extraction == "randomized" else "attention block"
+    sample = f"one sequence of the batch per step ({w.seqs[0].X.shape[0]} tokens), {what}"
     line = {"impl": "reference", "metric": "ATP layer prefill tokens/sec", "value": val, "unit": "tokens/s",
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": dict(workload_config(w, args.gpus), sample="one sequence of the batch per step"),
+            "config": dict(workload_config(w, args.gpus, args.extraction), sample="one sequence of the batch per step"),
             "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -147,6 +165,8 @@ def main():
     ap.add_argument("--rank", type=int, default=0, help="number of principal keys r (0: the workload's default)")
     ap.add_argument("--seed", type=int, default=2000)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--extraction", default="randomized", choices=["randomized", "alternating"],
+                    help="alternating: time the attention block with the paper's Algorithm 1 as the extraction")
     ap.add_argument("--power-iters", type=int, default=-1)
     ap.add_argument("--jacobi-block", type=int, default=0)
     ap.add_argument("--jacobi-inner", type=int, default=0)
@@ -195,8 +215,22 @@ def main():
                                        max_sweeps=args.max_sweeps))
     out_rows, out_cols = None, None
 
-    def step(i):
-        return layer.forward(Xsets[i % nsets])
+    if args.extraction == "alternating":
+        V0 = torch.from_numpy(np.concatenate(alt_start_vectors(w, pdist.rank_seed(args.seed, rank)))).to(dev)
+        bufs = {}
+
+        def step(i):
+            X = Xsets[i % nsets]
+            if "U" not in bufs:
+                bufs["U"], bufs["Xr"] = atp.atp_alternating_basis(ctx, X, V0, lengths, ranks, inner=ALT_INNER)
+            else:
+                atp.atp_alternating_basis(ctx, X, V0, lengths, ranks, inner=ALT_INNER, out=(bufs["U"], bufs["Xr"]))
+            bufs["O"] = atp.atp_attention(ctx, X, bufs["U"], bufs["Xr"], weights["W_Q"], weights["W_K"], weights["W_V"],
+                                          w.heads, lengths, ranks, out=bufs.get("O"))
+            return bufs["O"]
+    else:
+        def step(i):
+            return layer.forward(Xsets[i % nsets])
 
     for i in range(args.warmup):
         y = step(i)
@@ -280,21 +314,23 @@ def main():
     cpu = None
     if not args.no_cpu_baseline and world == 1:
         import oracle
+        v0_cpu = alt_start_vectors(w, args.seed) if args.extraction == "alternating" else None
         t0 = time.perf_counter()
         n = 0
         toks = 0
         while n < len(w.seqs) and (time.perf_counter() - t0 < 15.0 or n == 0):
-            oracle_step(w, n)
+            oracle_step(w, n, args.extraction, v0_cpu)
             toks += w.seqs[n].X.shape[0]
             n += 1
         dt = time.perf_counter() - t0
         cpu = {"value": toks / dt, "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle",
-               "sample": f"{n} of {len(w.seqs)} sequences ({toks} tokens), full layer, {dt:.1f} s"}
+               "sample": f"{n} of {len(w.seqs)} sequences ({toks} tokens), "
+                         f"{'full layer' if args.extraction == 'randomized' else 'attention block'}, {dt:.1f} s"}
 
     line = {"metric": "ATP layer prefill tokens/sec", "value": value, "unit": "tokens/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
-            "config": workload_config(w, world),
+            "config": workload_config(w, world, args.extraction),
             "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)
     pdist.finish()
