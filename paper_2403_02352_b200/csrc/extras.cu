@@ -68,7 +68,7 @@ __global__ void __launch_bounds__(256) alt_u_kernel(const __grid_constant__ AltB
     if (lane == 0) q.u[l] = vv > 0.0 ? (float)(acc / vv) : 0.f;
 }
 
-// v = R^T u / |u|^2; a CTA owns 128 columns, its two halves split the rows.
+// v = R^T u / |u|^2; a CTA owns 64 columns, its four quarters split the rows.
 __global__ void __launch_bounds__(256) alt_v_kernel(const __grid_constant__ AltBatch batch, int d, int comp)
 {
     pdl_trigger();
@@ -76,18 +76,27 @@ __global__ void __launch_bounds__(256) alt_v_kernel(const __grid_constant__ AltB
     const AltSeq &q = batch.s[blockIdx.y];
     if (comp >= q.r) return;
     __shared__ double red[8];
-    __shared__ double half_sum[128];
+    __shared__ double quarter[3][64];
     double part = 0.0;
     for (int l = threadIdx.x; l < q.L; l += 256) { const double x = q.u[l]; part += x * x; }
     const double uu = block_sum_256(part, red);
-    const int c = threadIdx.x & 127, h = threadIdx.x >> 7;
-    const int k = blockIdx.x * 128 + c;
+    const int c = threadIdx.x & 63, h = threadIdx.x >> 6;
+    const int k = blockIdx.x * 64 + c;
     double acc = 0.0;
-    if (k < d)
-        for (int l = h; l < q.L; l += 2) acc = fma((double)q.R[(size_t)l * d + k], (double)q.u[l], acc);
-    if (h == 1) half_sum[c] = acc;
+    if (k < d) {
+        int l = h;
+        for (; l + 28 < q.L; l += 32) {            // eight loads in flight per thread
+            float rv[8], uv[8];
+#pragma unroll
+            for (int t = 0; t < 8; ++t) { rv[t] = q.R[(size_t)(l + 4 * t) * d + k]; uv[t] = q.u[l + 4 * t]; }
+#pragma unroll
+            for (int t = 0; t < 8; ++t) acc = fma((double)rv[t], (double)uv[t], acc);
+        }
+        for (; l < q.L; l += 4) acc = fma((double)q.R[(size_t)l * d + k], (double)q.u[l], acc);
+    }
+    if (h > 0) quarter[h - 1][c] = acc;
     __syncthreads();
-    if (h == 0 && k < d) q.v[k] = uu > 0.0 ? (float)((acc + half_sum[c]) / uu) : 0.f;
+    if (h == 0 && k < d) q.v[k] = uu > 0.0 ? (float)((acc + quarter[0][c] + quarter[1][c] + quarter[2][c]) / uu) : 0.f;
 }
 
 // R <- R - u v^T, and the finished component: U[:, comp] = u / |u|, X'[comp, :] = v |u|.
@@ -153,7 +162,7 @@ static atp_status alternating_impl(atp_ctx *ctx, const atp_mat *X, const std::ve
         alt_copy_kernel<T><<<dim3(std::min(1024, (int)(((size_t)maxL * d + 255) / 256)), b.count), 256, 0, ctx->stream>>>(
             b, (const T *)X->data, (int)X->ld, d, row0_dev + i0);
         ATP_LAUNCHED(ctx);
-        const dim3 grows((maxL + 7) / 8, b.count), gcols((d + 127) / 128, b.count);
+        const dim3 grows((maxL + 7) / 8, b.count), gcols((d + 63) / 64, b.count);
         for (int comp = 0; comp < maxr; ++comp) {
             for (int j = 0; j < inner; ++j) {
                 ATP_KERNEL(ctx, "alt_u", 0, mat_bytes);
