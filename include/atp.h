@@ -145,8 +145,12 @@ ATP_API atp_status atp_input_norm(atp_ctx *ctx, const atp_mat *X, const atp_mat 
  * vectors U_r (L_b x r_b, orthonormal columns) and X_r = U_r^T X = [sigma_1 v_1; ..; sigma_r v_r]
  * (r_b x d), components sorted by sigma descending, i.e. the minimiser of Eq. 9. Computed by a
  * randomised range finder with subspace iteration, block Gram-Schmidt orthonormalisation and a
- * one-sided Jacobi rotation of the projected rows (not by a full SVD), so the subspace is the
- * optimal one up to the range finder's error; opts->power_iters trades passes over X for that.
+ * block Jacobi rotation of the small projected problem (one-sided on the projected rows for f32
+ * input, two-sided on their Gram matrix, in two passes, for bf16 input) - not by a full SVD - so
+ * the subspace is the optimal one up to the range finder's error; opts->power_iters trades passes
+ * over X for that. The Jacobi sweeps stop on a device-side convergence test (largest scaled
+ * off-diagonal <= 1e-6 for f32, 3e-5 for bf16); opts->max_sweeps bounds them, and a sequence that
+ * has not converged by then raises ATP_ERR_NOT_CONVERGED on the device status word.
  * Sign of each component: sum of the column of U_r >= 0; if that sum is within 1e-6*sqrt(L_b) of
  * zero, the largest-magnitude entry of the row of X_r is positive.
  *   X      in   sum(L_b) x d                      (f32 or bf16)

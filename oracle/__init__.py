@@ -83,6 +83,24 @@ def attention(X, U_r, X_r, W_Q, W_K, W_V, heads, q_mode=0, scale=0.0):
     return O
 
 
+def attention_rope(X, U_r, X_r, W_Q, W_K, W_V, heads, positions=None, rope_base=10000.0, q_mode=0, scale=0.0):
+    """Attention on principal keys with rotary positions (Sec. 4.2): K = U_r K' rotated row by row,
+    K'_rot = U_r^T K_rot are the principal keys; queries rotated; positions default to 0..L-1."""
+    U_r = _c(U_r); X_r = _c(X_r); W_Q = _c(W_Q); W_K = _c(W_K); W_V = _c(W_V); X = _c(X)
+    L, r = U_r.shape
+    d = X_r.shape[1]
+    dp = W_Q.shape[1]
+    O = np.empty((L, dp))
+    pos = None if positions is None else np.ascontiguousarray(positions, dtype=np.int32)
+    rc = _load().oracle_attention_rope(_p(X), _p(U_r), _p(X_r), _p(W_Q), _p(W_K), _p(W_V),
+                                       L, d, dp, r, int(heads), int(q_mode), ctypes.c_double(scale),
+                                       None if pos is None else pos.ctypes.data_as(ctypes.c_void_p),
+                                       ctypes.c_double(rope_base), _p(O))
+    if rc < 0:
+        raise ValueError("invalid attention arguments")
+    return O
+
+
 ACT = {None: 0, "none": 0, "gelu": 1, "swiglu": 2}
 
 

@@ -17,6 +17,8 @@
  *   oracle_attention         Q,K,V = U {Q',K',V'} (Eq. 6), then attention of every query on the
  *                            r principal keys/values: the procedure of Eq. 1 with K', V' in place
  *                            of K, V (Sec. 4.1 closing paragraph, Fig. 2 caption)
+ *   oracle_attention_rope    the same with rotary positions: keys rotated, then projected back on
+ *                            U (Sec. 4.2, "Combine with Position Encoding")
  *   oracle_lowrank_linear    linear layers applied to the r-row representation (Sec. 1, Sec. 4.3)
  *   oracle_norm              the "Norm" box of Fig. 3 (RMSNorm / LayerNorm, unit gain)
  *   oracle_alternating_svd   Algorithm 1 (appendix B), the paper's own approximate extraction
@@ -328,6 +330,96 @@ ORACLE_API int oracle_attention(const double *X, const double *U_r, const double
         free(s);
     }
     free(Qp); free(Kp); free(Vp); free(Q);
+    return 0;
+}
+
+/* ------------------------------------------------------------------ */
+/* Rotary position embedding (Sec. 4.2, "Combine with Position          */
+/* Encoding"): k = x W^K R_i with R_i the rotary matrix of position i.   */
+/* R_i is block diagonal, one 2x2 rotation per pair of consecutive      */
+/* coordinates (2j, 2j+1) of a head, by the angle i * base^(-2j/d_h)     */
+/* (the RoFormer definition). Applied in place to the rows of M (L x dp).*/
+/* ------------------------------------------------------------------ */
+static void rope_rows(double *M, int L, int dp, int heads, const int *pos, double base)
+{
+    int dh = dp / heads;
+    for (int l = 0; l < L; ++l) {
+        double p = pos ? (double)pos[l] : (double)l;
+        for (int h = 0; h < heads; ++h) {
+            double *x = M + (size_t)l * dp + (size_t)h * dh;
+            for (int j = 0; j < dh / 2; ++j) {
+                double ang = p * pow(base, -2.0 * j / dh);
+                double c = cos(ang), sn = sin(ang);
+                double a = x[2 * j], b = x[2 * j + 1];
+                x[2 * j] = a * c - b * sn;
+                x[2 * j + 1] = a * sn + b * c;
+            }
+        }
+    }
+}
+
+/* ------------------------------------------------------------------ */
+/* Attention on principal keys with rotary positions. The paper's       */
+/* recipe: rotate the full keys K = U_r K' row by row, then "project     */
+/* the key matrix into a low-dimension space with U": K'_rot = U_r^T     */
+/* K_rot (r x dp) are the principal keys; queries are rotated the same   */
+/* way; values are untouched. pos: L positions (NULL: 0..L-1).           */
+/* ------------------------------------------------------------------ */
+ORACLE_API int oracle_attention_rope(const double *X, const double *U_r, const double *X_r,
+                                     const double *W_Q, const double *W_K, const double *W_V,
+                                     int L, int d, int dp, int r, int heads, int q_mode, double scale,
+                                     const int *pos, double rope_base, double *O)
+{
+    if (heads < 1 || dp % heads != 0 || (dp / heads) % 2 != 0 || !(rope_base > 0.0)) return -1;
+    if (q_mode == 1 && !X) return -1;
+    int dh = dp / heads;
+    if (scale <= 0.0) scale = 1.0 / sqrt((double)dh);
+    double *Qp = (double *)malloc(sizeof(double) * (size_t)r * dp);
+    double *Kp = (double *)malloc(sizeof(double) * (size_t)r * dp);
+    double *Vp = (double *)malloc(sizeof(double) * (size_t)r * dp);
+    double *Q = (double *)malloc(sizeof(double) * (size_t)L * dp);
+    double *K = (double *)malloc(sizeof(double) * (size_t)L * dp);
+    matmul(X_r, W_K, Kp, r, d, dp);
+    matmul(X_r, W_V, Vp, r, d, dp);
+    if (q_mode == 0) {
+        matmul(X_r, W_Q, Qp, r, d, dp);
+        matmul(U_r, Qp, Q, L, r, dp);
+    } else {
+        matmul(X, W_Q, Q, L, d, dp);
+    }
+    matmul(U_r, Kp, K, L, r, dp);                 /* K = U_r K' (Eq. 6) */
+    rope_rows(K, L, dp, heads, pos, rope_base);
+    rope_rows(Q, L, dp, heads, pos, rope_base);
+    for (int i = 0; i < r; ++i)                   /* K'_rot = U_r^T K_rot */
+        for (int c = 0; c < dp; ++c) {
+            double acc = 0.0;
+            for (int l = 0; l < L; ++l) acc += U_r[(size_t)l * r + i] * K[(size_t)l * dp + c];
+            Kp[(size_t)i * dp + c] = acc;
+        }
+    double *s = (double *)malloc(sizeof(double) * (size_t)r);
+    for (int l = 0; l < L; ++l) {
+        for (int h = 0; h < heads; ++h) {
+            const double *q = Q + (size_t)l * dp + (size_t)h * dh;
+            double mx = -INFINITY;
+            for (int i = 0; i < r; ++i) {
+                const double *k = Kp + (size_t)i * dp + (size_t)h * dh;
+                double acc = 0.0;
+                for (int c = 0; c < dh; ++c) acc += q[c] * k[c];
+                s[i] = acc * scale;
+                if (s[i] > mx) mx = s[i];
+            }
+            double den = 0.0;
+            for (int i = 0; i < r; ++i) { s[i] = exp(s[i] - mx); den += s[i]; }
+            double *o = O + (size_t)l * dp + (size_t)h * dh;
+            for (int c = 0; c < dh; ++c) o[c] = 0.0;
+            for (int i = 0; i < r; ++i) {
+                double p = s[i] / den;
+                const double *v = Vp + (size_t)i * dp + (size_t)h * dh;
+                for (int c = 0; c < dh; ++c) o[c] += p * v[c];
+            }
+        }
+    }
+    free(s); free(Qp); free(Kp); free(Vp); free(Q); free(K);
     return 0;
 }
 

@@ -353,3 +353,67 @@ def test_bf16_rounding_is_exact_and_idempotent():
     assert np.abs(b - a).max() <= np.abs(a).max() * 2.0 ** -8
     import torch
     assert np.all(torch.from_numpy(a).to(torch.bfloat16).float().numpy() == b)
+
+
+# ------------------------------------------------------------------ rotary positions (Sec. 4.2)
+def _naive_rope(M, heads, pos, base):
+    """Independent restatement: complex multiplication of consecutive coordinate pairs by e^{i pos theta_j}."""
+    L, dp = M.shape
+    dh = dp // heads
+    out = np.empty_like(M)
+    theta = base ** (-2.0 * np.arange(dh // 2) / dh)
+    for h in range(heads):
+        blk = M[:, h * dh:(h + 1) * dh]
+        z = (blk[:, 0::2] + 1j * blk[:, 1::2]) * np.exp(1j * np.outer(pos, theta))
+        out[:, h * dh + 0:(h + 1) * dh:2] = z.real
+        out[:, h * dh + 1:(h + 1) * dh:2] = z.imag
+    return out
+
+
+def _naive_attention(Q, K, V, heads, scale):
+    L, dp = Q.shape
+    dh = dp // heads
+    O = np.empty((L, dp))
+    for h in range(heads):
+        sl = slice(h * dh, (h + 1) * dh)
+        S = Q[:, sl] @ K[:, sl].T * scale
+        P = np.exp(S - S.max(axis=1, keepdims=True))
+        P /= P.sum(axis=1, keepdims=True)
+        O[:, sl] = P @ V[:, sl]
+    return O
+
+
+def test_attention_rope_pins():
+    rng = np.random.default_rng(123)
+    L, d, heads, dh = 24, 20, 2, 8
+    dp = heads * dh
+    X = rng.standard_normal((L, d))
+    WQ, WK, WV = (rng.standard_normal((d, dp)) / math.sqrt(d) for _ in range(3))
+    pos = rng.integers(0, 50, L)
+    # (1) U = I, r = L: textbook rotary attention on the full keys, written independently
+    I = np.eye(L)
+    got = oracle.attention_rope(X, I, X, WQ, WK, WV, heads, positions=pos, rope_base=100.0)
+    want = _naive_attention(_naive_rope(X @ WQ, heads, pos, 100.0), _naive_rope(X @ WK, heads, pos, 100.0), X @ WV,
+                            heads, 1 / math.sqrt(dh))
+    assert np.abs(got - want).max() < 1e-12
+    # (2) with U = I the result depends on relative positions only: a common shift changes nothing
+    got2 = oracle.attention_rope(X, I, X, WQ, WK, WV, heads, positions=pos + 17, rope_base=100.0)
+    assert np.abs(got2 - got).max() < 1e-10
+    # (3) all positions zero: no rotation, equals the plain principal-key attention for any basis
+    U, Xr, _ = oracle.principal_basis(X, 6)
+    a = oracle.attention_rope(X, U, Xr, WQ, WK, WV, heads, positions=np.zeros(L, dtype=int))
+    b = oracle.attention(X, U, Xr, WQ, WK, WV, heads)
+    assert np.abs(a - b).max() < 1e-12
+    # (4) truncated basis: the principal keys are U^T applied to the rotated keys, checked by composing the pieces
+    Kp = U.T @ _naive_rope(U @ (Xr @ WK), heads, np.arange(L), 10000.0)
+    Qr = _naive_rope(U @ (Xr @ WQ), heads, np.arange(L), 10000.0)
+    want = _naive_attention(Qr, Kp, Xr @ WV, heads, 1 / math.sqrt(dh))
+    got = oracle.attention_rope(X, U, Xr, WQ, WK, WV, heads)          # default positions 0..L-1, base 10000
+    assert np.abs(got - want).max() < 1e-12
+    # (5) exact-query option rotates X W_Q
+    got = oracle.attention_rope(X, U, Xr, WQ, WK, WV, heads, q_mode=1)
+    want = _naive_attention(_naive_rope(X @ WQ, heads, np.arange(L), 10000.0), Kp, Xr @ WV, heads, 1 / math.sqrt(dh))
+    assert np.abs(got - want).max() < 1e-12
+    # odd head width is rejected
+    with pytest.raises(ValueError):
+        oracle.attention_rope(X, U, Xr, WQ[:, :6], WK[:, :6], WV[:, :6], 2)
