@@ -109,6 +109,12 @@ typedef struct {
     uint32_t struct_size;
     int32_t q_mode;        /* atp_q_mode; LOWRANK: Q = U_r (X_r W_Q) (Eq. 6); FULL: Q = X W_Q  */
     float scale;           /* logit scale; <= 0: 1/sqrt(d_h)                                   */
+    float rope_base;       /* 0: no positions. > 1: rotary positions (Sec. 4.2, "Combine with
+                              Position Encoding"): the full keys K = U_r K' and the queries are
+                              rotated row by row - the coordinate pair (2j, 2j+1) of every head by
+                              position * rope_base^(-2j/d_h) - and the principal keys become
+                              K'_rot = U_r^T K_rot. Values are not rotated.                      */
+    const int32_t *positions; /* DEVICE, sum(L_b) ints, or NULL: a row's index in its sequence  */
 } atp_attn_opts;
 
 typedef struct {

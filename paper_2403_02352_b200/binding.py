@@ -49,7 +49,8 @@ class BasisOpts(C.Structure):
 
 
 class AttnOpts(C.Structure):
-    _fields_ = [("struct_size", C.c_uint32), ("q_mode", C.c_int32), ("scale", C.c_float)]
+    _fields_ = [("struct_size", C.c_uint32), ("q_mode", C.c_int32), ("scale", C.c_float), ("rope_base", C.c_float),
+                ("positions", C.c_void_p)]
 
 
 class LinearOpts(C.Structure):
@@ -260,13 +261,16 @@ def atp_principal_basis(ctx: Context, X, lengths, ranks, oversample=-1, power_it
 
 
 def atp_attention(ctx: Context, X, U_r, X_r, W_Q, W_K, W_V, heads, lengths, ranks, q_mode="lowrank", scale=0.0,
-                  out=None, auto_workspace=True):
+                  out=None, auto_workspace=True, rope_base=0.0, positions=None):
     sd = SeqDesc(lengths, ranks)
     dp = W_Q.shape[1]
     O = _padded((sd.total_rows, dp), U_r) if out is None else out
     if auto_workspace:
         ctx.ensure_workspace(ctx.workspace_bytes(OP_ATTENTION, sd, X_r.shape[1], dp, _dt(X_r)))
-    opts = AttnOpts(C.sizeof(AttnOpts), Q_FULL if q_mode == "full" else Q_LOWRANK, scale)
+    if positions is not None and (positions.dtype != torch.int32 or not positions.is_cuda or positions.numel() != sd.total_rows):
+        raise ValueError("positions: CUDA int32 tensor with one entry per row")
+    opts = AttnOpts(C.sizeof(AttnOpts), Q_FULL if q_mode == "full" else Q_LOWRANK, scale, rope_base,
+                    C.c_void_p(positions.data_ptr()) if positions is not None else None)
     mx = mat(X)
     ms = [mat(t) for t in (U_r, X_r, W_Q, W_K, W_V, O)]
     _check(lib.atp_attention(ctx._h, C.byref(mx) if mx else None, C.byref(ms[0]), C.byref(ms[1]), C.byref(ms[2]),

@@ -123,13 +123,40 @@ attn_simt_kernel(const __grid_constant__ AttnBatch batch, int dh, int ldq, int l
     }
 }
 
-struct AttnPlan { float *Qp, *Kp, *Vp, *Q; __nv_bfloat16 *Qph, *Qpl, *Kh, *Kl, *Vb, *Qh, *Ql; float *nrm; };
+// Rotary positions (Sec. 4.2, position-encoding paragraph): every row of M (fp32, rows x dp) is rotated
+// by its position: the pair of coordinates (2j, 2j+1) of each head turns by pos * base^(-2j/d_h).
+// pos: per-row positions or nullptr (row index inside its sequence, given by seq_row0). The angle is
+// formed in fp64: at position 3e4 an fp32 angle would already be off by 2e-3 rad.
+struct RopeSeq { float *K, *Q; int L, row0; };
+struct RopeBatch { RopeSeq s[32]; int count; };
+__global__ void __launch_bounds__(256) rope_kernel(const __grid_constant__ RopeBatch batch, int dp, int dh, double log2_base,
+                                                   const int *pos)
+{
+    const RopeSeq &q = batch.s[blockIdx.y];
+    const int half = dp / 2;
+    const size_t n = (size_t)q.L * half;
+    for (size_t e = (size_t)blockIdx.x * 256 + threadIdx.x; e < n; e += (size_t)gridDim.x * 256) {
+        const int l = (int)(e / half), pr = (int)(e - (size_t)l * half);
+        const int j = pr % (dh / 2);
+        const double p = pos ? (double)pos[q.row0 + l] : (double)l;
+        double sn, c;
+        sincos(p * exp2(-2.0 * j / dh * log2_base), &sn, &c);
+        const float cf = (float)c, sf = (float)sn;
+        float *k = q.K + (size_t)l * dp + 2 * pr, *x = q.Q + (size_t)l * dp + 2 * pr;
+        const float ka = k[0], kb = k[1], xa = x[0], xb = x[1];
+        k[0] = ka * cf - kb * sf; k[1] = ka * sf + kb * cf;
+        x[0] = xa * cf - xb * sf; x[1] = xa * sf + xb * cf;
+    }
+}
+
+struct AttnPlan { float *Qp, *Kp, *Vp, *Q, *Kf; __nv_bfloat16 *Qph, *Qpl, *Kh, *Kl, *Vb, *Qh, *Ql; float *nrm; };
 static void plan_attn(Arena &ar, int64_t tr, int64_t tl, int64_t dp, int64_t nseq, AttnPlan &p)
 {
     p.Qp = ar.take<float>((size_t)tr * dp);
     p.Kp = ar.take<float>((size_t)tr * dp);
     p.Vp = ar.take<float>((size_t)tr * dp);
     p.Q = ar.take<float>((size_t)tl * dp);
+    p.Kf = ar.take<float>((size_t)tl * dp);                                     // full keys U_r K' (rotary positions only)
     p.Qph = ar.take<__nv_bfloat16>((size_t)tr * align_up((size_t)dp, 8));     // Q' as a bf16 hi/lo pair (tensor-core path)
     p.Qpl = ar.take<__nv_bfloat16>((size_t)tr * align_up((size_t)dp, 8));
     p.Kh = ar.take<__nv_bfloat16>((size_t)tr * align_up((size_t)dp, 8));      // fused tensor-core attention operands
@@ -152,9 +179,11 @@ size_t attention_workspace_bytes(const std::vector<SeqDims> &seqs, int64_t dp)
 template <typename T>
 static atp_status attention_impl(atp_ctx *ctx, const atp_mat *X, const atp_mat *U_r, const atp_mat *X_r,
                                  const atp_mat *WQ, const atp_mat *WK, const atp_mat *WV, int heads,
-                                 const std::vector<SeqDims> &seqs, int q_mode, float scale, atp_mat *O)
+                                 const std::vector<SeqDims> &seqs, int q_mode, float scale, float rope_base, const int *positions,
+                                 atp_mat *O)
 {
     const int d = (int)X_r->cols, dp = (int)WQ->cols, dh = dp / heads;
+    const bool rope = rope_base > 0.f;
     int64_t tr = 0, tl = 0;
     for (auto &s : seqs) { tr += s.r; tl += s.L; }
     Arena ar(ctx->workspace, ctx->workspace_bytes);
@@ -164,7 +193,7 @@ static atp_status attention_impl(atp_ctx *ctx, const atp_mat *X, const atp_mat *
     atp_status st;
     GemmEpi store{EPI_STORE, nullptr};
     if constexpr (std::is_same<T, __nv_bfloat16>::value) {
-        if (dh == 64 || dh == 128) {
+        if ((dh == 64 || dh == 128) && !rope) {
             // bf16, head width 64 or 128: everything on the tensor cores. K' and Q are produced as
             // bf16 hi/lo pairs by the GEMM epilogues, V' as bf16; the fused kernel does the rest.
             const int ldq = (int)align_up((size_t)dp, 8);
@@ -243,6 +272,65 @@ static atp_status attention_impl(atp_ctx *ctx, const atp_mat *X, const atp_mat *
         if ((st = launch_gemm_simt<T, T, float, false>(ctx, b, store)) != ATP_OK) return st;
     }
     }
+    if (rope) {
+        // K = U_r K' (Eq. 6), rows of K and Q rotated by their positions, principal keys K'_rot = U_r^T K_rot
+        std::vector<GemmProblem> up, down;
+        RopeBatch rb; rb.count = 0;
+        auto flush_rope = [&]() -> atp_status {
+            if (rb.count == 0) return ATP_OK;
+            int maxL = 0;
+            for (int i = 0; i < rb.count; ++i) maxL = std::max(maxL, rb.s[i].L);
+            ATP_KERNEL(ctx, "rope", 0, 0);
+            rope_kernel<<<dim3(std::min(512, ceil_div(maxL * (dp / 2), 256)), rb.count), 256, 0, ctx->stream>>>(
+                rb, dp, dh, log2((double)rope_base), positions);
+            ATP_LAUNCHED(ctx);
+            rb.count = 0;
+            return ATP_OK;
+        };
+        for (auto &sq : seqs)
+            if (sq.L > 0)
+                up.push_back(GemmProblem{(const T *)U_r->data + (size_t)sq.row0 * U_r->ld, pl.Kp + (size_t)sq.rank0 * dp,
+                                         pl.Kf + (size_t)sq.row0 * dp, nullptr, sq.L, dp, sq.r, (int)U_r->ld, dp, dp, 0});
+        st = for_each_chunk(up, [&](const GemmBatch &b) { return launch_gemm_simt<T, float, float, false>(ctx, b, store, 1, nullptr, 0, "gemm_simt_rope"); });
+        if (st != ATP_OK) return st;
+        for (auto &sq : seqs)
+            if (sq.L > 0) {
+                rb.s[rb.count++] = RopeSeq{pl.Kf + (size_t)sq.row0 * dp, pl.Q + (size_t)sq.row0 * dp, sq.L, sq.row0};
+                if (rb.count == 32 && (st = flush_rope()) != ATP_OK) return st;
+            }
+        if ((st = flush_rope()) != ATP_OK) return st;
+        for (auto &sq : seqs)
+            if (sq.L > 0)
+                down.push_back(GemmProblem{(const T *)U_r->data + (size_t)sq.row0 * U_r->ld, pl.Kf + (size_t)sq.row0 * dp,
+                                           pl.Kp + (size_t)sq.rank0 * dp, nullptr, sq.r, dp, sq.L, (int)U_r->ld, dp, dp, 0});
+        st = for_each_chunk(down, [&](const GemmBatch &b) { return launch_gemm_simt<T, float, float, true>(ctx, b, store, 1, nullptr, 0, "gemm_simt_rope"); });
+        if (st != ATP_OK) return st;
+    }
+    if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+        if (dh == 64 || dh == 128) {
+            // rotary positions with a tensor-core head width: the fp32 K'_rot, Q_rot and V' are cut into the
+            // bf16 (hi/lo) operands of the fused kernel
+            const int ldq = (int)align_up((size_t)dp, 8);
+            ATP_KERNEL(ctx, "f32_to_bf16", 0, (double)(2 * tr + tl) * dp * 8);
+            tc::f32_to_bf16_split_kernel<<<1024, 256, 0, ctx->stream>>>(pl.Kp, dp, pl.Kh, pl.Kl, ldq, (int)tr, dp);
+            ATP_LAUNCHED(ctx);
+            tc::f32_to_bf16_split_kernel<<<1024, 256, 0, ctx->stream>>>(pl.Q, dp, pl.Qh, pl.Ql, ldq, (int)tl, dp);
+            ATP_LAUNCHED(ctx);
+            tc::f32_to_bf16_split_kernel<<<1024, 256, 0, ctx->stream>>>(pl.Vp, dp, pl.Vb, pl.Qpl, ldq, (int)tr, dp);   // lo part unused
+            ATP_LAUNCHED(ctx);
+            std::vector<atc::HostSeq> hs;
+            float *nrm = pl.nrm;
+            for (auto &sq : seqs)
+                if (sq.L > 0) {
+                    float *qmax = nrm, *kmax = nrm + heads;
+                    nrm += heads + (size_t)heads * ceil_div(sq.r, 128);
+                    hs.push_back(atc::HostSeq{pl.Qh + (size_t)sq.row0 * ldq, pl.Ql + (size_t)sq.row0 * ldq, pl.Kh + (size_t)sq.rank0 * ldq,
+                                              pl.Kl + (size_t)sq.rank0 * ldq, pl.Vb + (size_t)sq.rank0 * ldq,
+                                              (T *)O->data + (size_t)sq.row0 * O->ld, sq.L, sq.r, ldq, ldq, (int)O->ld, dp, qmax, kmax});
+                }
+            return dh == 64 ? atc::launch<64>(ctx, hs, heads, scale) : atc::launch<128>(ctx, hs, heads, scale);
+        }
+    }
     size_t smem = ((size_t)dh * 68 * 2 + (size_t)64 * dh + 64 * 65) * sizeof(float);
     ATP_CUDA_OK(ctx, cudaFuncSetAttribute(attn_simt_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     for (size_t i = 0; i < seqs.size(); i += ATT_MAX_BATCH) {
@@ -274,11 +362,14 @@ extern "C" atp_status atp_attention(atp_ctx *ctx, const atp_mat *X, const atp_ma
     if ((st = check_mat(U_r)) != ATP_OK || (st = check_mat(X_r)) != ATP_OK || (st = check_mat(W_Q)) != ATP_OK ||
         (st = check_mat(W_K)) != ATP_OK || (st = check_mat(W_V)) != ATP_OK || (st = check_mat(O)) != ATP_OK)
         return st;
-    int q_mode = ATP_Q_LOWRANK; float scale = 0.f;
+    int q_mode = ATP_Q_LOWRANK; float scale = 0.f, rope_base = 0.f; const int32_t *positions = nullptr;
     if (opts) {
-        if (opts->struct_size < sizeof(atp_attn_opts)) return ATP_ERR_INVALID_ARG;
+        // the struct grew by the rotary fields: a caller built against the shorter layout gets no rotation
+        if (opts->struct_size < offsetof(atp_attn_opts, rope_base)) return ATP_ERR_INVALID_ARG;
         q_mode = opts->q_mode; scale = opts->scale;
+        if (opts->struct_size >= sizeof(atp_attn_opts)) { rope_base = opts->rope_base; positions = opts->positions; }
     }
+    if (rope_base < 0.f || (rope_base > 0.f && rope_base <= 1.f)) return ATP_ERR_INVALID_ARG;
     if (q_mode != ATP_Q_LOWRANK && q_mode != ATP_Q_FULL) return ATP_ERR_INVALID_ARG;
     if (q_mode == ATP_Q_FULL) {
         if (!X || (st = check_mat(X)) != ATP_OK) return st != ATP_OK ? st : ATP_ERR_INVALID_ARG;
@@ -300,6 +391,6 @@ extern "C" atp_status atp_attention(atp_ctx *ctx, const atp_mat *X, const atp_ma
     if (U_r->rows == 0) return ATP_OK;
     if (!(scale > 0.f)) scale = 1.0f / sqrtf((float)dh);
     ATP_CUDA_OK(ctx, cudaSetDevice(ctx->device));
-    if (dt == ATP_F32) return attention_impl<float>(ctx, X, U_r, X_r, W_Q, W_K, W_V, heads, sd, q_mode, scale, O);
-    return attention_impl<__nv_bfloat16>(ctx, X, U_r, X_r, W_Q, W_K, W_V, heads, sd, q_mode, scale, O);
+    if (dt == ATP_F32) return attention_impl<float>(ctx, X, U_r, X_r, W_Q, W_K, W_V, heads, sd, q_mode, scale, rope_base, positions, O);
+    return attention_impl<__nv_bfloat16>(ctx, X, U_r, X_r, W_Q, W_K, W_V, heads, sd, q_mode, scale, rope_base, positions, O);
 }

@@ -108,3 +108,50 @@ def test_svd_entropy_of_a_full_spectrum_from_the_basis_call(ctx):
     s = oracle.svd_jacobi(X)[1]
     want = oracle.svd_entropy(s)
     assert abs(float(mu[0]) - want) <= 1e-4 * max(1.0, want)
+
+
+# ------------------------------------------------------------------ rotary positions (Sec. 4.2)
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("q_mode", ["lowrank", "full"])
+@pytest.mark.parametrize("L,d,heads,dh,r", [(150, 128, 2, 64, 45), (70, 96, 3, 32, 70), (257, 256, 2, 128, 129)])
+def test_attention_with_rotary_positions_on_oracle_basis(ctx, dtype, q_mode, L, d, heads, dh, r):
+    rng = np.random.default_rng(900 + L + r)
+    X = _planted(rng, L, d, 10, dtype)
+    dp = heads * dh
+    W = [ai.finish(ai.gaussian_weight(rng, d, dp), dtype) for _ in range(3)]
+    U, Xr, _ = oracle.principal_basis(X, r)
+    U, Xr = ai.finish(U, dtype), ai.finish(Xr, dtype)
+    pos = rng.integers(0, 4000, L).astype(np.int32)
+    want = oracle.attention_rope(X, U, Xr, W[0], W[1], W[2], heads, positions=pos, rope_base=10000.0,
+                                 q_mode=1 if q_mode == "full" else 0)
+    got = _atp().atp_attention(ctx, to_dev(X, dtype), to_dev(U, dtype), to_dev(Xr, dtype), *(to_dev(w, dtype) for w in W),
+                               heads, [L], [r], q_mode=q_mode, rope_base=10000.0, positions=torch.from_numpy(pos).cuda())
+    ctx.poll()
+    assert rel_err(to_np(got), want) <= TOL[dtype]
+
+
+def test_rotary_positions_default_to_row_index_per_sequence_and_zero_positions_are_plain_attention(ctx):
+    rng = np.random.default_rng(31)
+    lengths, ranks, d, heads, dh = [40, 0, 75], [10, 0, 20], 64, 2, 32
+    dp = heads * dh
+    Xs = [_planted(rng, L, d, 6, "f32") if L else np.zeros((0, d)) for L in lengths]
+    W = [ai.finish(ai.gaussian_weight(rng, d, dp), "f32") for _ in range(3)]
+    bases = [oracle.principal_basis(x, r)[:2] if len(x) else (np.zeros((0, 0)), np.zeros((0, d))) for x, r in zip(Xs, ranks)]
+    maxr = max(ranks)
+    Upack = np.zeros((sum(lengths), maxr)); row = 0
+    for (U, _), L, r in zip(bases, lengths, ranks):
+        Upack[row:row + L, :r] = U; row += L
+    Xrpack = np.concatenate([b[1] for b in bases])
+    args = (to_dev(np.concatenate(Xs), "f32"), to_dev(Upack, "f32"), to_dev(Xrpack, "f32"), *(to_dev(w, "f32") for w in W))
+    got = to_np(_atp().atp_attention(ctx, *args, heads, lengths, ranks, rope_base=500.0))
+    zero = to_np(_atp().atp_attention(ctx, *args, heads, lengths, ranks, rope_base=500.0,
+                                      positions=torch.zeros(sum(lengths), dtype=torch.int32, device="cuda")))
+    plain = to_np(_atp().atp_attention(ctx, *args, heads, lengths, ranks))
+    ctx.poll()
+    assert rel_err(zero, plain) <= 1e-6
+    row = 0
+    for x, (U, Xr), L, r in zip(Xs, bases, lengths, ranks):
+        if L:
+            want = oracle.attention_rope(x, U, Xr, W[0], W[1], W[2], heads, rope_base=500.0)     # positions 0..L-1
+            assert rel_err(got[row:row + L], want) <= 1e-4
+        row += L
