@@ -302,8 +302,12 @@ def main():
         return "hbm", by / per_launch_s / 1e9, pk["hbm_gbs"], "GB/s"
 
     bound, achieved, peak, unit = rate(dom_name, dom)
+    # DRAM bytes per launch (read + write) of one ncu capture of the current kernels on the default workload
+    # (profiles/ncu_*_bert_large_bf16.md); taken with ncu's cache flush, so for these L2-resident kernels it is what
+    # a cold launch reads, not what a launch inside the step moves. Other kernels / workloads: no capture, null.
+    traffic = {"jac2_apply": 11.2e6, "jac2_local": 1.3e6}.get(dom_name) if args.workload == "bert_large_bf16" else None
     roofline = {"kernel": dom_name, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
-                "frac": achieved / peak, "traffic": None, "peak_source": pk["source"],
+                "frac": achieved / peak, "traffic": traffic, "peak_source": pk["source"],
                 "share_of_step": dom["ms"] / total_ms,
                 "kernels": {k: {"launches": v["launches"] // nprof, "ms_per_step": v["ms"] / nprof,
                                 "share": v["ms"] / total_ms, "bound": rate(k, v)[0], "achieved": rate(k, v)[1],
