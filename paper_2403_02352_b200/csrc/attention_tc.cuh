@@ -53,7 +53,7 @@ __device__ __forceinline__ float fast_exp2(float x)
 
 template <int DH> struct Cfg {
     static constexpr int TILE = 128 * DH * 2;                   // one 128-row operand tile (bf16)
-    static constexpr int NSLOT = (DH == 128) ? 3 : 6;           // K'_hi / K'_lo / V' tile slots
+    static constexpr int NSLOT = (DH == 128) ? 4 : 6;           // K'_hi / K'_lo / V' tile slots (a ring: the loads run ahead of the MMAs)
     static constexpr int NPBUF = (DH == 128) ? 1 : 2;           // P buffers (shared memory allows two at d_h = 64)
     static constexpr int P_BYTES = 128 * 128 * 2;               // one P buffer
     static constexpr int OFF_Q = 0;                             // Q hi, Q lo
@@ -63,7 +63,9 @@ template <int DH> struct Cfg {
     // q, slot full/empty, s_full[2], s_free[2], p_full[2], p_free[2], o_done, xchg
     static constexpr int NBAR = 1 + 2 * NSLOT + 2 + 2 + 2 + 2 + 1 + 1;
     static constexpr int OFF_XCH = OFF_BAR + 8 * NBAR + 16;     // float[2 parity][2 halves][128 rows]
-    static constexpr int SMEM = OFF_XCH + 2 * 2 * 128 * 4 + 1024;
+    // no slack for aligning the base: the kernel has no static shared memory, so its dynamic window starts
+    // on a 1024-byte boundary (checked at run time); with four 32 KB slots at d_h = 128 every byte counts
+    static constexpr int SMEM = OFF_XCH + 2 * 2 * 128 * 4;
 };
 
 // Warps 0-7: softmax (warp w and w + 4 share the TMEM lanes 32 (w & 3) .. and split the 128 keys of a
@@ -75,15 +77,18 @@ attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e
     using C_ = Cfg<DH>;
     constexpr int NS = C_::NSLOT, NP = C_::NPBUF;
     extern __shared__ uint8_t smem_raw[];
-    const uint32_t raw = smem_u32(smem_raw);
-    const uint32_t base = (raw + 1023u) & ~1023u;
-    uint8_t *gbase = smem_raw + (base - raw);
+    const uint32_t base = smem_u32(smem_raw);
+    uint8_t *gbase = smem_raw;
+    if (base & 1023u) {                                         // the swizzled tiles need 1024-byte alignment
+        if (threadIdx.x == 0 && dev_status) raise_status(dev_status, ATP_ERR_CUDA);
+        return;
+    }
     const uint32_t bar0 = base + C_::OFF_BAR;
     const uint32_t b_q = bar0, b_full = bar0 + 8, b_empty = b_full + 8 * NS, b_sfull = b_empty + 8 * NS, b_sfree = b_sfull + 16,
                    b_pfull = b_sfree + 16, b_pfree = b_pfull + 16, b_odone = b_pfree + 16, b_xchg = b_odone + 8;
     uint32_t *tmem_slot = (uint32_t *)(gbase + C_::OFF_BAR + 8 * C_::NBAR);
     float *xch = (float *)(gbase + C_::OFF_XCH);
-    __shared__ int abort_flag;
+    volatile int &abort_flag = *(volatile int *)(tmem_slot + 1);
 
     // work item: (sequence, query tile) from blockIdx.x, head from blockIdx.y
     int si = 0;
@@ -212,21 +217,31 @@ attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e
             tc_fence_after();
             const uint32_t t_s = t_s0 + 128 * (j & 1) + lane_addr + half * 64;
             const int kvalid = sq.r - j * 128 - half * 64;            // keys of this half-block that exist
-            // pass A: maximum of the raw scores of this half (the scale is positive: applied once)
-            float mx = -INFINITY;
+            // the 64 scores of this half go to registers in one go (both loads in flight), which frees the S
+            // buffer for the score products of block j + 2 before any arithmetic here
+            uint32_t sa[32], sb[32];
+            tmem_ld32_nowait(t_s, sa);
+            tmem_ld32_nowait(t_s + 32, sb);
+            tmem_ld_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(b_sfree + 8 * (j & 1));
+            // maximum of the raw scores (the scale is positive: applied once); four independent chains
+            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            if (kvalid >= 64) {
 #pragma unroll
-            for (int c = 0; c < 64; c += 32) {
-                uint32_t rr[32];
-                tmem_ld32(t_s + c, rr);
-                if (kvalid >= 64) {
+                for (int i = 0; i < 32; ++i) {
+                    mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(sa[i]));
+                    mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(sb[i]));
+                }
+            } else {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(rr[i]));
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (c + i < kvalid) mx = fmaxf(mx, __uint_as_float(rr[i]));
+                for (int i = 0; i < 32; ++i) {
+                    if (i < kvalid) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(sa[i]));
+                    if (32 + i < kvalid) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(sb[i]));
                 }
             }
+            float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
             // exchange with the thread that holds the other half of the row
             float *xb = xch + (j & 1) * 256;
             xb[half * 128 + row] = mx;
@@ -265,10 +280,10 @@ attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e
             // region); the row sum is taken from the unrounded values
             uint8_t *prow = gbase + C_::OFF_P + pb * C_::P_BYTES + half * 16384 + row * 128;
             const float neg_m = -m_used;
+            float ls[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int c = 0; c < 64; c += 32) {
-                uint32_t rr[32];
-                tmem_ld32(t_s + c, rr);
+                const uint32_t (&rr)[32] = (c == 0) ? sa : sb;
                 uint32_t packed[16];
 #pragma unroll
                 for (int i = 0; i < 32; i += 2) {
@@ -278,7 +293,7 @@ attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e
                         if (c + i >= kvalid) p0 = 0.f;
                         if (c + i + 1 >= kvalid) p1 = 0.f;
                     }
-                    l_sum += p0 + p1;
+                    ls[(i >> 1) & 3] += p0 + p1;
                     __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
                     packed[i >> 1] = *(uint32_t *)&h;
                 }
@@ -289,10 +304,11 @@ attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e
                     *(uint4 *)(prow + ((within ^ (row & 7)) << 4)) = val;
                 }
             }
+            l_sum += (ls[0] + ls[1]) + (ls[2] + ls[3]);
             tc_fence_before();
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA
             __syncwarp();
-            if (lane == 0) { mbar_arrive(b_sfree + 8 * (j & 1)); mbar_arrive(b_pfull + 8 * pb); }
+            if (lane == 0) mbar_arrive(b_pfull + 8 * pb);
         }
         // epilogue: O / l, with l summed over the two halves of the row
         if (ok) {
