@@ -53,13 +53,12 @@ __device__ __forceinline__ float fast_exp2(float x)
 
 template <int DH> struct Cfg {
     static constexpr int TILE = 128 * DH * 2;                   // one 128-row operand tile (bf16)
-    static constexpr int NSLOT = (DH == 128) ? 4 : 6;           // K'_hi / K'_lo / V' tile slots (a ring: the loads run ahead of the MMAs)
-    static constexpr int NPBUF = (DH == 128) ? 1 : 2;           // P buffers (shared memory allows two at d_h = 64)
-    static constexpr int P_BYTES = 128 * 128 * 2;               // one P buffer
+    static constexpr int NSLOT = (DH == 128) ? 5 : 6;           // K'_hi / K'_lo / V' tile slots (a ring: the loads run ahead of the MMAs)
+    static constexpr int NPBUF = 2;                             // P buffers, in tensor memory (64 columns each)
     static constexpr int OFF_Q = 0;                             // Q hi, Q lo
     static constexpr int OFF_SLOT = 2 * TILE;
-    static constexpr int OFF_P = OFF_SLOT + NSLOT * TILE;
-    static constexpr int OFF_BAR = OFF_P + NPBUF * P_BYTES;
+    static constexpr int OFF_P = OFF_SLOT + NSLOT * TILE;       // (no shared-memory P any more: barriers follow the slots)
+    static constexpr int OFF_BAR = OFF_P;
     // q, slot full/empty, s_full[2], s_free[2], p_full[2], p_free[2], o_done, xchg
     static constexpr int NBAR = 1 + 2 * NSLOT + 2 + 2 + 2 + 2 + 1 + 1;
     static constexpr int OFF_XCH = OFF_BAR + 8 * NBAR + 16;     // float[2 parity][2 halves][128 rows]
@@ -121,7 +120,7 @@ attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t t_s0 = tmem_base, t_o = tmem_base + 256;
+    const uint32_t t_s0 = tmem_base, t_o = tmem_base + 256, t_p0 = tmem_base + 384;   // S0 S1 | O | P0 P1
 
     if (warp == 8) {
         if (lane == 0) {
@@ -186,12 +185,11 @@ attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e
                 if (!mbar_wait(b_full + 8 * sv, (lv / NS) & 1, &abort_flag)) { ok = false; break; }
                 if (!mbar_wait(b_pfull + 8 * pb, pu & 1, &abort_flag)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t pv = base + C_::OFF_P + pb * C_::P_BYTES, vv = base + C_::OFF_SLOT + sv * C_::TILE;
+                const uint32_t tp = t_p0 + 64 * pb, vv = base + C_::OFF_SLOT + sv * C_::TILE;
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const uint64_t ap = smem_desc(pv + (kk >> 2) * 16384 + (kk & 3) * 32, 16, 1024);
+                for (int kk = 0; kk < 8; ++kk) {                 // A = P from tensor memory: 16 keys = 8 columns per step
                     const uint64_t bv = smem_desc(vv + kk * 2048, 16384, 1024);
-                    umma_bf16(t_o, ap, bv, idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
+                    umma_bf16_ts(t_o, tp + 8 * kk, bv, idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
                 }
                 umma_commit(b_empty + 8 * sv);
                 umma_commit(b_pfree + 8 * pb);
@@ -276,15 +274,14 @@ attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e
                 ok = wait_all(b_pfree + 8 * pb, (pu - 1) & 1);
                 if (!ok) break;
             }
-            // pass B: P = exp2(s * c - m) as bf16 into the swizzled K-major A tile (this half = one 64-key
-            // region); the row sum is taken from the unrounded values
-            uint8_t *prow = gbase + C_::OFF_P + pb * C_::P_BYTES + half * 16384 + row * 128;
+            // P = exp2(s * c - m) as bf16 pairs into tensor memory (this half = 32 columns of the P buffer: the A
+            // operand of the value MMA); the row sum is taken from the unrounded values
             const float neg_m = -m_used;
             float ls[4] = {0.f, 0.f, 0.f, 0.f};
+            uint32_t packed[32];
 #pragma unroll
             for (int c = 0; c < 64; c += 32) {
                 const uint32_t (&rr)[32] = (c == 0) ? sa : sb;
-                uint32_t packed[16];
 #pragma unroll
                 for (int i = 0; i < 32; i += 2) {
                     float p0 = fast_exp2(fmaf(__uint_as_float(rr[i]), scale_log2e, neg_m));
@@ -295,18 +292,12 @@ attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e
                     }
                     ls[(i >> 1) & 3] += p0 + p1;
                     __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-                    packed[i >> 1] = *(uint32_t *)&h;
-                }
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {                           // four 16-byte chunks of 8 keys
-                    const int within = (c >> 3) + q;                    // 0..7 inside the 64-key region
-                    uint4 val = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
-                    *(uint4 *)(prow + ((within ^ (row & 7)) << 4)) = val;
+                    packed[(c + i) >> 1] = *(uint32_t *)&h;
                 }
             }
             l_sum += (ls[0] + ls[1]) + (ls[2] + ls[3]);
+            tmem_st32(t_p0 + 64 * pb + lane_addr + half * 32, packed);
             tc_fence_before();
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA
             __syncwarp();
             if (lane == 0) mbar_arrive(b_pfull + 8 * pb);
         }
