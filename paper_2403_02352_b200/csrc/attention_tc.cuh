@@ -68,9 +68,9 @@ template <int DH> struct Cfg {
 };
 
 // Warps 0-7: softmax (warp w and w + 4 share the TMEM lanes 32 (w & 3) .. and split the 128 keys of a
-// block in halves), warp 8: TMA, warp 9: MMA.
+// block in halves), warp 8: TMA, warp 9: score MMAs, warp 10: value MMAs.
 template <int DH>
-__global__ void __launch_bounds__(320)
+__global__ void __launch_bounds__(352)
 attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e, float lo_thresh, int *dev_status)
 {
     using C_ = Cfg<DH>;
@@ -147,7 +147,6 @@ attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e
     } else if (warp == 9) {
         if (lane == 0) {
             constexpr uint32_t idesc_s = instr_desc(128, 128, false, false);
-            constexpr uint32_t idesc_o = instr_desc(128, DH, false, true);
             const uint32_t q_hi = base + C_::OFF_Q, q_lo = q_hi + C_::TILE;
             bool ok = mbar_wait(b_q, 0, &abort_flag);
             tc_fence_after();
@@ -177,9 +176,15 @@ attn_tc_kernel(const __grid_constant__ Batch batch, int heads, float scale_log2e
                 umma_commit(b_sfull + 8 * (j & 1));
                 return true;
             };
-            if (ok) ok = issue_s(0);
+            for (int j = 0; j < nblk && ok; ++j) ok = issue_s(j);
+        }
+    } else if (warp == 10) {
+        // the value MMAs have their own issuing thread: they are independent of the score MMAs of the next
+        // block (other accumulator), and two instruction streams let the tensor pipe take them in either order
+        if (lane == 0) {
+            constexpr uint32_t idesc_o = instr_desc(128, DH, false, true);
+            bool ok = true;
             for (int j = 0; j < nblk && ok; ++j) {
-                if (j + 1 < nblk) { ok = issue_s(j + 1); if (!ok) break; }
                 // O += P_j V_j
                 const int lv = 3 * j + 2, sv = lv % NS, pb = j % NP, pu = j / NP;
                 if (!mbar_wait(b_full + 8 * sv, (lv / NS) & 1, &abort_flag)) { ok = false; break; }
@@ -410,7 +415,7 @@ static atp_status launch(atp_ctx *ctx, const std::vector<HostSeq> &seqs, int hea
         ATP_KERNEL(ctx, "attn_tc", flops, bytes);
         // drop the lo products of a key block when scale * |q|max * |k|max * 2^-8 <= 2^-10 (logit error bound)
         const float lo_thresh = 0.25f / scale;
-        attn_tc_kernel<DH><<<dim3(b.total_tiles, heads), 320, C_::SMEM, ctx->stream>>>(b, heads, scale * 1.4426950408889634f, lo_thresh, ctx->dev_status);
+        attn_tc_kernel<DH><<<dim3(b.total_tiles, heads), 352, C_::SMEM, ctx->stream>>>(b, heads, scale * 1.4426950408889634f, lo_thresh, ctx->dev_status);
         ATP_LAUNCHED(ctx);
     }
     return ATP_OK;
