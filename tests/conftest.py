@@ -8,8 +8,20 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 
+def _ensure_library():
+    """The package refuses to import without libatp.so (no fallback path), so a fresh tree builds it first;
+    build.py is loaded by path for the same reason."""
+    import importlib.util
+    path = os.path.join(ROOT, "paper_2403_02352_b200", "build.py")
+    spec = importlib.util.spec_from_file_location("_atp_build", path)
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    mod.build()
+
+
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run on a B200)")
+    _ensure_library()
 
 
 def pytest_collection_modifyitems(config, items):
