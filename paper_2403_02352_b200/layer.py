@@ -17,12 +17,14 @@ from . import binding as B
 class AtpLayer:
     def __init__(self, ctx: B.Context, weights: Dict[str, torch.Tensor], lengths: Sequence[int], ranks: Sequence[int],
                  heads: int, ffn: Optional[str] = None, input_norm: Optional[str] = None, post_norm: str = "layer",
-                 power_iters: int = -1, oversample: int = -1, seed: int = 0, basis_kwargs: Optional[dict] = None):
+                 power_iters: int = -1, oversample: int = -1, seed: int = 0, basis_kwargs: Optional[dict] = None,
+                 q_mode: str = "lowrank", rope_base: float = 0.0):
         self.ctx, self.w = ctx, weights
         self.lengths, self.ranks = [int(x) for x in lengths], [int(x) for x in ranks]
         self.heads, self.ffn, self.input_norm, self.post_norm = heads, ffn, input_norm, post_norm
         self.power_iters, self.oversample, self.seed = power_iters, oversample, seed
         self.basis_kwargs = dict(basis_kwargs or {})
+        self.q_mode, self.rope_base = q_mode, rope_base
         self.has_wo = "W_O" in weights
         self.dtype = weights["W_Q"].dtype
         self.device = weights["W_Q"].device
@@ -80,7 +82,7 @@ class AtpLayer:
             Xin = B.atp_input_norm(c, X, None, kind=self.input_norm, out=self.Xn)
         self._basis(Xin, self.bX)
         B.atp_attention(c, Xin, self.bX[0], self.bX[1], w["W_Q"], w["W_K"], w["W_V"], self.heads, self.lengths,
-                        self.ranks, out=self.O, auto_workspace=False)
+                        self.ranks, out=self.O, auto_workspace=False, q_mode=self.q_mode, rope_base=self.rope_base)
         if not self.has_wo:
             return self.O
         self._basis(self.O, self.bO)
@@ -98,3 +100,25 @@ class AtpLayer:
             self._basis(self.F, self.bF)
             self._linear(self.bF, w["W_down"], self.Y)
         return self.Y
+
+
+class AtpStack:
+    """A chain of ATP layers (Sec. 4.2: the next encoder/decoder layer first attains the principal components
+    of the previous layer's output). Layer l maps X_l to Y_l = FFN(H_l) with H_l = Norm(X_l + A_l); the stack
+    closes the block the usual post-norm way, X_{l+1} = Norm(H_l + Y_l). Layers without an FFN pass their
+    output on unchanged. Every layer has its own weights; lengths, ranks and options are shared."""
+
+    def __init__(self, ctx: B.Context, layer_weights: Sequence[Dict[str, torch.Tensor]], lengths: Sequence[int],
+                 ranks: Sequence[int], heads: int, **layer_kwargs):
+        self.ctx = ctx
+        self.layers = [AtpLayer(ctx, w, lengths, ranks, heads, **layer_kwargs) for w in layer_weights]
+        first = self.layers[0]
+        rows = sum(first.lengths)
+        self.Xnext = [torch.empty((rows, (first.d + 7) // 8 * 8), dtype=first.dtype, device=first.device)[:, :first.d]
+                      for _ in self.layers]
+
+    def forward(self, X: torch.Tensor) -> torch.Tensor:
+        for layer, xn in zip(self.layers, self.Xnext):
+            Y = layer.forward(X)
+            X = B.atp_input_norm(self.ctx, layer.H, Y, kind=layer.post_norm, out=xn) if layer.ffn else Y
+        return X

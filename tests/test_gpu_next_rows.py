@@ -155,3 +155,33 @@ def test_rotary_positions_default_to_row_index_per_sequence_and_zero_positions_a
             want = oracle.attention_rope(x, U, Xr, W[0], W[1], W[2], heads, rope_base=500.0)     # positions 0..L-1
             assert rel_err(got[row:row + L], want) <= 1e-4
         row += L
+
+
+# ------------------------------------------------------------------ a chain of layers
+def test_stack_of_layers_equals_manual_chaining_and_options_reach_the_attention(ctx):
+    from paper_2403_02352_b200.layer import AtpLayer, AtpStack
+    atp = _atp()
+    rng = np.random.default_rng(404)
+    lengths, ranks, d, heads, dff = [96, 64], [24, 16], 64, 2, 128
+    X = to_dev(np.concatenate([_planted(rng, L, d, 8, "f32") for L in lengths]), "f32")
+
+    def weights():
+        w = {k: to_dev(ai.finish(ai.gaussian_weight(rng, d, d), "f32"), "f32") for k in ("W_Q", "W_K", "W_V", "W_O")}
+        w["W_1"] = to_dev(ai.finish(ai.gaussian_weight(rng, d, dff), "f32"), "f32")
+        w["W_2"] = to_dev(ai.finish(ai.gaussian_weight(rng, dff, d), "f32"), "f32")
+        return w
+
+    ws = [weights(), weights()]
+    for kw in (dict(), dict(q_mode="full", rope_base=10000.0)):
+        stack = AtpStack(ctx, ws, lengths, ranks, heads, ffn="gelu", **kw)
+        out = stack.forward(X).clone()
+        x = X
+        for w in ws:
+            layer = AtpLayer(ctx, w, lengths, ranks, heads, ffn="gelu", **kw)
+            y = layer.forward(x)
+            x = atp.atp_input_norm(ctx, layer.H, y, kind="layer")
+        ctx.poll()
+        assert torch.isfinite(out).all()
+        assert torch.equal(out, x)                 # same calls, same order: bit-identical
+    plain = AtpStack(ctx, ws, lengths, ranks, heads, ffn="gelu").forward(X)
+    assert not torch.equal(plain, out)             # the options changed the result
