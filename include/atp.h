@@ -103,6 +103,11 @@ typedef struct {
     int32_t jacobi_inner;  /* tuning: on-chip sweeps per block visit;   <= 0: default 1                */
     int32_t groups;        /* tuning: 0 / 1 = run the whole batch on the caller's stream; 2 = split the */
                            /* batch in two groups on internal streams (forked from and joined to it)   */
+    int32_t no_host_sync;  /* 0: the call reads the device's convergence flags while it enqueues sweeps */
+                           /* and stops early (it may block the calling thread, see above). Non-zero:   */
+                           /* nothing is read back; max_sweeps sweeps are enqueued, those of converged  */
+                           /* sequences return at once. The call then never waits and can be recorded   */
+                           /* by a stream capture; choose max_sweeps with that cost in mind.            */
 } atp_basis_opts;
 
 typedef struct {

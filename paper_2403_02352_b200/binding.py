@@ -45,7 +45,8 @@ class Seqs(C.Structure):
 
 class BasisOpts(C.Structure):
     _fields_ = [("struct_size", C.c_uint32), ("oversample", C.c_int32), ("power_iters", C.c_int32),
-                ("max_sweeps", C.c_int32), ("seed", C.c_uint64), ("jacobi_block", C.c_int32), ("jacobi_inner", C.c_int32), ("groups", C.c_int32)]
+                ("max_sweeps", C.c_int32), ("seed", C.c_uint64), ("jacobi_block", C.c_int32), ("jacobi_inner", C.c_int32), ("groups", C.c_int32),
+                ("no_host_sync", C.c_int32)]
 
 
 class AttnOpts(C.Structure):
@@ -235,7 +236,7 @@ def atp_input_norm(ctx: Context, X, residual=None, kind="rms", eps=1e-5, out=Non
 
 
 def atp_principal_basis(ctx: Context, X, lengths, ranks, oversample=-1, power_iters=-1, max_sweeps=0, seed=0,
-                        out=None, auto_workspace=True, jacobi_block=0, jacobi_inner=0, groups=0):
+                        out=None, auto_workspace=True, jacobi_block=0, jacobi_inner=0, groups=0, no_host_sync=False):
     """(U_r, X_r, sigma) for a packed batch; see include/atp.h."""
     sd = SeqDesc(lengths, ranks)
     d = X.shape[1]
@@ -253,7 +254,8 @@ def atp_principal_basis(ctx: Context, X, lengths, ranks, oversample=-1, power_it
         if ov > 64:      # the query assumes the default oversampling; scale generously for larger ones
             need = int(need * (1.0 + ov / 64.0))
         ctx.ensure_workspace(need)
-    opts = BasisOpts(C.sizeof(BasisOpts), oversample, power_iters, max_sweeps, seed, jacobi_block, jacobi_inner, groups)
+    opts = BasisOpts(C.sizeof(BasisOpts), oversample, power_iters, max_sweeps, seed, jacobi_block, jacobi_inner, groups,
+                     1 if no_host_sync else 0)
     mx, mu, mxr = mat(X), mat(U), mat(Xr)
     _check(lib.atp_principal_basis(ctx._h, C.byref(mx), C.byref(sd.c), C.byref(opts), C.byref(mu), C.byref(mxr),
                                    C.c_void_p(sig.data_ptr()) if sig is not None else None), "atp_principal_basis")

@@ -913,7 +913,7 @@ static atp_status orthonormalise(atp_ctx *ctx, BasisPlan &bp, size_t i0, size_t 
 
 template <typename T>
 static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<SeqDims> &sd, int oversample,
-                             int power_iters, int max_sweeps, uint64_t seed, int jbj, int jinner, int groups, atp_mat *U_r, atp_mat *X_r, float *sigma)
+                             int power_iters, int max_sweeps, uint64_t seed, int jbj, int jinner, int groups, bool no_host_sync, atp_mat *U_r, atp_mat *X_r, float *sigma)
 {
     const int d = (int)X->cols;
     Arena ar(ctx->workspace, ctx->workspace_bytes);
@@ -943,6 +943,10 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
     const size_t nseq = bp.seqs.size();
     const bool forked = groups == 2 && nseq >= 2 && ctx->aux[0] && ctx->aux[1] && !ctx->profiling;
     const size_t gsz = forked ? std::min<size_t>(BMAX, (nseq + 1) / 2) : BMAX;
+    // reading the convergence flags back lets the host stop enqueueing sweeps; without it (forked streams, or on
+    // request: stream capture, callers that must never block) the whole sweep budget is enqueued and the kernels
+    // of converged sequences return at once
+    const bool hsync = !forked && !no_host_sync;
     struct StreamGuard {
         atp_ctx *c; cudaStream_t saved;
         ~StreamGuard() { c->stream = saved; }
@@ -1053,7 +1057,7 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
             init_w_kernel<<<dim3(64, cnt), 256, 0, ctx->stream>>>(jb);
             ATP_LAUNCHED(ctx);
             for (int sw = 0; sw < max_sweeps; ++sw) {
-                if (sw >= 2 && !forked) {      // host stays at most two sweeps ahead; stop once converged
+                if (sw >= 2 && hsync) {      // host stays at most two sweeps ahead; stop once converged
                     const int slot = (sw - 2) & 3;
                     ATP_CUDA_OK(ctx, cudaEventSynchronize(ctx->ev_flag[slot]));
                     if (ctx->h_flags[slot]) break;
@@ -1067,7 +1071,7 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
                 jacobi_sweep_end_kernel<<<1, BMAX, 0, ctx->stream>>>(jb, tol_conv, sw == max_sweeps - 1, ctx->dev_status,
                                                                      ctx->d_flags + (sw & 3));
                 ATP_LAUNCHED(ctx);
-                if (!forked) {
+                if (hsync) {
                     ATP_CUDA_OK(ctx, cudaMemcpyAsync(ctx->h_flags + (sw & 3), ctx->d_flags + (sw & 3), sizeof(int),
                                                      cudaMemcpyDeviceToHost, ctx->stream));
                     ATP_CUDA_OK(ctx, cudaEventRecord(ctx->ev_flag[sw & 3], ctx->stream));
@@ -1148,7 +1152,7 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
                 for (int sw = 0; sw < nsw; ++sw) {
                     // Stop enqueueing once the device reported convergence. The flag of sweep sw - 2 is
                     // awaited here, so the host stays at most two sweeps ahead and the GPU never idles.
-                    if (sw >= 2 && !forked) {
+                    if (sw >= 2 && hsync) {
                         const int slot = (sw - 2) & 3;
                         ATP_CUDA_OK(ctx, cudaEventSynchronize(ctx->ev_flag[slot]));
                         if (ctx->h_flags[slot]) break;
@@ -1171,7 +1175,7 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
                     jac2_sweep_end_kernel<<<1, J2MAX, 0, ctx->stream>>>(jb, tolc, pass == 1 && sw == nsw - 1, ctx->dev_status,
                                                                         ctx->d_flags + (sw & 3));
                     ATP_LAUNCHED(ctx);
-                    if (!forked) {
+                    if (hsync) {
                         ATP_CUDA_OK(ctx, cudaMemcpyAsync(ctx->h_flags + (sw & 3), ctx->d_flags + (sw & 3), sizeof(int),
                                                          cudaMemcpyDeviceToHost, ctx->stream));
                         ATP_CUDA_OK(ctx, cudaEventRecord(ctx->ev_flag[sw & 3], ctx->stream));
@@ -1234,8 +1238,11 @@ extern "C" atp_status atp_principal_basis(atp_ctx *ctx, const atp_mat *X, const 
     atp_status st;
     if ((st = check_mat(X)) != ATP_OK || (st = check_mat(U_r)) != ATP_OK || (st = check_mat(X_r)) != ATP_OK) return st;
     int oversample = 64, power_iters = 2, max_sweeps = 24, jbj = 16, jinner = 1, groups = 0; uint64_t seed = 0x243F6A8885A308D3ull;
+    bool no_host_sync = false;
     if (opts) {
-        if (opts->struct_size < sizeof(atp_basis_opts)) return ATP_ERR_INVALID_ARG;
+        // the struct grew by no_host_sync: the shorter layout is still accepted
+        if (opts->struct_size < offsetof(atp_basis_opts, no_host_sync)) return ATP_ERR_INVALID_ARG;
+        if (opts->struct_size >= sizeof(atp_basis_opts)) no_host_sync = opts->no_host_sync != 0;
         if (opts->oversample >= 0) oversample = opts->oversample;
         if (opts->power_iters >= 0) power_iters = opts->power_iters;
         if (opts->max_sweeps > 0) max_sweeps = opts->max_sweeps;
@@ -1258,8 +1265,8 @@ extern "C" atp_status atp_principal_basis(atp_ctx *ctx, const atp_mat *X, const 
     if (U_r->rows != X->rows || U_r->cols < maxr || X_r->rows != tr || X_r->cols != X->cols) return ATP_ERR_INVALID_ARG;
     if (X->rows == 0) return ATP_OK;
     ATP_CUDA_OK(ctx, cudaSetDevice(ctx->device));
-    if (X->dtype == ATP_F32) return basis_impl<float>(ctx, X, sd, oversample, power_iters, max_sweeps, seed, jbj, jinner, groups, U_r, X_r, sigma);
-    return basis_impl<__nv_bfloat16>(ctx, X, sd, oversample, power_iters, max_sweeps, seed, jbj, jinner, groups, U_r, X_r, sigma);
+    if (X->dtype == ATP_F32) return basis_impl<float>(ctx, X, sd, oversample, power_iters, max_sweeps, seed, jbj, jinner, groups, no_host_sync, U_r, X_r, sigma);
+    return basis_impl<__nv_bfloat16>(ctx, X, sd, oversample, power_iters, max_sweeps, seed, jbj, jinner, groups, no_host_sync, U_r, X_r, sigma);
 }
 
 // ------------------------------------------------------------------------------------------------

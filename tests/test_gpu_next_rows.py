@@ -185,3 +185,34 @@ def test_stack_of_layers_equals_manual_chaining_and_options_reach_the_attention(
         assert torch.equal(out, x)                 # same calls, same order: bit-identical
     plain = AtpStack(ctx, ws, lengths, ranks, heads, ffn="gelu").forward(X)
     assert not torch.equal(plain, out)             # the options changed the result
+
+
+# ------------------------------------------------------------------ basis without host read-back, in a CUDA graph
+def test_basis_without_host_sync_matches_and_can_be_captured(ctx):
+    atp = _atp()
+    rng = np.random.default_rng(77)
+    lengths, ranks, d = [160, 96], [40, 24], 128
+    X = to_dev(np.concatenate([_planted(rng, L, d, 12, "bf16") for L in lengths]), "bf16")
+    U0, X0, s0 = atp.atp_principal_basis(ctx, X, lengths, ranks)
+    U1, X1, s1 = atp.atp_principal_basis(ctx, X, lengths, ranks, no_host_sync=True, max_sweeps=16)
+    ctx.poll()
+    assert torch.equal(U0, U1) and torch.equal(X0, X1) and torch.equal(s0, s1)
+    # the same call recorded by a stream capture and replayed on fresh outputs
+    out = (torch.zeros_like(U0), torch.zeros_like(X0), torch.zeros_like(s0))
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        ctx.use_current_stream()
+        atp.atp_principal_basis(ctx, X, lengths, ranks, no_host_sync=True, max_sweeps=16, out=out, auto_workspace=False)
+        torch.cuda.synchronize()
+        for t in out:
+            t.zero_()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            ctx.use_current_stream()
+            atp.atp_principal_basis(ctx, X, lengths, ranks, no_host_sync=True, max_sweeps=16, out=out, auto_workspace=False)
+        g.replay()
+        torch.cuda.synchronize()
+    ctx.use_current_stream()
+    ctx.poll()
+    assert torch.equal(out[0], U0) and torch.equal(out[1], X0) and torch.equal(out[2], s0)
