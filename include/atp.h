@@ -22,7 +22,8 @@
  *     atp_destroy().
  *   - Calls only enqueue work and return; they never wait for results, except
  *     atp_poll_device_status(). atp_principal_basis reads back its own convergence flags while it
- *     enqueues Jacobi sweeps: the calling thread may block until the GPU is within two sweeps of it.
+ *     enqueues Jacobi sweeps: the calling thread may block until the GPU is within two sweeps of it
+ *     (atp_basis_opts.no_host_sync turns that off).
  *     Work is ordered on the context's stream (atp_set_stream); atp_principal_basis can fork part of
  *     a batch onto two internal streams (opts->groups) and joins them back before it returns.
  *   - Errors the host can detect are returned at once and nothing is launched. Conditions only
