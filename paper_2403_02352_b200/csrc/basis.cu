@@ -792,7 +792,7 @@ __global__ void __launch_bounds__(256) signfix_kernel(const __grid_constant__ Fi
 // ------------------------------------------------------------------------------------------------
 struct SeqPlan {
     SeqDims dims; int rt, npanel_L, npanel_d;
-    __nv_bfloat16 *Yb, *Yl, *Zb, *Zl; float *Y2; float *Y, *Z, *BW, *Wsel, *tsum, *sig, *Cc, *rinv, *G, *Wt, *Vbuf; double *gpart; int *ord, *flags, *conv, *vflag, *needfix; unsigned *maxoff; bool hist_ok;
+    __nv_bfloat16 *Yb, *Yl, *Zb, *Zl; float *Y2; float *Y, *Z, *BW, *Wsel, *tsum, *sig, *Cc, *rinv, *G, *Wt, *Vbuf; double *gpart; int *ord, *flags, *conv, *vflag, *needfix; unsigned *maxoff;
 };
 struct BasisPlan {
     std::vector<SeqPlan> seqs; float *omega; __nv_bfloat16 *omega_b; float *part; size_t part_stride, part_group; int group = 0; int rtmax; int splits;
@@ -843,17 +843,8 @@ static void plan_basis(Arena &ar, const std::vector<SeqDims> &sd, int d, int ove
         p.gpart = ar.take<double>((size_t)ceil_div(std::max(std::max(L, d), 1), GRAM_ROWS) * PB * PB);
         p.G = ar.take<float>((size_t)rt * rt);
         p.Wt = ar.take<float>((size_t)rt * rt);
-        {
-            // rotations published by jac2_local: one set per step of a sweep (block height 16: the sweep's
-            // rotations are replayed on W once, by jac2_wsweep) when that history stays below 64 MB, else
-            // (and with block height 32) one set that the next step overwrites
-            const int nb_all = (ceil_div(std::max(bp.rtmax, 1), 16) + 1) & ~1, nb_own = (ceil_div(std::max(rt, 1), 16) + 1) & ~1;
-            const size_t one = (size_t)(rt / 64 + 2) * 4096 + (size_t)(rt / 32 + 2) * 1024;
-            const size_t hist = (size_t)(nb_all - 1) * (nb_own / 2) * 1024;
-            p.hist_ok = hist * sizeof(float) <= ((size_t)64 << 20);
-            p.Vbuf = ar.take<float>(p.hist_ok ? std::max(hist, one) : one);
-            p.vflag = ar.take<int>(p.hist_ok ? (size_t)(nb_all - 1) * (nb_own / 2) + 4 : (size_t)(rt / 32 + 4));
-        }
+        p.Vbuf = ar.take<float>((size_t)(rt / 64 + 2) * 4096 + (size_t)(rt / 32 + 2) * 1024);
+        p.vflag = ar.take<int>(rt / 32 + 4);
         p.needfix = ar.take<int>(std::max(p.dims.r, 1));
         p.maxoff = ar.take<unsigned>(1);
         p.conv = ar.take<int>(1);
@@ -1112,10 +1103,8 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
             Jac2Batch jb; jb.count = cnt; Fin2Batch fb; fb.count = cnt;
             GemmBatch gg; gg.count = cnt;
             int maxnb = 2, maxrt = 0, maxr = 0;
-            bool hist_all = true;
             for (size_t i = i0; i < i1; ++i) {
                 SeqPlan &p = bp.seqs[i];
-                hist_all = hist_all && p.hist_ok;
                 int k = (int)(i - i0);
                 g.p[k] = GemmProblem{Xb(p), p.Y, p.BW, nullptr, p.rt > 0 ? d : 0, p.rt, p.dims.L, (int)X->ld, p.rt, p.rt, 0};
                 gg.p[k] = GemmProblem{p.BW, p.BW, p.G, nullptr, p.rt, p.rt, p.rt > 0 ? d : 0, p.rt, p.rt, p.rt, 0};
@@ -1149,14 +1138,6 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
             const size_t lsh = jbj == 32 ? JAC2_LOCAL_SMEM(64) : JAC2_LOCAL_SMEM(32);
             if (jbj == 32) ATP_CUDA_OK(ctx, cudaFuncSetAttribute(jac2_apply_kernel<32, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ash));
             if (jbj == 32) ATP_CUDA_OK(ctx, cudaFuncSetAttribute(jac2_local_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lsh));
-            // W once per sweep (jac2_wsweep) when the rotation history and a column chunk of W fit
-            int wcw = 0;
-            if (jbj == 16 && hist_all)
-                for (int c : {32, 16, 8})
-                    if (!wcw && JAC2_WSWEEP_SMEM(maxnb * 16, c) <= (size_t)200 * 1024) wcw = c;
-            const bool defer_w = wcw > 0;
-            const size_t wsh = defer_w ? JAC2_WSWEEP_SMEM(maxnb * 16, wcw) : 0;
-            if (defer_w) ATP_CUDA_OK(ctx, cudaFuncSetAttribute(jac2_wsweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)wsh));
             for (int pass = 0; pass < 2; ++pass) {
                 if ((st = launch_gemm_simt<float, float, float, true, false>(ctx, gg, store, 1, nullptr, 0, "gemm_simt_gram")) != ATP_OK) return st;
                 ATP_KERNEL(ctx, "jac2_init", 0, 0);
@@ -1180,20 +1161,14 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
                         // algorithmic work of a step when every pair rotates (converged pairs skip it)
                         const double nseq = cnt, bl = blk;
                         ATP_KERNEL(ctx, "jac2_local", nseq * npairs * jinner * (bl - 1) * (bl * bl * 6.0 + bl * bl * 3.0), 0);
-                        if (jbj == 32) launch_pdl(jac2_local_kernel<32>, dim3(npairs, cnt), dim3(1024), lsh, ctx->stream, jb, step, tolr, jinner, (int)(step > 0), 0);
-                        else launch_pdl(jac2_local_kernel<16>, dim3(npairs, cnt), dim3(256), lsh, ctx->stream, jb, step, tolr, jinner, (int)(step > 0), defer_w ? step : 0);
+                        if (jbj == 32) launch_pdl(jac2_local_kernel<32>, dim3(npairs, cnt), dim3(1024), lsh, ctx->stream, jb, step, tolr, jinner, (int)(step > 0));
+                        else launch_pdl(jac2_local_kernel<16>, dim3(npairs, cnt), dim3(256), lsh, ctx->stream, jb, step, tolr, jinner, (int)(step > 0));
                         ATP_LAUNCHED(ctx);
-                        const double wchunks = defer_w ? 0.0 : (double)ceil_div(maxrt, blk);
-                        ATP_KERNEL(ctx, "jac2_apply", nseq * npairs * (npairs * 4.0 + wchunks * 2.0) * bl * bl * bl,
-                                   nseq * npairs * (npairs * 2.0 + wchunks * 2.0) * bl * bl * 4.0);
-                        dim3 ag(npairs * (npairs + 1) / 2 + (defer_w ? 0 : npairs * ceil_div(maxrt, blk)), 1, cnt);
-                        if (jbj == 32) launch_pdl(jac2_apply_kernel<32, 4>, ag, dim3(256), ash, ctx->stream, jb, step, 0, 1);
-                        else launch_pdl(jac2_apply_kernel<16, 2>, ag, dim3(128), ash, ctx->stream, jb, step, defer_w ? step : 0, defer_w ? 0 : 1);
-                        ATP_LAUNCHED(ctx);
-                    }
-                    if (defer_w) {
-                        ATP_KERNEL(ctx, "jac2_wsweep", (double)cnt * (maxnb - 1) * npairs * 2.0 * blk * blk * maxrt, (double)cnt * 8.0 * maxrt * maxrt);
-                        launch_pdl(jac2_wsweep_kernel, dim3(ceil_div(maxrt, wcw), cnt), dim3(256), wsh, ctx->stream, jb, maxnb - 1, wcw);
+                        ATP_KERNEL(ctx, "jac2_apply", nseq * npairs * (npairs * 4.0 + ceil_div(maxrt, blk) * 2.0) * bl * bl * bl,
+                                   nseq * npairs * (npairs * 2.0 + ceil_div(maxrt, blk) * 2.0) * bl * bl * 4.0);
+                        dim3 ag(npairs * (npairs + 1) / 2 + npairs * ceil_div(maxrt, blk), 1, cnt);
+                        if (jbj == 32) launch_pdl(jac2_apply_kernel<32, 4>, ag, dim3(256), ash, ctx->stream, jb, step);
+                        else launch_pdl(jac2_apply_kernel<16, 2>, ag, dim3(128), ash, ctx->stream, jb, step);
                         ATP_LAUNCHED(ctx);
                     }
                     ATP_KERNEL(ctx, "jac2_sweep_end", 0, 0);

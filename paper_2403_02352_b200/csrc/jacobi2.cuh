@@ -77,7 +77,7 @@ __device__ __forceinline__ float2 jac2_rotation(float gpp, float gqq, float gpq,
 #define JAC2_LOCAL_SMEM(BLK) ((size_t)(3 * (BLK) * ((BLK) + 1)) * sizeof(float))
 template <int BJ2>
 __global__ void __launch_bounds__(BJ2 * BJ2)
-jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_rot, int max_inner, int cross_only, int vslot)
+jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_rot, int max_inner, int cross_only)
 {
     constexpr int BLK = 2 * BJ2, HP = BLK / 2, NT = HP * HP;
     pdl_trigger();
@@ -129,7 +129,7 @@ jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_r
     for (int w = 1; w < NT / 32; ++w) mo = fmaxf(mo, red[w]);
     if (tid == 0) atomicMax(sq.maxoff, __float_as_uint(mo));
     if (mo <= tol_rot) {
-        if (tid == 0) sq.vflag[vslot * npairs + pair] = 0;
+        if (tid == 0) sq.vflag[pair] = 0;
         return;
     }
     const int ba = tid / HP, bb = tid % HP;            // 2x2 block (pair ba rows, pair bb columns)
@@ -168,9 +168,9 @@ jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_r
             __syncthreads();
         }
     }
-    float *dst = sq.Vbuf + ((size_t)vslot * npairs + pair) * BLK * BLK;   // vslot: 0, or the step when a sweep's rotations are kept
+    float *dst = sq.Vbuf + (size_t)pair * BLK * BLK;
     for (int e = tid; e < BLK * BLK; e += NT) dst[e] = V[e % BLK][e / BLK];   // transposed: what jac2_apply reads
-    if (tid == 0) sq.vflag[vslot * npairs + pair] = 1;
+    if (tid == 0) sq.vflag[pair] = 1;
 }
 
 // grid: (npairs (npairs + 1) / 2 + npairs ceil(rt/BLK), 1, batch); dynamic shared memory: JAC2_APPLY_SMEM(BLK) bytes.
@@ -181,7 +181,7 @@ jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_r
 #define JAC2_APPLY_SMEM(BLK) ((size_t)(4 * (BLK) * ((BLK) + 4)) * sizeof(float))
 template <int BJ2, int MR>
 __global__ void __launch_bounds__(BJ2 * BJ2 / MR, BJ2 == 16 ? 12 : 1)      // 12 CTAs per SM: one wave at batch 16, r~ = 320
-jac2_apply_kernel(const __grid_constant__ Jac2Batch batch, int step, int vslot, int with_w)
+jac2_apply_kernel(const __grid_constant__ Jac2Batch batch, int step)
 {
     constexpr int BLK = 2 * BJ2, NT = BLK * BLK / (4 * MR), LD4 = BLK + 4, Q = BLK / 4;   // Q: 4-vectors per row
     pdl_trigger();
@@ -189,7 +189,7 @@ jac2_apply_kernel(const __grid_constant__ Jac2Batch batch, int step, int vslot, 
     const int npairs = sq.nb / 2;
     // blockIdx.x enumerates the blocks (p, q >= p) of the upper triangle row by row, then the
     // (pair, column chunk) blocks of Wt
-    const int ntri = npairs * (npairs + 1) / 2, nw = with_w ? (sq.rt + BLK - 1) / BLK : 0;   // with_w = 0: W is updated once per sweep by jac2_wsweep
+    const int ntri = npairs * (npairs + 1) / 2, nw = (sq.rt + BLK - 1) / BLK;
     int idx = blockIdx.x;
     const bool in_range = idx < ntri + npairs * nw;
     if (!in_range) idx = 0;
@@ -206,9 +206,8 @@ jac2_apply_kernel(const __grid_constant__ Jac2Batch batch, int step, int vslot, 
     if (!in_range) return;
     // the three flags travel together (one memory latency), then the decision
     const int conv = *sq.conv;
-    const int fp = sq.vflag[vslot * npairs + p];
-    const int fq = gblock ? sq.vflag[vslot * npairs + q] : 0;
-    const float *Vb = sq.Vbuf + (size_t)vslot * npairs * BLK * BLK;
+    const int fp = sq.vflag[p];
+    const int fq = gblock ? sq.vflag[q] : 0;
     if (conv) return;
     if (gblock ? (!fp && !fq) : !fp) return;
     const int tid = threadIdx.x;
@@ -231,11 +230,11 @@ jac2_apply_kernel(const __grid_constant__ Jac2Batch batch, int step, int vslot, 
     for (int f = tid; f < BLK * Q; f += NT) {
         const int i = f / Q, c = (f % Q) * 4;
         // the published rotations are stored transposed: element (k, r) of the copy is Vt[r][k]
-        float4 vp = fp ? *(const float4 *)(Vb + (size_t)p * BLK * BLK + i * BLK + c)
+        float4 vp = fp ? *(const float4 *)(sq.Vbuf + (size_t)p * BLK * BLK + i * BLK + c)
                        : make_float4(i == c ? 1.f : 0.f, i == c + 1 ? 1.f : 0.f, i == c + 2 ? 1.f : 0.f, i == c + 3 ? 1.f : 0.f);
         *(float4 *)&VpT[i * LD4 + c] = vp;
         if (gblock) {
-            float4 vq = fq ? *(const float4 *)(Vb + (size_t)q * BLK * BLK + i * BLK + c)
+            float4 vq = fq ? *(const float4 *)(sq.Vbuf + (size_t)q * BLK * BLK + i * BLK + c)
                            : make_float4(i == c ? 1.f : 0.f, i == c + 1 ? 1.f : 0.f, i == c + 2 ? 1.f : 0.f, i == c + 3 ? 1.f : 0.f);
             *(float4 *)&VqT[i * LD4 + c] = vq;
         }
@@ -321,79 +320,6 @@ jac2_apply_kernel(const __grid_constant__ Jac2Batch batch, int step, int vslot, 
                 for (int i = 0; i < MR; ++i) if (gi0 + i < rt) dst[i] = acc[i][j];
             }
         }
-    }
-}
-
-// W <- (product of a sweep's rotations) W, once per sweep instead of once per step (block height 16 only).
-// A CTA keeps a chunk of cw columns of W (all rows) in shared memory and replays the nsteps x npairs
-// rotations that jac2_local kept (slot = step): per step every warp takes pairs, stages the pair's 32x32
-// rotation in its own shared-memory buffer and updates the 32 rows of the pair, one column per lane
-// (32 accumulators, the rotation read as broadcast 16-byte vectors). W makes one round trip to L2 per
-// sweep; in the per-step kernel it made one per step and its 32x32 products ran at a tenth of the
-// multiply-add rate. grid: (ceil(rt / cw), batch), 256 threads, shared memory JAC2_WSWEEP_SMEM(rows, cw).
-#define JAC2_WSWEEP_SMEM(rows, cw) (((size_t)(rows) * (cw) + 8 * 1024) * sizeof(float))
-__global__ void __launch_bounds__(256)
-jac2_wsweep_kernel(const __grid_constant__ Jac2Batch batch, int nsteps, int cw)
-{
-    constexpr int BJ2 = 16, BLK = 32;
-    pdl_trigger();
-    pdl_wait();
-    const Jac2Seq &sq = batch.s[blockIdx.y];
-    const int rt = sq.rt, nb = sq.nb, npairs = nb / 2;
-    const int c0 = blockIdx.x * cw;
-    if (c0 >= rt || *sq.conv) return;
-    extern __shared__ __align__(16) float wsm[];
-    const int rows = nb * BJ2;                          // padded row count
-    float *Wc = wsm;                                    // [rows][cw]
-    float *Vs = wsm + (size_t)rows * cw;                // [8 warps][32][32]
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    for (int e = tid; e < rows * cw; e += 256) {
-        const int r = e / cw, c = e - r * cw;
-        Wc[e] = (r < rt && c0 + c < rt) ? sq.Wt[(size_t)r * rt + c0 + c] : 0.f;
-    }
-    __syncthreads();
-    float *Vw = Vs + warp * 1024;
-    for (int st = 0; st < nsteps; ++st) {
-        for (int p = warp; p < npairs; p += 8) {
-            if (!sq.vflag[st * npairs + p]) continue;   // warp-uniform
-            int I, J;
-            rr_pair2(nb, st % (nb - 1), p, I, J);
-            const float4 *src = (const float4 *)(sq.Vbuf + ((size_t)st * npairs + p) * BLK * BLK);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) ((float4 *)Vw)[lane + 32 * i] = src[lane + 32 * i];   // Vw[k][r] = Vt[r][k]
-            __syncwarp();
-            if (lane < cw) {
-                float w[BLK], out[BLK];
-#pragma unroll
-                for (int k = 0; k < BLK; ++k) {
-                    const int row = (k < BJ2) ? I * BJ2 + k : J * BJ2 + (k - BJ2);
-                    w[k] = Wc[row * cw + lane];
-                    out[k] = 0.f;
-                }
-#pragma unroll
-                for (int k = 0; k < BLK; ++k) {
-#pragma unroll
-                    for (int r4 = 0; r4 < BLK / 4; ++r4) {
-                        const float4 v = *(const float4 *)&Vw[k * BLK + 4 * r4];
-                        out[4 * r4] = fmaf(v.x, w[k], out[4 * r4]);
-                        out[4 * r4 + 1] = fmaf(v.y, w[k], out[4 * r4 + 1]);
-                        out[4 * r4 + 2] = fmaf(v.z, w[k], out[4 * r4 + 2]);
-                        out[4 * r4 + 3] = fmaf(v.w, w[k], out[4 * r4 + 3]);
-                    }
-                }
-#pragma unroll
-                for (int k = 0; k < BLK; ++k) {
-                    const int row = (k < BJ2) ? I * BJ2 + k : J * BJ2 + (k - BJ2);
-                    Wc[row * cw + lane] = out[k];
-                }
-            }
-            __syncwarp();
-        }
-        __syncthreads();                                // the next step pairs the rows differently
-    }
-    for (int e = tid; e < rows * cw; e += 256) {
-        const int r = e / cw, c = e - r * cw;
-        if (r < rt && c0 + c < rt) sq.Wt[(size_t)r * rt + c0 + c] = Wc[e];
     }
 }
 
