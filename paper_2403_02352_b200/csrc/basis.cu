@@ -792,7 +792,7 @@ __global__ void __launch_bounds__(256) signfix_kernel(const __grid_constant__ Fi
 // ------------------------------------------------------------------------------------------------
 struct SeqPlan {
     SeqDims dims; int rt, npanel_L, npanel_d;
-    __nv_bfloat16 *Yb, *Yl, *Zb, *Zl; float *Y2; float *Y, *Z, *BW, *Wsel, *tsum, *sig, *Cc, *rinv, *G, *Wt, *Vbuf; double *gpart; int *ord, *flags, *conv, *vflag, *needfix; unsigned *maxoff; bool hist_ok;
+    __nv_bfloat16 *Yb, *Yl, *Zb, *Zl; float *Y2; float *Y, *Z, *BW, *Wsel, *tsum, *sig, *Cc, *rinv, *G, *Wt, *Vbuf; double *gpart; int *ord, *flags, *conv, *vflag, *needfix; unsigned *maxoff;
 };
 struct BasisPlan {
     std::vector<SeqPlan> seqs; float *omega; __nv_bfloat16 *omega_b; float *part; size_t part_stride, part_group; int group = 0; int rtmax; int splits;
@@ -843,17 +843,8 @@ static void plan_basis(Arena &ar, const std::vector<SeqDims> &sd, int d, int ove
         p.gpart = ar.take<double>((size_t)ceil_div(std::max(std::max(L, d), 1), GRAM_ROWS) * PB * PB);
         p.G = ar.take<float>((size_t)rt * rt);
         p.Wt = ar.take<float>((size_t)rt * rt);
-        {
-            // rotations published by jac2_local: one set per step of a sweep (block height 16: the update of W
-            // then runs on its own stream, behind the iteration) when that history stays below 64 MB, else
-            // (and with block height 32) one set that the next step overwrites
-            const int nb_all = (ceil_div(std::max(bp.rtmax, 1), 16) + 1) & ~1, nb_own = (ceil_div(std::max(rt, 1), 16) + 1) & ~1;
-            const size_t one = (size_t)(rt / 64 + 2) * 4096 + (size_t)(rt / 32 + 2) * 1024;
-            const size_t hist = (size_t)(nb_all - 1) * (nb_own / 2) * 1024;
-            p.hist_ok = hist * sizeof(float) <= ((size_t)64 << 20);
-            p.Vbuf = ar.take<float>(p.hist_ok ? std::max(hist, one) : one);
-            p.vflag = ar.take<int>(p.hist_ok ? (size_t)(nb_all - 1) * (nb_own / 2) + 4 : (size_t)(rt / 32 + 4));
-        }
+        p.Vbuf = ar.take<float>((size_t)(rt / 64 + 2) * 4096 + (size_t)(rt / 32 + 2) * 1024);
+        p.vflag = ar.take<int>(rt / 32 + 4);
         p.needfix = ar.take<int>(std::max(p.dims.r, 1));
         p.maxoff = ar.take<unsigned>(1);
         p.conv = ar.take<int>(1);
@@ -1112,10 +1103,8 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
             Jac2Batch jb; jb.count = cnt; Fin2Batch fb; fb.count = cnt;
             GemmBatch gg; gg.count = cnt;
             int maxnb = 2, maxrt = 0, maxr = 0;
-            bool hist_all = true;
             for (size_t i = i0; i < i1; ++i) {
                 SeqPlan &p = bp.seqs[i];
-                hist_all = hist_all && p.hist_ok;
                 int k = (int)(i - i0);
                 g.p[k] = GemmProblem{Xb(p), p.Y, p.BW, nullptr, p.rt > 0 ? d : 0, p.rt, p.dims.L, (int)X->ld, p.rt, p.rt, 0};
                 gg.p[k] = GemmProblem{p.BW, p.BW, p.G, nullptr, p.rt, p.rt, p.rt > 0 ? d : 0, p.rt, p.rt, p.rt, 0};
@@ -1149,10 +1138,6 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
             const size_t lsh = jbj == 32 ? JAC2_LOCAL_SMEM(64) : JAC2_LOCAL_SMEM(32);
             if (jbj == 32) ATP_CUDA_OK(ctx, cudaFuncSetAttribute(jac2_apply_kernel<32, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ash));
             if (jbj == 32) ATP_CUDA_OK(ctx, cudaFuncSetAttribute(jac2_local_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lsh));
-            // The update of W (the accumulated rotations) does not feed back into the iteration on G: with block
-            // height 16 and the rotations of every step of a sweep kept (slot = step), it runs on an auxiliary
-            // stream, forked after each local kernel and joined at the end of the sweep, off the critical chain.
-            const bool side_w = jbj == 16 && hist_all && !forked && ctx->aux[0];
             for (int pass = 0; pass < 2; ++pass) {
                 if ((st = launch_gemm_simt<float, float, float, true, false>(ctx, gg, store, 1, nullptr, 0, "gemm_simt_gram")) != ATP_OK) return st;
                 ATP_KERNEL(ctx, "jac2_init", 0, 0);
@@ -1176,33 +1161,15 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
                         // algorithmic work of a step when every pair rotates (converged pairs skip it)
                         const double nseq = cnt, bl = blk;
                         ATP_KERNEL(ctx, "jac2_local", nseq * npairs * jinner * (bl - 1) * (bl * bl * 6.0 + bl * bl * 3.0), 0);
-                        if (jbj == 32) launch_pdl(jac2_local_kernel<32>, dim3(npairs, cnt), dim3(1024), lsh, ctx->stream, jb, step, tolr, jinner, (int)(step > 0), 0);
-                        else launch_pdl(jac2_local_kernel<16>, dim3(npairs, cnt), dim3(256), lsh, ctx->stream, jb, step, tolr, jinner, (int)(step > 0), side_w ? step : 0);
+                        if (jbj == 32) launch_pdl(jac2_local_kernel<32>, dim3(npairs, cnt), dim3(1024), lsh, ctx->stream, jb, step, tolr, jinner, (int)(step > 0));
+                        else launch_pdl(jac2_local_kernel<16>, dim3(npairs, cnt), dim3(256), lsh, ctx->stream, jb, step, tolr, jinner, (int)(step > 0));
                         ATP_LAUNCHED(ctx);
-                        const int nwc = ceil_div(maxrt, blk);
-                        if (side_w) {
-                            ATP_CUDA_OK(ctx, cudaEventRecord(ctx->ev_fork, ctx->stream));
-                            ATP_CUDA_OK(ctx, cudaStreamWaitEvent(ctx->aux[0], ctx->ev_fork, 0));
-                            const cudaStream_t cur = ctx->stream;
-                            ctx->stream = ctx->aux[0];
-                            ATP_KERNEL(ctx, "jac2_apply_w", nseq * npairs * nwc * 2.0 * bl * bl * bl, nseq * npairs * nwc * 2.0 * bl * bl * 4.0);
-                            launch_pdl(jac2_apply_kernel<16, 2>, dim3(npairs * nwc, 1, cnt), dim3(128), ash, ctx->stream, jb, step, step, 2);
-                            ctx->launches++;
-                            prof_end(ctx);
-                            ctx->stream = cur;
-                            if (cudaGetLastError() != cudaSuccess) return ATP_ERR_CUDA;
-                        }
-                        const double wchunks = side_w ? 0.0 : (double)nwc;
-                        ATP_KERNEL(ctx, "jac2_apply", nseq * npairs * (npairs * 4.0 + wchunks * 2.0) * bl * bl * bl,
-                                   nseq * npairs * (npairs * 2.0 + wchunks * 2.0) * bl * bl * 4.0);
-                        dim3 ag(npairs * (npairs + 1) / 2 + (side_w ? 0 : npairs * nwc), 1, cnt);
-                        if (jbj == 32) launch_pdl(jac2_apply_kernel<32, 4>, ag, dim3(256), ash, ctx->stream, jb, step, 0, 1);
-                        else launch_pdl(jac2_apply_kernel<16, 2>, ag, dim3(128), ash, ctx->stream, jb, step, side_w ? step : 0, side_w ? 0 : 1);
+                        ATP_KERNEL(ctx, "jac2_apply", nseq * npairs * (npairs * 4.0 + ceil_div(maxrt, blk) * 2.0) * bl * bl * bl,
+                                   nseq * npairs * (npairs * 2.0 + ceil_div(maxrt, blk) * 2.0) * bl * bl * 4.0);
+                        dim3 ag(npairs * (npairs + 1) / 2 + npairs * ceil_div(maxrt, blk), 1, cnt);
+                        if (jbj == 32) launch_pdl(jac2_apply_kernel<32, 4>, ag, dim3(256), ash, ctx->stream, jb, step);
+                        else launch_pdl(jac2_apply_kernel<16, 2>, ag, dim3(128), ash, ctx->stream, jb, step);
                         ATP_LAUNCHED(ctx);
-                    }
-                    if (side_w) {                     // W of this sweep complete before the convergence test and whatever follows
-                        ATP_CUDA_OK(ctx, cudaEventRecord(ctx->ev_join[0], ctx->aux[0]));
-                        ATP_CUDA_OK(ctx, cudaStreamWaitEvent(ctx->stream, ctx->ev_join[0], 0));
                     }
                     ATP_KERNEL(ctx, "jac2_sweep_end", 0, 0);
                     jac2_sweep_end_kernel<<<1, J2MAX, 0, ctx->stream>>>(jb, tolc, pass == 1 && sw == nsw - 1, ctx->dev_status,

@@ -77,7 +77,7 @@ __device__ __forceinline__ float2 jac2_rotation(float gpp, float gqq, float gpq,
 #define JAC2_LOCAL_SMEM(BLK) ((size_t)(3 * (BLK) * ((BLK) + 1)) * sizeof(float))
 template <int BJ2>
 __global__ void __launch_bounds__(BJ2 * BJ2)
-jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_rot, int max_inner, int cross_only, int vslot)
+jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_rot, int max_inner, int cross_only)
 {
     constexpr int BLK = 2 * BJ2, HP = BLK / 2, NT = HP * HP;
     pdl_trigger();
@@ -129,7 +129,7 @@ jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_r
     for (int w = 1; w < NT / 32; ++w) mo = fmaxf(mo, red[w]);
     if (tid == 0) atomicMax(sq.maxoff, __float_as_uint(mo));
     if (mo <= tol_rot) {
-        if (tid == 0) sq.vflag[vslot * npairs + pair] = 0;
+        if (tid == 0) sq.vflag[pair] = 0;
         return;
     }
     const int ba = tid / HP, bb = tid % HP;            // 2x2 block (pair ba rows, pair bb columns)
@@ -168,9 +168,9 @@ jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_r
             __syncthreads();
         }
     }
-    float *dst = sq.Vbuf + ((size_t)vslot * npairs + pair) * BLK * BLK;   // vslot: 0, or the step when a sweep's rotations are kept
+    float *dst = sq.Vbuf + (size_t)pair * BLK * BLK;
     for (int e = tid; e < BLK * BLK; e += NT) dst[e] = V[e % BLK][e / BLK];   // transposed: what jac2_apply reads
-    if (tid == 0) sq.vflag[vslot * npairs + pair] = 1;
+    if (tid == 0) sq.vflag[pair] = 1;
 }
 
 // grid: (npairs (npairs + 1) / 2 + npairs ceil(rt/BLK), 1, batch); dynamic shared memory: JAC2_APPLY_SMEM(BLK) bytes.
@@ -181,7 +181,7 @@ jac2_local_kernel(const __grid_constant__ Jac2Batch batch, int step, float tol_r
 #define JAC2_APPLY_SMEM(BLK) ((size_t)(4 * (BLK) * ((BLK) + 4)) * sizeof(float))
 template <int BJ2, int MR>
 __global__ void __launch_bounds__(BJ2 * BJ2 / MR, BJ2 == 16 ? 12 : 1)      // 12 CTAs per SM: one wave at batch 16, r~ = 320
-jac2_apply_kernel(const __grid_constant__ Jac2Batch batch, int step, int vslot, int with_w)
+jac2_apply_kernel(const __grid_constant__ Jac2Batch batch, int step)
 {
     constexpr int BLK = 2 * BJ2, NT = BLK * BLK / (4 * MR), LD4 = BLK + 4, Q = BLK / 4;   // Q: 4-vectors per row
     pdl_trigger();
@@ -189,9 +189,7 @@ jac2_apply_kernel(const __grid_constant__ Jac2Batch batch, int step, int vslot, 
     const int npairs = sq.nb / 2;
     // blockIdx.x enumerates the blocks (p, q >= p) of the upper triangle row by row, then the
     // (pair, column chunk) blocks of Wt
-    // with_w: 1 = blocks of G and of W in one launch; 0 = G only, 2 = W only (the W update is off the critical
-    // path of the iteration and can run on another stream)
-    const int ntri = with_w == 2 ? 0 : npairs * (npairs + 1) / 2, nw = with_w ? (sq.rt + BLK - 1) / BLK : 0;
+    const int ntri = npairs * (npairs + 1) / 2, nw = (sq.rt + BLK - 1) / BLK;
     int idx = blockIdx.x;
     const bool in_range = idx < ntri + npairs * nw;
     if (!in_range) idx = 0;
@@ -208,9 +206,8 @@ jac2_apply_kernel(const __grid_constant__ Jac2Batch batch, int step, int vslot, 
     if (!in_range) return;
     // the three flags travel together (one memory latency), then the decision
     const int conv = *sq.conv;
-    const int fp = sq.vflag[vslot * npairs + p];
-    const int fq = gblock ? sq.vflag[vslot * npairs + q] : 0;
-    const float *Vb = sq.Vbuf + (size_t)vslot * npairs * BLK * BLK;
+    const int fp = sq.vflag[p];
+    const int fq = gblock ? sq.vflag[q] : 0;
     if (conv) return;
     if (gblock ? (!fp && !fq) : !fp) return;
     const int tid = threadIdx.x;
@@ -233,11 +230,11 @@ jac2_apply_kernel(const __grid_constant__ Jac2Batch batch, int step, int vslot, 
     for (int f = tid; f < BLK * Q; f += NT) {
         const int i = f / Q, c = (f % Q) * 4;
         // the published rotations are stored transposed: element (k, r) of the copy is Vt[r][k]
-        float4 vp = fp ? *(const float4 *)(Vb + (size_t)p * BLK * BLK + i * BLK + c)
+        float4 vp = fp ? *(const float4 *)(sq.Vbuf + (size_t)p * BLK * BLK + i * BLK + c)
                        : make_float4(i == c ? 1.f : 0.f, i == c + 1 ? 1.f : 0.f, i == c + 2 ? 1.f : 0.f, i == c + 3 ? 1.f : 0.f);
         *(float4 *)&VpT[i * LD4 + c] = vp;
         if (gblock) {
-            float4 vq = fq ? *(const float4 *)(Vb + (size_t)q * BLK * BLK + i * BLK + c)
+            float4 vq = fq ? *(const float4 *)(sq.Vbuf + (size_t)q * BLK * BLK + i * BLK + c)
                            : make_float4(i == c ? 1.f : 0.f, i == c + 1 ? 1.f : 0.f, i == c + 2 ? 1.f : 0.f, i == c + 3 ? 1.f : 0.f);
             *(float4 *)&VqT[i * LD4 + c] = vq;
         }
