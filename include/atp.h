@@ -100,7 +100,8 @@ typedef struct {
     int32_t power_iters;   /* subspace (power) iterations;        < 0: default 2              */
     int32_t max_sweeps;    /* Jacobi sweep limit;                 <= 0: default 24            */
     uint64_t seed;         /* seed of the +-1 test matrix                                      */
-    int32_t jacobi_block;  /* tuning: rows per Jacobi block, 16 or 32; 0: default 16 (bf16 path only)  */
+    int32_t jacobi_block;  /* tuning: rows per block of the two-sided Jacobi, 16 or 32; 0: default 16; */
+                           /* 1: one-sided Jacobi on the projected rows themselves (no Gram matrix)      */
     int32_t jacobi_inner;  /* tuning: on-chip sweeps per block visit;   <= 0: default 1                */
     int32_t groups;        /* tuning: 0 / 1 = run the whole batch on the caller's stream; 2 = split the */
                            /* batch in two groups on internal streams (forked from and joined to it)   */
@@ -157,8 +158,9 @@ ATP_API atp_status atp_input_norm(atp_ctx *ctx, const atp_mat *X, const atp_mat 
  * vectors U_r (L_b x r_b, orthonormal columns) and X_r = U_r^T X = [sigma_1 v_1; ..; sigma_r v_r]
  * (r_b x d), components sorted by sigma descending, i.e. the minimiser of Eq. 9. Computed by a
  * randomised range finder with subspace iteration, block Gram-Schmidt orthonormalisation and a
- * block Jacobi rotation of the small projected problem (one-sided on the projected rows for f32
- * input, two-sided on their Gram matrix, in two passes, for bf16 input) - not by a full SVD - so
+ * block Jacobi rotation of the small projected problem (two-sided on the Gram matrix of the
+ * projected rows, in two passes; one-sided on the rows themselves with opts->jacobi_block = 1) -
+ * not by a full SVD - so
  * the subspace is the optimal one up to the range finder's error; opts->power_iters trades passes
  * over X for that. The Jacobi sweeps stop on a device-side convergence test (largest scaled
  * off-diagonal <= 1e-6 for f32, 3e-5 for bf16); opts->max_sweeps bounds them, and a sequence that

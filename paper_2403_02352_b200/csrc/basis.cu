@@ -933,7 +933,7 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
     }
     const float tol_conv = (X->dtype == ATP_F32) ? 1e-6f : 3e-5f;
     const float tol_rot = tol_conv * 0.25f;
-    const bool two_sided = (X->dtype == ATP_BF16) && jbj != 1;    // fp32 inputs keep the one-sided rotation of B itself
+    const bool two_sided = jbj != 1;    // jacobi_block = 1 selects the one-sided rotation of B itself
     GemmEpi store{EPI_STORE, nullptr};
 
     // The chains below are many small dependent launches (latency-bound). On request (groups = 2) the

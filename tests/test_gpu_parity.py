@@ -137,6 +137,15 @@ def test_basis_invariants_noisy(ctx, dtype, L, d, r, k):
     _check_t1(X, U, Xr, sig, dtype, 3e-2)
 
 
+@pytest.mark.parametrize("jb", [1, 32])
+def test_basis_invariants_other_jacobi_variants_fp32(ctx, jb):
+    """jacobi_block = 1: the one-sided rotation of the projected rows themselves; 32: 64x64 diagonal blocks."""
+    rng = np.random.default_rng(91 + jb)
+    X = _noisy(rng, 300, 200, 16, "f32")
+    (U, Xr, sig), = _run_basis(ctx, [(X, 40)], "f32", jacobi_block=jb)
+    _check_t1(X, U, Xr, sig, "f32", 3e-2)
+
+
 def test_basis_more_power_iterations_approach_the_optimum(ctx):
     rng = np.random.default_rng(5)
     X = _noisy(rng, 256, 192, 10, "f32")
