@@ -56,8 +56,9 @@ atp_status atp_create(atp_ctx **out, int device)
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return ATP_ERR_CUDA; }
     ctx->sm_count = prop.multiProcessorCount;
-    if (cudaMalloc(&ctx->dev_status, sizeof(int)) != cudaSuccess) { delete ctx; return ATP_ERR_CUDA; }
-    if (cudaMemset(ctx->dev_status, 0, sizeof(int)) != cudaSuccess) { cudaFree(ctx->dev_status); delete ctx; return ATP_ERR_CUDA; }
+    // two words: [0] the sticky status, [1] the abort flag shared by the bounded waits of persistent kernels
+    if (cudaMalloc(&ctx->dev_status, 2 * sizeof(int)) != cudaSuccess) { delete ctx; return ATP_ERR_CUDA; }
+    if (cudaMemset(ctx->dev_status, 0, 2 * sizeof(int)) != cudaSuccess) { cudaFree(ctx->dev_status); delete ctx; return ATP_ERR_CUDA; }
     bool ok = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) == cudaSuccess;
     for (int i = 0; i < 2 && ok; ++i)
         ok = cudaStreamCreateWithFlags(&ctx->aux[i], cudaStreamNonBlocking) == cudaSuccess &&
@@ -108,10 +109,10 @@ atp_status atp_poll_device_status(atp_ctx *ctx)
     if (!ctx) return ATP_ERR_INVALID_ARG;
     ATP_CUDA_OK(ctx, cudaSetDevice(ctx->device));
     ATP_CUDA_OK(ctx, cudaStreamSynchronize(ctx->stream));
-    int st = 0;
-    ATP_CUDA_OK(ctx, cudaMemcpy(&st, ctx->dev_status, sizeof(int), cudaMemcpyDeviceToHost));
-    if (st != 0) ATP_CUDA_OK(ctx, cudaMemset(ctx->dev_status, 0, sizeof(int)));
-    return (atp_status)st;
+    int st[2] = {0, 0};
+    ATP_CUDA_OK(ctx, cudaMemcpy(st, ctx->dev_status, 2 * sizeof(int), cudaMemcpyDeviceToHost));
+    if (st[0] != 0 || st[1] != 0) ATP_CUDA_OK(ctx, cudaMemset(ctx->dev_status, 0, 2 * sizeof(int)));
+    return (atp_status)st[0];
 }
 
 int64_t atp_launch_count(const atp_ctx *ctx) { return ctx ? ctx->launches : -1; }

@@ -9,7 +9,7 @@
 //   4. sort by sigma, fix signs, write U_r = Y W and X_r.
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
-#include "jacobi2.cuh"
+#include "jacobi3.cuh"
 #include <type_traits>
 #include <math.h>
 #include <algorithm>
@@ -680,7 +680,7 @@ __global__ void __launch_bounds__(256) select_kernel(const __grid_constant__ Fin
 // ---- finalisation of the two-sided path ----------------------------------------------------------
 struct Fin2Seq {
     const float *G; const float *Wt; const float *Y; float *sig; int *ord; float *tsum; float *Wsel; int *needfix;
-    void *Xr; void *U; float *sigma_out; int rt, r, d, L, ldy, ldxr, ldu;
+    void *Xr; void *U; float *sigma_out; int rt, r, d, L, ldy, ldxr, ldu, ldg;
 };
 struct Fin2Batch { Fin2Seq s[BMAX]; int count; };
 
@@ -695,7 +695,7 @@ __global__ void __launch_bounds__(1024) sigma_sort2_kernel(const __grid_constant
     int *idx = (int *)(sh + npow);
     const int tid = threadIdx.x;
     for (int i = tid; i < npow; i += 1024) {
-        key[i] = (i < sq.rt) ? sqrtf(fmaxf(sq.G[(size_t)i * sq.rt + i], 0.f)) : -1.f;
+        key[i] = (i < sq.rt) ? sqrtf(fmaxf(sq.G[(size_t)i * sq.ldg + i], 0.f)) : -1.f;
         idx[i] = i;
     }
     __syncthreads();
@@ -733,7 +733,7 @@ __global__ void __launch_bounds__(128) select2_kernel(const __grid_constant__ Fi
     const int a = blockIdx.x;
     if (a >= sq.r) return;
     const int i = sq.ord[a];
-    const float *w = sq.Wt + (size_t)i * sq.rt;
+    const float *w = sq.Wt + (size_t)i * sq.ldg;
     __shared__ float redf[4];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     float s = 0.f;
@@ -791,7 +791,7 @@ __global__ void __launch_bounds__(256) signfix_kernel(const __grid_constant__ Fi
 
 // ------------------------------------------------------------------------------------------------
 struct SeqPlan {
-    SeqDims dims; int rt, npanel_L, npanel_d;
+    SeqDims dims; int rt, np, npanel_L, npanel_d; unsigned *jsync;
     __nv_bfloat16 *Yb, *Yl, *Zb, *Zl; float *Y2; float *Y, *Z, *BW, *Wsel, *tsum, *sig, *Cc, *rinv, *G, *Wt, *Vbuf; double *gpart; int *ord, *flags, *conv, *vflag, *needfix; unsigned *maxoff;
 };
 struct BasisPlan {
@@ -806,6 +806,9 @@ static int pick_splits(int K, int nseq)
     int s = std::min(std::min(want, K / 64), 16);
     return s < 1 ? 1 : s;
 }
+
+// Size of the Jacobi matrices: rt rounded up to a whole number of 64-row block pairs.
+static int jacobi_padded(int rt) { return rt <= 0 ? 0 : (rt + 63) / 64 * 64; }
 
 static void plan_basis(Arena &ar, const std::vector<SeqDims> &sd, int d, int oversample, BasisPlan &bp)
 {
@@ -841,10 +844,12 @@ static void plan_basis(Arena &ar, const std::vector<SeqDims> &sd, int d, int ove
         p.rinv = ar.take<float>(PB * PB + PB);
         p.flags = ar.take<int>(PB);
         p.gpart = ar.take<double>((size_t)ceil_div(std::max(std::max(L, d), 1), GRAM_ROWS) * PB * PB);
-        p.G = ar.take<float>((size_t)rt * rt);
-        p.Wt = ar.take<float>((size_t)rt * rt);
-        p.Vbuf = ar.take<float>((size_t)(rt / 64 + 2) * 4096 + (size_t)(rt / 32 + 2) * 1024);
-        p.vflag = ar.take<int>(rt / 32 + 4);
+        p.np = jacobi_padded(rt);
+        p.G = ar.take<float>((size_t)p.np * p.np);
+        p.Wt = ar.take<float>((size_t)p.np * p.np);
+        p.Vbuf = ar.take<float>((size_t)(p.np / 64 + 1) * 4096);
+        p.vflag = ar.take<int>(p.np / 64 + 4);
+        p.jsync = ar.take<unsigned>(8);
         p.needfix = ar.take<int>(std::max(p.dims.r, 1));
         p.maxoff = ar.take<unsigned>(1);
         p.conv = ar.take<int>(1);
@@ -1100,20 +1105,19 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
         } else {
             // Bt = X^T Y (d x r~, i.e. B^T), G = Bt^T Bt, two-sided block Jacobi on G, then
             // X_r = Wsel^T Bt^T and U_r = Y Wsel
-            Jac2Batch jb; jb.count = cnt; Fin2Batch fb; fb.count = cnt;
+            j3::Batch jb; jb.count = cnt; Fin2Batch fb; fb.count = cnt;
             GemmBatch gg; gg.count = cnt;
-            int maxnb = 2, maxrt = 0, maxr = 0;
+            int maxrt = 0, maxr = 0;
             for (size_t i = i0; i < i1; ++i) {
                 SeqPlan &p = bp.seqs[i];
                 int k = (int)(i - i0);
                 g.p[k] = GemmProblem{Xb(p), p.Y, p.BW, nullptr, p.rt > 0 ? d : 0, p.rt, p.dims.L, (int)X->ld, p.rt, p.rt, 0};
-                gg.p[k] = GemmProblem{p.BW, p.BW, p.G, nullptr, p.rt, p.rt, p.rt > 0 ? d : 0, p.rt, p.rt, p.rt, 0};
-                int nb = ceil_div(std::max(p.rt, 1), jbj); nb += nb & 1;
-                jb.s[k] = Jac2Seq{p.G, p.Wt, p.Vbuf, p.vflag, p.rt, nb, p.maxoff, p.conv};
+                gg.p[k] = GemmProblem{p.BW, p.BW, p.G, nullptr, p.rt, p.rt, p.rt > 0 ? d : 0, p.rt, p.rt, p.np, 0};
+                jb.s[k] = j3::Seq{p.G, p.Wt, p.Vbuf, p.vflag, p.jsync, p.rt, p.np, p.np / j3::JB, 0, 0};
                 fb.s[k] = Fin2Seq{p.G, p.Wt, p.Y, p.sig, p.ord, p.tsum, p.Wsel, p.needfix,
                                   (T *)X_r->data + (size_t)p.dims.rank0 * X_r->ld, (T *)U_r->data + (size_t)p.dims.row0 * U_r->ld,
-                                  sigma ? sigma + p.dims.rank0 : nullptr, p.rt, p.dims.r, d, p.dims.L, p.rt, (int)X_r->ld, (int)U_r->ld};
-                maxnb = std::max(maxnb, nb); maxrt = std::max(maxrt, p.rt); maxr = std::max(maxr, p.dims.r);
+                                  sigma ? sigma + p.dims.rank0 : nullptr, p.rt, p.dims.r, d, p.dims.L, p.rt, (int)X_r->ld, (int)U_r->ld, p.np};
+                maxrt = std::max(maxrt, p.rt); maxr = std::max(maxr, p.dims.r);
             }
             if (maxrt == 0) continue;
             if constexpr (std::is_same<T, __nv_bfloat16>::value) {
@@ -1132,63 +1136,26 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
             // orthogonal all the same, so (Bt, Y) <- (Bt W1, Y W1) loses nothing; the rotated rows are
             // graded and nearly orthogonal, their Gram matrix carries errors relative to the row norms,
             // and a short second pass on it finishes the job (a one-sided Jacobi in two strokes).
-            const int npairs = maxnb / 2;
-            const int blk = 2 * jbj;
-            const size_t ash = jbj == 32 ? JAC2_APPLY_SMEM(64) : JAC2_APPLY_SMEM(32);
-            const size_t lsh = jbj == 32 ? JAC2_LOCAL_SMEM(64) : JAC2_LOCAL_SMEM(32);
-            if (jbj == 32) ATP_CUDA_OK(ctx, cudaFuncSetAttribute(jac2_apply_kernel<32, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ash));
-            if (jbj == 32) ATP_CUDA_OK(ctx, cudaFuncSetAttribute(jac2_local_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lsh));
+            // Each pass is one persistent kernel that stops on its own convergence test: nothing is
+            // read back by the host.
             for (int pass = 0; pass < 2; ++pass) {
                 if ((st = launch_gemm_simt<float, float, float, true, false>(ctx, gg, store, 1, nullptr, 0, "gemm_simt_gram")) != ATP_OK) return st;
-                ATP_KERNEL(ctx, "jac2_init", 0, 0);
-                jac2_init_kernel<<<dim3(64, cnt), 256, 0, ctx->stream>>>(jb);
-                ATP_LAUNCHED(ctx);
-                // the second pass continues the same iteration on the rotated data: split the sweep budget
                 // pass 0 only has to make the rows graded and roughly orthogonal (scaled off-diagonals below
-                // 1e-2; on ill-conditioned input it stalls at the noise floor of G, hence the cap of 8 sweeps)
-                const int nsw = pass == 0 ? std::min(8, (max_sweeps + 1) / 2) : max_sweeps - std::min(8, (max_sweeps + 1) / 2);
+                // 1e-2; on ill-conditioned input it stalls at the noise floor of G, hence the cap of 8 sweeps);
+                // the second pass continues the same iteration on the rotated data with the rest of the budget
+                const int nsw0 = std::min(8, (max_sweeps + 1) / 2);
+                const int nsw = pass == 0 ? nsw0 : std::max(1, max_sweeps - nsw0);
                 const float tolc = pass == 0 ? fmaxf(tol_conv, 1e-2f) : tol_conv;
-                const float tolr = tolc * 0.25f;
-                for (int sw = 0; sw < nsw; ++sw) {
-                    // Stop enqueueing once the device reported convergence. The flag of sweep sw - 2 is
-                    // awaited here, so the host stays at most two sweeps ahead and the GPU never idles.
-                    if (sw >= 2 && hsync) {
-                        const int slot = (sw - 2) & 3;
-                        ATP_CUDA_OK(ctx, cudaEventSynchronize(ctx->ev_flag[slot]));
-                        if (ctx->h_flags[slot]) break;
-                    }
-                    for (int step = 0; step < maxnb - 1; ++step) {
-                        // algorithmic work of a step when every pair rotates (converged pairs skip it)
-                        const double nseq = cnt, bl = blk;
-                        ATP_KERNEL(ctx, "jac2_local", nseq * npairs * jinner * (bl - 1) * (bl * bl * 6.0 + bl * bl * 3.0), 0);
-                        if (jbj == 32) launch_pdl(jac2_local_kernel<32>, dim3(npairs, cnt), dim3(1024), lsh, ctx->stream, jb, step, tolr, jinner, (int)(step > 0));
-                        else launch_pdl(jac2_local_kernel<16>, dim3(npairs, cnt), dim3(256), lsh, ctx->stream, jb, step, tolr, jinner, (int)(step > 0));
-                        ATP_LAUNCHED(ctx);
-                        ATP_KERNEL(ctx, "jac2_apply", nseq * npairs * (npairs * 4.0 + ceil_div(maxrt, blk) * 2.0) * bl * bl * bl,
-                                   nseq * npairs * (npairs * 2.0 + ceil_div(maxrt, blk) * 2.0) * bl * bl * 4.0);
-                        dim3 ag(npairs * (npairs + 1) / 2 + npairs * ceil_div(maxrt, blk), 1, cnt);
-                        if (jbj == 32) launch_pdl(jac2_apply_kernel<32, 4>, ag, dim3(256), ash, ctx->stream, jb, step);
-                        else launch_pdl(jac2_apply_kernel<16, 2>, ag, dim3(128), ash, ctx->stream, jb, step);
-                        ATP_LAUNCHED(ctx);
-                    }
-                    ATP_KERNEL(ctx, "jac2_sweep_end", 0, 0);
-                    jac2_sweep_end_kernel<<<1, J2MAX, 0, ctx->stream>>>(jb, tolc, pass == 1 && sw == nsw - 1, ctx->dev_status,
-                                                                        ctx->d_flags + (sw & 3));
-                    ATP_LAUNCHED(ctx);
-                    if (hsync) {
-                        ATP_CUDA_OK(ctx, cudaMemcpyAsync(ctx->h_flags + (sw & 3), ctx->d_flags + (sw & 3), sizeof(int),
-                                                         cudaMemcpyDeviceToHost, ctx->stream));
-                        ATP_CUDA_OK(ctx, cudaEventRecord(ctx->ev_flag[sw & 3], ctx->stream));
-                    }
-                }
+                // fp32 inputs: the block products stay on the fp32 units (the threshold is below split-precision rounding)
+                if ((st = j3::launch<std::is_same<T, __nv_bfloat16>::value>(ctx, jb, tolc, tolc * 0.25f, nsw, pass == 1)) != ATP_OK) return st;
                 if (pass == 0) {
                     GemmBatch r1, r2; r1.count = r2.count = cnt;
                     for (size_t i = i0; i < i1; ++i) {
                         SeqPlan &p = bp.seqs[i];
                         int k = (int)(i - i0);
                         // Bt2 = Bt Wt^T (d x r~),  Y2 = Y Wt^T (L x r~);  Wt rows are the eigenvectors
-                        r1.p[k] = GemmProblem{p.BW, p.Wt, p.Z, nullptr, p.rt > 0 ? d : 0, p.rt, p.rt, p.rt, p.rt, p.rt, 0};
-                        r2.p[k] = GemmProblem{p.Y, p.Wt, p.Y2, nullptr, p.dims.L, p.rt, p.rt, p.rt, p.rt, p.rt, 0};
+                        r1.p[k] = GemmProblem{p.BW, p.Wt, p.Z, nullptr, p.rt > 0 ? d : 0, p.rt, p.rt, p.rt, p.np, p.rt, 0};
+                        r2.p[k] = GemmProblem{p.Y, p.Wt, p.Y2, nullptr, p.dims.L, p.rt, p.rt, p.rt, p.np, p.rt, 0};
                         gg.p[k].A = p.Z; gg.p[k].B = p.Z;
                         fb.s[k].Y = p.Y2;
                     }

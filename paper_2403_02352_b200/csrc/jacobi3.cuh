@@ -1,0 +1,484 @@
+// Persistent two-sided block Jacobi eigensolver for the Gram matrix G = B B^T of the projected input
+// (Rayleigh-Ritz step of the basis extraction, Sec. 4.2: the rotation that diagonalises G turns the
+// orthonormal range basis into singular vectors, X' = [sigma_i v_i]).
+//
+// One cooperative launch diagonalises every sequence of a batch. Each sequence owns a fixed group of
+// CTAs that loops over sweeps and steps on its own and leaves when its matrix has converged; the
+// CTAs of a group meet at a counter in global memory (bounded spin) instead of at kernel boundaries.
+// Blocks of 32 rows; a step handles n/64 disjoint block pairs (round-robin order) in two phases:
+//   pivot : per pair, the 64 x 64 pivot block is rotated on chip by cyclic Jacobi. The rows live at
+//           64 "positions"; positions (2k, 2k+1) are rotated in every round and a fixed permutation
+//           of the positions between rounds brings new partners together (circle method for the
+//           first step of a sweep, which rotates all pairs of the 64 rows once; a cyclic shift of the
+//           second block's rows in the other steps, which rotates each cross pair once). All
+//           addresses are loop invariants; a round is one thread's instruction stream plus one
+//           block barrier. The accumulated row transform Vt (64 x 64) is published.
+//   apply : every 64 x 64 block (p, q) of G becomes Vt_p G_pq Vt_q^T (upper triangle computed, mirror
+//           stored), rows of Wt become Vt_p Wt. The 64^3 products run on the tensor cores in split
+//           precision (three TF32 mma products per fp32 product), which keeps fp32 accuracy.
+// G and Wt are stored with a leading dimension padded to a multiple of 64; the padding of G is zero
+// (zero diagonal entries are never rotated), the padding of Wt is the identity.
+#pragma once
+#include "common.cuh"
+#include <mutex>
+#include <algorithm>
+
+namespace j3 {
+
+constexpr int JB = 32;            // block height
+constexpr int BLK = 64;           // pivot block = one pair of blocks
+constexpr int NT = 256;           // threads per CTA
+constexpr int LDA = 68;           // shared-memory row stride (floats) of A-operand style tiles
+constexpr int LDB = 72;           // shared-memory row stride of B-operand style tiles
+constexpr int MAXSEQ = 32;        // sequences per launch
+constexpr unsigned SPIN_LIMIT = 1u << 22;
+
+struct Seq {
+    float *G, *Wt, *Vbuf;         // G, Wt: np x np (ld = np); Vbuf: npairs x 64 x 64
+    int *vflag;                   // npairs: the pair rotated in this step
+    unsigned *sync;               // [0]: group barrier counter (monotonic); [1..3]: largest scaled
+                                  // off-diagonal entry of a sweep, slot sweep % 3; [4]: sweeps used
+    int n, np, nb;                // size, padded size (multiple of 64), number of 32-row blocks (even)
+    int cta0, ncta;               // the group of CTAs that owns this sequence
+};
+struct Batch { Seq s[MAXSEQ]; int count; };
+
+// Bytes of dynamic shared memory: four 64 x LDA tiles (pivot phase: two copies of A and of V;
+// apply phase: Vt_p, Vt_q, T and the G block at stride LDB).
+constexpr size_t SMEM_BYTES = (size_t)(3 * BLK * LDA + BLK * LDB) * sizeof(float);
+
+__device__ __forceinline__ void rr_pair(int nb, int step, int t, int &I, int &J)
+{
+    const int m = nb - 1;
+    if (t == 0) { I = m; J = step % m; }
+    else { I = (step + t) % m; J = (step - t + m) % m; }
+    if (I > J) { const int x = I; I = J; J = x; }
+}
+
+// Group barrier: every CTA of the group adds one, then waits until the counter reaches `target`.
+// Returns false when the wait ran out or another CTA flagged an abort.
+__device__ __forceinline__ bool group_barrier(unsigned *bar, unsigned target, int *abort_flag)
+{
+    __syncthreads();
+    __shared__ int ok_s;
+    if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(bar, 1u);
+        int ok = 0;
+        for (unsigned i = 0; i < SPIN_LIMIT; ++i) {
+            const unsigned v = *(volatile unsigned *)bar;
+            if ((int)(v - target) >= 0) { ok = 1; break; }
+            if ((i & 255u) == 255u && *(volatile int *)abort_flag) break;
+            __nanosleep(32);
+        }
+        if (!ok) *(volatile int *)abort_flag = 1;
+        __threadfence();
+        ok_s = ok;
+    }
+    __syncthreads();
+    return ok_s != 0;
+}
+
+// Rotation (c, s) that annihilates the (p, q) entry of a symmetric matrix; identity when the entry is
+// already small against its diagonal. With a = g_qq - g_pp, b = 2 g_pq, r = sqrt(a^2 + b^2):
+//   cos 2t = |a| / r,  c = sqrt((1 + cos 2t) / 2),  s = sign(a) b / (2 r c)      (|t| <= pi/4).
+__device__ __forceinline__ float2 rotation(float gpp, float gqq, float gpq, float tol_rot)
+{
+    float c = 1.f, s = 0.f;
+    if (gpq != 0.f && gpq * gpq > tol_rot * tol_rot * fmaxf(gpp, 0.f) * fmaxf(gqq, 0.f)) {
+        float a = gqq - gpp, b = 2.f * gpq;
+        const float m = fmaxf(fabsf(a), fabsf(b));
+        const float sc = m < 1e-18f ? 0x1p60f : (m > 1e18f ? 0x1p-60f : 1.f);
+        a *= sc; b *= sc;
+        const float rh = rsqrtf(fmaf(a, a, b * b));
+        const float c2 = fmaf(0.5f * fabsf(a), rh, 0.5f);
+        const float rc = rsqrtf(c2);
+        c = c2 * rc;
+        s = copysignf(0.5f, a) * b * rh * rc;
+    }
+    return make_float2(c, s);
+}
+
+// Position permutation applied between rounds.
+//   full  : circle method, position 0 fixed, the other 63 positions form one cycle
+//           2 -> 4 -> ... -> 62 -> 63 -> 61 -> ... -> 3 -> 1 -> 2
+//   cross : even positions (rows of the first block) stay, odd positions shift by one pair
+__device__ __forceinline__ int perm_pos(int pos, bool cross)
+{
+    if (cross) return (pos & 1) ? ((pos + 2) & (BLK - 1)) : pos;
+    if (pos == 0) return 0;
+    if (pos & 1) return pos == 1 ? 2 : pos - 2;
+    return pos == BLK - 2 ? BLK - 1 : pos + 2;
+}
+// local row (0..31: first block, 32..63: second block) that starts at a position
+__device__ __forceinline__ int loc_of_pos(int pos) { return (pos >> 1) + ((pos & 1) ? JB : 0); }
+
+__device__ __forceinline__ int pos_of_loc(int l) { return l < JB ? 2 * l : 2 * (l - JB) + 1; }
+// global row / column of local index l of the pair (I, J)
+__device__ __forceinline__ int glob_of_loc(int I, int J, int l) { return (l < JB ? I : J) * JB + (l & (JB - 1)); }
+
+// ---- pivot phase -------------------------------------------------------------------------------
+// Rotates the 64 x 64 pivot block of the pair (I, J) on chip and publishes the accumulated row
+// transform Vt (new rows = Vt * old rows, logical order) to vout. 256 threads; thread (ta, tb) owns
+// the 4 x 4 element block at rows 4 ta, columns 4 tb of the position-indexed matrices, i.e. two row
+// pairs and two column pairs. It derives the rotations of its column pairs from the diagonal 4 x 4
+// block (tb, tb) and receives those of its row pairs by shuffle from the lane whose tb equals its ta.
+// Returns the largest scaled off-diagonal entry found in the block before rotating (block-uniform);
+// when it is <= tol_rot nothing is rotated and nothing is published.
+__device__ float pivot_solve(float *sm, const float *G, int np, int I, int J, bool cross, float tol_rot,
+                             float *vout, bool &rotated)
+{
+    __shared__ float red[NT / 32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    float *Ab0 = sm, *Ab1 = sm + BLK * LDA, *Vb0 = sm + 2 * BLK * LDA, *Vb1 = sm + 3 * BLK * LDA;
+    // coalesced 16-byte loads in logical order, scattered to the positions
+    for (int f = tid; f < BLK * (BLK / 4); f += NT) {
+        const int li = f >> 4, lj = (f & 15) * 4;
+        const float4 v = __ldcg((const float4 *)(G + (size_t)glob_of_loc(I, J, li) * np + glob_of_loc(I, J, lj)));
+        float *dst = Ab0 + pos_of_loc(li) * LDA;
+        dst[pos_of_loc(lj)] = v.x; dst[pos_of_loc(lj + 1)] = v.y; dst[pos_of_loc(lj + 2)] = v.z; dst[pos_of_loc(lj + 3)] = v.w;
+    }
+    for (int e = tid; e < BLK * BLK; e += NT) Vb0[(e >> 6) * LDA + (e & 63)] = ((e >> 6) == (e & 63)) ? 1.f : 0.f;
+    __syncthreads();
+    float mo = 0.f;
+    for (int e = tid; e < BLK * BLK; e += NT) {
+        const int i = e >> 6, j = e & 63;
+        if (i != j) {
+            const float dd = fmaxf(Ab0[i * LDA + i], 0.f) * fmaxf(Ab0[j * LDA + j], 0.f);
+            if (dd > 0.f) mo = fmaxf(mo, fabsf(Ab0[i * LDA + j]) * rsqrtf(dd));
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mo = fmaxf(mo, __shfl_xor_sync(0xffffffffu, mo, o));
+    if (lane == 0) red[warp] = mo;
+    __syncthreads();
+    mo = red[0];
+#pragma unroll
+    for (int w = 1; w < NT / 32; ++w) mo = fmaxf(mo, red[w]);
+    rotated = mo > tol_rot;
+    if (!rotated) return mo;
+
+    const int ta = tid >> 4, tb = tid & 15;
+    const int src_lane = (lane & 16) | ta;               // same warp, its tb equals this thread's ta
+    int prow[4], pcol[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { prow[i] = perm_pos(4 * ta + i, cross) * LDA; pcol[i] = perm_pos(4 * tb + i, cross); }
+    const int own = (4 * ta) * LDA + 4 * tb, dia = (4 * tb) * LDA + 4 * tb;
+    const int rounds = cross ? JB : BLK - 1;
+    for (int rd = 0; rd < rounds; ++rd) {
+        const float *Ao = (rd & 1) ? Ab1 : Ab0, *Vo = (rd & 1) ? Vb1 : Vb0;
+        float *An = (rd & 1) ? Ab0 : Ab1, *Vn = (rd & 1) ? Vb0 : Vb1;
+        const float2 d0 = *(const float2 *)(Ao + dia);                       // (0,0) (0,1)
+        const float d11 = Ao[dia + LDA + 1];
+        const float2 d2 = *(const float2 *)(Ao + dia + 2 * LDA + 2);         // (2,2) (2,3)
+        const float d33 = Ao[dia + 3 * LDA + 3];
+        float g[4][4], v[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float4 a = *(const float4 *)(Ao + own + i * LDA);
+            g[i][0] = a.x; g[i][1] = a.y; g[i][2] = a.z; g[i][3] = a.w;
+            const float4 b = *(const float4 *)(Vo + own + i * LDA);
+            v[i][0] = b.x; v[i][1] = b.y; v[i][2] = b.z; v[i][3] = b.w;
+        }
+        const float2 cb0 = rotation(d0.x, d11, d0.y, tol_rot);
+        const float2 cb1 = rotation(d2.x, d33, d2.y, tol_rot);
+        float2 ca0, ca1;
+        ca0.x = __shfl_sync(0xffffffffu, cb0.x, src_lane); ca0.y = __shfl_sync(0xffffffffu, cb0.y, src_lane);
+        ca1.x = __shfl_sync(0xffffffffu, cb1.x, src_lane); ca1.y = __shfl_sync(0xffffffffu, cb1.y, src_lane);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {                    // rows: (0,1) with ca0, (2,3) with ca1
+            float x = g[0][j], y = g[1][j];
+            g[0][j] = ca0.x * x - ca0.y * y; g[1][j] = ca0.y * x + ca0.x * y;
+            x = g[2][j]; y = g[3][j];
+            g[2][j] = ca1.x * x - ca1.y * y; g[3][j] = ca1.y * x + ca1.x * y;
+            x = v[0][j]; y = v[1][j];
+            v[0][j] = ca0.x * x - ca0.y * y; v[1][j] = ca0.y * x + ca0.x * y;
+            x = v[2][j]; y = v[3][j];
+            v[2][j] = ca1.x * x - ca1.y * y; v[3][j] = ca1.y * x + ca1.x * y;
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {                    // columns: (0,1) with cb0, (2,3) with cb1
+            float x = g[i][0], y = g[i][1];
+            g[i][0] = cb0.x * x - cb0.y * y; g[i][1] = cb0.y * x + cb0.x * y;
+            x = g[i][2]; y = g[i][3];
+            g[i][2] = cb1.x * x - cb1.y * y; g[i][3] = cb1.y * x + cb1.x * y;
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) An[prow[i] + pcol[j]] = g[i][j];
+            *(float4 *)(Vn + prow[i] + 4 * tb) = make_float4(v[i][0], v[i][1], v[i][2], v[i][3]);
+        }
+        __syncthreads();
+    }
+    // after `rounds` rounds every row is back at its starting position
+    const float *Vf = (rounds & 1) ? Vb1 : Vb0;
+    for (int e = tid; e < BLK * BLK; e += NT) vout[e] = Vf[pos_of_loc(e >> 6) * LDA + pos_of_loc(e & 63)];
+    return mo;
+}
+
+// ---- apply phase -------------------------------------------------------------------------------
+__device__ __forceinline__ void split_tf32(float x, uint32_t &hi, uint32_t &lo)
+{
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(hi) : "f"(x));
+    const float rest = x - __uint_as_float(hi);
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(lo) : "f"(rest));
+}
+__device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], const uint32_t (&b)[2])
+{
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+
+// acc (this warp's 16 x 32 part of a 64 x 64 result, rows m0.., columns n0..) = As * Bop, K = 64, in
+// split precision: x = hi + lo with both parts in TF32, product = lo*hi + hi*lo + hi*hi (the lo*lo term
+// is below fp32 rounding). As[m][k] at stride LDA; Bop[k][n] = Bs[k * ldb + n], or Bs[n * ldb + k] when
+// B_TRANS. Strides LDA = 68 and LDB = 72 make every fragment load conflict-free.
+template <bool B_TRANS>
+__device__ __forceinline__ void product64(const float *As, const float *Bs, int ldb, int m0, int n0, float (&acc)[4][4])
+{
+    const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[nt][i] = 0.f;
+#pragma unroll 2
+    for (int k0 = 0; k0 < BLK; k0 += 8) {
+        uint32_t ah[4], al[4];
+        split_tf32(As[(m0 + g) * LDA + k0 + t], ah[0], al[0]);
+        split_tf32(As[(m0 + g + 8) * LDA + k0 + t], ah[1], al[1]);
+        split_tf32(As[(m0 + g) * LDA + k0 + t + 4], ah[2], al[2]);
+        split_tf32(As[(m0 + g + 8) * LDA + k0 + t + 4], ah[3], al[3]);
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+            const int n = n0 + nt * 8 + g;
+            uint32_t bh[2], bl[2];
+            if (B_TRANS) {
+                split_tf32(Bs[n * ldb + k0 + t], bh[0], bl[0]);
+                split_tf32(Bs[n * ldb + k0 + t + 4], bh[1], bl[1]);
+            } else {
+                split_tf32(Bs[(k0 + t) * ldb + n], bh[0], bl[0]);
+                split_tf32(Bs[(k0 + t + 4) * ldb + n], bh[1], bl[1]);
+            }
+            mma_tf32(acc[nt], al, bh);
+            mma_tf32(acc[nt], ah, bl);
+            mma_tf32(acc[nt], ah, bh);
+        }
+    }
+}
+
+// The same product on the fp32 FMA units, with the ownership layout of the tensor-core version (this
+// thread: rows m0 + g and m0 + g + 8, columns n0 + 8 nt + 2 t, + 1). Used for fp32 inputs, whose
+// convergence threshold (1e-6) sits below the rounding of the split-precision product (~2^-21).
+template <bool B_TRANS>
+__device__ __forceinline__ void product64_fma(const float *As, const float *Bs, int ldb, int m0, int n0, float (&acc)[4][4])
+{
+    const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[nt][i] = 0.f;
+#pragma unroll 2
+    for (int k0 = 0; k0 < BLK; k0 += 4) {
+        const float4 a0 = *(const float4 *)(As + (m0 + g) * LDA + k0);
+        const float4 a1 = *(const float4 *)(As + (m0 + g + 8) * LDA + k0);
+        const float av0[4] = {a0.x, a0.y, a0.z, a0.w}, av1[4] = {a1.x, a1.y, a1.z, a1.w};
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) {
+                const int n = n0 + nt * 8 + 2 * t;
+                float b0, b1;
+                if (B_TRANS) { b0 = Bs[n * ldb + k0 + kk]; b1 = Bs[(n + 1) * ldb + k0 + kk]; }
+                else { const float2 b = *(const float2 *)(Bs + (k0 + kk) * ldb + n); b0 = b.x; b1 = b.y; }
+                acc[nt][0] = fmaf(av0[kk], b0, acc[nt][0]); acc[nt][1] = fmaf(av0[kk], b1, acc[nt][1]);
+                acc[nt][2] = fmaf(av1[kk], b0, acc[nt][2]); acc[nt][3] = fmaf(av1[kk], b1, acc[nt][3]);
+            }
+        }
+    }
+}
+
+// One block of the update. Items [0, ntri): block (p, q >= p) of G, enumerated row by row; items
+// [ntri, ntri + npairs * nw): rows of pair p of Wt, column chunk of 64.
+template <bool TENSOR>
+__device__ void apply_item(float *sm, const Seq &sq, int step, int idx, int npairs, int ntri, int nw)
+{
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+    const bool gblock = idx < ntri;
+    int p = 0, q = 0, chunk = 0;
+    if (gblock) {
+        while (idx >= npairs - p) { idx -= npairs - p; ++p; }
+        q = p + idx;
+    } else {
+        idx -= ntri;
+        p = idx / nw; chunk = idx - p * nw;
+    }
+    const int fp = __ldcg(sq.vflag + p);
+    const int fq = gblock ? __ldcg(sq.vflag + q) : 0;
+    if (!fp && !fq) return;
+    float *Vp = sm, *Vq = sm + BLK * LDA, *Tm = sm + 2 * BLK * LDA, *Bk = sm + 3 * BLK * LDA;
+    int Ip, Jp, Iq = 0, Jq = 0;
+    rr_pair(sq.nb, step, p, Ip, Jp);
+    if (gblock) rr_pair(sq.nb, step, q, Iq, Jq);
+    const int np = sq.np;
+    float *mat = gblock ? sq.G : sq.Wt;
+    auto gcol = [&](int c) -> int { return gblock ? glob_of_loc(Iq, Jq, c) : chunk * BLK + c; };
+    // the block goes to the B tile when a row transform comes first, else straight to the T tile
+    float *blk_dst = fp ? Bk : Tm;
+    const int blk_ld = fp ? LDB : LDA;
+    for (int f = tid; f < BLK * (BLK / 4); f += NT) {
+        const int i = f >> 4, c = (f & 15) * 4;
+        if (fp) *(float4 *)(Vp + i * LDA + c) = __ldcg((const float4 *)(sq.Vbuf + (size_t)p * BLK * BLK + i * BLK + c));
+        if (fq) *(float4 *)(Vq + i * LDA + c) = __ldcg((const float4 *)(sq.Vbuf + (size_t)q * BLK * BLK + i * BLK + c));
+        *(float4 *)(blk_dst + i * blk_ld + c) = __ldcg((const float4 *)(mat + (size_t)glob_of_loc(Ip, Jp, i) * np + gcol(c)));
+    }
+    __syncthreads();
+    const int m0 = (warp & 3) * 16, n0 = (warp >> 2) * 32;
+    float acc[4][4];
+    if (fp) {
+        if (TENSOR) product64<false>(Vp, Bk, LDB, m0, n0, acc);  // T = Vt_p * block
+        else product64_fma<false>(Vp, Bk, LDB, m0, n0, acc);
+        if (fq) {
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) {
+                const int c = n0 + nt * 8 + 2 * t;
+                *(float2 *)(Tm + (m0 + g) * LDA + c) = make_float2(acc[nt][0], acc[nt][1]);
+                *(float2 *)(Tm + (m0 + g + 8) * LDA + c) = make_float2(acc[nt][2], acc[nt][3]);
+            }
+            __syncthreads();
+        }
+    }
+    if (fq) {                                                    // out = T * Vt_q^T
+        if (TENSOR) product64<true>(Tm, Vq, LDA, m0, n0, acc);
+        else product64_fma<true>(Tm, Vq, LDA, m0, n0, acc);
+    }
+    const int gr0 = glob_of_loc(Ip, Jp, m0 + g), gr1 = glob_of_loc(Ip, Jp, m0 + g + 8);
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) {
+        const int gc = gcol(n0 + nt * 8 + 2 * t);                // gc, gc + 1 are contiguous
+        *(float2 *)(mat + (size_t)gr0 * np + gc) = make_float2(acc[nt][0], acc[nt][1]);
+        *(float2 *)(mat + (size_t)gr1 * np + gc) = make_float2(acc[nt][2], acc[nt][3]);
+        if (gblock && q != p) {                                  // mirror block
+            mat[(size_t)gc * np + gr0] = acc[nt][0]; mat[(size_t)(gc + 1) * np + gr0] = acc[nt][1];
+            mat[(size_t)gc * np + gr1] = acc[nt][2]; mat[(size_t)(gc + 1) * np + gr1] = acc[nt][3];
+        }
+    }
+    __syncthreads();                                             // tiles are reused by the next item
+}
+
+// ---- the kernel --------------------------------------------------------------------------------
+// status[0]: sticky device status word of the context; status[1]: abort flag of bounded waits.
+template <bool TENSOR>
+__global__ void __launch_bounds__(NT, 2)
+jacobi_persistent_kernel(const __grid_constant__ Batch batch, float tol_conv, float tol_rot, int max_sweeps,
+                         int raise_not_converged, int *status)
+{
+    extern __shared__ __align__(16) float j3sm[];
+    int si = 0;
+#pragma unroll 1
+    for (int i = 1; i < batch.count; ++i) if ((int)blockIdx.x >= batch.s[i].cta0) si = i;
+    const Seq &sq = batch.s[si];
+    const int rank = (int)blockIdx.x - sq.cta0;
+    if (rank >= sq.ncta || sq.np <= 0) return;
+    const int npairs = sq.nb / 2, nw = sq.np / BLK, ntri = npairs * (npairs + 1) / 2;
+    const int nsteps = sq.nb - 1;
+    int *abort_flag = status + 1;
+    unsigned target = 0;
+    bool converged = false, alive = true;
+    int sweep = 0;
+    for (; sweep < max_sweeps && alive; ++sweep) {
+        if (rank == 0 && threadIdx.x == 0) sq.sync[1 + (sweep + 1) % 3] = 0u;
+        for (int step = 0; step < nsteps && alive; ++step) {
+            for (int pr = rank; pr < npairs; pr += sq.ncta) {
+                int I, J;
+                rr_pair(sq.nb, step, pr, I, J);
+                bool rotated;
+                const float mo = pivot_solve(j3sm, sq.G, sq.np, I, J, step > 0, tol_rot,
+                                             sq.Vbuf + (size_t)pr * BLK * BLK, rotated);
+                if (threadIdx.x == 0) {
+                    sq.vflag[pr] = rotated ? 1 : 0;
+                    atomicMax(sq.sync + 1 + sweep % 3, __float_as_uint(mo));
+                }
+                __syncthreads();
+            }
+            target += (unsigned)sq.ncta;
+            alive = group_barrier(sq.sync, target, abort_flag);
+            if (!alive) break;
+            for (int it = rank; it < ntri + npairs * nw; it += sq.ncta) apply_item<TENSOR>(j3sm, sq, step, it, npairs, ntri, nw);
+            target += (unsigned)sq.ncta;
+            alive = group_barrier(sq.sync, target, abort_flag);
+        }
+        if (!alive) break;
+        const float mo = __uint_as_float(*(volatile unsigned *)(sq.sync + 1 + sweep % 3));
+        if (mo <= tol_conv) { converged = true; ++sweep; break; }
+    }
+    if (rank == 0 && threadIdx.x == 0) {
+        if (!alive) raise_status(status, ATP_ERR_TIMEOUT);
+        else if (!converged && raise_not_converged) raise_status(status, ATP_ERR_NOT_CONVERGED);
+        sq.sync[4] = (unsigned)sweep;
+    }
+}
+
+
+// Wt = identity, padding of G = 0, synchronisation words = 0. grid (x, count).
+__global__ void init_kernel(const __grid_constant__ Batch batch)
+{
+    const Seq &sq = batch.s[blockIdx.y];
+    const size_t n2 = (size_t)sq.np * sq.np;
+    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n2; e += (size_t)gridDim.x * blockDim.x) {
+        const int i = (int)(e / sq.np), j = (int)(e - (size_t)i * sq.np);
+        sq.Wt[e] = (i == j) ? 1.f : 0.f;
+        if (i >= sq.n || j >= sq.n) sq.G[e] = 0.f;
+    }
+    if (blockIdx.x == 0 && threadIdx.x < 8 && sq.np > 0) sq.sync[threadIdx.x] = 0u;
+}
+
+// Host side: hands every sequence a group of CTAs in proportion to the size of its update (at most one
+// CTA per block of the update, at least one) and launches the kernel cooperatively, so that all
+// groups are resident together and the group barriers cannot starve.
+template <bool TENSOR>
+static inline atp_status launch(atp_ctx *ctx, Batch &jb, float tol_conv, float tol_rot, int max_sweeps, bool raise_not_converged)
+{
+    if (jb.count <= 0) return ATP_OK;
+    static std::mutex mu;
+    static int occ_dev[64] = {};
+    int occ = 0;
+    {
+        std::lock_guard<std::mutex> lk(mu);
+        const int dv = ctx->device;
+        if (dv < 0 || dv >= 64 || occ_dev[dv] == 0) {
+            ATP_CUDA_OK(ctx, cudaFuncSetAttribute(jacobi_persistent_kernel<TENSOR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+            ATP_CUDA_OK(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, jacobi_persistent_kernel<TENSOR>, NT, SMEM_BYTES));
+            if (occ < 1) return ATP_ERR_CUDA;
+            if (dv >= 0 && dv < 64) occ_dev[dv] = occ;
+        } else occ = occ_dev[dv];
+    }
+    const int total = ctx->sm_count * std::min(occ, 2);
+    double wsum = 0;
+    for (int i = 0; i < jb.count; ++i) wsum += (double)jb.s[i].np * jb.s[i].np;
+    if (wsum <= 0) return ATP_OK;
+    int next = 0;
+    for (int i = 0; i < jb.count; ++i) {
+        Seq &q = jb.s[i];
+        const int npairs = q.nb / 2, items = npairs * (npairs + 1) / 2 + npairs * (q.np / BLK);
+        int c = (int)((double)total * ((double)q.np * q.np / wsum));
+        c = std::max(1, std::min(c, std::max(items, 1)));
+        if (q.np <= 0) c = 1;
+        q.cta0 = next; q.ncta = c;
+        next += c;
+    }
+    if (next > total) return ATP_ERR_INVALID_ARG;      // cannot happen: shares sum to at most `total`
+    ATP_KERNEL(ctx, "jacobi_init", 0, wsum * 4.0);
+    init_kernel<<<dim3(64, jb.count), 256, 0, ctx->stream>>>(jb);
+    ATP_LAUNCHED(ctx);
+    int *status = ctx->dev_status;
+    int ms = max_sweeps, rn = raise_not_converged ? 1 : 0;
+    void *args[] = {(void *)&jb, (void *)&tol_conv, (void *)&tol_rot, (void *)&ms, (void *)&rn, (void *)&status};
+    ATP_KERNEL(ctx, "jacobi_persistent", 0, 0);
+    ATP_CUDA_OK(ctx, cudaLaunchCooperativeKernel((const void *)jacobi_persistent_kernel<TENSOR>, dim3(next), dim3(NT), args, SMEM_BYTES, ctx->stream));
+    ATP_LAUNCHED(ctx);
+    return ATP_OK;
+}
+
+}  // namespace j3
