@@ -849,7 +849,7 @@ static void plan_basis(Arena &ar, const std::vector<SeqDims> &sd, int d, int ove
         p.Wt = ar.take<float>((size_t)p.np * p.np);
         p.Vbuf = ar.take<float>((size_t)(p.np / 64 + 1) * 4096);
         p.vflag = ar.take<int>(p.np / 64 + 4);
-        p.jsync = ar.take<unsigned>(8);
+        p.jsync = ar.take<unsigned>(64);
         p.needfix = ar.take<int>(std::max(p.dims.r, 1));
         p.maxoff = ar.take<unsigned>(1);
         p.conv = ar.take<int>(1);

@@ -36,8 +36,9 @@ constexpr unsigned SPIN_LIMIT = 1u << 22;
 struct Seq {
     float *G, *Wt, *Vbuf;         // G, Wt: np x np (ld = np); Vbuf: npairs x 64 x 64
     int *vflag;                   // npairs: the pair rotated in this step
-    unsigned *sync;               // [0]: group barrier counter (monotonic); [1..3]: largest scaled
-                                  // off-diagonal entry of a sweep, slot sweep % 3; [4]: sweeps used
+    unsigned *sync;               // 64 words. [0]: arrivals at the group barrier (monotonic); [32]: last
+                                  // barrier completed; [1..3]: largest scaled off-diagonal entry of a
+                                  // sweep, slot sweep % 3; [4]: sweeps used
     int n, np, nb;                // size, padded size (multiple of 64), number of 32-row blocks (even)
     int cta0, ncta;               // the group of CTAs that owns this sequence
 };
@@ -55,24 +56,33 @@ __device__ __forceinline__ void rr_pair(int nb, int step, int t, int &I, int &J)
     if (I > J) { const int x = I; I = J; J = x; }
 }
 
-// Group barrier: every CTA of the group adds one, then waits until the counter reaches `target`.
-// Returns false when the wait ran out or another CTA flagged an abort.
-__device__ __forceinline__ bool group_barrier(unsigned *bar, unsigned target, int *abort_flag)
+// Group barrier number `gen` (1, 2, ...) of a group of `ncta` CTAs: every CTA adds one to the arrival
+// counter sync[0]; the last one to arrive publishes `gen` in sync[32] (another cache line, so that
+// the pollers do not slow the arrivals down); the others poll that word. Bounded: returns false when
+// the wait ran out or another CTA flagged an abort.
+__device__ __forceinline__ bool group_barrier(unsigned *sync, unsigned gen, unsigned ncta, int *abort_flag)
 {
     __syncthreads();
     __shared__ int ok_s;
     if (threadIdx.x == 0) {
-        __threadfence();
-        atomicAdd(bar, 1u);
-        int ok = 0;
-        for (unsigned i = 0; i < SPIN_LIMIT; ++i) {
-            const unsigned v = *(volatile unsigned *)bar;
-            if ((int)(v - target) >= 0) { ok = 1; break; }
-            if ((i & 255u) == 255u && *(volatile int *)abort_flag) break;
-            __nanosleep(32);
+        int ok = 1;
+        if (ncta > 1) {
+            __threadfence();
+            const unsigned old = atomicAdd(sync, 1u);
+            volatile unsigned *flag = sync + 32;
+            if (old + 1u == gen * ncta) {
+                __threadfence();
+                *flag = gen;
+            } else {
+                ok = 0;
+                for (unsigned i = 0; i < SPIN_LIMIT; ++i) {
+                    if ((int)(*flag - gen) >= 0) { ok = 1; break; }
+                    if ((i & 1023u) == 1023u && *(volatile int *)abort_flag) break;
+                }
+                if (!ok) *(volatile int *)abort_flag = 1;
+            }
+            __threadfence();
         }
-        if (!ok) *(volatile int *)abort_flag = 1;
-        __threadfence();
         ok_s = ok;
     }
     __syncthreads();
@@ -99,53 +109,137 @@ __device__ __forceinline__ float2 rotation(float gpp, float gqq, float gpq, floa
     return make_float2(c, s);
 }
 
-// Position permutation applied between rounds.
-//   full  : circle method, position 0 fixed, the other 63 positions form one cycle
-//           2 -> 4 -> ... -> 62 -> 63 -> 61 -> ... -> 3 -> 1 -> 2
-//   cross : even positions (rows of the first block) stay, odd positions shift by one pair
-__device__ __forceinline__ int perm_pos(int pos, bool cross)
-{
-    if (cross) return (pos & 1) ? ((pos + 2) & (BLK - 1)) : pos;
-    if (pos == 0) return 0;
-    if (pos & 1) return pos == 1 ? 2 : pos - 2;
-    return pos == BLK - 2 ? BLK - 1 : pos + 2;
-}
-// local row (0..31: first block, 32..63: second block) that starts at a position
-__device__ __forceinline__ int loc_of_pos(int pos) { return (pos >> 1) + ((pos & 1) ? JB : 0); }
+// ---- pivot phase -------------------------------------------------------------------------------
+// The 64 rows of a pivot block sit in 32 "even" and 32 "odd" slots. A phase of width m rotates, in m
+// rounds, every even slot k with the odd slots of its own group of m: in round rd with slot
+// base(k) + ((k - rd) mod m). The data never moves between rounds, only the pairing shifts, so every
+// thread keeps its elements in registers:
+//   thread (warp w, lane l) owns the even rows 4w..4w+3 and column slot l of the four quadrants
+//     ee[a] = A[E(4w+a)][E(l)]   eo[a] = A[E(4w+a)][O(s(l))]
+//     oe[a] = A[O(s(4w+a))][E(l)]   oo[a] = A[O(s(4w+a))][O(s(l))]         s = current pairing
+//   and the same rows of the accumulated transform Vt (two logical columns l, l + 32).
+// The 2 x 2 problem of pair k is complete in the thread with 4w+a = l, which derives the rotation and
+// publishes it; everybody applies the rotations of its four row pairs and of its column pair. Moving
+// to the next pairing shifts the odd quadrants by one slot: along the columns by a lane shuffle,
+// along the rows inside the thread, except the last of its four rows, which goes to the next warp
+// through shared memory (4 floats per thread and round).
+// Slot -> logical row (0..31 first block, 32..63 second block) for a phase of width m: the logical
+// rows are cut in groups of 2m; the first m of a group are even slots, the last m odd slots. Width 32
+// pairs every row of the first block with every row of the second; widths 16, 8, 4, 2, 1 pair the rows
+// inside the blocks; together the 63 rounds rotate each of the 2016 pairs exactly once.
+constexpr int LDP = 65;           // row stride of the logical A and Vt copies in shared memory
+__device__ __forceinline__ int slot_even(int i, int m) { return 2 * m * (i / m) + (i % m); }
 
-__device__ __forceinline__ int pos_of_loc(int l) { return l < JB ? 2 * l : 2 * (l - JB) + 1; }
+__device__ void cross_phase(float *As, float *Vs, float2 *rot, float4 *xch, int m, float tol_rot)
+{
+    const int tid = threadIdx.x, w = tid >> 5, l = tid & 31;
+    float ee[4], eo[4], oe[4], oo[4], ve[4][2], vo[4][2];
+    const int cE = slot_even(l, m), cO = cE + m;
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+        const int rE = slot_even(4 * w + a, m) * LDP, rO = rE + m * LDP;
+        ee[a] = As[rE + cE]; eo[a] = As[rE + cO]; oe[a] = As[rO + cE]; oo[a] = As[rO + cO];
+        ve[a][0] = Vs[rE + l]; ve[a][1] = Vs[rE + l + 32];
+        vo[a][0] = Vs[rO + l]; vo[a][1] = Vs[rO + l + 32];
+    }
+    const int ad = l - 4 * w;                                   // 0..3: this thread completes pair 4w + ad
+    const int src_lane = (l & ~(m - 1)) | ((l - 1) & (m - 1));  // previous column slot of the group
+    const int wg = m >= 8 ? m / 4 : 1;                          // warps per row group
+    const int wprev = (w & ~(wg - 1)) | ((w - 1) & (wg - 1));
+    for (int rd = 0; rd < m; ++rd) {
+        float2 *rt = rot + (rd & 1) * 32;
+        if ((unsigned)ad < 4u) {
+            const float x = ad == 0 ? ee[0] : ad == 1 ? ee[1] : ad == 2 ? ee[2] : ee[3];
+            const float y = ad == 0 ? oo[0] : ad == 1 ? oo[1] : ad == 2 ? oo[2] : oo[3];
+            const float z = ad == 0 ? eo[0] : ad == 1 ? eo[1] : ad == 2 ? eo[2] : eo[3];
+            rt[l] = rotation(x, y, z, tol_rot);
+        }
+        __syncthreads();
+        const float2 cb = rt[l];
+#pragma unroll
+        for (int a = 0; a < 4; ++a) {
+            const float2 ca = rt[4 * w + a];
+            const float r0 = ca.x * ee[a] - ca.y * oe[a], r1 = ca.x * eo[a] - ca.y * oo[a];
+            const float r2 = ca.y * ee[a] + ca.x * oe[a], r3 = ca.y * eo[a] + ca.x * oo[a];
+            ee[a] = cb.x * r0 - cb.y * r1; eo[a] = cb.y * r0 + cb.x * r1;
+            oe[a] = cb.x * r2 - cb.y * r3; oo[a] = cb.y * r2 + cb.x * r3;
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                const float x = ve[a][c], y = vo[a][c];
+                ve[a][c] = ca.x * x - ca.y * y; vo[a][c] = ca.y * x + ca.x * y;
+            }
+        }
+        if (m == 1) break;
+        // next pairing: odd rows shift by one slot inside their group ...
+        float4 in;
+        if (m >= 8) {
+            xch[tid] = make_float4(oe[3], oo[3], vo[3][0], vo[3][1]);
+            __syncthreads();
+            in = xch[wprev * 32 + l];
+        } else if (m == 4) {
+            in = make_float4(oe[3], oo[3], vo[3][0], vo[3][1]);
+        }
+        if (m >= 4) {
+#pragma unroll
+            for (int a = 3; a > 0; --a) { oe[a] = oe[a - 1]; oo[a] = oo[a - 1]; vo[a][0] = vo[a - 1][0]; vo[a][1] = vo[a - 1][1]; }
+            oe[0] = in.x; oo[0] = in.y; vo[0][0] = in.z; vo[0][1] = in.w;
+        } else {                                                // m == 2: rows (0,1) and (2,3) swap
+#pragma unroll
+            for (int a = 0; a < 4; a += 2) {
+                float t;
+                t = oe[a]; oe[a] = oe[a + 1]; oe[a + 1] = t;
+                t = oo[a]; oo[a] = oo[a + 1]; oo[a + 1] = t;
+                t = vo[a][0]; vo[a][0] = vo[a + 1][0]; vo[a + 1][0] = t;
+                t = vo[a][1]; vo[a][1] = vo[a + 1][1]; vo[a + 1][1] = t;
+            }
+        }
+        // ... and so do the odd columns
+#pragma unroll
+        for (int a = 0; a < 4; ++a) {
+            eo[a] = __shfl_sync(0xffffffffu, eo[a], src_lane);
+            oo[a] = __shfl_sync(0xffffffffu, oo[a], src_lane);
+        }
+    }
+    // after m shifts (none for m = 1) every element is back where it was loaded from
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+        const int rE = slot_even(4 * w + a, m) * LDP, rO = rE + m * LDP;
+        As[rE + cE] = ee[a]; As[rE + cO] = eo[a]; As[rO + cE] = oe[a]; As[rO + cO] = oo[a];
+        Vs[rE + l] = ve[a][0]; Vs[rE + l + 32] = ve[a][1];
+        Vs[rO + l] = vo[a][0]; Vs[rO + l + 32] = vo[a][1];
+    }
+    __syncthreads();
+}
+
 // global row / column of local index l of the pair (I, J)
 __device__ __forceinline__ int glob_of_loc(int I, int J, int l) { return (l < JB ? I : J) * JB + (l & (JB - 1)); }
 
-// ---- pivot phase -------------------------------------------------------------------------------
 // Rotates the 64 x 64 pivot block of the pair (I, J) on chip and publishes the accumulated row
-// transform Vt (new rows = Vt * old rows, logical order) to vout. 256 threads; thread (ta, tb) owns
-// the 4 x 4 element block at rows 4 ta, columns 4 tb of the position-indexed matrices, i.e. two row
-// pairs and two column pairs. It derives the rotations of its column pairs from the diagonal 4 x 4
-// block (tb, tb) and receives those of its row pairs by shuffle from the lane whose tb equals its ta.
-// Returns the largest scaled off-diagonal entry found in the block before rotating (block-uniform);
-// when it is <= tol_rot nothing is rotated and nothing is published.
-__device__ float pivot_solve(float *sm, const float *G, int np, int I, int J, bool cross, float tol_rot,
+// transform Vt (new rows = Vt * old rows, logical order) to vout. cross_only: the 32 rounds that pair
+// the two blocks' rows; otherwise all 63 rounds. Returns the largest scaled off-diagonal entry found
+// in the block before rotating (block-uniform); when it is <= tol_rot nothing is rotated or published.
+__device__ float pivot_solve(float *sm, const float *G, int np, int I, int J, bool cross_only, float tol_rot,
                              float *vout, bool &rotated)
 {
     __shared__ float red[NT / 32];
+    __shared__ float2 rot[64];
+    __shared__ float4 xch[NT];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    float *Ab0 = sm, *Ab1 = sm + BLK * LDA, *Vb0 = sm + 2 * BLK * LDA, *Vb1 = sm + 3 * BLK * LDA;
-    // coalesced 16-byte loads in logical order, scattered to the positions
+    float *As = sm, *Vs = sm + BLK * LDP;
     for (int f = tid; f < BLK * (BLK / 4); f += NT) {
         const int li = f >> 4, lj = (f & 15) * 4;
         const float4 v = __ldcg((const float4 *)(G + (size_t)glob_of_loc(I, J, li) * np + glob_of_loc(I, J, lj)));
-        float *dst = Ab0 + pos_of_loc(li) * LDA;
-        dst[pos_of_loc(lj)] = v.x; dst[pos_of_loc(lj + 1)] = v.y; dst[pos_of_loc(lj + 2)] = v.z; dst[pos_of_loc(lj + 3)] = v.w;
+        float *dst = As + li * LDP + lj;
+        dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
     }
-    for (int e = tid; e < BLK * BLK; e += NT) Vb0[(e >> 6) * LDA + (e & 63)] = ((e >> 6) == (e & 63)) ? 1.f : 0.f;
+    for (int e = tid; e < BLK * BLK; e += NT) Vs[(e >> 6) * LDP + (e & 63)] = ((e >> 6) == (e & 63)) ? 1.f : 0.f;
     __syncthreads();
     float mo = 0.f;
     for (int e = tid; e < BLK * BLK; e += NT) {
         const int i = e >> 6, j = e & 63;
         if (i != j) {
-            const float dd = fmaxf(Ab0[i * LDA + i], 0.f) * fmaxf(Ab0[j * LDA + j], 0.f);
-            if (dd > 0.f) mo = fmaxf(mo, fabsf(Ab0[i * LDA + j]) * rsqrtf(dd));
+            const float dd = fmaxf(As[i * LDP + i], 0.f) * fmaxf(As[j * LDP + j], 0.f);
+            if (dd > 0.f) mo = fmaxf(mo, fabsf(As[i * LDP + j]) * rsqrtf(dd));
         }
     }
 #pragma unroll
@@ -157,63 +251,10 @@ __device__ float pivot_solve(float *sm, const float *G, int np, int I, int J, bo
     for (int w = 1; w < NT / 32; ++w) mo = fmaxf(mo, red[w]);
     rotated = mo > tol_rot;
     if (!rotated) return mo;
-
-    const int ta = tid >> 4, tb = tid & 15;
-    const int src_lane = (lane & 16) | ta;               // same warp, its tb equals this thread's ta
-    int prow[4], pcol[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) { prow[i] = perm_pos(4 * ta + i, cross) * LDA; pcol[i] = perm_pos(4 * tb + i, cross); }
-    const int own = (4 * ta) * LDA + 4 * tb, dia = (4 * tb) * LDA + 4 * tb;
-    const int rounds = cross ? JB : BLK - 1;
-    for (int rd = 0; rd < rounds; ++rd) {
-        const float *Ao = (rd & 1) ? Ab1 : Ab0, *Vo = (rd & 1) ? Vb1 : Vb0;
-        float *An = (rd & 1) ? Ab0 : Ab1, *Vn = (rd & 1) ? Vb0 : Vb1;
-        const float2 d0 = *(const float2 *)(Ao + dia);                       // (0,0) (0,1)
-        const float d11 = Ao[dia + LDA + 1];
-        const float2 d2 = *(const float2 *)(Ao + dia + 2 * LDA + 2);         // (2,2) (2,3)
-        const float d33 = Ao[dia + 3 * LDA + 3];
-        float g[4][4], v[4][4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const float4 a = *(const float4 *)(Ao + own + i * LDA);
-            g[i][0] = a.x; g[i][1] = a.y; g[i][2] = a.z; g[i][3] = a.w;
-            const float4 b = *(const float4 *)(Vo + own + i * LDA);
-            v[i][0] = b.x; v[i][1] = b.y; v[i][2] = b.z; v[i][3] = b.w;
-        }
-        const float2 cb0 = rotation(d0.x, d11, d0.y, tol_rot);
-        const float2 cb1 = rotation(d2.x, d33, d2.y, tol_rot);
-        float2 ca0, ca1;
-        ca0.x = __shfl_sync(0xffffffffu, cb0.x, src_lane); ca0.y = __shfl_sync(0xffffffffu, cb0.y, src_lane);
-        ca1.x = __shfl_sync(0xffffffffu, cb1.x, src_lane); ca1.y = __shfl_sync(0xffffffffu, cb1.y, src_lane);
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {                    // rows: (0,1) with ca0, (2,3) with ca1
-            float x = g[0][j], y = g[1][j];
-            g[0][j] = ca0.x * x - ca0.y * y; g[1][j] = ca0.y * x + ca0.x * y;
-            x = g[2][j]; y = g[3][j];
-            g[2][j] = ca1.x * x - ca1.y * y; g[3][j] = ca1.y * x + ca1.x * y;
-            x = v[0][j]; y = v[1][j];
-            v[0][j] = ca0.x * x - ca0.y * y; v[1][j] = ca0.y * x + ca0.x * y;
-            x = v[2][j]; y = v[3][j];
-            v[2][j] = ca1.x * x - ca1.y * y; v[3][j] = ca1.y * x + ca1.x * y;
-        }
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {                    // columns: (0,1) with cb0, (2,3) with cb1
-            float x = g[i][0], y = g[i][1];
-            g[i][0] = cb0.x * x - cb0.y * y; g[i][1] = cb0.y * x + cb0.x * y;
-            x = g[i][2]; y = g[i][3];
-            g[i][2] = cb1.x * x - cb1.y * y; g[i][3] = cb1.y * x + cb1.x * y;
-        }
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-#pragma unroll
-            for (int j = 0; j < 4; ++j) An[prow[i] + pcol[j]] = g[i][j];
-            *(float4 *)(Vn + prow[i] + 4 * tb) = make_float4(v[i][0], v[i][1], v[i][2], v[i][3]);
-        }
-        __syncthreads();
-    }
-    // after `rounds` rounds every row is back at its starting position
-    const float *Vf = (rounds & 1) ? Vb1 : Vb0;
-    for (int e = tid; e < BLK * BLK; e += NT) vout[e] = Vf[pos_of_loc(e >> 6) * LDA + pos_of_loc(e & 63)];
+    cross_phase(As, Vs, rot, xch, 32, tol_rot);
+    if (!cross_only)
+        for (int m = 16; m >= 1; m >>= 1) cross_phase(As, Vs, rot, xch, m, tol_rot);
+    for (int e = tid; e < BLK * BLK; e += NT) vout[e] = Vs[(e >> 6) * LDP + (e & 63)];
     return mo;
 }
 
@@ -384,7 +425,7 @@ jacobi_persistent_kernel(const __grid_constant__ Batch batch, float tol_conv, fl
     const int npairs = sq.nb / 2, nw = sq.np / BLK, ntri = npairs * (npairs + 1) / 2;
     const int nsteps = sq.nb - 1;
     int *abort_flag = status + 1;
-    unsigned target = 0;
+    unsigned gen = 0;
     bool converged = false, alive = true;
     int sweep = 0;
     for (; sweep < max_sweeps && alive; ++sweep) {
@@ -402,12 +443,10 @@ jacobi_persistent_kernel(const __grid_constant__ Batch batch, float tol_conv, fl
                 }
                 __syncthreads();
             }
-            target += (unsigned)sq.ncta;
-            alive = group_barrier(sq.sync, target, abort_flag);
+            alive = group_barrier(sq.sync, ++gen, (unsigned)sq.ncta, abort_flag);
             if (!alive) break;
             for (int it = rank; it < ntri + npairs * nw; it += sq.ncta) apply_item<TENSOR>(j3sm, sq, step, it, npairs, ntri, nw);
-            target += (unsigned)sq.ncta;
-            alive = group_barrier(sq.sync, target, abort_flag);
+            alive = group_barrier(sq.sync, ++gen, (unsigned)sq.ncta, abort_flag);
         }
         if (!alive) break;
         const float mo = __uint_as_float(*(volatile unsigned *)(sq.sync + 1 + sweep % 3));
@@ -431,7 +470,7 @@ __global__ void init_kernel(const __grid_constant__ Batch batch)
         sq.Wt[e] = (i == j) ? 1.f : 0.f;
         if (i >= sq.n || j >= sq.n) sq.G[e] = 0.f;
     }
-    if (blockIdx.x == 0 && threadIdx.x < 8 && sq.np > 0) sq.sync[threadIdx.x] = 0u;
+    if (blockIdx.x == 0 && threadIdx.x < 64 && sq.np > 0) sq.sync[threadIdx.x] = 0u;
 }
 
 // Host side: hands every sequence a group of CTAs in proportion to the size of its update (at most one
