@@ -59,8 +59,13 @@ ORACLE_API int oracle_num_threads(void) {
 /* a_i = sigma_i * w_i with w_i orthonormal and row i of G is the     */
 /* matching singular vector on the other side.                        */
 /* ------------------------------------------------------------------ */
-static int jacobi_rows(double *A, double *G, int n, int m, double tol, int max_sweeps)
+/* max_rounds > 0 stops the iteration after that many rounds (a round rotates n/2 disjoint pairs; a    */
+/* sweep is n-1 rounds). It exists only so that a timing run can measure a bounded part of a large    */
+/* problem; the arithmetic of a round is the same and *rounds_done (nullable) reports what was run.   */
+static int jacobi_rows(double *A, double *G, int n, int m, double tol, int max_sweeps, long max_rounds, long *rounds_done)
 {
+    long rounds = 0;
+    int stopped = 0;
     int np = n + (n & 1);              /* pad to even for the round-robin schedule */
     int *idx = (int *)malloc(sizeof(int) * np);
     for (int i = 0; i < np; ++i) idx[i] = i;
@@ -76,6 +81,8 @@ static int jacobi_rows(double *A, double *G, int n, int m, double tol, int max_s
         }
         double tiny = nmax * 1e-300;
         for (int round = 0; round < np - 1; ++round) {
+            if (max_rounds > 0 && rounds >= max_rounds) { stopped = 1; break; }
+            ++rounds;
 #pragma omp parallel for schedule(dynamic, 4) reduction(max : worst)
             for (int t = 0; t < np / 2; ++t) {
                 int p = idx[t], q = idx[np - 1 - t];
@@ -112,9 +119,11 @@ static int jacobi_rows(double *A, double *G, int n, int m, double tol, int max_s
             for (int i = np - 1; i > 1; --i) idx[i] = idx[i - 1];
             idx[1] = last;
         }
+        if (stopped) break;
         if (worst < tol) { ++sweeps; break; }
     }
     free(idx);
+    if (rounds_done) *rounds_done = rounds;
     return sweeps;
 }
 
@@ -123,7 +132,22 @@ static int jacobi_rows(double *A, double *G, int n, int m, double tol, int max_s
  * Returns the number of sweeps used (60 if the tolerance was not met).
  * Singular vectors that belong to sigma = 0 are completed to an orthonormal set.
  */
+static int svd_jacobi_impl(const double *X, int L, int d, double *U, double *S, double *Vt, long max_rounds, long *rounds_done);
+
 ORACLE_API int oracle_svd_jacobi(const double *X, int L, int d, double *U, double *S, double *Vt)
+{
+    return svd_jacobi_impl(X, L, d, U, S, Vt, 0, NULL);
+}
+
+/* The same routine stopped after max_rounds rounds (see jacobi_rows): for timing a bounded sample of a
+ * large decomposition. Its outputs are those of an unfinished iteration and are not a decomposition. */
+ORACLE_API int oracle_svd_jacobi_capped(const double *X, int L, int d, double *U, double *S, double *Vt,
+                                        long max_rounds, long *rounds_done)
+{
+    return svd_jacobi_impl(X, L, d, U, S, Vt, max_rounds, rounds_done);
+}
+
+static int svd_jacobi_impl(const double *X, int L, int d, double *U, double *S, double *Vt, long max_rounds, long *rounds_done)
 {
     int n = L < d ? L : d;
     int m = L < d ? d : L;
@@ -137,7 +161,7 @@ ORACLE_API int oracle_svd_jacobi(const double *X, int L, int d, double *U, doubl
             for (int j = 0; j < d; ++j) A[(size_t)j * L + i] = X[(size_t)i * d + j];
     }
     for (int i = 0; i < n; ++i) G[(size_t)i * n + i] = 1.0;
-    int sweeps = jacobi_rows(A, G, n, m, 1e-14, 60);
+    int sweeps = jacobi_rows(A, G, n, m, 1e-14, 60, max_rounds, rounds_done);
 
     double *sig = (double *)malloc(sizeof(double) * n);
     int *ord = (int *)malloc(sizeof(int) * n);

@@ -376,11 +376,10 @@ template <int DH>
 static atp_status launch(atp_ctx *ctx, const std::vector<HostSeq> &seqs, int heads, float scale)
 {
     using C_ = Cfg<DH>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        ATP_CUDA_OK(ctx, cudaFuncSetAttribute(attn_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::SMEM));
-        attr_set = true;
-    }
+    static PerDeviceOnce attr_once;        // the shared-memory opt-in is a per-device attribute
+    ATP_CUDA_OK(ctx, attr_once.run(ctx->device, [] {
+        return cudaFuncSetAttribute(attn_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::SMEM);
+    }));
     size_t i = 0;
     while (i < seqs.size()) {
         Batch b; b.count = 0; b.total_tiles = 0;

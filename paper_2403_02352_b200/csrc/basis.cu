@@ -678,9 +678,13 @@ __global__ void __launch_bounds__(256) select_kernel(const __grid_constant__ Fin
 }
 
 // ---- finalisation of the two-sided path ----------------------------------------------------------
+constexpr int COLSUM_SLABS = 16;
 struct Fin2Seq {
     const float *G; const float *Wt; const float *Y; float *sig; int *ord; float *tsum; float *Wsel; int *needfix;
     void *Xr; void *U; float *sigma_out; int rt, r, d, L, ldy, ldxr, ldu, ldg;
+    // bf16 inputs: Y is held as a hi/lo pair (leading dimension ldy), and Wsel is written as one (ldws)
+    const __nv_bfloat16 *Yh, *Yl; __nv_bfloat16 *Wselh, *Wsell; int ldws;
+    float *tpart;                 // COLSUM_SLABS x rt partial column sums
 };
 struct Fin2Batch { Fin2Seq s[BMAX]; int count; };
 
@@ -694,6 +698,11 @@ __global__ void __launch_bounds__(1024) sigma_sort2_kernel(const __grid_constant
     float *key = sh;
     int *idx = (int *)(sh + npow);
     const int tid = threadIdx.x;
+    for (int k = tid; k < sq.rt; k += 1024) {       // column sums of Y from the slab sums, fixed order
+        float t = 0.f;
+        for (int sl = 0; sl < COLSUM_SLABS; ++sl) t += sq.tpart[(size_t)sl * sq.rt + k];
+        sq.tsum[k] = t;
+    }
     for (int i = tid; i < npow; i += 1024) {
         key[i] = (i < sq.rt) ? sqrtf(fmaxf(sq.G[(size_t)i * sq.ldg + i], 0.f)) : -1.f;
         idx[i] = i;
@@ -716,14 +725,28 @@ __global__ void __launch_bounds__(1024) sigma_sort2_kernel(const __grid_constant
     for (int i = tid; i < sq.rt; i += 1024) { sq.sig[i] = key[i]; sq.ord[i] = idx[i]; }
 }
 
-__global__ void colsum2_kernel(const __grid_constant__ Fin2Batch batch)
+// Column sums of Y (L x r~): t[k] = sum_l Y[l][k]. grid (column chunks of 32, row slabs, batch); 8 warps of a
+// CTA take interleaved rows of the slab, lanes take columns; the slab sums go to tpart and are added up in a
+// fixed order by sigma_sort2_kernel (same result on every run).
+__global__ void __launch_bounds__(256) colsum2_kernel(const __grid_constant__ Fin2Batch batch)
 {
-    const Fin2Seq &sq = batch.s[blockIdx.y];
-    int k = blockIdx.x * blockDim.x + threadIdx.x;
-    if (k >= sq.rt) return;
+    const Fin2Seq &sq = batch.s[blockIdx.z];
+    const int k = blockIdx.x * 32 + (threadIdx.x & 31), w = threadIdx.x >> 5;
+    const int rows = (sq.L + COLSUM_SLABS - 1) / COLSUM_SLABS, l0 = blockIdx.y * rows, l1 = min(sq.L, l0 + rows);
     float s = 0.f;
-    for (int l = 0; l < sq.L; ++l) s += sq.Y[(size_t)l * sq.ldy + k];
-    sq.tsum[k] = s;
+    if (k < sq.rt) {
+        if (sq.Yh) for (int l = l0 + w; l < l1; l += 8) s += __bfloat162float(sq.Yh[(size_t)l * sq.ldy + k]) + __bfloat162float(sq.Yl[(size_t)l * sq.ldy + k]);
+        else for (int l = l0 + w; l < l1; l += 8) s += sq.Y[(size_t)l * sq.ldy + k];
+    }
+    __shared__ float part[8][33];
+    part[w][threadIdx.x & 31] = s;
+    __syncthreads();
+    if (w == 0 && k < sq.rt) {
+        float t = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) t += part[i][threadIdx.x];
+        sq.tpart[(size_t)blockIdx.y * sq.rt + k] = t;
+    }
 }
 
 // One CTA per kept component: sign from the column sum of U (= tsum . w), Wsel column, sigma.
@@ -744,7 +767,16 @@ __global__ void __launch_bounds__(128) select2_kernel(const __grid_constant__ Fi
     __syncthreads();
     float colsum = redf[0] + redf[1] + redf[2] + redf[3];
     float sgn = colsum < 0.f ? -1.f : 1.f;
-    for (int k = tid; k < sq.rt; k += 128) sq.Wsel[(size_t)k * sq.r + a] = sgn * w[k];
+    if (sq.Wselh) {
+        for (int k = tid; k < sq.rt; k += 128) {
+            const float v = sgn * w[k];
+            const __nv_bfloat16 h = __float2bfloat16_rn(v);
+            sq.Wselh[(size_t)k * sq.ldws + a] = h;
+            sq.Wsell[(size_t)k * sq.ldws + a] = __float2bfloat16_rn(v - __bfloat162float(h));
+        }
+    } else {
+        for (int k = tid; k < sq.rt; k += 128) sq.Wsel[(size_t)k * sq.r + a] = sgn * w[k];
+    }
     if (tid == 0) {
         sq.needfix[a] = fabsf(colsum) < 1e-6f * sqrtf((float)sq.L);
         if (sq.sigma_out) sq.sigma_out[a] = sq.sig[a];
@@ -791,7 +823,8 @@ __global__ void __launch_bounds__(256) signfix_kernel(const __grid_constant__ Fi
 
 // ------------------------------------------------------------------------------------------------
 struct SeqPlan {
-    SeqDims dims; int rt, np, npanel_L, npanel_d; unsigned *jsync;
+    SeqDims dims; int rt, np, npanel_L, npanel_d; unsigned *jsync, *jdone; float *tpart;
+    __nv_bfloat16 *Bth, *Btl, *Y2h, *Y2l, *Wth, *Wtl, *Wsh, *Wsl;
     __nv_bfloat16 *Yb, *Yl, *Zb, *Zl; float *Y2; float *Y, *Z, *BW, *Wsel, *tsum, *sig, *Cc, *rinv, *G, *Wt, *Vbuf; double *gpart; int *ord, *flags, *conv, *vflag, *needfix; unsigned *maxoff;
 };
 struct BasisPlan {
@@ -847,8 +880,17 @@ static void plan_basis(Arena &ar, const std::vector<SeqDims> &sd, int d, int ove
         p.np = jacobi_padded(rt);
         p.G = ar.take<float>((size_t)p.np * p.np);
         p.Wt = ar.take<float>((size_t)p.np * p.np);
-        p.Vbuf = ar.take<float>((size_t)(p.np / 64 + 1) * 4096);
-        p.vflag = ar.take<int>(p.np / 64 + 4);
+        p.Vbuf = ar.take<float>((size_t)2 * (p.np / 64 + 1) * 4096);
+        p.vflag = ar.take<int>(2 * (p.np / 64) + 4);
+        p.tpart = ar.take<float>((size_t)COLSUM_SLABS * std::max(rt, 1));
+        {   // bf16 hi/lo operands of the tensor-core products around the rotation (bf16 inputs only)
+            const size_t ldr = align_up((size_t)std::max(rt, 1), 8), ldw = align_up((size_t)std::max(p.dims.r, 1), 8);
+            p.Bth = ar.take<__nv_bfloat16>((size_t)d * ldr); p.Btl = ar.take<__nv_bfloat16>((size_t)d * ldr);
+            p.Y2h = ar.take<__nv_bfloat16>((size_t)L * ldr); p.Y2l = ar.take<__nv_bfloat16>((size_t)L * ldr);
+            p.Wth = ar.take<__nv_bfloat16>((size_t)p.np * p.np); p.Wtl = ar.take<__nv_bfloat16>((size_t)p.np * p.np);
+            p.Wsh = ar.take<__nv_bfloat16>((size_t)std::max(rt, 1) * ldw); p.Wsl = ar.take<__nv_bfloat16>((size_t)std::max(rt, 1) * ldw);
+        }
+        p.jdone = ar.take<unsigned>((size_t)(p.np / 64) * (p.np / 64 + 1) / 2 + 4);
         p.jsync = ar.take<unsigned>(64);
         p.needfix = ar.take<int>(std::max(p.dims.r, 1));
         p.maxoff = ar.take<unsigned>(1);
@@ -1105,29 +1147,36 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
         } else {
             // Bt = X^T Y (d x r~, i.e. B^T), G = Bt^T Bt, two-sided block Jacobi on G, then
             // X_r = Wsel^T Bt^T and U_r = Y Wsel
+            constexpr bool kBf16 = std::is_same<T, __nv_bfloat16>::value;
             j3::Batch jb; jb.count = cnt; Fin2Batch fb; fb.count = cnt;
             GemmBatch gg; gg.count = cnt;
-            int maxrt = 0, maxr = 0;
+            int maxrt = 0, maxr = 0, maxL = 0;
             for (size_t i = i0; i < i1; ++i) {
                 SeqPlan &p = bp.seqs[i];
                 int k = (int)(i - i0);
+                const int ldr = (int)align_up((size_t)std::max(p.rt, 1), 8), ldw = (int)align_up((size_t)std::max(p.dims.r, 1), 8);
                 g.p[k] = GemmProblem{Xb(p), p.Y, p.BW, nullptr, p.rt > 0 ? d : 0, p.rt, p.dims.L, (int)X->ld, p.rt, p.rt, 0};
                 gg.p[k] = GemmProblem{p.BW, p.BW, p.G, nullptr, p.rt, p.rt, p.rt > 0 ? d : 0, p.rt, p.rt, p.np, 0};
-                jb.s[k] = j3::Seq{p.G, p.Wt, p.Vbuf, p.vflag, p.jsync, p.rt, p.np, p.np / j3::JB, 0, 0};
+                jb.s[k] = j3::Seq{p.G, p.Wt, p.Vbuf, p.vflag, p.jdone, p.jsync, p.rt, p.np, p.np / j3::JB, 0, 0};
                 fb.s[k] = Fin2Seq{p.G, p.Wt, p.Y, p.sig, p.ord, p.tsum, p.Wsel, p.needfix,
                                   (T *)X_r->data + (size_t)p.dims.rank0 * X_r->ld, (T *)U_r->data + (size_t)p.dims.row0 * U_r->ld,
-                                  sigma ? sigma + p.dims.rank0 : nullptr, p.rt, p.dims.r, d, p.dims.L, p.rt, (int)X_r->ld, (int)U_r->ld, p.np};
-                maxrt = std::max(maxrt, p.rt); maxr = std::max(maxr, p.dims.r);
+                                  sigma ? sigma + p.dims.rank0 : nullptr, p.rt, p.dims.r, d, p.dims.L, kBf16 ? ldr : p.rt, (int)X_r->ld, (int)U_r->ld, p.np,
+                                  nullptr, nullptr, kBf16 ? p.Wsh : nullptr, kBf16 ? p.Wsl : nullptr, ldw, p.tpart};
+                maxrt = std::max(maxrt, p.rt); maxr = std::max(maxr, p.dims.r); maxL = std::max(maxL, p.dims.L);
             }
             if (maxrt == 0) continue;
-            if constexpr (std::is_same<T, __nv_bfloat16>::value) {
-                std::vector<tc::HostProblem> hp;
-                for (size_t i = i0; i < i1; ++i) {      // Bt = X^T (Yb + Yl)
+            // bf16 inputs: every product around the rotation runs on the tensor cores with both operands cut
+            // into bf16 hi/lo pairs (three MMA products, about 16 mantissa bits per operand); the projected
+            // rows Bt, the rotated Bt2 / Y2 and the selected rotation Wsel only ever exist as such pairs.
+            // fp32 inputs: the same products on the fp32 units.
+            std::vector<tc::HostProblem> hp;
+            if constexpr (kBf16) {
+                for (size_t i = i0; i < i1; ++i) {      // Bt = X^T (Yb + Yl), d x r~, kept as hi/lo
                     SeqPlan &p = bp.seqs[i];
                     int ldb = (int)align_up((size_t)p.rt, 8);
-                    hp.push_back(tc::HostProblem{Xb(p), p.Yb, p.Yl, p.BW, nullptr, nullptr, d, p.rt, p.dims.L, (int)X->ld, ldb, p.rt, 0});
+                    hp.push_back(tc::HostProblem{Xb(p), p.Yb, p.Yl, p.Bth, p.Btl, nullptr, d, p.rt, p.dims.L, (int)X->ld, ldb, ldb, 0});
                 }
-                if ((st = tc::launch<true, true, tc::OUT_F32>(ctx, hp, store)) != ATP_OK) return st;
+                if ((st = tc::launch<true, true, tc::OUT_BF16_SPLIT>(ctx, hp, store)) != ATP_OK) return st;
             } else {
                 if ((st = launch_gemm_simt<T, float, float, true>(ctx, g, store)) != ATP_OK) return st;
             }
@@ -1139,7 +1188,20 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
             // Each pass is one persistent kernel that stops on its own convergence test: nothing is
             // read back by the host.
             for (int pass = 0; pass < 2; ++pass) {
-                if ((st = launch_gemm_simt<float, float, float, true, false>(ctx, gg, store, 1, nullptr, 0, "gemm_simt_gram")) != ATP_OK) return st;
+                if constexpr (kBf16) {
+                    hp.clear();
+                    for (size_t i = i0; i < i1; ++i) {  // G = Bt^T Bt
+                        SeqPlan &p = bp.seqs[i];
+                        int ldb = (int)align_up((size_t)p.rt, 8);
+                        const __nv_bfloat16 *bh = pass == 0 ? p.Bth : p.Zb, *bl = pass == 0 ? p.Btl : p.Zl;
+                        tc::HostProblem h{bh, bh, bl, p.G, nullptr, nullptr, p.rt, p.rt, d, ldb, ldb, p.np, 0};
+                        h.A2 = bl;
+                        hp.push_back(h);
+                    }
+                    if ((st = tc::launch<true, true, tc::OUT_F32, false, true>(ctx, hp, store, "gemm_tc_gram")) != ATP_OK) return st;
+                } else {
+                    if ((st = launch_gemm_simt<float, float, float, true, false>(ctx, gg, store, 1, nullptr, 0, "gemm_simt_gram")) != ATP_OK) return st;
+                }
                 // pass 0 only has to make the rows graded and roughly orthogonal (scaled off-diagonals below
                 // 1e-2; on ill-conditioned input it stalls at the noise floor of G, hence the cap of 8 sweeps);
                 // the second pass continues the same iteration on the rotated data with the rest of the budget
@@ -1147,43 +1209,88 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
                 const int nsw = pass == 0 ? nsw0 : std::max(1, max_sweeps - nsw0);
                 const float tolc = pass == 0 ? fmaxf(tol_conv, 1e-2f) : tol_conv;
                 // fp32 inputs: the block products stay on the fp32 units (the threshold is below split-precision rounding)
-                if ((st = j3::launch<std::is_same<T, __nv_bfloat16>::value>(ctx, jb, tolc, tolc * 0.25f, nsw, pass == 1)) != ATP_OK) return st;
+                if ((st = j3::launch<kBf16>(ctx, jb, tolc, tolc * 0.25f, nsw, pass == 1)) != ATP_OK) return st;
                 if (pass == 0) {
-                    GemmBatch r1, r2; r1.count = r2.count = cnt;
-                    for (size_t i = i0; i < i1; ++i) {
-                        SeqPlan &p = bp.seqs[i];
-                        int k = (int)(i - i0);
-                        // Bt2 = Bt Wt^T (d x r~),  Y2 = Y Wt^T (L x r~);  Wt rows are the eigenvectors
-                        r1.p[k] = GemmProblem{p.BW, p.Wt, p.Z, nullptr, p.rt > 0 ? d : 0, p.rt, p.rt, p.rt, p.np, p.rt, 0};
-                        r2.p[k] = GemmProblem{p.Y, p.Wt, p.Y2, nullptr, p.dims.L, p.rt, p.rt, p.rt, p.np, p.rt, 0};
-                        gg.p[k].A = p.Z; gg.p[k].B = p.Z;
-                        fb.s[k].Y = p.Y2;
+                    // Bt2 = Bt Wt^T (d x r~),  Y2 = Y Wt^T (L x r~);  Wt rows are the eigenvectors
+                    if constexpr (kBf16) {
+                        SplitBatch sb; sb.count = cnt;
+                        double bytes = 0; int maxel = 0;
+                        for (size_t i = i0; i < i1; ++i) {
+                            SeqPlan &p = bp.seqs[i];
+                            sb.s[i - i0] = SplitSeq{p.Wt, p.Wth, p.Wtl, p.np, p.np, p.rt, p.rt};
+                            bytes += (double)p.rt * p.rt * 8; maxel = std::max(maxel, p.rt * p.rt);
+                        }
+                        ATP_KERNEL(ctx, "f32_to_bf16", 0, bytes);
+                        launch_pdl(split_bf16_batch_kernel, dim3(std::min(256, ceil_div(maxel, 1024)), sb.count), dim3(256), 0, ctx->stream, sb);
+                        ATP_LAUNCHED(ctx);
+                        std::vector<tc::HostProblem> h1, h2;
+                        for (size_t i = i0; i < i1; ++i) {
+                            SeqPlan &p = bp.seqs[i];
+                            int ldb = (int)align_up((size_t)p.rt, 8);
+                            tc::HostProblem a{p.Bth, p.Wth, p.Wtl, p.Zb, p.Zl, nullptr, d, p.rt, p.rt, ldb, p.np, ldb, 0};
+                            a.A2 = p.Btl;
+                            h1.push_back(a);
+                            tc::HostProblem c{p.Yb, p.Wth, p.Wtl, p.Y2h, p.Y2l, nullptr, p.dims.L, p.rt, p.rt, ldb, p.np, ldb, 0};
+                            c.A2 = p.Yl;
+                            h2.push_back(c);
+                            fb.s[i - i0].Yh = p.Y2h; fb.s[i - i0].Yl = p.Y2l;
+                        }
+                        if ((st = tc::launch<false, true, tc::OUT_BF16_SPLIT, true, true>(ctx, h1, store, "gemm_tc_rot")) != ATP_OK) return st;
+                        if ((st = tc::launch<false, true, tc::OUT_BF16_SPLIT, true, true>(ctx, h2, store, "gemm_tc_rot")) != ATP_OK) return st;
+                    } else {
+                        GemmBatch r1, r2; r1.count = r2.count = cnt;
+                        for (size_t i = i0; i < i1; ++i) {
+                            SeqPlan &p = bp.seqs[i];
+                            int k = (int)(i - i0);
+                            r1.p[k] = GemmProblem{p.BW, p.Wt, p.Z, nullptr, p.rt > 0 ? d : 0, p.rt, p.rt, p.rt, p.np, p.rt, 0};
+                            r2.p[k] = GemmProblem{p.Y, p.Wt, p.Y2, nullptr, p.dims.L, p.rt, p.rt, p.rt, p.np, p.rt, 0};
+                            gg.p[k].A = p.Z; gg.p[k].B = p.Z;
+                            fb.s[k].Y = p.Y2;
+                        }
+                        if ((st = launch_gemm_simt<float, float, float, false, true>(ctx, r1, store, 1, nullptr, 0, "gemm_simt_rot")) != ATP_OK) return st;
+                        if ((st = launch_gemm_simt<float, float, float, false, true>(ctx, r2, store, 1, nullptr, 0, "gemm_simt_rot")) != ATP_OK) return st;
                     }
-                    if ((st = launch_gemm_simt<float, float, float, false, true>(ctx, r1, store, 1, nullptr, 0, "gemm_simt_rot")) != ATP_OK) return st;
-                    if ((st = launch_gemm_simt<float, float, float, false, true>(ctx, r2, store, 1, nullptr, 0, "gemm_simt_rot")) != ATP_OK) return st;
                 }
             }
             int npow = 1; while (npow < maxrt) npow <<= 1;
+            ATP_KERNEL(ctx, "colsum", 0, 0);
+            colsum2_kernel<<<dim3(ceil_div(maxrt, 32), COLSUM_SLABS, cnt), 256, 0, ctx->stream>>>(fb);
+            ATP_LAUNCHED(ctx);
             ATP_KERNEL(ctx, "sigma_sort", 0, 0);
             sigma_sort2_kernel<<<cnt, 1024, (size_t)npow * 8, ctx->stream>>>(fb);
-            ATP_LAUNCHED(ctx);
-            ATP_KERNEL(ctx, "colsum", 0, 0);
-            colsum2_kernel<<<dim3(ceil_div(maxrt, 128), cnt), 128, 0, ctx->stream>>>(fb);
             ATP_LAUNCHED(ctx);
             ATP_KERNEL(ctx, "select", 0, 0);
             select2_kernel<<<dim3(maxr, cnt), 128, 0, ctx->stream>>>(fb);
             ATP_LAUNCHED(ctx);
-            for (size_t i = i0; i < i1; ++i) {
-                SeqPlan &p = bp.seqs[i];
-                int k = (int)(i - i0);
-                // X_r = Wsel^T Bt2^T  and  U_r = Y2 Wsel  (Bt2, Y2: rotated by the first pass)
-                g.p[k] = GemmProblem{p.Wsel, p.Z, (T *)X_r->data + (size_t)p.dims.rank0 * X_r->ld, nullptr,
-                                     p.dims.r, p.rt > 0 ? d : 0, p.rt, p.dims.r, p.rt, (int)X_r->ld, 0};
-                gg.p[k] = GemmProblem{p.Y2, p.Wsel, (T *)U_r->data + (size_t)p.dims.row0 * U_r->ld, nullptr,
-                                      p.dims.L, p.dims.r, p.rt, p.rt, p.dims.r, (int)U_r->ld, 0};
+            // X_r = Wsel^T Bt2^T  and  U_r = Y2 Wsel  (Bt2, Y2: rotated by the first pass)
+            if constexpr (kBf16) {
+                std::vector<tc::HostProblem> h1, h2;
+                for (size_t i = i0; i < i1; ++i) {
+                    SeqPlan &p = bp.seqs[i];
+                    int ldb = (int)align_up((size_t)p.rt, 8), ldw = (int)align_up((size_t)std::max(p.dims.r, 1), 8);
+                    tc::HostProblem a{p.Wsh, p.Zb, p.Zl, (T *)X_r->data + (size_t)p.dims.rank0 * X_r->ld, nullptr, nullptr,
+                                      p.dims.r, d, p.rt, ldw, ldb, (int)X_r->ld, 0};
+                    a.A2 = p.Wsl;
+                    h1.push_back(a);
+                    tc::HostProblem c{p.Y2h, p.Wsh, p.Wsl, (T *)U_r->data + (size_t)p.dims.row0 * U_r->ld, nullptr, nullptr,
+                                      p.dims.L, p.dims.r, p.rt, ldb, ldw, (int)U_r->ld, 0};
+                    c.A2 = p.Y2l;
+                    h2.push_back(c);
+                }
+                if ((st = tc::launch<true, true, tc::OUT_BF16, true, true>(ctx, h1, store, "gemm_tc_out")) != ATP_OK) return st;
+                if ((st = tc::launch<false, true, tc::OUT_BF16, false, true>(ctx, h2, store, "gemm_tc_out")) != ATP_OK) return st;
+            } else {
+                for (size_t i = i0; i < i1; ++i) {
+                    SeqPlan &p = bp.seqs[i];
+                    int k = (int)(i - i0);
+                    g.p[k] = GemmProblem{p.Wsel, p.Z, (T *)X_r->data + (size_t)p.dims.rank0 * X_r->ld, nullptr,
+                                         p.dims.r, p.rt > 0 ? d : 0, p.rt, p.dims.r, p.rt, (int)X_r->ld, 0};
+                    gg.p[k] = GemmProblem{p.Y2, p.Wsel, (T *)U_r->data + (size_t)p.dims.row0 * U_r->ld, nullptr,
+                                          p.dims.L, p.dims.r, p.rt, p.rt, p.dims.r, (int)U_r->ld, 0};
+                }
+                if ((st = launch_gemm_simt<float, float, T, true, true>(ctx, g, store, 1, nullptr, 0, "gemm_simt_out")) != ATP_OK) return st;
+                if ((st = launch_gemm_simt<float, float, T, false>(ctx, gg, store, 1, nullptr, 0, "gemm_simt_out")) != ATP_OK) return st;
             }
-            if ((st = launch_gemm_simt<float, float, T, true, true>(ctx, g, store, 1, nullptr, 0, "gemm_simt_out")) != ATP_OK) return st;
-            if ((st = launch_gemm_simt<float, float, T, false>(ctx, gg, store, 1, nullptr, 0, "gemm_simt_out")) != ATP_OK) return st;
             ATP_KERNEL(ctx, "signfix", 0, 0);
             signfix_kernel<T><<<dim3(maxr, cnt), 256, 0, ctx->stream>>>(fb);
             ATP_LAUNCHED(ctx);

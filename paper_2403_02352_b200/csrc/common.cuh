@@ -5,6 +5,7 @@
 #include <stdint.h>
 #include <stddef.h>
 #include <vector>
+#include <mutex>
 #include "atp.h"
 
 // One record per kernel launch while profiling is on (see atp_profile_start).
@@ -81,6 +82,22 @@ static inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 blo
     cfg.attrs = at; cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
 }
+
+// Runs a per-device set-up step (a kernel attribute, an address look-up) once for every device
+// ordinal, whichever context or thread comes first; a failed step is retried by the next caller.
+struct PerDeviceOnce {
+    static constexpr int MAX_DEV = 64;
+    std::mutex mu;
+    bool done[MAX_DEV] = {};
+    template <typename F> cudaError_t run(int device, F step)
+    {
+        std::lock_guard<std::mutex> lk(mu);
+        if (device >= 0 && device < MAX_DEV && done[device]) return cudaSuccess;
+        const cudaError_t e = step();
+        if (e == cudaSuccess && device >= 0 && device < MAX_DEV) done[device] = true;
+        return e;
+    }
+};
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }

@@ -1,8 +1,10 @@
 // Batched bf16 GEMM on the 5th-generation tensor cores (tcgen05.mma, accumulator in TMEM, operands
 // staged in shared memory by TMA with the 128-byte swizzle): C = epilogue(op(A) * B).
 //   A: M x K row-major (K-major operand) or K x M row-major (M-major operand), bf16
-//   B: K x N row-major (N-major operand), bf16; optionally a second matrix B_lo of the same shape
-//      whose product is accumulated on top (split precision: B = B_hi + B_lo)
+//   B: K x N row-major (N-major operand) or N x K row-major (K-major operand), bf16; optionally a
+//      second matrix B_lo of the same shape whose product is accumulated on top (split precision:
+//      B = B_hi + B_lo), and a second matrix A_lo as well: A_hi B_hi + A_hi B_lo + A_lo B_hi carries
+//      about 16 mantissa bits of both operands, for fp32 data cut into bf16 hi/lo pairs
 //   C: M x N row-major, fp32 or bf16, or a bf16 hi/lo pair; D (optional): M x N fp32
 // One CTA computes one 128 x 128 tile: warp 4 issues the TMA loads, warp 5 allocates TMEM and issues
 // the MMAs, warps 0-3 read the accumulator back (tcgen05.ld) and run the epilogue. Extents come
@@ -20,7 +22,7 @@ constexpr int MAX_PROB = 16;
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 
 struct Problem {
-    CUtensorMap ta, tb, tb2;     // tb2 only with a split B
+    CUtensorMap ta, ta2, tb, tb2; // ta2 / tb2 only with a split A / B
     void *C; void *C2; const float *D;
     int M, N, K, ldc, ldd;
     int tile0, tiles_n;          // first linear tile index of this problem, tiles along N
@@ -141,19 +143,21 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool a_mn_major,
            ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
-template <bool SPLIT_B> struct Cfg {
-    static constexpr int STAGES = SPLIT_B ? 4 : 3;
+template <bool SPLIT_B, bool SPLIT_A = false> struct Cfg {
+    static constexpr int STAGES = SPLIT_A ? 3 : (SPLIT_B ? 4 : 3);
     static constexpr int A_BYTES = BM * BK * 2;                 // 16 KB
     static constexpr int B_BYTES = BK * BN * 2;                 // 16 KB
-    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES * (SPLIT_B ? 2 : 1);
+    static constexpr int B_OFF = A_BYTES * (SPLIT_A ? 2 : 1);
+    static constexpr int STAGE_BYTES = B_OFF + B_BYTES * (SPLIT_B ? 2 : 1);
     static constexpr int SMEM = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
-template <bool A_MN, bool SPLIT_B, int OUT>
+template <bool A_MN, bool SPLIT_B, int OUT, bool B_KMAJ = false, bool SPLIT_A = false>
 __global__ void __launch_bounds__(192)
 gemm_tc_kernel(const __grid_constant__ Batch batch, GemmEpi epi, int *dev_status)
 {
-    using C_ = Cfg<SPLIT_B>;
+    using C_ = Cfg<SPLIT_B, SPLIT_A>;
+    static_assert(!SPLIT_A || SPLIT_B, "a split A comes with a split B");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;                // swizzled tiles need 1024-byte alignment
@@ -191,42 +195,52 @@ gemm_tc_kernel(const __grid_constant__ Batch batch, GemmEpi epi, int *dev_status
                 const int s = kt % C_::STAGES;
                 if (kt >= C_::STAGES && !mbar_wait(bars + 8 * (C_::STAGES + s), ((kt / C_::STAGES) - 1) & 1, &abort_flag)) break;
                 const uint32_t full = bars + 8 * s;
-                const uint32_t sa = base + s * C_::STAGE_BYTES, sb = sa + C_::A_BYTES;
+                const uint32_t sa = base + s * C_::STAGE_BYTES, sb = sa + C_::B_OFF;
                 mbar_expect_tx(full, C_::STAGE_BYTES);
                 const int k0 = kt * BK;
                 if (!A_MN) {
                     tma_load_2d(sa, &pr.ta, k0, m0, full);                       // box {64 k, 128 m}
+                    if (SPLIT_A) tma_load_2d(sa + C_::A_BYTES, &pr.ta2, k0, m0, full);
                 } else {
                     tma_load_2d(sa, &pr.ta, m0, k0, full);                       // box {64 m, 64 k} x 2
                     tma_load_2d(sa + 8192, &pr.ta, m0 + 64, k0, full);
+                    if (SPLIT_A) {
+                        tma_load_2d(sa + C_::A_BYTES, &pr.ta2, m0, k0, full);
+                        tma_load_2d(sa + C_::A_BYTES + 8192, &pr.ta2, m0 + 64, k0, full);
+                    }
                 }
-                tma_load_2d(sb, &pr.tb, n0, k0, full);                           // box {64 n, 64 k} x 2
-                tma_load_2d(sb + 8192, &pr.tb, n0 + 64, k0, full);
-                if (SPLIT_B) {
-                    tma_load_2d(sb + C_::B_BYTES, &pr.tb2, n0, k0, full);
-                    tma_load_2d(sb + C_::B_BYTES + 8192, &pr.tb2, n0 + 64, k0, full);
+                if (B_KMAJ) {
+                    tma_load_2d(sb, &pr.tb, k0, n0, full);                       // box {64 k, 128 n}
+                    if (SPLIT_B) tma_load_2d(sb + C_::B_BYTES, &pr.tb2, k0, n0, full);
+                } else {
+                    tma_load_2d(sb, &pr.tb, n0, k0, full);                       // box {64 n, 64 k} x 2
+                    tma_load_2d(sb + 8192, &pr.tb, n0 + 64, k0, full);
+                    if (SPLIT_B) {
+                        tma_load_2d(sb + C_::B_BYTES, &pr.tb2, n0, k0, full);
+                        tma_load_2d(sb + C_::B_BYTES + 8192, &pr.tb2, n0 + 64, k0, full);
+                    }
                 }
             }
         }
     } else if (warp == 5) {
         if (lane == 0) {
-            constexpr uint32_t idesc = instr_desc(BM, BN, A_MN, true);
+            constexpr uint32_t idesc = instr_desc(BM, BN, A_MN, !B_KMAJ);
             bool ok = true;
             for (int kt = 0; kt < num_kt && ok; ++kt) {
                 const int s = kt % C_::STAGES;
                 ok = mbar_wait(bars + 8 * s, (kt / C_::STAGES) & 1, &abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t sa = base + s * C_::STAGE_BYTES, sb = sa + C_::A_BYTES;
+                const uint32_t sa = base + s * C_::STAGE_BYTES, sb = sa + C_::B_OFF;
 #pragma unroll
                 for (int kk = 0; kk < BK / 16; ++kk) {
-                    const uint64_t ad = A_MN ? smem_desc(sa + kk * 2048, 8192, 1024) : smem_desc(sa + kk * 32, 16, 1024);
-                    const uint64_t bd = smem_desc(sb + kk * 2048, 8192, 1024);
-                    umma_bf16(tmem_base, ad, bd, idesc, (kt > 0 || kk > 0) ? 1u : 0u);
-                    if (SPLIT_B) {
-                        const uint64_t bd2 = smem_desc(sb + C_::B_BYTES + kk * 2048, 8192, 1024);
-                        umma_bf16(tmem_base, ad, bd2, idesc, 1u);
-                    }
+                    auto adesc = [&](uint32_t a0) { return A_MN ? smem_desc(a0 + kk * 2048, 8192, 1024) : smem_desc(a0 + kk * 32, 16, 1024); };
+                    auto bdesc = [&](uint32_t b0) { return B_KMAJ ? smem_desc(b0 + kk * 32, 16, 1024) : smem_desc(b0 + kk * 2048, 8192, 1024); };
+                    const uint64_t ad = adesc(sa), bd = bdesc(sb);
+                    // small terms first, the hi * hi product last
+                    if (SPLIT_A) umma_bf16(tmem_base, adesc(sa + C_::A_BYTES), bd, idesc, (kt > 0 || kk > 0) ? 1u : 0u);
+                    if (SPLIT_B) umma_bf16(tmem_base, ad, bdesc(sb + C_::B_BYTES), idesc, (SPLIT_A || kt > 0 || kk > 0) ? 1u : 0u);
+                    umma_bf16(tmem_base, ad, bd, idesc, (SPLIT_B || kt > 0 || kk > 0) ? 1u : 0u);
                 }
                 umma_commit(bars + 8 * (C_::STAGES + s));        // frees the stage once these MMAs have read it
             }
@@ -342,6 +356,7 @@ static inline bool make_map(CUtensorMap *m, const void *ptr, uint64_t rows, uint
 struct HostProblem {
     const void *A; const void *B; const void *B2; void *C; void *C2; const float *D;
     int M, N, K, lda, ldb, ldc, ldd;
+    const void *A2 = nullptr;     // low part of a split A
 };
 
 static inline bool operands_ok(const HostProblem &h)
@@ -350,15 +365,14 @@ static inline bool operands_ok(const HostProblem &h)
     return al(h.A) && al(h.B) && (!h.B2 || al(h.B2)) && (h.lda % 8 == 0) && (h.ldb % 8 == 0) && h.M > 0 && h.N > 0 && h.K > 0;
 }
 
-template <bool A_MN, bool SPLIT_B, int OUT>
-static atp_status launch(atp_ctx *ctx, const std::vector<HostProblem> &probs, GemmEpi epi)
+template <bool A_MN, bool SPLIT_B, int OUT, bool B_KMAJ = false, bool SPLIT_A = false>
+static atp_status launch(atp_ctx *ctx, const std::vector<HostProblem> &probs, GemmEpi epi, const char *tag = nullptr)
 {
-    using C_ = Cfg<SPLIT_B>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        ATP_CUDA_OK(ctx, cudaFuncSetAttribute(gemm_tc_kernel<A_MN, SPLIT_B, OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::SMEM));
-        attr_set = true;
-    }
+    using C_ = Cfg<SPLIT_B, SPLIT_A>;
+    static PerDeviceOnce attr_once;        // the shared-memory opt-in is a per-device attribute
+    ATP_CUDA_OK(ctx, attr_once.run(ctx->device, [] {
+        return cudaFuncSetAttribute(gemm_tc_kernel<A_MN, SPLIT_B, OUT, B_KMAJ, SPLIT_A>, cudaFuncAttributeMaxDynamicSharedMemorySize, C_::SMEM);
+    }));
     size_t i = 0;
     while (i < probs.size()) {
         Batch b; b.count = 0; b.total_tiles = 0;
@@ -368,20 +382,22 @@ static atp_status launch(atp_ctx *ctx, const std::vector<HostProblem> &probs, Ge
             if (h.M <= 0 || h.N <= 0 || h.K <= 0) continue;
             Problem &p = b.p[b.count];
             bool ok = A_MN ? make_map(&p.ta, h.A, h.K, h.M, h.lda, 64) : make_map(&p.ta, h.A, h.M, h.K, h.lda, BM);
-            ok = ok && make_map(&p.tb, h.B, h.K, h.N, h.ldb, 64);
-            if (SPLIT_B) ok = ok && make_map(&p.tb2, h.B2, h.K, h.N, h.ldb, 64);
+            if (SPLIT_A) ok = ok && h.A2 && (A_MN ? make_map(&p.ta2, h.A2, h.K, h.M, h.lda, 64) : make_map(&p.ta2, h.A2, h.M, h.K, h.lda, BM));
+            auto bmap = [&](CUtensorMap *m, const void *ptr) { return B_KMAJ ? make_map(m, ptr, h.N, h.K, h.ldb, BN) : make_map(m, ptr, h.K, h.N, h.ldb, 64); };
+            ok = ok && bmap(&p.tb, h.B);
+            if (SPLIT_B) ok = ok && h.B2 && bmap(&p.tb2, h.B2);
             if (!ok) return ATP_ERR_INVALID_ARG;
             p.C = h.C; p.C2 = h.C2; p.D = h.D; p.M = h.M; p.N = h.N; p.K = h.K; p.ldc = h.ldc; p.ldd = h.ldd;
             p.tiles_n = ceil_div(h.N, BN);
             p.tile0 = b.total_tiles;
             b.total_tiles += ceil_div(h.M, BM) * p.tiles_n;
             b.count++;
-            flops += 2.0 * h.M * h.N * h.K * (SPLIT_B ? 2 : 1);
+            flops += 2.0 * h.M * h.N * h.K * (SPLIT_A ? 3 : (SPLIT_B ? 2 : 1));
             bytes += 2.0 * ((double)h.M * h.K + (double)h.K * h.N * (SPLIT_B ? 2 : 1)) + (double)h.M * h.N * (OUT == OUT_F32 ? 4 : (OUT == OUT_BF16 ? 2 : 4));
         }
         if (b.count == 0) continue;
-        ATP_KERNEL(ctx, SPLIT_B ? "gemm_tc_split" : "gemm_tc", flops, bytes);
-        gemm_tc_kernel<A_MN, SPLIT_B, OUT><<<b.total_tiles, 192, C_::SMEM, ctx->stream>>>(b, epi, ctx->dev_status);
+        ATP_KERNEL(ctx, tag ? tag : (SPLIT_A ? "gemm_tc_split3" : (SPLIT_B ? "gemm_tc_split" : "gemm_tc")), flops, bytes);
+        gemm_tc_kernel<A_MN, SPLIT_B, OUT, B_KMAJ, SPLIT_A><<<b.total_tiles, 192, C_::SMEM, ctx->stream>>>(b, epi, ctx->dev_status);
         ATP_LAUNCHED(ctx);
     }
     return ATP_OK;

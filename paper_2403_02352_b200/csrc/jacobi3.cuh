@@ -34,11 +34,12 @@ constexpr int MAXSEQ = 32;        // sequences per launch
 constexpr unsigned SPIN_LIMIT = 1u << 22;
 
 struct Seq {
-    float *G, *Wt, *Vbuf;         // G, Wt: np x np (ld = np); Vbuf: npairs x 64 x 64
-    int *vflag;                   // npairs: the pair rotated in this step
+    float *G, *Wt, *Vbuf;         // G, Wt: np x np (ld = np); Vbuf: 2 x npairs x 64 x 64 (by step parity)
+    int *vflag;                   // 2 x npairs: the pair rotated in this step
+    unsigned *done;               // per block (p, q >= p) of G: number of the last step that updated it
     unsigned *sync;               // 64 words. [0]: arrivals at the group barrier (monotonic); [32]: last
-                                  // barrier completed; [1..3]: largest scaled off-diagonal entry of a
-                                  // sweep, slot sweep % 3; [4]: sweeps used
+                                  // barrier completed; [1..4]: largest scaled off-diagonal entry of a
+                                  // sweep, slot sweep % 4; [5]: sweeps used; [16..17]: work tickets of the update, by step parity
     int n, np, nb;                // size, padded size (multiple of 64), number of 32-row blocks (even)
     int cta0, ncta;               // the group of CTAs that owns this sequence
 };
@@ -343,7 +344,7 @@ __device__ __forceinline__ void product64_fma(const float *As, const float *Bs, 
 // One block of the update. Items [0, ntri): block (p, q >= p) of G, enumerated row by row; items
 // [ntri, ntri + npairs * nw): rows of pair p of Wt, column chunk of 64.
 template <bool TENSOR>
-__device__ void apply_item(float *sm, const Seq &sq, int step, int idx, int npairs, int ntri, int nw)
+__device__ void apply_item(float *sm, const Seq &sq, const float *Vbuf, const int *vflag, int step, int idx, int npairs, int ntri, int nw)
 {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     const bool gblock = idx < ntri;
@@ -355,8 +356,8 @@ __device__ void apply_item(float *sm, const Seq &sq, int step, int idx, int npai
         idx -= ntri;
         p = idx / nw; chunk = idx - p * nw;
     }
-    const int fp = __ldcg(sq.vflag + p);
-    const int fq = gblock ? __ldcg(sq.vflag + q) : 0;
+    const int fp = __ldcg(vflag + p);
+    const int fq = gblock ? __ldcg(vflag + q) : 0;
     if (!fp && !fq) return;
     float *Vp = sm, *Vq = sm + BLK * LDA, *Tm = sm + 2 * BLK * LDA, *Bk = sm + 3 * BLK * LDA;
     int Ip, Jp, Iq = 0, Jq = 0;
@@ -370,8 +371,8 @@ __device__ void apply_item(float *sm, const Seq &sq, int step, int idx, int npai
     const int blk_ld = fp ? LDB : LDA;
     for (int f = tid; f < BLK * (BLK / 4); f += NT) {
         const int i = f >> 4, c = (f & 15) * 4;
-        if (fp) *(float4 *)(Vp + i * LDA + c) = __ldcg((const float4 *)(sq.Vbuf + (size_t)p * BLK * BLK + i * BLK + c));
-        if (fq) *(float4 *)(Vq + i * LDA + c) = __ldcg((const float4 *)(sq.Vbuf + (size_t)q * BLK * BLK + i * BLK + c));
+        if (fp) *(float4 *)(Vp + i * LDA + c) = __ldcg((const float4 *)(Vbuf + (size_t)p * BLK * BLK + i * BLK + c));
+        if (fq) *(float4 *)(Vq + i * LDA + c) = __ldcg((const float4 *)(Vbuf + (size_t)q * BLK * BLK + i * BLK + c));
         *(float4 *)(blk_dst + i * blk_ld + c) = __ldcg((const float4 *)(mat + (size_t)glob_of_loc(Ip, Jp, i) * np + gcol(c)));
     }
     __syncthreads();
@@ -409,56 +410,153 @@ __device__ void apply_item(float *sm, const Seq &sq, int step, int idx, int npai
 }
 
 // ---- the kernel --------------------------------------------------------------------------------
+// Schedule of a group. The pivot blocks of step s+1 lie inside 3 blocks of the update of step s (the
+// two diagonal blocks of the pairs their rows come from, and the block that couples those pairs).
+// Every step therefore runs
+//   1. the "critical" blocks of its update first (all diagonal blocks and the coupling blocks of the
+//      next step's pairs), spread over the whole group, each marking itself done;
+//   2. then, side by side, the pivot solves of the NEXT step (each waits for its 3 blocks) and the
+//      rest of the update, handed out by a ticket counter so that the pivot CTAs join in when they
+//      are through;
+//   3. one group barrier.
+// Vt and the rotated-flags are double buffered by step parity, because step s+1's pivots publish while
+// step s's update still reads.
 // status[0]: sticky device status word of the context; status[1]: abort flag of bounded waits.
+constexpr int MAXPAIRS = 72;                  // np <= 4608
+__device__ __forceinline__ int tri_index(int p, int q, int npairs) { return p * npairs - p * (p - 1) / 2 + (q - p); }
+
 template <bool TENSOR>
 __global__ void __launch_bounds__(NT, 2)
 jacobi_persistent_kernel(const __grid_constant__ Batch batch, float tol_conv, float tol_rot, int max_sweeps,
                          int raise_not_converged, int *status)
 {
     extern __shared__ __align__(16) float j3sm[];
+    __shared__ short pair_of[2 * MAXPAIRS];
+    __shared__ unsigned char is_crit[MAXPAIRS * (MAXPAIRS + 1) / 2];
+    __shared__ short crit_list[2 * MAXPAIRS];
+    __shared__ int ncrit_s, ticket_s, wait_ok_s;
     int si = 0;
 #pragma unroll 1
     for (int i = 1; i < batch.count; ++i) if ((int)blockIdx.x >= batch.s[i].cta0) si = i;
     const Seq &sq = batch.s[si];
-    const int rank = (int)blockIdx.x - sq.cta0;
+    const int rank = (int)blockIdx.x - sq.cta0, tid = threadIdx.x;
     if (rank >= sq.ncta || sq.np <= 0) return;
-    const int npairs = sq.nb / 2, nw = sq.np / BLK, ntri = npairs * (npairs + 1) / 2;
+    const int npairs = sq.nb / 2, nw = sq.np / BLK, ntri = npairs * (npairs + 1) / 2, total = ntri + npairs * nw;
     const int nsteps = sq.nb - 1;
     int *abort_flag = status + 1;
-    unsigned gen = 0;
+    unsigned gen = 0, gstep = 0;
     bool converged = false, alive = true;
+
+    auto pivot_item = [&](int sweep, int step, int pr, int par) {
+        int I, J;
+        rr_pair(sq.nb, step, pr, I, J);
+        bool rotated;
+        const float mo = pivot_solve(j3sm, sq.G, sq.np, I, J, step > 0, tol_rot,
+                                     sq.Vbuf + ((size_t)par * npairs + pr) * BLK * BLK, rotated);
+        if (tid == 0) {
+            sq.vflag[par * npairs + pr] = rotated ? 1 : 0;
+            atomicMax(sq.sync + 1 + sweep % 4, __float_as_uint(mo));
+        }
+        __syncthreads();
+    };
+
+    // prologue: the pivots of the very first step
+    for (int pr = rank; pr < npairs; pr += sq.ncta) pivot_item(0, 0, pr, 0);
+    alive = group_barrier(sq.sync, ++gen, (unsigned)sq.ncta, abort_flag);
+
     int sweep = 0;
     for (; sweep < max_sweeps && alive; ++sweep) {
-        if (rank == 0 && threadIdx.x == 0) sq.sync[1 + (sweep + 1) % 3] = 0u;
-        for (int step = 0; step < nsteps && alive; ++step) {
-            for (int pr = rank; pr < npairs; pr += sq.ncta) {
+        if (rank == 0 && tid == 0) sq.sync[1 + (sweep + 2) % 4] = 0u;      // slot of sweep + 2, last read two sweeps ago
+        for (int step = 0; step < nsteps && alive; ++step, ++gstep) {
+            const int par = (int)(gstep & 1u);
+            const bool has_next = !(sweep == max_sweeps - 1 && step == nsteps - 1);
+            const int nstep = step + 1 == nsteps ? 0 : step + 1, nsweep = sweep + (step + 1 == nsteps ? 1 : 0);
+            const float *Vcur = sq.Vbuf + (size_t)par * npairs * BLK * BLK;
+            const int *fcur = sq.vflag + par * npairs;
+            // tables of this step: block -> pair, critical blocks
+            if (tid < npairs) {
                 int I, J;
-                rr_pair(sq.nb, step, pr, I, J);
-                bool rotated;
-                const float mo = pivot_solve(j3sm, sq.G, sq.np, I, J, step > 0, tol_rot,
-                                             sq.Vbuf + (size_t)pr * BLK * BLK, rotated);
-                if (threadIdx.x == 0) {
-                    sq.vflag[pr] = rotated ? 1 : 0;
-                    atomicMax(sq.sync + 1 + sweep % 3, __float_as_uint(mo));
-                }
-                __syncthreads();
+                rr_pair(sq.nb, step, tid, I, J);
+                pair_of[I] = (short)tid; pair_of[J] = (short)tid;
             }
-            alive = group_barrier(sq.sync, ++gen, (unsigned)sq.ncta, abort_flag);
-            if (!alive) break;
-            for (int it = rank; it < ntri + npairs * nw; it += sq.ncta) apply_item<TENSOR>(j3sm, sq, step, it, npairs, ntri, nw);
-            alive = group_barrier(sq.sync, ++gen, (unsigned)sq.ncta, abort_flag);
+            for (int e = tid; e < ntri; e += NT) is_crit[e] = 0;
+            __syncthreads();
+            if (tid == 0) {
+                int nc = 0;
+                for (int p = 0; p < npairs; ++p) { const int idx = tri_index(p, p, npairs); is_crit[idx] = 1; crit_list[nc++] = (short)idx; }
+                if (has_next)
+                    for (int t = 0; t < npairs; ++t) {
+                        int I2, J2;
+                        rr_pair(sq.nb, nstep, t, I2, J2);
+                        const int p1 = pair_of[I2], p2 = pair_of[J2];
+                        if (p1 != p2) {
+                            const int idx = tri_index(min(p1, p2), max(p1, p2), npairs);
+                            if (!is_crit[idx]) { is_crit[idx] = 1; crit_list[nc++] = (short)idx; }
+                        }
+                    }
+                ncrit_s = nc;
+                if (rank == 0) sq.sync[16 + (par ^ 1)] = 0u;          // tickets of the next step
+            }
+            __syncthreads();
+            // 1. critical blocks
+            for (int k = rank; k < ncrit_s; k += sq.ncta) {
+                const int idx = crit_list[k];
+                apply_item<TENSOR>(j3sm, sq, Vcur, fcur, step, idx, npairs, ntri, nw);
+                if (tid == 0) { __threadfence(); *(volatile unsigned *)(sq.done + idx) = gstep + 1u; }
+            }
+            // 2a. pivots of the next step
+            if (has_next)
+                for (int pr = rank; pr < npairs && alive; pr += sq.ncta) {
+                    if (tid == 0) {
+                        int I2, J2;
+                        rr_pair(sq.nb, nstep, pr, I2, J2);
+                        const int p1 = pair_of[I2], p2 = pair_of[J2];
+                        const int dep[3] = {tri_index(p1, p1, npairs), tri_index(p2, p2, npairs),
+                                            tri_index(min(p1, p2), max(p1, p2), npairs)};
+                        int ok = 1;
+                        for (int k = 0; k < 3 && ok; ++k) {
+                            ok = 0;
+                            for (unsigned i = 0; i < SPIN_LIMIT; ++i) {
+                                if (*(volatile unsigned *)(sq.done + dep[k]) == gstep + 1u) { ok = 1; break; }
+                                if ((i & 1023u) == 1023u && *(volatile int *)abort_flag) break;
+                            }
+                        }
+                        if (!ok) *(volatile int *)abort_flag = 1;
+                        __threadfence();
+                        wait_ok_s = ok;
+                    }
+                    __syncthreads();
+                    if (!wait_ok_s) { alive = false; break; }
+                    pivot_item(nsweep, nstep, pr, par ^ 1);
+                }
+            // 2b. the rest of the update, by tickets (the next one is requested while a block is processed)
+            if (alive) {
+                if (tid == 0) ticket_s = (int)atomicAdd(sq.sync + 16 + par, 1u);
+                __syncthreads();
+                int t = ticket_s;
+                while (t < total) {
+                    int tn = 0;
+                    if (tid == 0) tn = (int)atomicAdd(sq.sync + 16 + par, 1u);
+                    if (!(t < ntri && is_crit[t])) apply_item<TENSOR>(j3sm, sq, Vcur, fcur, step, t, npairs, ntri, nw);
+                    __syncthreads();
+                    if (tid == 0) ticket_s = tn;
+                    __syncthreads();
+                    t = ticket_s;
+                }
+            }
+            // 3.
+            alive = group_barrier(sq.sync, ++gen, (unsigned)sq.ncta, abort_flag) && alive;
         }
         if (!alive) break;
-        const float mo = __uint_as_float(*(volatile unsigned *)(sq.sync + 1 + sweep % 3));
+        const float mo = __uint_as_float(*(volatile unsigned *)(sq.sync + 1 + sweep % 4));
         if (mo <= tol_conv) { converged = true; ++sweep; break; }
     }
-    if (rank == 0 && threadIdx.x == 0) {
+    if (rank == 0 && tid == 0) {
         if (!alive) raise_status(status, ATP_ERR_TIMEOUT);
         else if (!converged && raise_not_converged) raise_status(status, ATP_ERR_NOT_CONVERGED);
-        sq.sync[4] = (unsigned)sweep;
+        sq.sync[5] = (unsigned)sweep;
     }
 }
-
 
 // Wt = identity, padding of G = 0, synchronisation words = 0. grid (x, count).
 __global__ void init_kernel(const __grid_constant__ Batch batch)
@@ -470,7 +568,11 @@ __global__ void init_kernel(const __grid_constant__ Batch batch)
         sq.Wt[e] = (i == j) ? 1.f : 0.f;
         if (i >= sq.n || j >= sq.n) sq.G[e] = 0.f;
     }
-    if (blockIdx.x == 0 && threadIdx.x < 64 && sq.np > 0) sq.sync[threadIdx.x] = 0u;
+    if (blockIdx.x == 0 && sq.np > 0) {
+        if (threadIdx.x < 64) sq.sync[threadIdx.x] = 0u;
+        const int npairs = sq.nb / 2;
+        for (int e = threadIdx.x; e < npairs * (npairs + 1) / 2; e += blockDim.x) sq.done[e] = 0u;
+    }
 }
 
 // Host side: hands every sequence a group of CTAs in proportion to the size of its update (at most one

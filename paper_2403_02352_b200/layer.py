@@ -74,31 +74,45 @@ class AtpLayer:
         return B.atp_lowrank_linear(self.ctx, basis[0], basis[1], W, self.lengths, self.ranks, act=act, W_gate=W_gate,
                                     out=out, auto_workspace=False)
 
-    def forward(self, X: torch.Tensor) -> torch.Tensor:
-        """Returns the layer output (Y with an FFN, else the projected attention output, else O)."""
+    def forward(self, X: torch.Tensor, stage_events: Optional[list] = None) -> torch.Tensor:
+        """Returns the layer output (Y with an FFN, else the projected attention output, else O).
+        stage_events: a list that receives (stage name, start event, end event) per library call, recorded on
+        the current stream (for per-stage timing; None: nothing is recorded)."""
         c, w = self.ctx, self.w
+
+        def timed(name, fn):
+            if stage_events is None:
+                return fn()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            out = fn()
+            b.record()
+            stage_events.append((name, a, b))
+            return out
+
         Xin = X
         if self.input_norm:
-            Xin = B.atp_input_norm(c, X, None, kind=self.input_norm, out=self.Xn)
-        self._basis(Xin, self.bX)
-        B.atp_attention(c, Xin, self.bX[0], self.bX[1], w["W_Q"], w["W_K"], w["W_V"], self.heads, self.lengths,
-                        self.ranks, out=self.O, auto_workspace=False, q_mode=self.q_mode, rope_base=self.rope_base)
+            Xin = timed("norm_in", lambda: B.atp_input_norm(c, X, None, kind=self.input_norm, out=self.Xn))
+        timed("basis_X", lambda: self._basis(Xin, self.bX))
+        timed("attention", lambda: B.atp_attention(c, Xin, self.bX[0], self.bX[1], w["W_Q"], w["W_K"], w["W_V"], self.heads,
+                                                   self.lengths, self.ranks, out=self.O, auto_workspace=False,
+                                                   q_mode=self.q_mode, rope_base=self.rope_base))
         if not self.has_wo:
             return self.O
-        self._basis(self.O, self.bO)
-        self._linear(self.bO, w["W_O"], self.A)
+        timed("basis_O", lambda: self._basis(self.O, self.bO))
+        timed("linear_WO", lambda: self._linear(self.bO, w["W_O"], self.A))
         if not self.ffn:
             return self.A
-        B.atp_input_norm(c, X, self.A, kind=self.post_norm, out=self.H)        # H = Norm(X + A)
-        self._basis(self.H, self.bH)
+        timed("norm_post", lambda: B.atp_input_norm(c, X, self.A, kind=self.post_norm, out=self.H))   # H = Norm(X + A)
+        timed("basis_H", lambda: self._basis(self.H, self.bH))
         if self.ffn == "gelu":
-            self._linear(self.bH, w["W_1"], self.F, act="gelu")
-            self._basis(self.F, self.bF)
-            self._linear(self.bF, w["W_2"], self.Y)
+            timed("linear_ffn_in", lambda: self._linear(self.bH, w["W_1"], self.F, act="gelu"))
+            timed("basis_F", lambda: self._basis(self.F, self.bF))
+            timed("linear_ffn_out", lambda: self._linear(self.bF, w["W_2"], self.Y))
         else:
-            self._linear(self.bH, w["W_up"], self.F, act="swiglu", W_gate=w["W_gate"])
-            self._basis(self.F, self.bF)
-            self._linear(self.bF, w["W_down"], self.Y)
+            timed("linear_ffn_in", lambda: self._linear(self.bH, w["W_up"], self.F, act="swiglu", W_gate=w["W_gate"]))
+            timed("basis_F", lambda: self._basis(self.F, self.bF))
+            timed("linear_ffn_out", lambda: self._linear(self.bF, w["W_down"], self.Y))
         return self.Y
 
 
