@@ -57,6 +57,30 @@ def svd_jacobi(X):
     return U, S, Vt, int(sweeps)
 
 
+def svd_jacobi_capped(X, max_rounds):
+    """The same Jacobi iteration stopped after `max_rounds` rounds (a round rotates n/2 disjoint pairs, a sweep
+    is n-1 rounds): for timing a bounded part of a large decomposition. Returns the number of rounds run; the
+    unfinished factors are discarded."""
+    X = _c(X)
+    L, d = X.shape
+    n = min(L, d)
+    U = np.empty((L, n)); S = np.empty(n); Vt = np.empty((n, d))
+    done = ctypes.c_long(0)
+    _load().oracle_svd_jacobi_capped(_p(X), L, d, _p(U), _p(S), _p(Vt), ctypes.c_long(int(max_rounds)), ctypes.byref(done))
+    return int(done.value)
+
+
+def project_rows(X, U_r, nrows=None):
+    """Leading `nrows` rows of X_r = U_r^T X (all r by default)."""
+    X = _c(X); U_r = _c(U_r)
+    L, d = X.shape
+    r = U_r.shape[1]
+    nrows = r if nrows is None else int(nrows)
+    X_r = np.empty((nrows, d))
+    _load().oracle_project_rows(_p(X), _p(U_r), L, d, r, nrows, _p(X_r))
+    return X_r
+
+
 def principal_basis(X, r, return_all_sigma=False):
     """Eq. 5 / Sec. 4.2: (U_r, X_r, sigma) of the exact truncated SVD, canonical signs."""
     X = _c(X)
@@ -170,3 +194,20 @@ def layer_forward(X, weights, r, heads, ffn=None, input_norm=None, post_norm="la
         Y = lowrank_linear(Uf, Fr, weights["W_down"])
     st.update(H=H, F=F, Y=Y)
     return Y
+
+
+def stack_forward(X, layer_weights, r, heads, ffn=None, input_norm=None, post_norm="layer", stages=None):
+    """A chain of ATP layers for a single sequence (Sec. 4.2: the next encoder/decoder layer follows the same
+    procedure and first attains the principal components of the previous layer's output; Fig. 3). Layer l maps
+    X_l to Y_l = FFN(H_l), H_l = Norm(X_l + A_l) (layer_forward); the block is closed the post-norm way,
+    X_{l+1} = Norm(H_l + Y_l). Layers without a FeedForward pass their output on unchanged. `stages` (a list)
+    receives one dict of intermediates per layer. Returns the input of the layer after the last one."""
+    x = np.asarray(X, dtype=np.float64)
+    for wts in layer_weights:
+        st = {}
+        y = layer_forward(x, wts, r, heads, ffn=ffn, input_norm=input_norm, post_norm=post_norm, stages=st)
+        x = norm(st["H"], residual=y, kind=post_norm) if ffn else y
+        if stages is not None:
+            st["X_next"] = x
+            stages.append(st)
+    return x

@@ -236,6 +236,22 @@ static int svd_jacobi_impl(const double *X, int L, int d, double *U, double *S, 
 /* row of X_r is made positive instead.                                */
 /* sigma_all (nullable) receives all min(L,d) singular values.         */
 /* ------------------------------------------------------------------ */
+/* Rows [0, nrows) of X_r = U_r^T X (Sec. 4.2: X' = U^T X), written as the product it is defined by.   */
+/* U_r is L x r; nrows < r computes only the leading rows (used to time a bounded part of the product). */
+ORACLE_API void oracle_project_rows(const double *X, const double *U_r, int L, int d, int r, int nrows, double *X_r)
+{
+#pragma omp parallel for schedule(static)
+    for (int a = 0; a < nrows; ++a) {
+        double *row = X_r + (size_t)a * d;
+        for (int k = 0; k < d; ++k) row[k] = 0.0;
+        for (int i = 0; i < L; ++i) {
+            double u = U_r[(size_t)i * r + a];
+            const double *x = X + (size_t)i * d;
+            for (int k = 0; k < d; ++k) row[k] += u * x[k];
+        }
+    }
+}
+
 ORACLE_API int oracle_principal_basis(const double *X, int L, int d, int r, double *U_r, double *X_r,
                                       double *sigma, double *sigma_all)
 {
@@ -249,17 +265,7 @@ ORACLE_API int oracle_principal_basis(const double *X, int L, int d, int r, doub
         for (int a = 0; a < r; ++a) U_r[(size_t)i * r + a] = U[(size_t)i * n + a];
     if (sigma) for (int a = 0; a < r; ++a) sigma[a] = S[a];
     if (sigma_all) for (int a = 0; a < n; ++a) sigma_all[a] = S[a];
-    /* X_r = U_r^T X, written as the product it is defined by */
-#pragma omp parallel for schedule(static)
-    for (int a = 0; a < r; ++a) {
-        double *row = X_r + (size_t)a * d;
-        for (int k = 0; k < d; ++k) row[k] = 0.0;
-        for (int i = 0; i < L; ++i) {
-            double u = U_r[(size_t)i * r + a];
-            const double *x = X + (size_t)i * d;
-            for (int k = 0; k < d; ++k) row[k] += u * x[k];
-        }
-    }
+    oracle_project_rows(X, U_r, L, d, r, r, X_r);
     for (int a = 0; a < r; ++a) {
         double sum = 0.0;
         for (int i = 0; i < L; ++i) sum += U_r[(size_t)i * r + a];

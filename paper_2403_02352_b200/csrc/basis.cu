@@ -95,40 +95,43 @@ __global__ void __launch_bounds__(256) panel_gram_kernel(const __grid_constant__
 //   3. everybody below subtracts L_i L_k^T from G (columns right of jb) or L_i X_b from X (columns up
 //      to jb): 64 independent multiply-adds per thread.
 // Two block barriers per four columns.
-__global__ void __launch_bounds__(256) panel_chol_kernel(const __grid_constant__ PanelBatch batch)
+__global__ void __launch_bounds__(1024) panel_chol_kernel(const __grid_constant__ PanelBatch batch)
 {
     pdl_trigger();
     pdl_wait();
     const PanelSeq &sq = batch.s[blockIdx.x];
     const int n = sq.pb;
     if (n <= 0) return;
+    __shared__ double Gs[PB * PB];     // the summed Gram matrix
     __shared__ double rs[PB];          // 1 / sqrt(diagonal of the Gram matrix)
     __shared__ double lcol4[PB][4];    // block column jb of L (rows below the diagonal block)
     __shared__ double xrow4[4][PB];    // block row jb of L^-1
     __shared__ double Lbb[4][4];       // the factored diagonal block (strictly lower part)
     __shared__ double rinv4[4];        // 1 / L_jj, 0 for a dependent column
     __shared__ int dep[PB];
+    const int nchunks = (sq.n + GRAM_ROWS - 1) / GRAM_ROWS;
+    {   // all 1024 threads: four entries each, chunk by chunk (a fixed order), coalesced
+        const int e = threadIdx.x;
+        double acc[4] = {0.0, 0.0, 0.0, 0.0};
+#pragma unroll 4
+        for (int c = 0; c < nchunks; ++c) {
+            const double *src = sq.gpart + (size_t)c * PB * PB + e;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) acc[q] += src[q * 1024];
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) Gs[e + q * 1024] = acc[q];
+    }
+    __syncthreads();
+    if (threadIdx.x >= 256) return;    // the factorisation runs on 256 threads, which meet at a barrier of their own
+    auto bar256 = [] { asm volatile("bar.sync 1, 256;" ::: "memory"); };
     const int tid = threadIdx.x;
     const int br = tid >> 4, bc = tid & 15;
-    const int nchunks = (sq.n + GRAM_ROWS - 1) / GRAM_ROWS;
     double g[4][4], x[4][4];
 #pragma unroll
     for (int a = 0; a < 4; ++a)
 #pragma unroll
-        for (int b = 0; b < 4; ++b) { g[a][b] = 0.0; x[a][b] = (br == bc && a == b) ? 1.0 : 0.0; }
-    // chunk by chunk (a fixed order), the eight 16-byte loads of a chunk in flight together
-    const double2 *gp = (const double2 *)(sq.gpart + (size_t)(4 * br) * PB + 4 * bc);
-#pragma unroll 2
-    for (int c = 0; c < nchunks; ++c) {
-        double2 v[4][2];
-#pragma unroll
-        for (int a = 0; a < 4; ++a) {
-            v[a][0] = gp[((size_t)c * PB * PB + (size_t)a * PB) / 2];
-            v[a][1] = gp[((size_t)c * PB * PB + (size_t)a * PB) / 2 + 1];
-        }
-#pragma unroll
-        for (int a = 0; a < 4; ++a) { g[a][0] += v[a][0].x; g[a][1] += v[a][0].y; g[a][2] += v[a][1].x; g[a][3] += v[a][1].y; }
-    }
+        for (int b = 0; b < 4; ++b) { g[a][b] = Gs[(4 * br + a) * PB + 4 * bc + b]; x[a][b] = (br == bc && a == b) ? 1.0 : 0.0; }
     if (br == bc) {
 #pragma unroll
         for (int a = 0; a < 4; ++a) {
@@ -137,7 +140,7 @@ __global__ void __launch_bounds__(256) panel_chol_kernel(const __grid_constant__
             dep[i] = 0;
         }
     }
-    __syncthreads();
+    bar256();
 #pragma unroll
     for (int a = 0; a < 4; ++a)
 #pragma unroll
@@ -177,7 +180,7 @@ __global__ void __launch_bounds__(256) panel_chol_kernel(const __grid_constant__
                 for (int c = 0; c < 4; ++c) Lbb[r][c] = (c < r) ? g[r][c] : 0.0;
             }
         }
-        __syncthreads();
+        bar256();
         if (bc == jb && br > jb) {
             // 2a. rows of L below the diagonal block: l_c = (g_c - sum_{k<c} l_k L_bb[c][k]) / L_cc
 #pragma unroll
@@ -208,7 +211,7 @@ __global__ void __launch_bounds__(256) panel_chol_kernel(const __grid_constant__
                 }
             }
         }
-        __syncthreads();
+        bar256();
         if (br > jb && bc <= br) {
             // 3. trailing update
             double la[4][4];
@@ -250,7 +253,7 @@ __global__ void __launch_bounds__(256) panel_chol_kernel(const __grid_constant__
         w.x = (float)(rk * x[0][b]); w.y = (float)(rk * x[1][b]); w.z = (float)(rk * x[2][b]); w.w = (float)(rk * x[3][b]);
         *(float4 *)(sq.rinv + k * PB + 4 * br) = w;
     }
-    __syncthreads();
+    bar256();
     if (tid < PB) sq.flags[tid] = (tid < n) ? (dep[tid] || !(rs[tid] > 0.0)) : 0;
 }
 
@@ -947,7 +950,7 @@ static atp_status orthonormalise(atp_ctx *ctx, BasisPlan &bp, size_t i0, size_t 
             launch_pdl(panel_gram_kernel, dim3(ceil_div(maxn, GRAM_ROWS), pb.count), dim3(256), 0, ctx->stream, pb);
             ATP_LAUNCHED(ctx);
             ATP_KERNEL(ctx, "panel_chol", 0, 0);
-            launch_pdl(panel_chol_kernel, dim3(pb.count), dim3(256), 0, ctx->stream, pb);
+            launch_pdl(panel_chol_kernel, dim3(pb.count), dim3(1024), 0, ctx->stream, pb);
             ATP_LAUNCHED(ctx);
             ATP_KERNEL(ctx, "panel_apply", 0, 0);
             launch_pdl(panel_apply_kernel, dim3(ceil_div(maxn, 64), pb.count), dim3(256), 0, ctx->stream, pb,
