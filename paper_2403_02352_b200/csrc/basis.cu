@@ -10,12 +10,11 @@
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
 #include "jacobi3.cuh"
+#include "orth.cuh"
 #include <type_traits>
 #include <math.h>
 #include <algorithm>
 
-constexpr int PB = 64;            // orthonormalisation panel width
-constexpr int GRAM_ROWS = 64;     // rows per CTA of the panel Gram kernel
 constexpr int BJ = 32;            // Jacobi block height (pairs are 64 rows)
 constexpr int BMAX = 32;          // sequences per launch
 
@@ -33,294 +32,6 @@ __global__ void fill_omega_kernel(float *om, size_t n, uint64_t seed)
 {
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
         om[i] = (mix64(seed, i) & 1) ? 1.f : -1.f;
-}
-
-struct PanelSeq { float *P; int n, pb, ld; double *gpart; float *rinv; int *flags; };
-struct PanelBatch { PanelSeq s[BMAX]; int count; };
-
-// Partial Gram matrices of a panel: G_chunk = P_chunk^T P_chunk, fp64 accumulation.
-__global__ void __launch_bounds__(256) panel_gram_kernel(const __grid_constant__ PanelBatch batch)
-{
-    pdl_trigger();
-    pdl_wait();
-    const PanelSeq &sq = batch.s[blockIdx.y];
-    const int r0 = blockIdx.x * GRAM_ROWS;
-    if (sq.pb <= 0 || r0 >= sq.n) return;
-    const int r1 = min(sq.n, r0 + GRAM_ROWS);
-    __shared__ __align__(16) float Ps[32][PB + 4];
-    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-    double acc[4][4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = 0.0;
-    for (int rr = r0; rr < r1; rr += 32) {
-        for (int e = tid; e < 32 * PB; e += 256) {
-            int row = e >> 6, c = e & 63;
-            float v = 0.f;
-            if (rr + row < r1 && c < sq.pb) v = sq.P[(size_t)(rr + row) * sq.ld + c];
-            Ps[row][c] = v;
-        }
-        __syncthreads();
-#pragma unroll 4
-        for (int k = 0; k < 32; ++k) {
-            float4 a = *(const float4 *)&Ps[k][ty * 4];
-            float4 b = *(const float4 *)&Ps[k][tx * 4];
-            double av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-#pragma unroll
-                for (int j = 0; j < 4; ++j) acc[i][j] = fma(av[i], bv[j], acc[i][j]);
-        }
-        __syncthreads();
-    }
-    double *dst = sq.gpart + (size_t)blockIdx.x * PB * PB;
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) dst[(ty * 4 + i) * PB + tx * 4 + j] = acc[i][j];
-}
-
-// Sums the partial Gram matrices in order, scales to unit diagonal, Cholesky-factors in fp64,
-// D^-1 G D^-1 = L L^T, and inverts the factor: writes W = D^-1 L^-T (upper triangular, fp32, PB x PB
-// row-major), so that P W has orthonormal columns. A column whose scaled pivot falls below 1e-10 (its
-// part outside the span of the earlier columns is below 1e-5 of its norm) is flagged as dependent:
-// the apply kernel replaces it by a pseudo-random vector, which the second Gram-Schmidt pass
-// orthonormalises.
-// Right-looking by blocks of four columns, in registers: thread (br, bc) owns the 4 x 4 blocks of G
-// and of X (X starts as the identity and ends as L^-1) at rows 4 br, columns 4 bc. Block step jb:
-//   1. the owner of the diagonal block factors it (four pivots) and publishes L_bb and 1 / L_jj;
-//   2. the owners of the block column below it solve for their rows of L, the owners of block row jb of
-//      X apply L_bb^-1 to it; both publish;
-//   3. everybody below subtracts L_i L_k^T from G (columns right of jb) or L_i X_b from X (columns up
-//      to jb): 64 independent multiply-adds per thread.
-// Two block barriers per four columns.
-__global__ void __launch_bounds__(1024) panel_chol_kernel(const __grid_constant__ PanelBatch batch)
-{
-    pdl_trigger();
-    pdl_wait();
-    const PanelSeq &sq = batch.s[blockIdx.x];
-    const int n = sq.pb;
-    if (n <= 0) return;
-    __shared__ double Gs[PB * PB];     // the summed Gram matrix
-    __shared__ double rs[PB];          // 1 / sqrt(diagonal of the Gram matrix)
-    __shared__ double lcol4[PB][4];    // block column jb of L (rows below the diagonal block)
-    __shared__ double xrow4[4][PB];    // block row jb of L^-1
-    __shared__ double Lbb[4][4];       // the factored diagonal block (strictly lower part)
-    __shared__ double rinv4[4];        // 1 / L_jj, 0 for a dependent column
-    __shared__ int dep[PB];
-    const int nchunks = (sq.n + GRAM_ROWS - 1) / GRAM_ROWS;
-    {   // all 1024 threads: four entries each, chunk by chunk (a fixed order), coalesced
-        const int e = threadIdx.x;
-        double acc[4] = {0.0, 0.0, 0.0, 0.0};
-#pragma unroll 4
-        for (int c = 0; c < nchunks; ++c) {
-            const double *src = sq.gpart + (size_t)c * PB * PB + e;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) acc[q] += src[q * 1024];
-        }
-#pragma unroll
-        for (int q = 0; q < 4; ++q) Gs[e + q * 1024] = acc[q];
-    }
-    __syncthreads();
-    if (threadIdx.x >= 256) return;    // the factorisation runs on 256 threads, which meet at a barrier of their own
-    auto bar256 = [] { asm volatile("bar.sync 1, 256;" ::: "memory"); };
-    const int tid = threadIdx.x;
-    const int br = tid >> 4, bc = tid & 15;
-    double g[4][4], x[4][4];
-#pragma unroll
-    for (int a = 0; a < 4; ++a)
-#pragma unroll
-        for (int b = 0; b < 4; ++b) { g[a][b] = Gs[(4 * br + a) * PB + 4 * bc + b]; x[a][b] = (br == bc && a == b) ? 1.0 : 0.0; }
-    if (br == bc) {
-#pragma unroll
-        for (int a = 0; a < 4; ++a) {
-            const int i = 4 * br + a;
-            rs[i] = (i < n && g[a][a] > 0.0) ? rsqrt(g[a][a]) : 0.0;
-            dep[i] = 0;
-        }
-    }
-    bar256();
-#pragma unroll
-    for (int a = 0; a < 4; ++a)
-#pragma unroll
-        for (int b = 0; b < 4; ++b) {
-            const double ra = rs[4 * br + a], rb = rs[4 * bc + b];
-            g[a][b] = (br == bc && a == b) ? (ra > 0.0 ? 1.0 : 0.0) : g[a][b] * ra * rb;
-        }
-    const int nblk = (n + 3) >> 2;
-    for (int jb = 0; jb < nblk; ++jb) {
-        if (br == jb && bc == jb) {
-            // 1. the diagonal block, column by column; a dependent column gets a unit pivot and zeros below
-            double ri[4];
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                double piv = g[c][c];
-#pragma unroll
-                for (int k = 0; k < c; ++k) piv = fma(-g[c][k], g[c][k], piv);
-                const bool bad = !(piv > 1e-10);
-                // 1/sqrt in fp64 from the fp32 approximation and two Newton steps (piv is in (1e-10, ~1])
-                double y = (double)rsqrtf((float)piv);
-                y = y * (1.5 - 0.5 * piv * y * y);
-                y = y * (1.5 - 0.5 * piv * y * y);
-                ri[c] = bad ? 0.0 : y;
-                if (bad && 4 * jb + c < n) dep[4 * jb + c] = 1;
-#pragma unroll
-                for (int r = c + 1; r < 4; ++r) {
-                    double v = g[r][c];
-#pragma unroll
-                    for (int k = 0; k < c; ++k) v = fma(-g[r][k], g[c][k], v);
-                    g[r][c] = v * ri[c];
-                }
-            }
-#pragma unroll
-            for (int r = 0; r < 4; ++r) {
-                rinv4[r] = ri[r];
-#pragma unroll
-                for (int c = 0; c < 4; ++c) Lbb[r][c] = (c < r) ? g[r][c] : 0.0;
-            }
-        }
-        bar256();
-        if (bc == jb && br > jb) {
-            // 2a. rows of L below the diagonal block: l_c = (g_c - sum_{k<c} l_k L_bb[c][k]) / L_cc
-#pragma unroll
-            for (int a = 0; a < 4; ++a) {
-                double l[4];
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    double v = g[a][c];
-#pragma unroll
-                    for (int k = 0; k < c; ++k) v = fma(-l[k], Lbb[c][k], v);
-                    l[c] = v * rinv4[c];
-                    lcol4[4 * br + a][c] = l[c];
-                }
-            }
-        }
-        if (br == jb && bc <= jb) {
-            // 2b. block row jb of X: forward substitution with L_bb (a dependent column keeps its scale)
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const double sc = rinv4[c] > 0.0 ? rinv4[c] : 1.0;
-#pragma unroll
-                for (int b = 0; b < 4; ++b) {
-                    double v = x[c][b];
-#pragma unroll
-                    for (int k = 0; k < c; ++k) v = fma(-Lbb[c][k], x[k][b], v);
-                    x[c][b] = v * sc;
-                    xrow4[c][4 * bc + b] = x[c][b];
-                }
-            }
-        }
-        bar256();
-        if (br > jb && bc <= br) {
-            // 3. trailing update
-            double la[4][4];
-#pragma unroll
-            for (int a = 0; a < 4; ++a)
-#pragma unroll
-                for (int c = 0; c < 4; ++c) la[a][c] = lcol4[4 * br + a][c];
-            if (bc > jb) {
-#pragma unroll
-                for (int b = 0; b < 4; ++b) {
-                    double lb[4];
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) lb[c] = lcol4[4 * bc + b][c];
-#pragma unroll
-                    for (int a = 0; a < 4; ++a)
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) g[a][b] = fma(-la[a][c], lb[c], g[a][b]);
-                }
-            } else {
-#pragma unroll
-                for (int b = 0; b < 4; ++b) {
-                    double xb[4];
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) xb[c] = xrow4[c][4 * bc + b];
-#pragma unroll
-                    for (int a = 0; a < 4; ++a)
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) x[a][b] = fma(-la[a][c], xb[c], x[a][b]);
-                }
-            }
-        }
-    }
-    // W[k][c] = (L^-1)[c][k] / D_k ; this thread holds (L^-1)[4 br + a][4 bc + b]
-#pragma unroll
-    for (int b = 0; b < 4; ++b) {
-        const int k = 4 * bc + b;
-        const double rk = rs[k];
-        float4 w;
-        w.x = (float)(rk * x[0][b]); w.y = (float)(rk * x[1][b]); w.z = (float)(rk * x[2][b]); w.w = (float)(rk * x[3][b]);
-        *(float4 *)(sq.rinv + k * PB + 4 * br) = w;
-    }
-    bar256();
-    if (tid < PB) sq.flags[tid] = (tid < n) ? (dep[tid] || !(rs[tid] > 0.0)) : 0;
-}
-
-// P <- P W in place (W = D^-1 L^-T from panel_chol_kernel): a 64 x 64 x 64 product per CTA, 4 x 4
-// register tiles. Flagged columns are refilled with hash noise.
-__global__ void __launch_bounds__(256) panel_apply_kernel(const __grid_constant__ PanelBatch batch, uint64_t seed)
-{
-    pdl_trigger();
-    pdl_wait();
-    const PanelSeq &sq = batch.s[blockIdx.y];
-    const int r0 = blockIdx.x * 64;
-    if (sq.pb <= 0 || r0 >= sq.n) return;
-    __shared__ __align__(16) float Ws[PB][PB + 4];
-    __shared__ float Ps[64][PB + 1];
-    __shared__ int fl[PB];
-    const int tid = threadIdx.x;
-    const bool vec = (sq.ld & 3) == 0 && ((size_t)sq.P & 15) == 0;
-    for (int f = tid; f < 64 * (PB / 4); f += 256) {
-        const int row = f >> 4, c = (f & 15) * 4;
-        *(float4 *)&Ws[row][c] = *(const float4 *)(sq.rinv + row * PB + c);
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (r0 + row < sq.n) {
-            const float *src = sq.P + (size_t)(r0 + row) * sq.ld + c;
-            if (vec && c + 3 < sq.pb) v = *(const float4 *)src;
-            else {
-                if (c < sq.pb) v.x = src[0];
-                if (c + 1 < sq.pb) v.y = src[1];
-                if (c + 2 < sq.pb) v.z = src[2];
-                if (c + 3 < sq.pb) v.w = src[3];
-            }
-        }
-        Ps[row][c] = v.x; Ps[row][c + 1] = v.y; Ps[row][c + 2] = v.z; Ps[row][c + 3] = v.w;
-    }
-    if (tid < PB) fl[tid] = sq.flags[tid];
-    __syncthreads();
-    const int rr = (tid >> 4) * 4, c0 = (tid & 15) * 4;
-    float acc[4][4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
-#pragma unroll 8
-    for (int k = 0; k < PB; ++k) {
-        const float4 b = *(const float4 *)&Ws[k][c0];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const float a = Ps[rr + i][k];
-            acc[i][0] = fmaf(a, b.x, acc[i][0]); acc[i][1] = fmaf(a, b.y, acc[i][1]);
-            acc[i][2] = fmaf(a, b.z, acc[i][2]); acc[i][3] = fmaf(a, b.w, acc[i][3]);
-        }
-    }
-    const float rscale = rsqrtf((float)sq.n * (1.f / 3.f));      // replacement columns of about unit norm
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int grow = r0 + rr + i;
-        if (grow >= sq.n) continue;
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-            if (fl[c0 + j])
-                acc[i][j] = rscale * hash_uniform(seed, ((uint64_t)blockIdx.y << 40) ^ ((uint64_t)grow << 8) ^ (uint64_t)(c0 + j));
-        float *dst = sq.P + (size_t)grow * sq.ld + c0;
-        if (vec && c0 + 3 < sq.pb) *(float4 *)dst = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
-        else {
-#pragma unroll
-            for (int j = 0; j < 4; ++j) if (c0 + j < sq.pb) dst[j] = acc[i][j];
-        }
-    }
 }
 
 // fp32 -> bf16 hi/lo pair (hi = bf16(x), lo = bf16(x - hi)) for every sequence of a batch.
@@ -828,25 +539,17 @@ __global__ void __launch_bounds__(256) signfix_kernel(const __grid_constant__ Fi
 struct SeqPlan {
     SeqDims dims; int rt, np, npanel_L, npanel_d; unsigned *jsync, *jdone; float *tpart;
     __nv_bfloat16 *Bth, *Btl, *Y2h, *Y2l, *Wth, *Wtl, *Wsh, *Wsl;
+    float *oCpart, *oC, *oDpart, *oW; double *ogpart, *ogpart2; unsigned *osync; int ocap;
     __nv_bfloat16 *Yb, *Yl, *Zb, *Zl; float *Y2; float *Y, *Z, *BW, *Wsel, *tsum, *sig, *Cc, *rinv, *G, *Wt, *Vbuf; double *gpart; int *ord, *flags, *conv, *vflag, *needfix; unsigned *maxoff;
 };
 struct BasisPlan {
     std::vector<SeqPlan> seqs; float *omega; __nv_bfloat16 *omega_b; float *part; size_t part_stride, part_group; int group = 0; int rtmax; int splits;
 };
 
-// Split-K factor of the thin projections C = Q^T P (few output tiles, long K): enough slices to put
-// about two CTAs on every SM, each at least 64 deep.
-static int pick_splits(int K, int nseq)
-{
-    int want = (296 + std::max(nseq, 1) - 1) / std::max(nseq, 1);
-    int s = std::min(std::min(want, K / 64), 16);
-    return s < 1 ? 1 : s;
-}
-
 // Size of the Jacobi matrices: rt rounded up to a whole number of 64-row block pairs.
 static int jacobi_padded(int rt) { return rt <= 0 ? 0 : (rt + 63) / 64 * 64; }
 
-static void plan_basis(Arena &ar, const std::vector<SeqDims> &sd, int d, int oversample, BasisPlan &bp)
+static void plan_basis(Arena &ar, const std::vector<SeqDims> &sd, int d, int oversample, int sm_count, BasisPlan &bp)
 {
     bp.seqs.clear(); bp.rtmax = 0;
     int maxdim = d; size_t maxpart = 0;
@@ -861,7 +564,6 @@ static void plan_basis(Arena &ar, const std::vector<SeqDims> &sd, int d, int ove
     }
     bp.omega = ar.take<float>((size_t)d * bp.rtmax);
     bp.omega_b = ar.take<__nv_bfloat16>((size_t)d * align_up((size_t)bp.rtmax, 8));
-    bp.splits = pick_splits(maxdim, (int)std::min<size_t>(sd.size(), BMAX));
     for (auto &p : bp.seqs) {
         int L = p.dims.L, rt = p.rt;
         p.Y = ar.take<float>((size_t)L * rt);
@@ -876,10 +578,14 @@ static void plan_basis(Arena &ar, const std::vector<SeqDims> &sd, int d, int ove
         p.tsum = ar.take<float>(rt);
         p.sig = ar.take<float>(rt);
         p.ord = ar.take<int>(rt);
-        p.Cc = ar.take<float>((size_t)rt * PB);
-        p.rinv = ar.take<float>(PB * PB + PB);
-        p.flags = ar.take<int>(PB);
-        p.gpart = ar.take<double>((size_t)ceil_div(std::max(std::max(L, d), 1), GRAM_ROWS) * PB * PB);
+        {   // tile scratch of the orthonormalisation kernel
+            p.ocap = orth::max_ctas_per_seq(sm_count, (int)std::min<size_t>(sd.size(), BMAX));
+            const orth::Scratch sc = orth::scratch_tiles(L, rt, p.ocap);
+            p.oCpart = ar.take<float>(sc.cpart * 4096); p.oC = ar.take<float>(sc.c * 4096);
+            p.oDpart = ar.take<float>(sc.dpart * 4096); p.oW = ar.take<float>(4096);
+            p.ogpart = ar.take<double>(sc.gpart * 4096); p.ogpart2 = ar.take<double>((size_t)orth::NRED * 4096);
+            p.flags = ar.take<int>(64); p.osync = ar.take<unsigned>(64);
+        }
         p.np = jacobi_padded(rt);
         p.G = ar.take<float>((size_t)p.np * p.np);
         p.Wt = ar.take<float>((size_t)p.np * p.np);
@@ -900,65 +606,30 @@ static void plan_basis(Arena &ar, const std::vector<SeqDims> &sd, int d, int ove
         p.conv = ar.take<int>(1);
         maxpart = std::max(maxpart, (size_t)rt * PB);
     }
-    bp.part_stride = maxpart;
-    bp.part_group = (size_t)bp.splits * std::min<size_t>(bp.seqs.size(), BMAX) * maxpart;
-    bp.part = ar.take<float>(2 * bp.part_group);        // one region per concurrent group
 }
 
-size_t basis_workspace_bytes(const std::vector<SeqDims> &sd, int d, int oversample)
+size_t basis_workspace_bytes(const std::vector<SeqDims> &sd, int d, int oversample, int sm_count)
 {
     Arena ar(nullptr, (size_t)-1);
     BasisPlan bp;
-    plan_basis(ar, sd, d, oversample, bp);
+    plan_basis(ar, sd, d, oversample, sm_count, bp);
     return ar.off;
 }
 
-// Orthonormalise the columns of M_b (n_b x rt_b, ld = rt_b) for the sequences [i0, i1).
-// reps: Gram-Schmidt passes per panel. Two give orthonormality to working precision and repair
-// dependent columns; one is enough for an intermediate iterate of the subspace iteration.
-static atp_status orthonormalise(atp_ctx *ctx, BasisPlan &bp, size_t i0, size_t i1, bool z_side, int d, uint64_t seed, int reps)
+// Orthonormalise the columns of Y_b (L_b x rt_b, ld = rt_b) for the sequences [i0, i1): one persistent kernel
+// (orth.cuh). reps: Gram-Schmidt repetitions per panel; two give orthonormality to working precision and repair
+// dependent columns. With TENSOR the finished columns also go out as the bf16 hi/lo pair (Yb, Yl).
+template <bool TENSOR>
+static atp_status orthonormalise(atp_ctx *ctx, BasisPlan &bp, size_t i0, size_t i1, uint64_t seed, int reps)
 {
-    int maxpan = 0, maxn = 0;
+    orth::Batch ob; ob.count = (int)(i1 - i0);
     for (size_t i = i0; i < i1; ++i) {
-        maxpan = std::max(maxpan, ceil_div(bp.seqs[i].rt, PB));
-        maxn = std::max(maxn, z_side ? d : bp.seqs[i].dims.L);
+        SeqPlan &p = bp.seqs[i];
+        ob.s[i - i0] = orth::Seq{p.Y, p.dims.L, p.rt, p.rt, TENSOR ? p.Yb : nullptr, TENSOR ? p.Yl : nullptr,
+                                 (int)align_up((size_t)std::max(p.rt, 1), 8), p.oCpart, p.oC, p.oDpart, p.oW, p.ogpart, p.ogpart2,
+                                 p.flags, p.osync, 0, p.ocap, 0};
     }
-    atp_status st;
-    for (int pj = 0; pj < maxpan; ++pj) {
-        const int j0 = pj * PB;
-        for (int rep = 0; rep < reps; ++rep) {
-            GemmBatch proj, upd; PanelBatch pb;
-            proj.count = upd.count = pb.count = (int)(i1 - i0);
-            for (size_t i = i0; i < i1; ++i) {
-                SeqPlan &p = bp.seqs[i];
-                float *M = z_side ? p.Z : p.Y;
-                int n = z_side ? d : p.dims.L;
-                int w = std::min(PB, p.rt - j0);
-                if (w <= 0 || n <= 0) { w = 0; n = 0; }
-                int k = (int)(i - i0);
-                // C = Qprev^T P  (j0 x w), then P -= Qprev C
-                proj.p[k] = GemmProblem{M, M + j0, p.Cc, nullptr, w > 0 ? j0 : 0, w, n, p.rt, p.rt, PB, 0};
-                upd.p[k] = GemmProblem{M, p.Cc, M + j0, M + j0, n, w, w > 0 ? j0 : 0, p.rt, PB, p.rt, p.rt};
-                pb.s[k] = PanelSeq{M + j0, n, w, p.rt, p.gpart, p.rinv, p.flags};
-            }
-            if (j0 > 0) {
-                if ((st = launch_gemm_simt<float, float, float, true>(ctx, proj, GemmEpi{EPI_STORE, nullptr}, bp.splits,
-                                                                      bp.part + bp.group * bp.part_group, bp.part_stride, "gemm_simt_proj")) != ATP_OK) return st;
-                if ((st = launch_gemm_simt<float, float, float, false>(ctx, upd, GemmEpi{EPI_D_MINUS, nullptr}, 1, nullptr, 0, "gemm_simt_upd")) != ATP_OK) return st;
-            }
-            ATP_KERNEL(ctx, "panel_gram", 0, 0);
-            launch_pdl(panel_gram_kernel, dim3(ceil_div(maxn, GRAM_ROWS), pb.count), dim3(256), 0, ctx->stream, pb);
-            ATP_LAUNCHED(ctx);
-            ATP_KERNEL(ctx, "panel_chol", 0, 0);
-            launch_pdl(panel_chol_kernel, dim3(pb.count), dim3(1024), 0, ctx->stream, pb);
-            ATP_LAUNCHED(ctx);
-            ATP_KERNEL(ctx, "panel_apply", 0, 0);
-            launch_pdl(panel_apply_kernel, dim3(ceil_div(maxn, 64), pb.count), dim3(256), 0, ctx->stream, pb,
-                       (uint64_t)(seed + 7919ull * (uint64_t)(pj * 2 + rep) + (z_side ? 104729ull : 0ull)));
-            ATP_LAUNCHED(ctx);
-        }
-    }
-    return ATP_OK;
+    return orth::launch<TENSOR>(ctx, ob, reps, seed);
 }
 
 template <typename T>
@@ -968,7 +639,7 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
     const int d = (int)X->cols;
     Arena ar(ctx->workspace, ctx->workspace_bytes);
     BasisPlan bp;
-    plan_basis(ar, sd, d, oversample, bp);
+    plan_basis(ar, sd, d, oversample, ctx->sm_count, bp);
     if (ar.overflow || !ctx->workspace) return ATP_ERR_WORKSPACE_TOO_SMALL;
     atp_status st;
     if (X->dtype == ATP_BF16) {
@@ -1018,31 +689,16 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
             // orthonormalised in fp32 and handed to the next pass as bf16 copies.
             const int ldo = (int)align_up((size_t)bp.rtmax, 8);
             // The orthonormal iterate goes to the next pass as a bf16 hi/lo pair (about 16 mantissa
-            // bits): a single bf16 rounding of Y would leak sigma_1 * 2^-9 / sqrt(L) of the leading
-            // direction into every column and bury directions that are 10^3..10^4 times weaker.
-            auto to_bf16 = [&]() -> atp_status {
-                SplitBatch sb; sb.count = (int)(i1 - i0);
-                double bytes = 0; int maxel = 0;
-                for (size_t i = i0; i < i1; ++i) {
-                    SeqPlan &p = bp.seqs[i];
-                    sb.s[i - i0] = SplitSeq{p.Y, p.Yb, p.Yl, p.rt, (int)align_up((size_t)p.rt, 8), p.dims.L, p.rt};
-                    bytes += (double)p.dims.L * p.rt * 8;
-                    maxel = std::max(maxel, p.dims.L * p.rt);
-                }
-                if (maxel == 0) return ATP_OK;
-                ATP_KERNEL(ctx, "f32_to_bf16", 0, bytes);
-                launch_pdl(split_bf16_batch_kernel, dim3(std::min(64, ceil_div(maxel, 1024)), sb.count), dim3(256), 0, ctx->stream, sb);
-                ATP_LAUNCHED(ctx);
-                return ATP_OK;
-            };
+            // bits, written by the orthonormalisation kernel): a single bf16 rounding of Y would leak
+            // sigma_1 * 2^-9 / sqrt(L) of the leading direction into every column and bury directions
+            // that are 10^3..10^4 times weaker.
             std::vector<tc::HostProblem> hp;
             for (size_t i = i0; i < i1; ++i) {
                 SeqPlan &p = bp.seqs[i];
                 hp.push_back(tc::HostProblem{Xb(p), bp.omega_b, nullptr, p.Y, nullptr, nullptr, p.dims.L, p.rt, d, (int)X->ld, ldo, p.rt, 0});
             }
             if ((st = tc::launch<false, false, tc::OUT_F32>(ctx, hp, store)) != ATP_OK) return st;
-            if ((st = orthonormalise(ctx, bp, i0, i1, false, d, seed, 2)) != ATP_OK) return st;
-            if ((st = to_bf16()) != ATP_OK) return st;
+            if ((st = orthonormalise<std::is_same<T, __nv_bfloat16>::value>(ctx, bp, i0, i1, seed, 2)) != ATP_OK) return st;
             for (int it = 0; it < power_iters; ++it) {
                 hp.clear();
                 for (size_t i = i0; i < i1; ++i) {      // Z = X^T Y, kept as a bf16 hi/lo pair (only the next pass reads it)
@@ -1058,9 +714,8 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
                     hp.push_back(tc::HostProblem{Xb(p), p.Zb, p.Zl, p.Y, nullptr, nullptr, p.dims.L, p.rt, d, (int)X->ld, ldb, p.rt, 0});
                 }
                 if ((st = tc::launch<false, true, tc::OUT_F32>(ctx, hp, store)) != ATP_OK) return st;
-                if ((st = orthonormalise(ctx, bp, i0, i1, false, d, seed + 2000003ull * (it + 1), 2)) != ATP_OK) return st;
-                if ((st = to_bf16()) != ATP_OK) return st;
-            }
+                if ((st = orthonormalise<std::is_same<T, __nv_bfloat16>::value>(ctx, bp, i0, i1, seed + 2000003ull * (it + 1), 2)) != ATP_OK) return st;
+                }
         } else {
             // Y = X Omega
             for (size_t i = i0; i < i1; ++i) {
@@ -1068,7 +723,7 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
                 g.p[i - i0] = GemmProblem{Xb(p), bp.omega, p.Y, nullptr, p.dims.L, p.rt, d, (int)X->ld, bp.rtmax, p.rt, 0};
             }
             if ((st = launch_gemm_simt<T, float, float, false>(ctx, g, store)) != ATP_OK) return st;
-            if ((st = orthonormalise(ctx, bp, i0, i1, false, d, seed, 2)) != ATP_OK) return st;
+            if ((st = orthonormalise<std::is_same<T, __nv_bfloat16>::value>(ctx, bp, i0, i1, seed, 2)) != ATP_OK) return st;
             for (int it = 0; it < power_iters; ++it) {
                 // Z = X^T Y ; Y = X Z ; orth(Y).  Z is not orthonormalised: Y has orthonormal, QR-ordered
                 // columns, so cond(Z) ~ sigma_1 / sigma_r~ and cond(X Z) is its square, which the fp64
@@ -1083,7 +738,7 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
                     g.p[i - i0] = GemmProblem{Xb(p), p.Z, p.Y, nullptr, p.dims.L, p.rt, d, (int)X->ld, p.rt, p.rt, 0};
                 }
                 if ((st = launch_gemm_simt<T, float, float, false>(ctx, g, store)) != ATP_OK) return st;
-                if ((st = orthonormalise(ctx, bp, i0, i1, false, d, seed + 2000003ull * (it + 1), 2)) != ATP_OK) return st;
+                if ((st = orthonormalise<std::is_same<T, __nv_bfloat16>::value>(ctx, bp, i0, i1, seed + 2000003ull * (it + 1), 2)) != ATP_OK) return st;
             }
         }
         if (!two_sided) {
@@ -1362,7 +1017,7 @@ extern "C" atp_status atp_workspace_bytes(atp_ctx *ctx, int op, const atp_seqs *
     if (st != ATP_OK) return st;
     if (d < 1 || d > 0x7fffffff) return ATP_ERR_INVALID_ARG;
     switch (op) {
-        case ATP_OP_BASIS: *bytes = basis_workspace_bytes(sd, (int)d, 64) + 256; return ATP_OK;
+        case ATP_OP_BASIS: *bytes = basis_workspace_bytes(sd, (int)d, 64, ctx->sm_count) + 256; return ATP_OK;
         case ATP_OP_ATTENTION: if (d_out < 1) return ATP_ERR_INVALID_ARG; *bytes = attention_workspace_bytes(sd, d_out) + 256; return ATP_OK;
         case ATP_OP_LINEAR: if (d_out < 1) return ATP_ERR_INVALID_ARG; *bytes = linear_workspace_bytes(sd, d_out) + 256; return ATP_OK;
         case ATP_OP_ALTERNATING: *bytes = alternating_workspace_bytes(sd, (int)d) + 256; return ATP_OK;

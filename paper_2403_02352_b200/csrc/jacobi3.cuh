@@ -310,6 +310,44 @@ __device__ __forceinline__ void product64(const float *As, const float *Bs, int 
     }
 }
 
+// General form for other kernels: acc += op(A) * op(B) over K = 64, NPASS = 3 (split precision, as above) or
+// 1 (plain TF32, ~2^-11 relative per term). A_TRANS: A[m][k] = As[k * lda + m] (use stride LDB = 72);
+// otherwise As[m * lda + k] (stride LDA = 68). B as in product64.
+template <bool A_TRANS, bool B_TRANS, int NPASS>
+__device__ __forceinline__ void product64_acc(const float *As, int lda, const float *Bs, int ldb, int m0, int n0, float (&acc)[4][4])
+{
+    const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+#pragma unroll 2
+    for (int k0 = 0; k0 < BLK; k0 += 8) {
+        float af[4];
+        if (A_TRANS) {
+            af[0] = As[(k0 + t) * lda + m0 + g]; af[1] = As[(k0 + t) * lda + m0 + g + 8];
+            af[2] = As[(k0 + t + 4) * lda + m0 + g]; af[3] = As[(k0 + t + 4) * lda + m0 + g + 8];
+        } else {
+            af[0] = As[(m0 + g) * lda + k0 + t]; af[1] = As[(m0 + g + 8) * lda + k0 + t];
+            af[2] = As[(m0 + g) * lda + k0 + t + 4]; af[3] = As[(m0 + g + 8) * lda + k0 + t + 4];
+        }
+        uint32_t ah[4], al[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (NPASS == 3) split_tf32(af[i], ah[i], al[i]);
+            else { ah[i] = __float_as_uint(af[i]); al[i] = 0u; }
+        }
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+            const int n = n0 + nt * 8 + g;
+            float b0, b1;
+            if (B_TRANS) { b0 = Bs[n * ldb + k0 + t]; b1 = Bs[n * ldb + k0 + t + 4]; }
+            else { b0 = Bs[(k0 + t) * ldb + n]; b1 = Bs[(k0 + t + 4) * ldb + n]; }
+            uint32_t bh[2], bl[2];
+            if (NPASS == 3) { split_tf32(b0, bh[0], bl[0]); split_tf32(b1, bh[1], bl[1]); }
+            else { bh[0] = __float_as_uint(b0); bh[1] = __float_as_uint(b1); }
+            if (NPASS == 3) { mma_tf32(acc[nt], al, bh); mma_tf32(acc[nt], ah, bl); }
+            mma_tf32(acc[nt], ah, bh);
+        }
+    }
+}
+
 // The same product on the fp32 FMA units, with the ownership layout of the tensor-core version (this
 // thread: rows m0 + g and m0 + g + 8, columns n0 + 8 nt + 2 t, + 1). Used for fp32 inputs, whose
 // convergence threshold (1e-6) sits below the rounding of the split-precision product (~2^-21).

@@ -1,0 +1,329 @@
+// Persistent block Gram-Schmidt: orthonormalises the columns of the range-finder iterates (Sec. 4.2:
+// the basis U must satisfy U^T U = I) for every sequence of a batch in ONE cooperative launch.
+//
+// Panels of 64 columns, left to right; every panel runs `reps` times through
+//   project   C = Q^T P against the finished columns Q (split over row ranges, partials summed in a fixed order)
+//   update    P <- P - Q C
+//   Gram      S = P^T P accumulated in fp64, scaled, Cholesky-factored and inverted in fp64 (panel_chol.cuh)
+//   apply     P <- P (D^-1 L^-T); columns found dependent are replaced by hash noise, which the next
+//             repetition orthonormalises
+// Two repetitions give orthonormality to working precision (the second also repairs the explicit inverse,
+// which is only norm-wise stable). Each sequence owns a group of CTAs; the phases of a panel are separated by
+// the group's barrier (bounded spin, see jacobi3.cuh) instead of kernel boundaries, and every phase is a list
+// of independent 64 x 64 tile jobs dealt out round-robin. The 64^3 tile products run on the tensor cores in
+// split TF32 precision (three products, ~2^-21): plain TF32 is not enough even for the first repetition, because
+// what a projection leaves of an ill-conditioned panel is far below 2^-11 of the panel. fp32 inputs keep every
+// product on the fp32 units.
+#pragma once
+#include "jacobi3.cuh"
+#include "panel_chol.cuh"
+
+namespace orth {
+
+using j3::BLK; using j3::NT; using j3::LDA; using j3::LDB;
+constexpr int MAXSEQ = 32;
+constexpr int NRED = 16;          // second-level partial Gram sums
+
+struct Seq {
+    float *M; int n, rt, ld;                  // the iterate: n x rt, fp32, leading dimension ld
+    __nv_bfloat16 *hi, *lo; int ldh;          // nullable: the finished columns also go out as a bf16 hi/lo pair
+    float *Cpart, *C, *Dpart, *W;             // tile scratch (see scratch_tiles)
+    double *gpart, *gpart2;
+    int *flags;
+    unsigned *sync;                           // 64 words: group barrier (jacobi3.cuh)
+    int cta0, ncta, index;                    // CTA group (on entry to launch(): ncta = the cap the scratch was
+                                              // sized for); index of the sequence in its batch (noise stream)
+};
+struct Batch { Seq s[MAXSEQ]; int count; };
+
+// Number of 64 x 64 fp32 tiles of Cpart / C / Dpart, fp64 tiles of gpart, for a sequence of n rows and rt
+// columns handled by at most `ncta` CTAs.
+struct Scratch { size_t cpart, c, dpart, gpart; };
+static inline Scratch scratch_tiles(int n, int rt, int ncta)
+{
+    const size_t nt = (size_t)(n + 63) / 64, nj = (size_t)(rt + 63) / 64;
+    return Scratch{(size_t)ncta + nj + 1, nj + 1, (size_t)ncta + nt + 1, nt + 1};
+}
+
+// 64 x 64 tile of a row-major fp32 matrix -> shared memory (stride lds), zero beyond rv rows / cv columns.
+__device__ __forceinline__ void load_tile(float *dst, int lds, const float *src, int ld, int rv, int cv, bool vec)
+{
+    for (int f = threadIdx.x; f < 64 * 16; f += NT) {
+        const int r = f >> 4, c = (f & 15) * 4;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (r < rv) {
+            const float *p = src + (size_t)r * ld + c;
+            if (vec && c + 3 < cv) v = __ldcg((const float4 *)p);
+            else {
+                if (c < cv) v.x = __ldcg(p);
+                if (c + 1 < cv) v.y = __ldcg(p + 1);
+                if (c + 2 < cv) v.z = __ldcg(p + 2);
+                if (c + 3 < cv) v.w = __ldcg(p + 3);
+            }
+        }
+        float *d = dst + r * lds + c;
+        d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
+    }
+}
+
+// acc += op(A) B on the units chosen by PREC: 0 fp32 FMA, 1 plain TF32, 3 split TF32.
+template <int PREC, bool A_TRANS>
+__device__ __forceinline__ void tile_mac(const float *As, int lda, const float *Bs, int ldb, int m0, int n0, float (&acc)[4][4])
+{
+    if (PREC == 3) j3::product64_acc<A_TRANS, false, 3>(As, lda, Bs, ldb, m0, n0, acc);
+    else if (PREC == 1) j3::product64_acc<A_TRANS, false, 1>(As, lda, Bs, ldb, m0, n0, acc);
+    else {
+        const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+#pragma unroll 4
+        for (int k = 0; k < BLK; ++k) {
+            const float a0 = A_TRANS ? As[k * lda + m0 + g] : As[(m0 + g) * lda + k];
+            const float a1 = A_TRANS ? As[k * lda + m0 + g + 8] : As[(m0 + g + 8) * lda + k];
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) {
+                const float2 b = *(const float2 *)(Bs + k * ldb + n0 + nt * 8 + 2 * t);
+                acc[nt][0] = fmaf(a0, b.x, acc[nt][0]); acc[nt][1] = fmaf(a0, b.y, acc[nt][1]);
+                acc[nt][2] = fmaf(a1, b.x, acc[nt][2]); acc[nt][3] = fmaf(a1, b.y, acc[nt][3]);
+            }
+        }
+    }
+}
+
+// This thread's part of a 64 x 64 accumulator tile (rows m0 + g, + 8; columns n0 + 8 nt + 2 t, + 1).
+__device__ __forceinline__ void store_acc(float *dst, int ld, int m0, int n0, const float (&acc)[4][4])
+{
+    const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) {
+        const int c = n0 + nt * 8 + 2 * t;
+        *(float2 *)(dst + (size_t)(m0 + g) * ld + c) = make_float2(acc[nt][0], acc[nt][1]);
+        *(float2 *)(dst + (size_t)(m0 + g + 8) * ld + c) = make_float2(acc[nt][2], acc[nt][3]);
+    }
+}
+
+// TENSOR: bf16 inputs (tensor-core products); otherwise fp32 FMA everywhere.
+template <bool TENSOR>
+__global__ void __launch_bounds__(NT, 2)
+orth_persistent_kernel(const __grid_constant__ Batch batch, int reps, uint64_t seed, int *status)
+{
+    extern __shared__ __align__(16) float osm[];
+    __shared__ __align__(16) double Gs[PB * PB];
+    float *sA = osm, *sB = osm + BLK * LDB;                   // two tiles at stride LDB (covers LDA too)
+    int si = 0;
+#pragma unroll 1
+    for (int i = 1; i < batch.count; ++i) if ((int)blockIdx.x >= batch.s[i].cta0) si = i;
+    const Seq &sq = batch.s[si];
+    const int rank = (int)blockIdx.x - sq.cta0, tid = threadIdx.x, warp = tid >> 5;
+    if (rank >= sq.ncta || sq.n <= 0 || sq.rt <= 0) return;
+    const int m0 = (warp & 3) * 16, n0 = (warp >> 2) * 32;
+    const int n = sq.n, rt = sq.rt, ld = sq.ld, ncta = sq.ncta;
+    const int ntile = (n + 63) / 64, npanel = (rt + 63) / 64;
+    const bool vec = (ld & 3) == 0 && ((size_t)sq.M & 15) == 0;
+    int *abort_flag = status + 1;
+    unsigned gen = 0;
+    bool alive = true;
+    // Every product needs fp32-like accuracy: a panel of an ill-conditioned iterate lies almost entirely in the span
+    // of the finished columns, and what the projection leaves (1e-4 of the panel or less) is the information kept.
+    constexpr int P_ROUGH = TENSOR ? 3 : 0, P_FINE = TENSOR ? 3 : 0;
+    auto barrier = [&]() { alive = j3::group_barrier(sq.sync, ++gen, (unsigned)ncta, abort_flag) && alive; };
+
+    for (int pj = 0; pj < npanel && alive; ++pj) {
+        const int j0 = pj * 64, w = min(64, rt - j0), nj = pj;            // nj finished panels
+        for (int rep = 0; rep < reps && alive; ++rep) {
+            int G = 1;
+            if (nj > 0) {
+                // ---- project: partial C[jb] over row ranges
+                const int KS = max(1, min(ntile, (ncta + nj - 1) / nj));
+                const int tper = (ntile + KS - 1) / KS;
+                for (int it = rank; it < nj * KS; it += ncta) {
+                    const int jb = it / KS, ks = it - jb * KS;
+                    float acc[4][4] = {};
+                    for (int t = ks * tper; t < min(ntile, (ks + 1) * tper); ++t) {
+                        const int rv = min(64, n - t * 64);
+                        load_tile(sA, LDB, sq.M + (size_t)t * 64 * ld + jb * 64, ld, rv, 64, vec);
+                        load_tile(sB, LDB, sq.M + (size_t)t * 64 * ld + j0, ld, rv, w, vec);
+                        __syncthreads();
+                        if (rep == 0) tile_mac<P_ROUGH, true>(sA, LDB, sB, LDB, m0, n0, acc);
+                        else tile_mac<P_FINE, true>(sA, LDB, sB, LDB, m0, n0, acc);
+                        __syncthreads();
+                    }
+                    store_acc(sq.Cpart + (size_t)it * 4096, 64, m0, n0, acc);
+                }
+                barrier();
+                if (!alive) break;
+                // ---- sum the partials in order: C[jb]
+                for (int jb = rank; jb < nj; jb += ncta)
+                    for (int e = tid; e < 4096; e += NT) {
+                        float s = 0.f;
+                        for (int ks = 0; ks < KS; ++ks) s += __ldcg(sq.Cpart + ((size_t)jb * KS + ks) * 4096 + e);
+                        sq.C[(size_t)jb * 4096 + e] = s;
+                    }
+                barrier();
+                if (!alive) break;
+                // ---- update: partial D[t][g] = sum over a range of jb of Q[t][:, jb] C[jb]
+                G = max(1, min(nj, (ncta + ntile - 1) / ntile));
+                const int jper = (nj + G - 1) / G;
+                for (int it = rank; it < ntile * G; it += ncta) {
+                    const int t = it / G, g = it - t * G;
+                    const int rv = min(64, n - t * 64);
+                    float acc[4][4] = {};
+                    for (int jb = g * jper; jb < min(nj, (g + 1) * jper); ++jb) {
+                        load_tile(sA, LDA, sq.M + (size_t)t * 64 * ld + jb * 64, ld, rv, 64, vec);
+                        load_tile(sB, LDB, sq.C + (size_t)jb * 4096, 64, 64, 64, true);
+                        __syncthreads();
+                        tile_mac<P_ROUGH, false>(sA, LDA, sB, LDB, m0, n0, acc);
+                        __syncthreads();
+                    }
+                    store_acc(sq.Dpart + (size_t)it * 4096, 64, m0, n0, acc);
+                }
+                barrier();
+                if (!alive) break;
+            }
+            // ---- P[t] -= sum_g D[t][g] (fixed order), written back; partial Gram matrix of the tile in fp64
+            for (int t = rank; t < ntile; t += ncta) {
+                const int rv = min(64, n - t * 64);
+                load_tile(sA, LDA, sq.M + (size_t)t * 64 * ld + j0, ld, rv, w, vec);
+                __syncthreads();
+                if (nj > 0) {
+                    for (int e = tid; e < 4096; e += NT) {
+                        const int r = e >> 6, c = e & 63;
+                        float s = 0.f;
+                        for (int g = 0; g < G; ++g) s += __ldcg(sq.Dpart + ((size_t)t * G + g) * 4096 + e);
+                        const float v = sA[r * LDA + c] - s;
+                        sA[r * LDA + c] = (r < rv && c < w) ? v : 0.f;
+                        if (r < rv && c < w) sq.M[((size_t)t * 64 + r) * ld + j0 + c] = v;
+                    }
+                    __syncthreads();
+                }
+                const int tx = tid & 15, ty = tid >> 4;
+                double acc[4][4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) acc[i][j] = 0.0;
+#pragma unroll 4
+                for (int k = 0; k < 64; ++k) {
+                    const float4 a = *(const float4 *)&sA[k * LDA + ty * 4];
+                    const float4 b = *(const float4 *)&sA[k * LDA + tx * 4];
+                    const double av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) acc[i][j] = fma(av[i], bv[j], acc[i][j]);
+                }
+                double *dst = sq.gpart + (size_t)t * 4096;
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) dst[(ty * 4 + i) * 64 + tx * 4 + j] = acc[i][j];
+                __syncthreads();
+            }
+            barrier();
+            if (!alive) break;
+            // ---- two-level ordered sum of the partial Gram matrices
+            const int nred = min(NRED, ntile), cper = (ntile + nred - 1) / nred;
+            for (int q = rank; q < nred; q += ncta)
+                for (int e = tid; e < 4096; e += NT) {
+                    double s = 0.0;
+                    for (int c = q * cper; c < min(ntile, (q + 1) * cper); ++c) s += __ldcg(sq.gpart + (size_t)c * 4096 + e);
+                    sq.gpart2[(size_t)q * 4096 + e] = s;
+                }
+            barrier();
+            if (!alive) break;
+            // ---- Cholesky factor and its inverse (one CTA)
+            if (rank == 0) {
+                for (int e = tid; e < 4096; e += NT) {
+                    double s = 0.0;
+                    for (int q = 0; q < nred; ++q) s += __ldcg(sq.gpart2 + (size_t)q * 4096 + e);
+                    Gs[e] = s;
+                }
+                __syncthreads();
+                chol_invert_64(Gs, w, sq.W, sq.flags);
+                __syncthreads();
+            }
+            barrier();
+            if (!alive) break;
+            // ---- apply: P[t] <- P[t] W, dependent columns refilled, finished columns also as bf16 hi/lo
+            const bool last = rep == reps - 1;
+            const uint64_t nseed = seed + 7919ull * (uint64_t)(pj * 2 + rep);
+            const float rscale = rsqrtf((float)n * (1.f / 3.f));         // replacement columns of about unit norm
+            for (int t = rank; t < ntile; t += ncta) {
+                const int rv = min(64, n - t * 64);
+                load_tile(sA, LDA, sq.M + (size_t)t * 64 * ld + j0, ld, rv, w, vec);
+                load_tile(sB, LDB, sq.W, 64, 64, 64, true);
+                __syncthreads();
+                float acc[4][4] = {};
+                tile_mac<P_FINE, false>(sA, LDA, sB, LDB, m0, n0, acc);
+                const int lane = tid & 31, g = lane >> 2, tq = lane & 3;
+#pragma unroll
+                for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int r = m0 + g + (i >= 2 ? 8 : 0), c = n0 + nt * 8 + 2 * tq + (i & 1);
+                        if (r >= rv || c >= w) continue;
+                        const int grow = t * 64 + r;
+                        float v = acc[nt][i];
+                        if (__ldcg(sq.flags + c))
+                            v = rscale * hash_uniform(nseed, ((uint64_t)sq.index << 40) ^ ((uint64_t)grow << 8) ^ (uint64_t)c);
+                        sq.M[(size_t)grow * ld + j0 + c] = v;
+                        if (last && sq.hi) {
+                            const __nv_bfloat16 h = __float2bfloat16_rn(v);
+                            sq.hi[(size_t)grow * sq.ldh + j0 + c] = h;
+                            sq.lo[(size_t)grow * sq.ldh + j0 + c] = __float2bfloat16_rn(v - __bfloat162float(h));
+                        }
+                    }
+                __syncthreads();
+            }
+            barrier();
+        }
+    }
+    if (rank == 0 && tid == 0 && !alive) raise_status(status, ATP_ERR_TIMEOUT);
+}
+
+__global__ void init_kernel(const __grid_constant__ Batch batch)
+{
+    const Seq &sq = batch.s[blockIdx.x];
+    if (threadIdx.x < 64 && sq.n > 0) sq.sync[threadIdx.x] = 0u;
+}
+
+constexpr size_t SMEM_BYTES = (size_t)(2 * BLK * LDB) * sizeof(float);
+
+// Largest number of CTAs a launch hands to one sequence (workspace sizing and launch agree on it).
+static inline int max_ctas_per_seq(int sm_count, int nseq) { return std::max(1, 2 * sm_count / std::max(nseq, 1)); }
+
+template <bool TENSOR>
+static inline atp_status launch(atp_ctx *ctx, Batch &ob, int reps, uint64_t seed)
+{
+    if (ob.count <= 0) return ATP_OK;
+    static PerDeviceOnce attr_once;
+    ATP_CUDA_OK(ctx, attr_once.run(ctx->device, [] {
+        return cudaFuncSetAttribute(orth_persistent_kernel<TENSOR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
+    }));
+    int occ = 0;
+    ATP_CUDA_OK(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, orth_persistent_kernel<TENSOR>, NT, SMEM_BYTES));
+    if (occ < 1) return ATP_ERR_CUDA;
+    const int total = ctx->sm_count * std::min(occ, 2);
+    double wsum = 0;
+    for (int i = 0; i < ob.count; ++i) wsum += (double)ob.s[i].n * ob.s[i].rt;
+    if (wsum <= 0) return ATP_OK;
+    int next = 0;
+    for (int i = 0; i < ob.count; ++i) {
+        Seq &q = ob.s[i];
+        const int ntile = (q.n + 63) / 64;
+        int c = (int)((double)total * ((double)q.n * q.rt / wsum));
+        c = std::max(1, std::min(std::min(c, q.ncta), 4 * std::max(ntile, 1)));    // q.ncta: the cap the scratch was sized for
+        q.cta0 = next; q.ncta = c; q.index = i;
+        next += c;
+    }
+    if (next > total) return ATP_ERR_INVALID_ARG;      // cannot happen: shares sum to at most `total`
+    ATP_KERNEL(ctx, "orth_init", 0, 0);
+    init_kernel<<<ob.count, 64, 0, ctx->stream>>>(ob);
+    ATP_LAUNCHED(ctx);
+    int *status = ctx->dev_status;
+    void *args[] = {(void *)&ob, (void *)&reps, (void *)&seed, (void *)&status};
+    ATP_KERNEL(ctx, "orth_persistent", 0, 0);
+    ATP_CUDA_OK(ctx, cudaLaunchCooperativeKernel((const void *)orth_persistent_kernel<TENSOR>, dim3(next), dim3(NT), args, SMEM_BYTES, ctx->stream));
+    ATP_LAUNCHED(ctx);
+    return ATP_OK;
+}
+
+}  // namespace orth

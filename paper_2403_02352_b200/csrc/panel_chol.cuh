@@ -1,0 +1,160 @@
+// Cholesky factorisation and inversion of a 64 x 64 Gram matrix in fp64, on 256 threads of a CTA.
+// Gs (shared memory, 64 x 64 doubles, row-major) holds G = P^T P of a panel of n <= 64 columns. The
+// matrix is scaled to unit diagonal, factored D^-1 G D^-1 = L L^T and the factor inverted; the result
+// W = D^-1 L^-T (upper triangular, fp32, 64 x 64 row-major) goes to rinv, so that P W has orthonormal
+// columns. A column whose scaled pivot falls below 1e-10 (its part outside the span of the earlier
+// columns is below 1e-5 of its norm) is flagged as dependent in flags[0..63].
+// Right-looking by blocks of four columns, in registers: thread (br, bc) owns the 4 x 4 blocks of G
+// and of X (X starts as the identity and ends as L^-1) at rows 4 br, columns 4 bc. Block step jb:
+//   1. the owner of the diagonal block factors it (four pivots) and publishes L_bb and 1 / L_jj;
+//   2. the owners of the block column below it solve for their rows of L, the owners of block row jb of
+//      X apply L_bb^-1 to it; both publish;
+//   3. everybody below subtracts L_i L_k^T from G (columns right of jb) or L_i X_b from X (columns up
+//      to jb): 64 independent multiply-adds per thread.
+// Two barriers per four columns (named barrier 1, 256 threads: exactly the threads 0..255 must call).
+#pragma once
+#include "common.cuh"
+
+constexpr int PB = 64;            // orthonormalisation panel width
+
+__device__ __forceinline__ void chol_invert_64(const double *Gs, int n, float *rinv, int *flags)
+{
+    __shared__ double rs[PB];          // 1 / sqrt(diagonal of the Gram matrix)
+    __shared__ double lcol4[PB][4];    // block column jb of L (rows below the diagonal block)
+    __shared__ double xrow4[4][PB];    // block row jb of L^-1
+    __shared__ double Lbb[4][4];       // the factored diagonal block (strictly lower part)
+    __shared__ double rinv4[4];        // 1 / L_jj, 0 for a dependent column
+    __shared__ int dep[PB];
+    auto bar256 = [] { asm volatile("bar.sync 1, 256;" ::: "memory"); };
+    const int tid = threadIdx.x;
+    const int br = tid >> 4, bc = tid & 15;
+    double g[4][4], x[4][4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) { g[a][b] = Gs[(4 * br + a) * PB + 4 * bc + b]; x[a][b] = (br == bc && a == b) ? 1.0 : 0.0; }
+    if (br == bc) {
+#pragma unroll
+        for (int a = 0; a < 4; ++a) {
+            const int i = 4 * br + a;
+            rs[i] = (i < n && g[a][a] > 0.0) ? rsqrt(g[a][a]) : 0.0;
+            dep[i] = 0;
+        }
+    }
+    bar256();
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const double ra = rs[4 * br + a], rb = rs[4 * bc + b];
+            g[a][b] = (br == bc && a == b) ? (ra > 0.0 ? 1.0 : 0.0) : g[a][b] * ra * rb;
+        }
+    const int nblk = (n + 3) >> 2;
+    for (int jb = 0; jb < nblk; ++jb) {
+        if (br == jb && bc == jb) {
+            // 1. the diagonal block, column by column; a dependent column gets a unit pivot and zeros below
+            double ri[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                double piv = g[c][c];
+#pragma unroll
+                for (int k = 0; k < c; ++k) piv = fma(-g[c][k], g[c][k], piv);
+                const bool bad = !(piv > 1e-10);
+                // 1/sqrt in fp64 from the fp32 approximation and two Newton steps (piv is in (1e-10, ~1])
+                double y = (double)rsqrtf((float)piv);
+                y = y * (1.5 - 0.5 * piv * y * y);
+                y = y * (1.5 - 0.5 * piv * y * y);
+                ri[c] = bad ? 0.0 : y;
+                if (bad && 4 * jb + c < n) dep[4 * jb + c] = 1;
+#pragma unroll
+                for (int r = c + 1; r < 4; ++r) {
+                    double v = g[r][c];
+#pragma unroll
+                    for (int k = 0; k < c; ++k) v = fma(-g[r][k], g[c][k], v);
+                    g[r][c] = v * ri[c];
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                rinv4[r] = ri[r];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) Lbb[r][c] = (c < r) ? g[r][c] : 0.0;
+            }
+        }
+        bar256();
+        if (bc == jb && br > jb) {
+            // 2a. rows of L below the diagonal block: l_c = (g_c - sum_{k<c} l_k L_bb[c][k]) / L_cc
+#pragma unroll
+            for (int a = 0; a < 4; ++a) {
+                double l[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    double v = g[a][c];
+#pragma unroll
+                    for (int k = 0; k < c; ++k) v = fma(-l[k], Lbb[c][k], v);
+                    l[c] = v * rinv4[c];
+                    lcol4[4 * br + a][c] = l[c];
+                }
+            }
+        }
+        if (br == jb && bc <= jb) {
+            // 2b. block row jb of X: forward substitution with L_bb (a dependent column keeps its scale)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const double sc = rinv4[c] > 0.0 ? rinv4[c] : 1.0;
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                    double v = x[c][b];
+#pragma unroll
+                    for (int k = 0; k < c; ++k) v = fma(-Lbb[c][k], x[k][b], v);
+                    x[c][b] = v * sc;
+                    xrow4[c][4 * bc + b] = x[c][b];
+                }
+            }
+        }
+        bar256();
+        if (br > jb && bc <= br) {
+            // 3. trailing update
+            double la[4][4];
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) la[a][c] = lcol4[4 * br + a][c];
+            if (bc > jb) {
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                    double lb[4];
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) lb[c] = lcol4[4 * bc + b][c];
+#pragma unroll
+                    for (int a = 0; a < 4; ++a)
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) g[a][b] = fma(-la[a][c], lb[c], g[a][b]);
+                }
+            } else {
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                    double xb[4];
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) xb[c] = xrow4[c][4 * bc + b];
+#pragma unroll
+                    for (int a = 0; a < 4; ++a)
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) x[a][b] = fma(-la[a][c], xb[c], x[a][b]);
+                }
+            }
+        }
+    }
+    // W[k][c] = (L^-1)[c][k] / D_k ; this thread holds (L^-1)[4 br + a][4 bc + b]
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+        const int k = 4 * bc + b;
+        const double rk = rs[k];
+        float4 w;
+        w.x = (float)(rk * x[0][b]); w.y = (float)(rk * x[1][b]); w.z = (float)(rk * x[2][b]); w.w = (float)(rk * x[3][b]);
+        *(float4 *)(rinv + k * PB + 4 * br) = w;
+    }
+    bar256();
+    if (tid < PB) flags[tid] = (tid < n) ? (dep[tid] || !(rs[tid] > 0.0)) : 0;
+}
+
