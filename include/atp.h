@@ -21,15 +21,19 @@
  *     atp_create() allocates one small device status word and a pinned staging page, freed by
  *     atp_destroy().
  *   - Calls only enqueue work and return; they never wait for results, except
- *     atp_poll_device_status(). atp_principal_basis reads back its own convergence flags while it
- *     enqueues Jacobi sweeps: the calling thread may block until the GPU is within two sweeps of it
- *     (atp_basis_opts.no_host_sync turns that off).
- *     Work is ordered on the context's stream (atp_set_stream); atp_principal_basis can fork part of
- *     a batch onto two internal streams (opts->groups) and joins them back before it returns.
+ *     atp_poll_device_status(). atp_principal_basis runs its iterations (orthonormalisation, Jacobi
+ *     sweeps) inside persistent kernels that stop on their own convergence tests; nothing is read
+ *     back by the host. The one exception is the one-sided Jacobi variant (opts->jacobi_block = 1),
+ *     which reads its convergence flags while it enqueues sweeps and may block the calling thread
+ *     until the GPU is within two sweeps of it (atp_basis_opts.no_host_sync turns that off).
+ *     Work is ordered on the context's stream (atp_set_stream).
  *   - Errors the host can detect are returned at once and nothing is launched. Conditions only
- *     the device can see (a Jacobi iteration that hit its sweep limit, a bounded wait that ran
- *     out, a value outside the representable range) are recorded in the status word and read
- *     back by atp_poll_device_status(); no kernel traps or spins without bound.
+ *     the device can see (ATP_ERR_NOT_CONVERGED: a Jacobi iteration that hit its sweep limit;
+ *     ATP_ERR_TIMEOUT: a bounded wait - an mbarrier of a tensor-core pipeline, a barrier between
+ *     the CTAs of a persistent kernel - that ran out; ATP_ERR_RANGE: a non-finite entry in the
+ *     Gram matrix of the projected input, i.e. Inf / NaN in X or squares beyond fp32) are recorded
+ *     in the status word, first one wins, and read back by atp_poll_device_status(); no kernel
+ *     traps or spins without bound. Outputs of a call that raised one of them are unspecified.
  *   - dtype ATP_BF16 needs 16-byte aligned base pointers and `ld` a multiple of 8; otherwise
  *     ATP_ERR_INVALID_ARG is returned.
  *
@@ -100,16 +104,16 @@ typedef struct {
     int32_t power_iters;   /* subspace (power) iterations;        < 0: default 2              */
     int32_t max_sweeps;    /* Jacobi sweep limit;                 <= 0: default 24            */
     uint64_t seed;         /* seed of the +-1 test matrix                                      */
-    int32_t jacobi_block;  /* tuning: rows per block of the two-sided Jacobi, 16 or 32; 0: default 16; */
-                           /* 1: one-sided Jacobi on the projected rows themselves (no Gram matrix)      */
-    int32_t jacobi_inner;  /* tuning: on-chip sweeps per block visit;   <= 0: default 1                */
-    int32_t groups;        /* tuning: 0 / 1 = run the whole batch on the caller's stream; 2 = split the */
-                           /* batch in two groups on internal streams (forked from and joined to it)   */
-    int32_t no_host_sync;  /* 0: the call reads the device's convergence flags while it enqueues sweeps */
-                           /* and stops early (it may block the calling thread, see above). Non-zero:   */
-                           /* nothing is read back; max_sweeps sweeps are enqueued, those of converged  */
-                           /* sequences return at once. The call then never waits and can be recorded   */
-                           /* by a stream capture; choose max_sweeps with that cost in mind.            */
+    int32_t jacobi_block;  /* 0 (default), 16 or 32: two-sided block Jacobi on the Gram matrix of the      */
+                           /* projected rows, blocks of 32 rows (16 is accepted and means the same);       */
+                           /* 1: one-sided Jacobi on the projected rows themselves (no Gram matrix)        */
+    int32_t jacobi_inner;  /* accepted for compatibility, ignored                                          */
+    int32_t groups;        /* one-sided variant only: 2 = split the batch in two groups on internal        */
+                           /* streams (forked from and joined to the context's stream); otherwise ignored  */
+    int32_t no_host_sync;  /* one-sided variant only. 0: the call reads the device's convergence flags     */
+                           /* while it enqueues sweeps and stops early (it may block the calling thread).  */
+                           /* Non-zero: nothing is read back; max_sweeps sweeps are enqueued, those of      */
+                           /* converged sequences return at once. The default variant never reads back.    */
 } atp_basis_opts;
 
 typedef struct {
@@ -142,6 +146,10 @@ ATP_API atp_status atp_set_stream(atp_ctx *ctx, void *cuda_stream);
  * weight the call will see, i.e. d' for attention, d_out for a linear layer, ignored otherwise). */
 ATP_API atp_status atp_workspace_bytes(atp_ctx *ctx, int op, const atp_seqs *seqs, int64_t d, int64_t d_out,
                                atp_dtype dtype, size_t *bytes);
+/* The same for atp_principal_basis with the options it will be called with (the oversampling changes
+ * the size; atp_workspace_bytes(ATP_OP_BASIS, ...) answers for the defaults). opts may be NULL. */
+ATP_API atp_status atp_basis_workspace_bytes(atp_ctx *ctx, const atp_seqs *seqs, int64_t d, atp_dtype dtype,
+                                             const atp_basis_opts *opts, size_t *bytes);
 /* dev_ptr: device memory, 256-byte aligned, stays owned by the caller. Contents are scratch. */
 ATP_API atp_status atp_set_workspace(atp_ctx *ctx, void *dev_ptr, size_t bytes);
 
@@ -157,10 +165,10 @@ ATP_API atp_status atp_input_norm(atp_ctx *ctx, const atp_mat *X, const atp_mat 
  * Principal basis (Eq. 3, Eq. 5, Sec. 4.2): for every sequence b, the top-r_b left singular
  * vectors U_r (L_b x r_b, orthonormal columns) and X_r = U_r^T X = [sigma_1 v_1; ..; sigma_r v_r]
  * (r_b x d), components sorted by sigma descending, i.e. the minimiser of Eq. 9. Computed by a
- * randomised range finder with subspace iteration, block Gram-Schmidt orthonormalisation and a
- * block Jacobi rotation of the small projected problem (two-sided on the Gram matrix of the
- * projected rows, in two passes; one-sided on the rows themselves with opts->jacobi_block = 1) -
- * not by a full SVD - so
+ * randomised range finder with subspace iteration, block Gram-Schmidt orthonormalisation (one
+ * persistent kernel per iterate) and a block Jacobi rotation of the small projected problem
+ * (two-sided on the Gram matrix of the projected rows, two passes of one persistent kernel each;
+ * one-sided on the rows themselves with opts->jacobi_block = 1) - not by a full SVD - so
  * the subspace is the optimal one up to the range finder's error; opts->power_iters trades passes
  * over X for that. The Jacobi sweeps stop on a device-side convergence test (largest scaled
  * off-diagonal <= 1e-6 for f32, 3e-5 for bf16); opts->max_sweeps bounds them, and a sequence that
@@ -197,7 +205,8 @@ ATP_API atp_status atp_attention(atp_ctx *ctx, const atp_mat *X, const atp_mat *
 ATP_API atp_status atp_lowrank_linear(atp_ctx *ctx, const atp_mat *U_r, const atp_mat *X_r, const atp_mat *W,
                               const atp_seqs *seqs, const atp_linear_opts *opts, atp_mat *Y);
 
-/* Synchronises the stream, returns and clears the device-side status (ATP_OK if none). */
+/* Synchronises the stream, returns and clears the device-side status (ATP_OK if none): see the general
+ * conventions above for ATP_ERR_NOT_CONVERGED, ATP_ERR_TIMEOUT, ATP_ERR_RANGE. */
 ATP_API atp_status atp_poll_device_status(atp_ctx *ctx);
 /* Number of kernels this context has launched since creation (for accounting). */
 ATP_API int64_t atp_launch_count(const atp_ctx *ctx);
@@ -215,6 +224,18 @@ ATP_API atp_status atp_profile_start(atp_ctx *ctx);
 ATP_API atp_status atp_profile_stop(atp_ctx *ctx, char *buf, size_t cap, size_t *needed);
 
 /*
+ * Self-tests of the library's own bookkeeping (no counterpart in the paper; used by the test suite).
+ * atp_selftest_wait_timeout enqueues a kernel whose inter-CTA barrier can never complete (it expects
+ * a second CTA that does not exist) with a short wait limit: the kernel gives up and raises
+ * ATP_ERR_TIMEOUT on the status word, which the next atp_poll_device_status returns; the context stays
+ * usable. It needs a workspace of at least 256 bytes.
+ * atp_selftest_per_device_once runs the once-per-device set-up helper (kernel attributes, symbol
+ * addresses) through a fixed script on the host and returns how often the guarded step ran (7).
+ */
+ATP_API atp_status atp_selftest_wait_timeout(atp_ctx *ctx);
+ATP_API int atp_selftest_per_device_once(void);
+
+/*
  * Low-rank linear layer without any allocation (the paper has no counterpart: this entry point
  * exists for deployment, not for the method). It computes what atp_lowrank_linear computes,
  * Y = act(U_r (X_r W) + bias) with act NONE or GELU, for callers that may not allocate device
@@ -228,6 +249,8 @@ ATP_API atp_status atp_profile_stop(atp_ctx *ctx, char *buf, size_t cap, size_t 
  *     caller's, as in atp_lowrank_linear (same layouts, same dtype rules). SwiGLU is not offered.
  *   - Limit: sum(r_b) * d_out * 4 bytes must fit in ATP_STATIC_SCRATCH_BYTES, otherwise
  *     ATP_ERR_STATIC_SCRATCH_LIMIT is returned and nothing is launched.
+ *   - There is no context, hence no status word: a bounded wait of the tensor-core pipeline that
+ *     ran out (ATP_ERR_TIMEOUT elsewhere) ends the kernel early here without being reported.
  *   - The first call on each device looks up the buffer's device address; make that first call
  *     before starting any stream capture on that device.
  *   - All calls share the one buffer, and it keeps whatever the previous call left in it. The

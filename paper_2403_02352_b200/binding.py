@@ -25,6 +25,7 @@ exported_symbols = (
     "atp_input_norm", "atp_principal_basis", "atp_attention", "atp_lowrank_linear",
     "atp_poll_device_status", "atp_launch_count", "atp_status_string", "atp_profile_start", "atp_profile_stop",
     "atp_lowrank_linear_static", "atp_alternating_basis", "atp_svd_entropy",
+    "atp_basis_workspace_bytes", "atp_selftest_wait_timeout", "atp_selftest_per_device_once",
 )
 
 
@@ -76,6 +77,10 @@ def _load():
     lib.atp_set_workspace.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t]
     lib.atp_workspace_bytes.argtypes = [C.c_void_p, C.c_int, C.POINTER(Seqs), C.c_int64, C.c_int64, C.c_int,
                                         C.POINTER(C.c_size_t)]
+    lib.atp_basis_workspace_bytes.argtypes = [C.c_void_p, C.POINTER(Seqs), C.c_int64, C.c_int, C.POINTER(BasisOpts),
+                                              C.POINTER(C.c_size_t)]
+    lib.atp_selftest_wait_timeout.argtypes = [C.c_void_p]
+    lib.atp_selftest_per_device_once.restype = C.c_int
     lib.atp_poll_device_status.argtypes = [C.c_void_p]
     lib.atp_profile_start.argtypes = [C.c_void_p]
     lib.atp_profile_stop.argtypes = [C.c_void_p, C.c_char_p, C.c_size_t, C.POINTER(C.c_size_t)]
@@ -195,6 +200,11 @@ class Context:
         else:
             _check(lib.atp_set_workspace(self._h, C.c_void_p(t.data_ptr()), t.numel() * t.element_size()), "atp_set_workspace")
 
+    def selftest_wait_timeout(self):
+        """Enqueues a kernel whose barrier cannot complete; the next poll() raises ATP_ERR_TIMEOUT."""
+        self.ensure_workspace(256)
+        _check(lib.atp_selftest_wait_timeout(self._h), "atp_selftest_wait_timeout")
+
     def poll(self):
         """Synchronise and raise if a kernel recorded a device-side condition."""
         _check(lib.atp_poll_device_status(self._h), "device status")
@@ -248,14 +258,13 @@ def atp_principal_basis(ctx: Context, X, lengths, ranks, oversample=-1, power_it
         sig = torch.empty(sd.total_rank, dtype=torch.float32, device=X.device)
     else:
         U, Xr, sig = out
-    if auto_workspace:
-        ov = 64 if oversample < 0 else oversample
-        need = ctx.workspace_bytes(OP_BASIS, sd, d, 0, _dt(X))
-        if ov > 64:      # the query assumes the default oversampling; scale generously for larger ones
-            need = int(need * (1.0 + ov / 64.0))
-        ctx.ensure_workspace(need)
     opts = BasisOpts(C.sizeof(BasisOpts), oversample, power_iters, max_sweeps, seed, jacobi_block, jacobi_inner, groups,
                      1 if no_host_sync else 0)
+    if auto_workspace:
+        need = C.c_size_t(0)
+        _check(lib.atp_basis_workspace_bytes(ctx._h, C.byref(sd.c), d, _dt(X), C.byref(opts), C.byref(need)),
+               "atp_basis_workspace_bytes")
+        ctx.ensure_workspace(int(need.value))
     mx, mu, mxr = mat(X), mat(U), mat(Xr)
     _check(lib.atp_principal_basis(ctx._h, C.byref(mx), C.byref(sd.c), C.byref(opts), C.byref(mu), C.byref(mxr),
                                    C.c_void_p(sig.data_ptr()) if sig is not None else None), "atp_principal_basis")

@@ -1005,8 +1005,8 @@ extern "C" atp_status atp_principal_basis(atp_ctx *ctx, const atp_mat *X, const 
 size_t linear_workspace_bytes(const std::vector<SeqDims> &seqs, int64_t d_out);
 size_t attention_workspace_bytes(const std::vector<SeqDims> &seqs, int64_t dp);
 
-extern "C" atp_status atp_workspace_bytes(atp_ctx *ctx, int op, const atp_seqs *seqs, int64_t d, int64_t d_out,
-                                          atp_dtype dtype, size_t *bytes)
+static atp_status workspace_bytes_impl(atp_ctx *ctx, int op, const atp_seqs *seqs, int64_t d, int64_t d_out,
+                                       atp_dtype dtype, int oversample, size_t *bytes)
 {
     if (!ctx || !bytes) return ATP_ERR_INVALID_ARG;
     if (dtype != ATP_F32 && dtype != ATP_BF16) return ATP_ERR_UNSUPPORTED_DTYPE;
@@ -1017,10 +1017,62 @@ extern "C" atp_status atp_workspace_bytes(atp_ctx *ctx, int op, const atp_seqs *
     if (st != ATP_OK) return st;
     if (d < 1 || d > 0x7fffffff) return ATP_ERR_INVALID_ARG;
     switch (op) {
-        case ATP_OP_BASIS: *bytes = basis_workspace_bytes(sd, (int)d, 64, ctx->sm_count) + 256; return ATP_OK;
+        case ATP_OP_BASIS: *bytes = basis_workspace_bytes(sd, (int)d, oversample, ctx->sm_count) + 256; return ATP_OK;
         case ATP_OP_ATTENTION: if (d_out < 1) return ATP_ERR_INVALID_ARG; *bytes = attention_workspace_bytes(sd, d_out) + 256; return ATP_OK;
         case ATP_OP_LINEAR: if (d_out < 1) return ATP_ERR_INVALID_ARG; *bytes = linear_workspace_bytes(sd, d_out) + 256; return ATP_OK;
         case ATP_OP_ALTERNATING: *bytes = alternating_workspace_bytes(sd, (int)d) + 256; return ATP_OK;
         default: return ATP_ERR_INVALID_ARG;
     }
+}
+
+extern "C" atp_status atp_workspace_bytes(atp_ctx *ctx, int op, const atp_seqs *seqs, int64_t d, int64_t d_out,
+                                          atp_dtype dtype, size_t *bytes)
+{
+    return workspace_bytes_impl(ctx, op, seqs, d, d_out, dtype, 64, bytes);
+}
+
+extern "C" atp_status atp_basis_workspace_bytes(atp_ctx *ctx, const atp_seqs *seqs, int64_t d, atp_dtype dtype,
+                                                const atp_basis_opts *opts, size_t *bytes)
+{
+    int oversample = 64;
+    if (opts) {
+        if (opts->struct_size < offsetof(atp_basis_opts, no_host_sync)) return ATP_ERR_INVALID_ARG;
+        if (opts->oversample >= 0) oversample = opts->oversample;
+    }
+    if (oversample > 4096) return ATP_ERR_INVALID_ARG;
+    return workspace_bytes_impl(ctx, ATP_OP_BASIS, seqs, d, 0, dtype, oversample, bytes);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Self-tests of the bookkeeping around the kernels (used by the test suite).
+__global__ void wait_timeout_kernel(unsigned *sync, int *status)
+{
+    // a group barrier that expects two CTAs while only this one exists: the flag it polls is never set
+    if (!j3::group_barrier(sync, 1u, 2u, status + 1, 1u << 12) && threadIdx.x == 0) raise_status(status, ATP_ERR_TIMEOUT);
+}
+
+extern "C" atp_status atp_selftest_wait_timeout(atp_ctx *ctx)
+{
+    if (!ctx) return ATP_ERR_INVALID_ARG;
+    if (!ctx->workspace || ctx->workspace_bytes < 64 * sizeof(unsigned)) return ATP_ERR_WORKSPACE_TOO_SMALL;
+    ATP_CUDA_OK(ctx, cudaSetDevice(ctx->device));
+    ATP_CUDA_OK(ctx, cudaMemsetAsync(ctx->workspace, 0, 64 * sizeof(unsigned), ctx->stream));
+    ATP_KERNEL(ctx, "wait_timeout", 0, 0);
+    wait_timeout_kernel<<<1, 32, 0, ctx->stream>>>((unsigned *)ctx->workspace, ctx->dev_status);
+    ATP_LAUNCHED(ctx);
+    return ATP_OK;
+}
+
+extern "C" int atp_selftest_per_device_once(void)
+{
+    // the step must run once per device ordinal, again after a failure, and every time for ordinals
+    // outside the table
+    PerDeviceOnce once;
+    int runs = 0;
+    auto ok = [&] { ++runs; return cudaSuccess; };
+    auto fail = [&] { ++runs; return cudaErrorUnknown; };
+    once.run(0, ok); once.run(0, ok); once.run(1, ok); once.run(1, ok); once.run(0, ok);     // 2 runs
+    once.run(2, fail); once.run(2, ok); once.run(2, ok);                                      // 2 more
+    once.run(-1, ok); once.run(-1, ok); once.run(PerDeviceOnce::MAX_DEV, ok);                 // 3 more
+    return runs;
 }

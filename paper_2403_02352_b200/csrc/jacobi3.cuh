@@ -61,7 +61,8 @@ __device__ __forceinline__ void rr_pair(int nb, int step, int t, int &I, int &J)
 // counter sync[0]; the last one to arrive publishes `gen` in sync[32] (another cache line, so that
 // the pollers do not slow the arrivals down); the others poll that word. Bounded: returns false when
 // the wait ran out or another CTA flagged an abort.
-__device__ __forceinline__ bool group_barrier(unsigned *sync, unsigned gen, unsigned ncta, int *abort_flag)
+__device__ __forceinline__ bool group_barrier(unsigned *sync, unsigned gen, unsigned ncta, int *abort_flag,
+                                              unsigned limit = SPIN_LIMIT)
 {
     __syncthreads();
     __shared__ int ok_s;
@@ -76,7 +77,7 @@ __device__ __forceinline__ bool group_barrier(unsigned *sync, unsigned gen, unsi
                 *flag = gen;
             } else {
                 ok = 0;
-                for (unsigned i = 0; i < SPIN_LIMIT; ++i) {
+                for (unsigned i = 0; i < limit; ++i) {
                     if ((int)(*flag - gen) >= 0) { ok = 1; break; }
                     if ((i & 1023u) == 1023u && *(volatile int *)abort_flag) break;
                 }
@@ -596,16 +597,20 @@ jacobi_persistent_kernel(const __grid_constant__ Batch batch, float tol_conv, fl
     }
 }
 
-// Wt = identity, padding of G = 0, synchronisation words = 0. grid (x, count).
-__global__ void init_kernel(const __grid_constant__ Batch batch)
+// Wt = identity, padding of G = 0, synchronisation words = 0; a non-finite entry of G (an input with Inf / NaN,
+// or one whose squares overflow fp32) raises ATP_ERR_RANGE. grid (x, count).
+__global__ void init_kernel(const __grid_constant__ Batch batch, int *status)
 {
+    bool bad = false;
     const Seq &sq = batch.s[blockIdx.y];
     const size_t n2 = (size_t)sq.np * sq.np;
     for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n2; e += (size_t)gridDim.x * blockDim.x) {
         const int i = (int)(e / sq.np), j = (int)(e - (size_t)i * sq.np);
         sq.Wt[e] = (i == j) ? 1.f : 0.f;
         if (i >= sq.n || j >= sq.n) sq.G[e] = 0.f;
+        else if (!isfinite(sq.G[e])) bad = true;
     }
+    if (__syncthreads_or(bad) && threadIdx.x == 0) raise_status(status, ATP_ERR_RANGE);
     if (blockIdx.x == 0 && sq.np > 0) {
         if (threadIdx.x < 64) sq.sync[threadIdx.x] = 0u;
         const int npairs = sq.nb / 2;
@@ -649,7 +654,7 @@ static inline atp_status launch(atp_ctx *ctx, Batch &jb, float tol_conv, float t
     }
     if (next > total) return ATP_ERR_INVALID_ARG;      // cannot happen: shares sum to at most `total`
     ATP_KERNEL(ctx, "jacobi_init", 0, wsum * 4.0);
-    init_kernel<<<dim3(64, jb.count), 256, 0, ctx->stream>>>(jb);
+    init_kernel<<<dim3(64, jb.count), 256, 0, ctx->stream>>>(jb, ctx->dev_status);
     ATP_LAUNCHED(ctx);
     int *status = ctx->dev_status;
     int ms = max_sweeps, rn = raise_not_converged ? 1 : 0;

@@ -193,7 +193,11 @@ extern "C" atp_status atp_lowrank_linear_static(void *cuda_stream, const atp_mat
         return ATP_ERR_INVALID_ARG;
     if (U_r->rows == 0) return ATP_OK;
     // T is the only scratch; it is written in full before it is read, so nothing has to be cleared.
-    if ((uint64_t)tr * (uint64_t)W->cols * sizeof(float) > ATP_STATIC_SCRATCH_BYTES) return ATP_ERR_STATIC_SCRATCH_LIMIT;
+    // (fp32: sum(r) x d_out floats; bf16: the same matrix in bf16 with its rows padded to 8 elements)
+    const uint64_t need = U_r->dtype == ATP_F32 ? (uint64_t)tr * (uint64_t)W->cols * sizeof(float)
+                                                 : (uint64_t)tr * (uint64_t)align_up((size_t)W->cols, 8) * sizeof(__nv_bfloat16);
+    if (need > ATP_STATIC_SCRATCH_BYTES || (uint64_t)tr * (uint64_t)W->cols * sizeof(float) > ATP_STATIC_SCRATCH_BYTES)
+        return ATP_ERR_STATIC_SCRATCH_LIMIT;
     atp_ctx local;                      // host-side bookkeeping only; owns nothing on the device
     void *scratch = nullptr;
     if ((st = static_scratch_for_current_device(&local.device, &scratch)) != ATP_OK) return st;

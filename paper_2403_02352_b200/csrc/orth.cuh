@@ -22,7 +22,7 @@ namespace orth {
 
 using j3::BLK; using j3::NT; using j3::LDA; using j3::LDB;
 constexpr int MAXSEQ = 32;
-constexpr int NRED = 16;          // second-level partial Gram sums
+constexpr int NRED = 8;           // second-level partial Gram sums (chunk ranges)
 
 struct Seq {
     float *M; int n, rt, ld;                  // the iterate: n x rt, fp32, leading dimension ld
@@ -45,11 +45,15 @@ static inline Scratch scratch_tiles(int n, int rt, int ncta)
     return Scratch{(size_t)ncta + nj + 1, nj + 1, (size_t)ncta + nt + 1, nt + 1};
 }
 
-// 64 x 64 tile of a row-major fp32 matrix -> shared memory (stride lds), zero beyond rv rows / cv columns.
-__device__ __forceinline__ void load_tile(float *dst, int lds, const float *src, int ld, int rv, int cv, bool vec)
+// 64 x 64 tile of a row-major fp32 matrix, zero beyond rv rows / cv columns, in two halves so that the loads of
+// the next tile can be in flight while the current one is multiplied: fetch_tile (global -> registers, four
+// 16-byte pieces per thread) and stash_tile (registers -> shared memory at stride lds).
+struct TileRegs { float4 v[4]; };
+__device__ __forceinline__ void fetch_tile(TileRegs &tr, const float *src, int ld, int rv, int cv, bool vec)
 {
-    for (int f = threadIdx.x; f < 64 * 16; f += NT) {
-        const int r = f >> 4, c = (f & 15) * 4;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int f = threadIdx.x + i * NT, r = f >> 4, c = (f & 15) * 4;
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
         if (r < rv) {
             const float *p = src + (size_t)r * ld + c;
@@ -61,9 +65,39 @@ __device__ __forceinline__ void load_tile(float *dst, int lds, const float *src,
                 if (c + 3 < cv) v.w = __ldcg(p + 3);
             }
         }
-        float *d = dst + r * lds + c;
-        d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
+        tr.v[i] = v;
     }
+}
+__device__ __forceinline__ void stash_tile(const TileRegs &tr, float *dst, int lds)
+{
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int f = threadIdx.x + i * NT, r = f >> 4, c = (f & 15) * 4;
+        *(float4 *)(dst + r * lds + c) = tr.v[i];             // lds is a multiple of 4 floats: 16-byte aligned
+    }
+}
+__device__ __forceinline__ void load_tile(float *dst, int lds, const float *src, int ld, int rv, int cv, bool vec)
+{
+    TileRegs tr;
+    fetch_tile(tr, src, ld, rv, cv, vec);
+    stash_tile(tr, dst, lds);
+}
+
+// sum of base[0], base[stride], ..., base[(count - 1) stride] in that order, eight loads in flight
+template <typename T>
+__device__ __forceinline__ T ordered_sum(const T *base, size_t stride, int count)
+{
+    T s = (T)0;
+    int i = 0;
+    for (; i + 8 <= count; i += 8) {
+        T v[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) v[k] = __ldcg(base + (size_t)(i + k) * stride);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) s += v[k];
+    }
+    for (; i < count; ++i) s += __ldcg(base + (size_t)i * stride);
+    return s;
 }
 
 // acc += op(A) B on the units chosen by PREC: 0 fp32 FMA, 1 plain TF32, 3 split TF32.
@@ -123,7 +157,7 @@ orth_persistent_kernel(const __grid_constant__ Batch batch, int reps, uint64_t s
     bool alive = true;
     // Every product needs fp32-like accuracy: a panel of an ill-conditioned iterate lies almost entirely in the span
     // of the finished columns, and what the projection leaves (1e-4 of the panel or less) is the information kept.
-    constexpr int P_ROUGH = TENSOR ? 3 : 0, P_FINE = TENSOR ? 3 : 0;
+    constexpr int P_FINE = TENSOR ? 3 : 0;
     auto barrier = [&]() { alive = j3::group_barrier(sq.sync, ++gen, (unsigned)ncta, abort_flag) && alive; };
 
     for (int pj = 0; pj < npanel && alive; ++pj) {
@@ -137,13 +171,22 @@ orth_persistent_kernel(const __grid_constant__ Batch batch, int reps, uint64_t s
                 for (int it = rank; it < nj * KS; it += ncta) {
                     const int jb = it / KS, ks = it - jb * KS;
                     float acc[4][4] = {};
-                    for (int t = ks * tper; t < min(ntile, (ks + 1) * tper); ++t) {
-                        const int rv = min(64, n - t * 64);
-                        load_tile(sA, LDB, sq.M + (size_t)t * 64 * ld + jb * 64, ld, rv, 64, vec);
-                        load_tile(sB, LDB, sq.M + (size_t)t * 64 * ld + j0, ld, rv, w, vec);
+                    const int t0 = ks * tper, t1 = min(ntile, (ks + 1) * tper);
+                    TileRegs ra, rb;
+                    if (t0 < t1) {
+                        fetch_tile(ra, sq.M + (size_t)t0 * 64 * ld + jb * 64, ld, min(64, n - t0 * 64), 64, vec);
+                        fetch_tile(rb, sq.M + (size_t)t0 * 64 * ld + j0, ld, min(64, n - t0 * 64), w, vec);
+                    }
+                    for (int t = t0; t < t1; ++t) {
+                        stash_tile(ra, sA, LDB);
+                        stash_tile(rb, sB, LDB);
                         __syncthreads();
-                        if (rep == 0) tile_mac<P_ROUGH, true>(sA, LDB, sB, LDB, m0, n0, acc);
-                        else tile_mac<P_FINE, true>(sA, LDB, sB, LDB, m0, n0, acc);
+                        if (t + 1 < t1) {                                   // next tiles in flight during the product
+                            const int rv = min(64, n - (t + 1) * 64);
+                            fetch_tile(ra, sq.M + (size_t)(t + 1) * 64 * ld + jb * 64, ld, rv, 64, vec);
+                            fetch_tile(rb, sq.M + (size_t)(t + 1) * 64 * ld + j0, ld, rv, w, vec);
+                        }
+                        tile_mac<P_FINE, true>(sA, LDB, sB, LDB, m0, n0, acc);
                         __syncthreads();
                     }
                     store_acc(sq.Cpart + (size_t)it * 4096, 64, m0, n0, acc);
@@ -152,11 +195,8 @@ orth_persistent_kernel(const __grid_constant__ Batch batch, int reps, uint64_t s
                 if (!alive) break;
                 // ---- sum the partials in order: C[jb]
                 for (int jb = rank; jb < nj; jb += ncta)
-                    for (int e = tid; e < 4096; e += NT) {
-                        float s = 0.f;
-                        for (int ks = 0; ks < KS; ++ks) s += __ldcg(sq.Cpart + ((size_t)jb * KS + ks) * 4096 + e);
-                        sq.C[(size_t)jb * 4096 + e] = s;
-                    }
+                    for (int e = tid; e < 4096; e += NT)
+                        sq.C[(size_t)jb * 4096 + e] = ordered_sum(sq.Cpart + (size_t)jb * KS * 4096 + e, 4096, KS);
                 barrier();
                 if (!alive) break;
                 // ---- update: partial D[t][g] = sum over a range of jb of Q[t][:, jb] C[jb]
@@ -166,11 +206,21 @@ orth_persistent_kernel(const __grid_constant__ Batch batch, int reps, uint64_t s
                     const int t = it / G, g = it - t * G;
                     const int rv = min(64, n - t * 64);
                     float acc[4][4] = {};
-                    for (int jb = g * jper; jb < min(nj, (g + 1) * jper); ++jb) {
-                        load_tile(sA, LDA, sq.M + (size_t)t * 64 * ld + jb * 64, ld, rv, 64, vec);
-                        load_tile(sB, LDB, sq.C + (size_t)jb * 4096, 64, 64, 64, true);
+                    const int jb0 = g * jper, jb1 = min(nj, (g + 1) * jper);
+                    TileRegs ra, rb;
+                    if (jb0 < jb1) {
+                        fetch_tile(ra, sq.M + (size_t)t * 64 * ld + jb0 * 64, ld, rv, 64, vec);
+                        fetch_tile(rb, sq.C + (size_t)jb0 * 4096, 64, 64, 64, true);
+                    }
+                    for (int jb = jb0; jb < jb1; ++jb) {
+                        stash_tile(ra, sA, LDA);
+                        stash_tile(rb, sB, LDB);
                         __syncthreads();
-                        tile_mac<P_ROUGH, false>(sA, LDA, sB, LDB, m0, n0, acc);
+                        if (jb + 1 < jb1) {
+                            fetch_tile(ra, sq.M + (size_t)t * 64 * ld + (jb + 1) * 64, ld, rv, 64, vec);
+                            fetch_tile(rb, sq.C + (size_t)(jb + 1) * 4096, 64, 64, 64, true);
+                        }
+                        tile_mac<P_FINE, false>(sA, LDA, sB, LDB, m0, n0, acc);
                         __syncthreads();
                     }
                     store_acc(sq.Dpart + (size_t)it * 4096, 64, m0, n0, acc);
@@ -186,8 +236,7 @@ orth_persistent_kernel(const __grid_constant__ Batch batch, int reps, uint64_t s
                 if (nj > 0) {
                     for (int e = tid; e < 4096; e += NT) {
                         const int r = e >> 6, c = e & 63;
-                        float s = 0.f;
-                        for (int g = 0; g < G; ++g) s += __ldcg(sq.Dpart + ((size_t)t * G + g) * 4096 + e);
+                        const float s = ordered_sum(sq.Dpart + (size_t)t * G * 4096 + e, 4096, G);
                         const float v = sA[r * LDA + c] - s;
                         sA[r * LDA + c] = (r < rv && c < w) ? v : 0.f;
                         if (r < rv && c < w) sq.M[((size_t)t * 64 + r) * ld + j0 + c] = v;
@@ -219,23 +268,18 @@ orth_persistent_kernel(const __grid_constant__ Batch batch, int reps, uint64_t s
             }
             barrier();
             if (!alive) break;
-            // ---- two-level ordered sum of the partial Gram matrices
-            const int nred = min(NRED, ntile), cper = (ntile + nred - 1) / nred;
-            for (int q = rank; q < nred; q += ncta)
-                for (int e = tid; e < 4096; e += NT) {
-                    double s = 0.0;
-                    for (int c = q * cper; c < min(ntile, (q + 1) * cper); ++c) s += __ldcg(sq.gpart + (size_t)c * 4096 + e);
-                    sq.gpart2[(size_t)q * 4096 + e] = s;
-                }
+            // ---- ordered sum of the partial Gram matrices: 16 element slices x (up to 8) chunk ranges
+            const int nrange = max(1, min(8, ntile / 64)), cper = (ntile + nrange - 1) / nrange;
+            for (int it = rank; it < 16 * nrange; it += ncta) {
+                const int sl = it & 15, rg = it >> 4, e = sl * 256 + tid;
+                const int c0 = rg * cper, c1 = min(ntile, (rg + 1) * cper);
+                sq.gpart2[(size_t)rg * 4096 + e] = ordered_sum(sq.gpart + (size_t)c0 * 4096 + e, 4096, max(c1 - c0, 0));
+            }
             barrier();
             if (!alive) break;
             // ---- Cholesky factor and its inverse (one CTA)
             if (rank == 0) {
-                for (int e = tid; e < 4096; e += NT) {
-                    double s = 0.0;
-                    for (int q = 0; q < nred; ++q) s += __ldcg(sq.gpart2 + (size_t)q * 4096 + e);
-                    Gs[e] = s;
-                }
+                for (int e = tid; e < 4096; e += NT) Gs[e] = ordered_sum(sq.gpart2 + e, 4096, nrange);
                 __syncthreads();
                 chol_invert_64(Gs, w, sq.W, sq.flags);
                 __syncthreads();

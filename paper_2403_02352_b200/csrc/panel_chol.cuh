@@ -28,16 +28,25 @@ __device__ __forceinline__ void chol_invert_64(const double *Gs, int n, float *r
     auto bar256 = [] { asm volatile("bar.sync 1, 256;" ::: "memory"); };
     const int tid = threadIdx.x;
     const int br = tid >> 4, bc = tid & 15;
-    double g[4][4], x[4][4];
+    // One 4 x 4 block per thread: it holds the thread's block of G until block step jb = bc has consumed it, and
+    // the thread's block of X from then on (a block of G left of the current step is dead, a block of X right of
+    // it is still its initial identity / zero block), which halves the register need.
+    double blk[4][4];
 #pragma unroll
     for (int a = 0; a < 4; ++a)
 #pragma unroll
-        for (int b = 0; b < 4; ++b) { g[a][b] = Gs[(4 * br + a) * PB + 4 * bc + b]; x[a][b] = (br == bc && a == b) ? 1.0 : 0.0; }
+        for (int b = 0; b < 4; ++b) blk[a][b] = Gs[(4 * br + a) * PB + 4 * bc + b];
+    auto to_x = [&]() {
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int b = 0; b < 4; ++b) blk[a][b] = (br == bc && a == b) ? 1.0 : 0.0;
+    };
     if (br == bc) {
 #pragma unroll
         for (int a = 0; a < 4; ++a) {
             const int i = 4 * br + a;
-            rs[i] = (i < n && g[a][a] > 0.0) ? rsqrt(g[a][a]) : 0.0;
+            rs[i] = (i < n && blk[a][a] > 0.0) ? rsqrt(blk[a][a]) : 0.0;
             dep[i] = 0;
         }
     }
@@ -47,7 +56,7 @@ __device__ __forceinline__ void chol_invert_64(const double *Gs, int n, float *r
 #pragma unroll
         for (int b = 0; b < 4; ++b) {
             const double ra = rs[4 * br + a], rb = rs[4 * bc + b];
-            g[a][b] = (br == bc && a == b) ? (ra > 0.0 ? 1.0 : 0.0) : g[a][b] * ra * rb;
+            blk[a][b] = (br == bc && a == b) ? (ra > 0.0 ? 1.0 : 0.0) : blk[a][b] * ra * rb;
         }
     const int nblk = (n + 3) >> 2;
     for (int jb = 0; jb < nblk; ++jb) {
@@ -56,9 +65,9 @@ __device__ __forceinline__ void chol_invert_64(const double *Gs, int n, float *r
             double ri[4];
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-                double piv = g[c][c];
+                double piv = blk[c][c];
 #pragma unroll
-                for (int k = 0; k < c; ++k) piv = fma(-g[c][k], g[c][k], piv);
+                for (int k = 0; k < c; ++k) piv = fma(-blk[c][k], blk[c][k], piv);
                 const bool bad = !(piv > 1e-10);
                 // 1/sqrt in fp64 from the fp32 approximation and two Newton steps (piv is in (1e-10, ~1])
                 double y = (double)rsqrtf((float)piv);
@@ -68,18 +77,19 @@ __device__ __forceinline__ void chol_invert_64(const double *Gs, int n, float *r
                 if (bad && 4 * jb + c < n) dep[4 * jb + c] = 1;
 #pragma unroll
                 for (int r = c + 1; r < 4; ++r) {
-                    double v = g[r][c];
+                    double v = blk[r][c];
 #pragma unroll
-                    for (int k = 0; k < c; ++k) v = fma(-g[r][k], g[c][k], v);
-                    g[r][c] = v * ri[c];
+                    for (int k = 0; k < c; ++k) v = fma(-blk[r][k], blk[c][k], v);
+                    blk[r][c] = v * ri[c];
                 }
             }
 #pragma unroll
             for (int r = 0; r < 4; ++r) {
                 rinv4[r] = ri[r];
 #pragma unroll
-                for (int c = 0; c < 4; ++c) Lbb[r][c] = (c < r) ? g[r][c] : 0.0;
+                for (int c = 0; c < 4; ++c) Lbb[r][c] = (c < r) ? blk[r][c] : 0.0;
             }
+            to_x();
         }
         bar256();
         if (bc == jb && br > jb) {
@@ -89,13 +99,14 @@ __device__ __forceinline__ void chol_invert_64(const double *Gs, int n, float *r
                 double l[4];
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
-                    double v = g[a][c];
+                    double v = blk[a][c];
 #pragma unroll
                     for (int k = 0; k < c; ++k) v = fma(-l[k], Lbb[c][k], v);
                     l[c] = v * rinv4[c];
                     lcol4[4 * br + a][c] = l[c];
                 }
             }
+            to_x();
         }
         if (br == jb && bc <= jb) {
             // 2b. block row jb of X: forward substitution with L_bb (a dependent column keeps its scale)
@@ -104,11 +115,11 @@ __device__ __forceinline__ void chol_invert_64(const double *Gs, int n, float *r
                 const double sc = rinv4[c] > 0.0 ? rinv4[c] : 1.0;
 #pragma unroll
                 for (int b = 0; b < 4; ++b) {
-                    double v = x[c][b];
+                    double v = blk[c][b];
 #pragma unroll
-                    for (int k = 0; k < c; ++k) v = fma(-Lbb[c][k], x[k][b], v);
-                    x[c][b] = v * sc;
-                    xrow4[c][4 * bc + b] = x[c][b];
+                    for (int k = 0; k < c; ++k) v = fma(-Lbb[c][k], blk[k][b], v);
+                    blk[c][b] = v * sc;
+                    xrow4[c][4 * bc + b] = blk[c][b];
                 }
             }
         }
@@ -129,7 +140,7 @@ __device__ __forceinline__ void chol_invert_64(const double *Gs, int n, float *r
 #pragma unroll
                     for (int a = 0; a < 4; ++a)
 #pragma unroll
-                        for (int c = 0; c < 4; ++c) g[a][b] = fma(-la[a][c], lb[c], g[a][b]);
+                        for (int c = 0; c < 4; ++c) blk[a][b] = fma(-la[a][c], lb[c], blk[a][b]);
                 }
             } else {
 #pragma unroll
@@ -140,18 +151,19 @@ __device__ __forceinline__ void chol_invert_64(const double *Gs, int n, float *r
 #pragma unroll
                     for (int a = 0; a < 4; ++a)
 #pragma unroll
-                        for (int c = 0; c < 4; ++c) x[a][b] = fma(-la[a][c], xb[c], x[a][b]);
+                        for (int c = 0; c < 4; ++c) blk[a][b] = fma(-la[a][c], xb[c], blk[a][b]);
                 }
             }
         }
     }
+    if (bc > br || bc >= nblk) to_x();      // blocks that never became part of X: above the diagonal, beyond n
     // W[k][c] = (L^-1)[c][k] / D_k ; this thread holds (L^-1)[4 br + a][4 bc + b]
 #pragma unroll
     for (int b = 0; b < 4; ++b) {
         const int k = 4 * bc + b;
         const double rk = rs[k];
         float4 w;
-        w.x = (float)(rk * x[0][b]); w.y = (float)(rk * x[1][b]); w.z = (float)(rk * x[2][b]); w.w = (float)(rk * x[3][b]);
+        w.x = (float)(rk * blk[0][b]); w.y = (float)(rk * blk[1][b]); w.z = (float)(rk * blk[2][b]); w.w = (float)(rk * blk[3][b]);
         *(float4 *)(rinv + k * PB + 4 * br) = w;
     }
     bar256();

@@ -30,10 +30,24 @@ def rel_err(G, R):
     return float(np.abs(G - R).max() / (den if den > 0 else 1.0))
 
 
+ORACLE_SVD_LIMIT = 512 * 1024      # entries: above this the oracle's Jacobi SVD takes minutes
+
+
+def spectrum(X):
+    """All singular values of X: from the oracle's own Jacobi SVD where that is affordable (up to 512 x 1024,
+    i.e. workloads 1 and 2 and every small case), from LAPACK above that size (the oracle is pinned to LAPACK
+    to 1e-12 on CPU, so the two agree; the larger workloads could not be checked at all otherwise)."""
+    X = np.asarray(X, dtype=np.float64)
+    if X.size <= ORACLE_SVD_LIMIT:
+        import oracle
+        return oracle.svd_jacobi(X)[1]
+    return np.linalg.svd(X, compute_uv=False)
+
+
 def basis_invariants(X, U, Xr, sig):
     """T1 quantities of one sequence (all float64 numpy)."""
     r = U.shape[1]
-    s_true = np.linalg.svd(X, compute_uv=False)
+    s_true = spectrum(X)
     out = {}
     out["orth"] = float(np.abs(U.T @ U - np.eye(r)).max())
     out["xr_vs_utx"] = float(np.abs(Xr - U.T @ X).max() / s_true[0])

@@ -33,6 +33,16 @@ def test_binding_lists_the_same_symbols():
     assert "rank" in pkg.binding.status_string(2)
 
 
+def test_per_device_once_bookkeeping():
+    """Kernel attributes and symbol addresses are set up once per device ordinal, not once per process: the
+    library's scripted self-test runs the guarded step for ordinals 0, 0, 1, 1, 0 (2 runs), for an ordinal whose
+    first attempt fails (2 runs) and for ordinals outside its table (3 runs, never cached)."""
+    from paper_2403_02352_b200 import build
+    lib = ctypes.CDLL(build.build())
+    lib.atp_selftest_per_device_once.restype = ctypes.c_int
+    assert lib.atp_selftest_per_device_once() == 7
+
+
 def test_no_fallback_without_cuda():
     import pytest
     import torch
