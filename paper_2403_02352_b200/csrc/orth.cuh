@@ -194,9 +194,11 @@ orth_persistent_kernel(const __grid_constant__ Batch batch, int reps, uint64_t s
                 barrier();
                 if (!alive) break;
                 // ---- sum the partials in order: C[jb]
-                for (int jb = rank; jb < nj; jb += ncta)
-                    for (int e = tid; e < 4096; e += NT)
+                for (int it = rank; it < nj * 4; it += ncta) {               // a quarter tile per job
+                    const int jb = it >> 2;
+                    for (int e = (it & 3) * 1024 + tid; e < ((it & 3) + 1) * 1024; e += NT)
                         sq.C[(size_t)jb * 4096 + e] = ordered_sum(sq.Cpart + (size_t)jb * KS * 4096 + e, 4096, KS);
+                }
                 barrier();
                 if (!alive) break;
                 // ---- update: partial D[t][g] = sum over a range of jb of Q[t][:, jb] C[jb]
@@ -234,12 +236,23 @@ orth_persistent_kernel(const __grid_constant__ Batch batch, int reps, uint64_t s
                 load_tile(sA, LDA, sq.M + (size_t)t * 64 * ld + j0, ld, rv, w, vec);
                 __syncthreads();
                 if (nj > 0) {
-                    for (int e = tid; e < 4096; e += NT) {
-                        const int r = e >> 6, c = e & 63;
-                        const float s = ordered_sum(sq.Dpart + (size_t)t * G * 4096 + e, 4096, G);
-                        const float v = sA[r * LDA + c] - s;
-                        sA[r * LDA + c] = (r < rv && c < w) ? v : 0.f;
-                        if (r < rv && c < w) sq.M[((size_t)t * 64 + r) * ld + j0 + c] = v;
+                    for (int e0 = tid; e0 < 4096; e0 += 4 * NT) {                // four elements, 4 G loads in flight
+                        float s[4] = {0.f, 0.f, 0.f, 0.f};
+                        const float *dp = sq.Dpart + (size_t)t * G * 4096 + e0;
+                        for (int g = 0; g < G; ++g) {
+                            float x[4];
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) x[q] = __ldcg(dp + (size_t)g * 4096 + q * NT);
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) s[q] += x[q];
+                        }
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const int e = e0 + q * NT, r = e >> 6, c = e & 63;
+                            const float v = sA[r * LDA + c] - s[q];
+                            sA[r * LDA + c] = (r < rv && c < w) ? v : 0.f;
+                            if (r < rv && c < w) sq.M[((size_t)t * 64 + r) * ld + j0 + c] = v;
+                        }
                     }
                     __syncthreads();
                 }
