@@ -24,7 +24,11 @@
  *   oracle_alternating_svd   Algorithm 1 (appendix B), the paper's own approximate extraction
  *   oracle_svd_entropy       Eq. 4
  *
- * Parity status: every function here is pinned by tests/test_oracle_pins.py
+ *   oracle_project_rows      X' = U^T X (Sec. 4.2), the product inside oracle_principal_basis
+ *   oracle_svd_jacobi_capped oracle_svd_jacobi stopped after a given number of rounds (timing aid only)
+ *
+ * Parity status: every function here is pinned by tests/test_oracle_pins.py and
+ * tests/test_oracle_layer_pins.py
  * (closed forms, planted spectra, Eckart-Young, reduction to textbook
  * attention, brute force on tiny inputs, LAPACK cross-check). The one value
  * that stays unpinned end to end is O on inputs whose cut r falls inside a

@@ -1,12 +1,14 @@
 // atp_principal_basis: top-r left singular vectors U_r and X_r = U_r^T X (Eq. 3, Eq. 5, Sec. 4.2),
 // i.e. the minimiser of Eq. 9, computed as
 //   1. randomised range finder  Y = X Omega  (+-1 test matrix) with subspace (power) iterations
-//      Z = orth(X^T Y), Y = orth(X Z), each orthonormalised by block Gram-Schmidt (two passes)
-//      with a Cholesky-QR of every 64-column panel (Gram matrix and Cholesky factor in fp64);
-//   2. projection  B = Y^T X  (r~ x d);
-//   3. one-sided block Jacobi on the rows of B (pairs of 32-row blocks, round-robin order): the
-//      rotated rows are sigma_i v_i^T and the accumulated rotations turn Y into singular vectors;
-//   4. sort by sigma, fix signs, write U_r = Y W and X_r.
+//      Z = X^T Y, Y = orth(X Z); every iterate is orthonormalised by one persistent block Gram-Schmidt
+//      kernel (orth.cuh: Cholesky-QR of every 64-column panel, Gram matrix and factor in fp64);
+//   2. projection  B^T = X^T Y  (d x r~) and its Gram matrix G = B B^T (r~ x r~);
+//   3. two-sided block Jacobi on G in two passes, one persistent kernel each (jacobi3.cuh): the
+//      accumulated rotation turns Y into singular vectors and the rows of B into sigma_i v_i^T
+//      (opts->jacobi_block = 1: one-sided block Jacobi on the rows of B instead, a launch chain);
+//   4. sort by sigma, fix signs, write U_r = Y W and X_r = W^T B.
+// This file holds the host flow, the finishing kernels and the one-sided variant.
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
 #include "jacobi3.cuh"
