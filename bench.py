@@ -94,6 +94,11 @@ class ClockSampler:
 
 ALT_INNER = 2        # rounds per component of Algorithm 1, as the paper runs it
 
+# DRAM bytes (read + write) of one launch of the dominant kernels, from one ncu pass on the same command
+# (profiles/ncu_metrics_llama7b_bf16_r2048.md); other workloads / kernels: no capture, null.
+NCU_DRAM_BYTES_PER_LAUNCH = {("llama7b_bf16", 2048, "jacobi_persistent"): 33.4e6,
+                             ("llama7b_bf16", 2048, "orth_persistent"): 68.6e6}
+
 
 def alt_start_vectors(w, seed):
     """The Gaussian start vectors of Algorithm 1 (one row per component), part of the seeded input."""
@@ -450,7 +455,7 @@ def main():
     if in_extraction and ext_bytes > 0:
         achieved = ext_bytes / dom_s / 1e9
         roofline = {"kernel": dom_name, "bound": "hbm", "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s",
-                    "frac": achieved / pk["hbm_gbs"], "traffic": None,
+                    "frac": achieved / pk["hbm_gbs"], "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get((args.workload, ranks[0], dom_name)),
                     "tensor_frac": ext_flops / dom_s / 1e12 / pk["bf16_tflops"],
                     "work": "algorithmic bytes / flops of the extraction calls of a step over this kernel's time per step"}
     else:
