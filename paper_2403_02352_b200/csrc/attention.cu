@@ -164,7 +164,7 @@ static void plan_attn(Arena &ar, int64_t tr, int64_t tl, int64_t dp, int64_t nse
     p.Vb = ar.take<__nv_bfloat16>((size_t)tr * align_up((size_t)dp, 8));
     p.Qh = ar.take<__nv_bfloat16>((size_t)tl * align_up((size_t)dp, 8));
     p.Ql = ar.take<__nv_bfloat16>((size_t)tl * align_up((size_t)dp, 8));
-    p.nrm = ar.take<float>((size_t)nseq * dp + (size_t)(tr / 128 + nseq) * dp);    // per head norms: queries, key blocks
+    p.nrm = ar.take<float>((size_t)(tl / 128 + nseq) * dp + (size_t)(tr / 128 + nseq) * dp);    // per head norms: query tiles, key blocks
 }
 size_t attention_workspace_bytes(const std::vector<SeqDims> &seqs, int64_t dp)
 {
@@ -219,8 +219,8 @@ static atp_status attention_impl(atp_ctx *ctx, const atp_mat *X, const atp_mat *
             float *nrm = pl.nrm;
             for (auto &s : seqs)
                 if (s.L > 0) {
-                    float *qmax = nrm, *kmax = nrm + heads;
-                    nrm += heads + (size_t)heads * ceil_div(s.r, 128);
+                    float *qmax = nrm, *kmax = nrm + (size_t)heads * ceil_div(s.L, 128);
+                    nrm += (size_t)heads * (ceil_div(s.L, 128) + ceil_div(s.r, 128));
                     hs.push_back(atc::HostSeq{pl.Qh + (size_t)s.row0 * ldq, pl.Ql + (size_t)s.row0 * ldq, pl.Kh + (size_t)s.rank0 * ldq,
                                               pl.Kl + (size_t)s.rank0 * ldq, pl.Vb + (size_t)s.rank0 * ldq,
                                               (T *)O->data + (size_t)s.row0 * O->ld, s.L, s.r, ldq, ldq, (int)O->ld, dp, qmax, kmax});
@@ -322,8 +322,8 @@ static atp_status attention_impl(atp_ctx *ctx, const atp_mat *X, const atp_mat *
             float *nrm = pl.nrm;
             for (auto &sq : seqs)
                 if (sq.L > 0) {
-                    float *qmax = nrm, *kmax = nrm + heads;
-                    nrm += heads + (size_t)heads * ceil_div(sq.r, 128);
+                    float *qmax = nrm, *kmax = nrm + (size_t)heads * ceil_div(sq.L, 128);
+                    nrm += (size_t)heads * (ceil_div(sq.L, 128) + ceil_div(sq.r, 128));
                     hs.push_back(atc::HostSeq{pl.Qh + (size_t)sq.row0 * ldq, pl.Ql + (size_t)sq.row0 * ldq, pl.Kh + (size_t)sq.rank0 * ldq,
                                               pl.Kl + (size_t)sq.rank0 * ldq, pl.Vb + (size_t)sq.rank0 * ldq,
                                               (T *)O->data + (size_t)sq.row0 * O->ld, sq.L, sq.r, ldq, ldq, (int)O->ld, dp, qmax, kmax});
