@@ -17,7 +17,7 @@
 
 constexpr int PB = 64;            // orthonormalisation panel width
 
-__device__ __forceinline__ void chol_invert_64(const double *Gs, int n, float *rinv, int *flags)
+__device__ __noinline__ void chol_invert_64(const double *Gs, int n, float *rinv, int *flags)
 {
     __shared__ double rs[PB];          // 1 / sqrt(diagonal of the Gram matrix)
     __shared__ double lcol4[PB][4];    // block column jb of L (rows below the diagonal block)
@@ -125,33 +125,19 @@ __device__ __forceinline__ void chol_invert_64(const double *Gs, int n, float *r
         }
         bar256();
         if (br > jb && bc <= br) {
-            // 3. trailing update
-            double la[4][4];
+            // 3. trailing update (operands re-read from shared memory per row: registers are scarce here)
+            const bool gpart = bc > jb;
 #pragma unroll
-            for (int a = 0; a < 4; ++a)
+            for (int b = 0; b < 4; ++b) {
+                double rb[4];
 #pragma unroll
-                for (int c = 0; c < 4; ++c) la[a][c] = lcol4[4 * br + a][c];
-            if (bc > jb) {
+                for (int c = 0; c < 4; ++c) rb[c] = gpart ? lcol4[4 * bc + b][c] : xrow4[c][4 * bc + b];
 #pragma unroll
-                for (int b = 0; b < 4; ++b) {
-                    double lb[4];
+                for (int a = 0; a < 4; ++a) {
+                    double acc = blk[a][b];
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) lb[c] = lcol4[4 * bc + b][c];
-#pragma unroll
-                    for (int a = 0; a < 4; ++a)
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) blk[a][b] = fma(-la[a][c], lb[c], blk[a][b]);
-                }
-            } else {
-#pragma unroll
-                for (int b = 0; b < 4; ++b) {
-                    double xb[4];
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) xb[c] = xrow4[c][4 * bc + b];
-#pragma unroll
-                    for (int a = 0; a < 4; ++a)
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) blk[a][b] = fma(-la[a][c], xb[c], blk[a][b]);
+                    for (int c = 0; c < 4; ++c) acc = fma(-lcol4[4 * br + a][c], rb[c], acc);
+                    blk[a][b] = acc;
                 }
             }
         }
