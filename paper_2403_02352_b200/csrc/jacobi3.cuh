@@ -34,9 +34,10 @@ constexpr int MAXSEQ = 32;        // sequences per launch
 constexpr unsigned SPIN_LIMIT = 1u << 22;
 
 struct Seq {
-    float *G, *Wt, *Vbuf;         // G, Wt: np x np (ld = np); Vbuf: 2 x npairs x 64 x 64 (by step parity)
+    float *G, *G2, *Wt, *Vbuf;    // G, G2, Wt: np x np (ld = np); G2: scratch, the update of a step reads one
+                                  // copy of the matrix and writes the other; Vbuf: 2 x npairs x 64 x 64 (by
+                                  // step parity)
     int *vflag;                   // 2 x npairs: the pair rotated in this step
-    unsigned *done;               // per block (p, q >= p) of G: number of the last step that updated it
     unsigned *sync;               // 64 words. [0]: arrivals at the group barrier (monotonic); [32]: last
                                   // barrier completed; [1..4]: largest scaled off-diagonal entry of a
                                   // sweep, slot sweep % 4; [5]: sweeps used; [16..17]: work tickets of the update, by step parity
@@ -45,9 +46,10 @@ struct Seq {
 };
 struct Batch { Seq s[MAXSEQ]; int count; };
 
-// Bytes of dynamic shared memory: four 64 x LDA tiles (pivot phase: two copies of A and of V;
-// apply phase: Vt_p, Vt_q, T and the G block at stride LDB).
-constexpr size_t SMEM_BYTES = (size_t)(3 * BLK * LDA + BLK * LDB) * sizeof(float);
+// Bytes of dynamic shared memory: four tile slots of 64 x LDB floats (pivot phase: the old blocks and the
+// transforms the pivot block is formed from, then A and Vt; apply phase: Vt_p, Vt_q, T and the G block).
+constexpr int SLOT = BLK * LDB;
+constexpr size_t SMEM_BYTES = (size_t)4 * SLOT * sizeof(float);
 
 __device__ __forceinline__ void rr_pair(int nb, int step, int t, int &I, int &J)
 {
@@ -216,24 +218,30 @@ __device__ void cross_phase(float *As, float *Vs, float2 *rot, float4 *xch, int 
 // global row / column of local index l of the pair (I, J)
 __device__ __forceinline__ int glob_of_loc(int I, int J, int l) { return (l < JB ? I : J) * JB + (l & (JB - 1)); }
 
-// Rotates the 64 x 64 pivot block of the pair (I, J) on chip and publishes the accumulated row
-// transform Vt (new rows = Vt * old rows, logical order) to vout. cross_only: the 32 rounds that pair
-// the two blocks' rows; otherwise all 63 rounds. Returns the largest scaled off-diagonal entry found
-// in the block before rotating (block-uniform); when it is <= tol_rot nothing is rotated or published.
-__device__ float pivot_solve(float *sm, const float *G, int np, int I, int J, bool cross_only, float tol_rot,
-                             float *vout, bool &rotated)
+// Copies the 64 x 64 pivot block of the pair (I, J) from G to the logical copy As (stride LDP).
+__device__ void pivot_load(float *sm, const float *G, int np, int I, int J)
+{
+    float *As = sm;
+    for (int f = threadIdx.x; f < BLK * (BLK / 4); f += NT) {
+        const int li = f >> 4, lj = (f & 15) * 4;
+        const float4 v = __ldcg((const float4 *)(G + (size_t)glob_of_loc(I, J, li) * np + glob_of_loc(I, J, lj)));
+        float *dst = As + li * LDP + lj;
+        dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
+    }
+}
+
+// Rotates the 64 x 64 pivot block held in As = sm (stride LDP, complete before the call: the routine starts with
+// a block barrier) and publishes the accumulated row transform Vt (new rows = Vt * old rows, logical order) to
+// vout. cross_only: the 32 rounds that pair the two blocks' rows; otherwise all 63 rounds. Returns the largest
+// scaled off-diagonal entry found in the block before rotating (block-uniform); when it is <= tol_rot nothing is
+// rotated or published.
+__device__ float pivot_rotate(float *sm, bool cross_only, float tol_rot, float *vout, bool &rotated)
 {
     __shared__ float red[NT / 32];
     __shared__ float2 rot[64];
     __shared__ float4 xch[NT];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     float *As = sm, *Vs = sm + BLK * LDP;
-    for (int f = tid; f < BLK * (BLK / 4); f += NT) {
-        const int li = f >> 4, lj = (f & 15) * 4;
-        const float4 v = __ldcg((const float4 *)(G + (size_t)glob_of_loc(I, J, li) * np + glob_of_loc(I, J, lj)));
-        float *dst = As + li * LDP + lj;
-        dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
-    }
     for (int e = tid; e < BLK * BLK; e += NT) Vs[(e >> 6) * LDP + (e & 63)] = ((e >> 6) == (e & 63)) ? 1.f : 0.f;
     __syncthreads();
     float mo = 0.f;
@@ -380,10 +388,84 @@ __device__ __forceinline__ void product64_fma(const float *As, const float *Bs, 
     }
 }
 
-// One block of the update. Items [0, ntri): block (p, q >= p) of G, enumerated row by row; items
-// [ntri, ntri + npairs * nw): rows of pair p of Wt, column chunk of 64.
+// Forms, on chip, the pivot block that a pair of the NEXT step will have once the current step's update is done,
+// from the state before that update. The pair's first block sits in half h1 of the current pair p1, its second in
+// half h2 of the current pair p2. With W1 / W2 the 32 rows of Vt_p1 / Vt_p2 that produce those blocks (rows of
+// the identity where the pair was not rotated: f1 / f2 = 0) and X_ab the old blocks between the pairs a and b,
+//   N = [ W1 X11 W1^T   W1 X12 W2^T ]
+//       [   (mirror)    W2 X22 W2^T ]
+// in three 64^3 products: [W1 X11; W2 X22] and W1 X12 first, then the multiplication by [W1; W2]^T from the
+// right. The result lands in As = sm (stride LDP). So the chain of pivot solves never waits for the update.
 template <bool TENSOR>
-__device__ void apply_item(float *sm, const Seq &sq, const float *Vbuf, const int *vflag, int step, int idx, int npairs, int ntri, int nw)
+__device__ void pivot_form(float *sm, const Seq &sq, const float *Gsrc, const float *Vcur, int step, int p1, int h1, int f1, int p2, int h2, int f2)
+{
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+    float *Wc = sm, *S1 = sm + SLOT, *S2 = sm + 2 * SLOT, *S3 = sm + 3 * SLOT;
+    int I1, J1, I2, J2;
+    rr_pair(sq.nb, step, p1, I1, J1);
+    rr_pair(sq.nb, step, p2, I2, J2);
+    const int np = sq.np;
+    for (int f = tid; f < BLK * (BLK / 4); f += NT) {
+        const int i = f >> 4, c = (f & 15) * 4;
+        const bool up = i < JB;
+        const int row = (up ? h1 : h2) * JB + (i & (JB - 1));
+        float4 w;
+        if (up ? f1 : f2) w = __ldcg((const float4 *)(Vcur + (size_t)(up ? p1 : p2) * BLK * BLK + row * BLK + c));
+        else w = make_float4(row == c ? 1.f : 0.f, row == c + 1 ? 1.f : 0.f, row == c + 2 ? 1.f : 0.f, row == c + 3 ? 1.f : 0.f);
+        *(float4 *)(Wc + i * LDA + c) = w;
+        const size_t r1 = (size_t)glob_of_loc(I1, J1, i) * np, r2 = (size_t)glob_of_loc(I2, J2, i) * np;
+        *(float4 *)(S1 + i * LDB + c) = __ldcg((const float4 *)(Gsrc + r1 + glob_of_loc(I1, J1, c)));
+        *(float4 *)(S2 + i * LDB + c) = __ldcg((const float4 *)(Gsrc + r2 + glob_of_loc(I2, J2, c)));
+        *(float4 *)(S3 + i * LDB + c) = __ldcg((const float4 *)(Gsrc + r1 + glob_of_loc(I2, J2, c)));
+    }
+    __syncthreads();
+    const int m0 = (warp & 3) * 16, n0 = (warp >> 2) * 32;
+    const bool up = m0 < JB;
+    const bool on_tensor = TENSOR;
+    float accd[4][4], acco[4][4];
+    if (on_tensor) product64<false>(Wc, up ? S1 : S2, LDB, m0, n0, accd);
+    else product64_fma<false>(Wc, up ? S1 : S2, LDB, m0, n0, accd);
+    if (up) {
+        if (on_tensor) product64<false>(Wc, S3, LDB, m0, n0, acco);
+        else product64_fma<false>(Wc, S3, LDB, m0, n0, acco);
+    }
+    __syncthreads();
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) {
+        const int c = n0 + nt * 8 + 2 * t;
+        *(float2 *)(S1 + (m0 + g) * LDA + c) = make_float2(accd[nt][0], accd[nt][1]);
+        *(float2 *)(S1 + (m0 + g + 8) * LDA + c) = make_float2(accd[nt][2], accd[nt][3]);
+        if (up) {
+            *(float2 *)(S2 + (m0 + g) * LDA + c) = make_float2(acco[nt][0], acco[nt][1]);
+            *(float2 *)(S2 + (m0 + g + 8) * LDA + c) = make_float2(acco[nt][2], acco[nt][3]);
+        }
+    }
+    __syncthreads();
+    const bool lower_left = !up && n0 == 0;                     // mirror of the upper right part
+    if (!lower_left) {
+        const float *Ta = (up && n0 != 0) ? S2 : S1;
+        if (on_tensor) product64<true>(Ta, Wc, LDA, m0, n0, accd);
+        else product64_fma<true>(Ta, Wc, LDA, m0, n0, accd);
+    }
+    __syncthreads();
+    float *As = sm;
+    if (!lower_left) {
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int i = m0 + g + (e >> 1) * 8, j = n0 + nt * 8 + 2 * t + (e & 1);
+                As[i * LDP + j] = accd[nt][e];
+                if (up && n0 != 0) As[j * LDP + i] = accd[nt][e];
+            }
+    }
+}
+
+// One block of the update. Items [0, ntri): block (p, q >= p) of G, enumerated row by row, read from Gsrc and
+// written (with its mirror) to Gdst, also when neither pair was rotated; items [ntri, ntri + npairs * nw): rows
+// of pair p of Wt, column chunk of 64, in place.
+template <bool TENSOR>
+__device__ void apply_item(float *sm, const Seq &sq, const float *Gsrc, float *Gdst, const float *Vbuf, const int *vflag, int step, int idx, int npairs, int ntri, int nw)
 {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     const bool gblock = idx < ntri;
@@ -397,13 +479,24 @@ __device__ void apply_item(float *sm, const Seq &sq, const float *Vbuf, const in
     }
     const int fp = __ldcg(vflag + p);
     const int fq = gblock ? __ldcg(vflag + q) : 0;
-    if (!fp && !fq) return;
+    if (!fp && !fq && !gblock) return;
     float *Vp = sm, *Vq = sm + BLK * LDA, *Tm = sm + 2 * BLK * LDA, *Bk = sm + 3 * BLK * LDA;
     int Ip, Jp, Iq = 0, Jq = 0;
     rr_pair(sq.nb, step, p, Ip, Jp);
     if (gblock) rr_pair(sq.nb, step, q, Iq, Jq);
     const int np = sq.np;
-    float *mat = gblock ? sq.G : sq.Wt;
+    if (!fp && !fq) {                                            // unchanged block: both mirror copies move over
+        for (int f = tid; f < BLK * (BLK / 4); f += NT) {
+            const int i = f >> 4, c = (f & 15) * 4;
+            const size_t a = (size_t)glob_of_loc(Ip, Jp, i) * np + glob_of_loc(Iq, Jq, c);
+            const size_t b = (size_t)glob_of_loc(Iq, Jq, i) * np + glob_of_loc(Ip, Jp, c);
+            *(float4 *)(Gdst + a) = __ldcg((const float4 *)(Gsrc + a));
+            if (q != p) *(float4 *)(Gdst + b) = __ldcg((const float4 *)(Gsrc + b));
+        }
+        return;
+    }
+    const float *msrc = gblock ? Gsrc : sq.Wt;
+    float *mat = gblock ? Gdst : sq.Wt;
     auto gcol = [&](int c) -> int { return gblock ? glob_of_loc(Iq, Jq, c) : chunk * BLK + c; };
     // the block goes to the B tile when a row transform comes first, else straight to the T tile
     float *blk_dst = fp ? Bk : Tm;
@@ -412,13 +505,14 @@ __device__ void apply_item(float *sm, const Seq &sq, const float *Vbuf, const in
         const int i = f >> 4, c = (f & 15) * 4;
         if (fp) *(float4 *)(Vp + i * LDA + c) = __ldcg((const float4 *)(Vbuf + (size_t)p * BLK * BLK + i * BLK + c));
         if (fq) *(float4 *)(Vq + i * LDA + c) = __ldcg((const float4 *)(Vbuf + (size_t)q * BLK * BLK + i * BLK + c));
-        *(float4 *)(blk_dst + i * blk_ld + c) = __ldcg((const float4 *)(mat + (size_t)glob_of_loc(Ip, Jp, i) * np + gcol(c)));
+        *(float4 *)(blk_dst + i * blk_ld + c) = __ldcg((const float4 *)(msrc + (size_t)glob_of_loc(Ip, Jp, i) * np + gcol(c)));
     }
     __syncthreads();
     const int m0 = (warp & 3) * 16, n0 = (warp >> 2) * 32;
+    const bool on_tensor = TENSOR;
     float acc[4][4];
     if (fp) {
-        if (TENSOR) product64<false>(Vp, Bk, LDB, m0, n0, acc);  // T = Vt_p * block
+        if (on_tensor) product64<false>(Vp, Bk, LDB, m0, n0, acc);  // T = Vt_p * block
         else product64_fma<false>(Vp, Bk, LDB, m0, n0, acc);
         if (fq) {
 #pragma unroll
@@ -431,7 +525,7 @@ __device__ void apply_item(float *sm, const Seq &sq, const float *Vbuf, const in
         }
     }
     if (fq) {                                                    // out = T * Vt_q^T
-        if (TENSOR) product64<true>(Tm, Vq, LDA, m0, n0, acc);
+        if (on_tensor) product64<true>(Tm, Vq, LDA, m0, n0, acc);
         else product64_fma<true>(Tm, Vq, LDA, m0, n0, acc);
     }
     const int gr0 = glob_of_loc(Ip, Jp, m0 + g), gr1 = glob_of_loc(Ip, Jp, m0 + g + 8);
@@ -449,20 +543,16 @@ __device__ void apply_item(float *sm, const Seq &sq, const float *Vbuf, const in
 }
 
 // ---- the kernel --------------------------------------------------------------------------------
-// Schedule of a group. The pivot blocks of step s+1 lie inside 3 blocks of the update of step s (the
-// two diagonal blocks of the pairs their rows come from, and the block that couples those pairs).
-// Every step therefore runs
-//   1. the "critical" blocks of its update first (all diagonal blocks and the coupling blocks of the
-//      next step's pairs), spread over the whole group, each marking itself done;
-//   2. then, side by side, the pivot solves of the NEXT step (each waits for its 3 blocks) and the
-//      rest of the update, handed out by a ticket counter so that the pivot CTAs join in when they
-//      are through;
-//   3. one group barrier.
-// Vt and the rotated-flags are double buffered by step parity, because step s+1's pivots publish while
-// step s's update still reads.
+// Schedule of a group. The pivot block of a pair of step s+1 is a function of the matrix before the update of
+// step s and of two transforms of step s (pivot_form), all of which are complete at the barrier that ends step
+// s-1. Every step therefore runs, side by side,
+//   1. the pivot solves of the NEXT step (a few CTAs; this chain of rotation rounds is the critical path), and
+//   2. the update of this step, its blocks handed out by a ticket counter so that the pivot CTAs join in when
+//      they are through,
+// followed by one group barrier. Vt and the rotated-flags are double buffered by step parity, because the
+// pivots of step s+1 publish while the update of step s still reads.
 // status[0]: sticky device status word of the context; status[1]: abort flag of bounded waits.
 constexpr int MAXPAIRS = 72;                  // np <= 4608
-__device__ __forceinline__ int tri_index(int p, int q, int npairs) { return p * npairs - p * (p - 1) / 2 + (q - p); }
 
 template <bool TENSOR>
 __global__ void __launch_bounds__(NT, 2)
@@ -470,10 +560,8 @@ jacobi_persistent_kernel(const __grid_constant__ Batch batch, float tol_conv, fl
                          int raise_not_converged, int *status)
 {
     extern __shared__ __align__(16) float j3sm[];
-    __shared__ short pair_of[2 * MAXPAIRS];
-    __shared__ unsigned char is_crit[MAXPAIRS * (MAXPAIRS + 1) / 2];
-    __shared__ short crit_list[2 * MAXPAIRS];
-    __shared__ int ncrit_s, ticket_s, wait_ok_s;
+    __shared__ short pair_of[2 * MAXPAIRS];       // block -> 2 * pair + half, for the current step
+    __shared__ int ticket_s;
     int si = 0;
 #pragma unroll 1
     for (int i = 1; i < batch.count; ++i) if ((int)blockIdx.x >= batch.s[i].cta0) si = i;
@@ -486,12 +574,10 @@ jacobi_persistent_kernel(const __grid_constant__ Batch batch, float tol_conv, fl
     unsigned gen = 0, gstep = 0;
     bool converged = false, alive = true;
 
-    auto pivot_item = [&](int sweep, int step, int pr, int par) {
-        int I, J;
-        rr_pair(sq.nb, step, pr, I, J);
+    // rotates the block held in shared memory for pair pr of (sweep, step); publishes to parity par
+    auto pivot_finish = [&](int sweep, int step, int pr, int par) {
         bool rotated;
-        const float mo = pivot_solve(j3sm, sq.G, sq.np, I, J, step > 0, tol_rot,
-                                     sq.Vbuf + ((size_t)par * npairs + pr) * BLK * BLK, rotated);
+        const float mo = pivot_rotate(j3sm, step > 0, tol_rot, sq.Vbuf + ((size_t)par * npairs + pr) * BLK * BLK, rotated);
         if (tid == 0) {
             sq.vflag[par * npairs + pr] = rotated ? 1 : 0;
             atomicMax(sq.sync + 1 + sweep % 4, __float_as_uint(mo));
@@ -499,8 +585,13 @@ jacobi_persistent_kernel(const __grid_constant__ Batch batch, float tol_conv, fl
         __syncthreads();
     };
 
-    // prologue: the pivots of the very first step
-    for (int pr = rank; pr < npairs; pr += sq.ncta) pivot_item(0, 0, pr, 0);
+    // prologue: the pivots of the very first step, straight from G
+    for (int pr = rank; pr < npairs; pr += sq.ncta) {
+        int I, J;
+        rr_pair(sq.nb, 0, pr, I, J);
+        pivot_load(j3sm, sq.G, sq.np, I, J);
+        pivot_finish(0, 0, pr, 0);
+    }
     alive = group_barrier(sq.sync, ++gen, (unsigned)sq.ncta, abort_flag);
 
     int sweep = 0;
@@ -512,83 +603,50 @@ jacobi_persistent_kernel(const __grid_constant__ Batch batch, float tol_conv, fl
             const int nstep = step + 1 == nsteps ? 0 : step + 1, nsweep = sweep + (step + 1 == nsteps ? 1 : 0);
             const float *Vcur = sq.Vbuf + (size_t)par * npairs * BLK * BLK;
             const int *fcur = sq.vflag + par * npairs;
-            // tables of this step: block -> pair, critical blocks
-            if (tid < npairs) {
-                int I, J;
-                rr_pair(sq.nb, step, tid, I, J);
-                pair_of[I] = (short)tid; pair_of[J] = (short)tid;
-            }
-            for (int e = tid; e < ntri; e += NT) is_crit[e] = 0;
-            __syncthreads();
-            if (tid == 0) {
-                int nc = 0;
-                for (int p = 0; p < npairs; ++p) { const int idx = tri_index(p, p, npairs); is_crit[idx] = 1; crit_list[nc++] = (short)idx; }
-                if (has_next)
-                    for (int t = 0; t < npairs; ++t) {
-                        int I2, J2;
-                        rr_pair(sq.nb, nstep, t, I2, J2);
-                        const int p1 = pair_of[I2], p2 = pair_of[J2];
-                        if (p1 != p2) {
-                            const int idx = tri_index(min(p1, p2), max(p1, p2), npairs);
-                            if (!is_crit[idx]) { is_crit[idx] = 1; crit_list[nc++] = (short)idx; }
-                        }
-                    }
-                ncrit_s = nc;
-                if (rank == 0) sq.sync[16 + (par ^ 1)] = 0u;          // tickets of the next step
-            }
-            __syncthreads();
-            // 1. critical blocks
-            for (int k = rank; k < ncrit_s; k += sq.ncta) {
-                const int idx = crit_list[k];
-                apply_item<TENSOR>(j3sm, sq, Vcur, fcur, step, idx, npairs, ntri, nw);
-                if (tid == 0) { __threadfence(); *(volatile unsigned *)(sq.done + idx) = gstep + 1u; }
-            }
-            // 2a. pivots of the next step
-            if (has_next)
-                for (int pr = rank; pr < npairs && alive; pr += sq.ncta) {
-                    if (tid == 0) {
-                        int I2, J2;
-                        rr_pair(sq.nb, nstep, pr, I2, J2);
-                        const int p1 = pair_of[I2], p2 = pair_of[J2];
-                        const int dep[3] = {tri_index(p1, p1, npairs), tri_index(p2, p2, npairs),
-                                            tri_index(min(p1, p2), max(p1, p2), npairs)};
-                        int ok = 1;
-                        for (int k = 0; k < 3 && ok; ++k) {
-                            ok = 0;
-                            for (unsigned i = 0; i < SPIN_LIMIT; ++i) {
-                                if (*(volatile unsigned *)(sq.done + dep[k]) == gstep + 1u) { ok = 1; break; }
-                                if ((i & 1023u) == 1023u && *(volatile int *)abort_flag) break;
-                            }
-                        }
-                        if (!ok) *(volatile int *)abort_flag = 1;
-                        __threadfence();
-                        wait_ok_s = ok;
-                    }
-                    __syncthreads();
-                    if (!wait_ok_s) { alive = false; break; }
-                    pivot_item(nsweep, nstep, pr, par ^ 1);
+            const float *Gsrc = par ? sq.G2 : sq.G;
+            float *Gdst = par ? sq.G : sq.G2;
+            if (rank == 0 && tid == 0) sq.sync[16 + (par ^ 1)] = 0u;      // tickets of the next step
+            // 1. pivots of the next step
+            if (has_next && rank < npairs) {
+                if (tid < npairs) {
+                    int I, J;
+                    rr_pair(sq.nb, step, tid, I, J);
+                    pair_of[I] = (short)(2 * tid); pair_of[J] = (short)(2 * tid + 1);
                 }
-            // 2b. the rest of the update, by tickets (the next one is requested while a block is processed)
-            if (alive) {
-                if (tid == 0) ticket_s = (int)atomicAdd(sq.sync + 16 + par, 1u);
                 __syncthreads();
-                int t = ticket_s;
-                while (t < total) {
-                    int tn = 0;
-                    if (tid == 0) tn = (int)atomicAdd(sq.sync + 16 + par, 1u);
-                    if (!(t < ntri && is_crit[t])) apply_item<TENSOR>(j3sm, sq, Vcur, fcur, step, t, npairs, ntri, nw);
-                    __syncthreads();
-                    if (tid == 0) ticket_s = tn;
-                    __syncthreads();
-                    t = ticket_s;
+                for (int pr = rank; pr < npairs; pr += sq.ncta) {
+                    int I2, J2;
+                    rr_pair(sq.nb, nstep, pr, I2, J2);
+                    const int p1 = pair_of[I2] >> 1, h1 = pair_of[I2] & 1, p2 = pair_of[J2] >> 1, h2 = pair_of[J2] & 1;
+                    const int f1 = __ldcg(fcur + p1), f2 = __ldcg(fcur + p2);
+                    if (!f1 && !f2) pivot_load(j3sm, Gsrc, sq.np, I2, J2);
+                    else pivot_form<TENSOR>(j3sm, sq, Gsrc, Vcur, step, p1, h1, f1, p2, h2, f2);
+                    pivot_finish(nsweep, nstep, pr, par ^ 1);
                 }
             }
-            // 3.
+            // 2. the update, by tickets (the next one is requested while a block is processed)
+            if (tid == 0) ticket_s = (int)atomicAdd(sq.sync + 16 + par, 1u);
+            __syncthreads();
+            int t = ticket_s;
+            while (t < total) {
+                int tn = 0;
+                if (tid == 0) tn = (int)atomicAdd(sq.sync + 16 + par, 1u);
+                apply_item<TENSOR>(j3sm, sq, Gsrc, Gdst, Vcur, fcur, step, t, npairs, ntri, nw);
+                __syncthreads();
+                if (tid == 0) ticket_s = tn;
+                __syncthreads();
+                t = ticket_s;
+            }
             alive = group_barrier(sq.sync, ++gen, (unsigned)sq.ncta, abort_flag) && alive;
         }
         if (!alive) break;
         const float mo = __uint_as_float(*(volatile unsigned *)(sq.sync + 1 + sweep % 4));
         if (mo <= tol_conv) { converged = true; ++sweep; break; }
+    }
+    if (alive && (gstep & 1u)) {                                  // the last update wrote G2: the result goes back to G
+        const size_t n4 = (size_t)sq.np * sq.np / 4;
+        for (size_t e = (size_t)rank * NT + tid; e < n4; e += (size_t)sq.ncta * NT)
+            ((float4 *)sq.G)[e] = __ldcg((const float4 *)sq.G2 + e);
     }
     if (rank == 0 && tid == 0) {
         if (!alive) raise_status(status, ATP_ERR_TIMEOUT);
@@ -613,8 +671,6 @@ __global__ void init_kernel(const __grid_constant__ Batch batch, int *status)
     if (__syncthreads_or(bad) && threadIdx.x == 0) raise_status(status, ATP_ERR_RANGE);
     if (blockIdx.x == 0 && sq.np > 0) {
         if (threadIdx.x < 64) sq.sync[threadIdx.x] = 0u;
-        const int npairs = sq.nb / 2;
-        for (int e = threadIdx.x; e < npairs * (npairs + 1) / 2; e += blockDim.x) sq.done[e] = 0u;
     }
 }
 
