@@ -269,11 +269,13 @@ __device__ float pivot_rotate(float *sm, bool cross_only, float tol_rot, float *
 }
 
 // ---- apply phase -------------------------------------------------------------------------------
+// x = hi + lo + (less than 2^-21 |x|) with hi and lo in TF32 (low 13 mantissa bits zero): hi is x cut to TF32, lo
+// the remainder cut the same way. Two logic operations and one subtraction; the cvt.rna.tf32 conversion would
+// round instead of cut, but it is a slow-path instruction and bounded the whole product (2997 -> 2273 cycles).
 __device__ __forceinline__ void split_tf32(float x, uint32_t &hi, uint32_t &lo)
 {
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(hi) : "f"(x));
-    const float rest = x - __uint_as_float(hi);
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(lo) : "f"(rest));
+    hi = __float_as_uint(x) & 0xffffe000u;
+    lo = __float_as_uint(x - __uint_as_float(hi)) & 0xffffe000u;
 }
 __device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], const uint32_t (&b)[2])
 {
@@ -461,85 +463,175 @@ __device__ void pivot_form(float *sm, const Seq &sq, const float *Gsrc, const fl
     }
 }
 
-// One block of the update. Items [0, ntri): block (p, q >= p) of G, enumerated row by row, read from Gsrc and
-// written (with its mirror) to Gdst, also when neither pair was rotated; items [ntri, ntri + npairs * nw): rows
-// of pair p of Wt, column chunk of 64, in place.
-template <bool TENSOR>
-__device__ void apply_item(float *sm, const Seq &sq, const float *Gsrc, float *Gdst, const float *Vbuf, const int *vflag, int step, int idx, int npairs, int ntri, int nw)
+// The update of a step is cut into strips. A strip of G: blocks (p, q0 .. q0 + cnt - 1) of the upper triangle,
+// read from Gsrc and written (with their mirrors) to Gdst, also when neither pair was rotated; a strip of Wt: the
+// rows of pair p, column chunks c0 .. c0 + cnt - 1 of 64, in place. Along a strip Vt_p stays in shared memory and
+// the next block is fetched into registers while the current one is multiplied.
+constexpr int SEG_G = 2, SEG_W = 3;
+
+__device__ __forceinline__ void store_tile_acc(float *dst, int ld, int m0, int n0, const float (&acc)[4][4])
 {
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-    const bool gblock = idx < ntri;
-    int p = 0, q = 0, chunk = 0;
-    if (gblock) {
-        while (idx >= npairs - p) { idx -= npairs - p; ++p; }
-        q = p + idx;
-    } else {
-        idx -= ntri;
-        p = idx / nw; chunk = idx - p * nw;
-    }
-    const int fp = __ldcg(vflag + p);
-    const int fq = gblock ? __ldcg(vflag + q) : 0;
-    if (!fp && !fq && !gblock) return;
-    float *Vp = sm, *Vq = sm + BLK * LDA, *Tm = sm + 2 * BLK * LDA, *Bk = sm + 3 * BLK * LDA;
-    int Ip, Jp, Iq = 0, Jq = 0;
-    rr_pair(sq.nb, step, p, Ip, Jp);
-    if (gblock) rr_pair(sq.nb, step, q, Iq, Jq);
-    const int np = sq.np;
-    if (!fp && !fq) {                                            // unchanged block: both mirror copies move over
-        for (int f = tid; f < BLK * (BLK / 4); f += NT) {
-            const int i = f >> 4, c = (f & 15) * 4;
-            const size_t a = (size_t)glob_of_loc(Ip, Jp, i) * np + glob_of_loc(Iq, Jq, c);
-            const size_t b = (size_t)glob_of_loc(Iq, Jq, i) * np + glob_of_loc(Ip, Jp, c);
-            *(float4 *)(Gdst + a) = __ldcg((const float4 *)(Gsrc + a));
-            if (q != p) *(float4 *)(Gdst + b) = __ldcg((const float4 *)(Gsrc + b));
-        }
-        return;
-    }
-    const float *msrc = gblock ? Gsrc : sq.Wt;
-    float *mat = gblock ? Gdst : sq.Wt;
-    auto gcol = [&](int c) -> int { return gblock ? glob_of_loc(Iq, Jq, c) : chunk * BLK + c; };
-    // the block goes to the B tile when a row transform comes first, else straight to the T tile
-    float *blk_dst = fp ? Bk : Tm;
-    const int blk_ld = fp ? LDB : LDA;
-    for (int f = tid; f < BLK * (BLK / 4); f += NT) {
-        const int i = f >> 4, c = (f & 15) * 4;
-        if (fp) *(float4 *)(Vp + i * LDA + c) = __ldcg((const float4 *)(Vbuf + (size_t)p * BLK * BLK + i * BLK + c));
-        if (fq) *(float4 *)(Vq + i * LDA + c) = __ldcg((const float4 *)(Vbuf + (size_t)q * BLK * BLK + i * BLK + c));
-        *(float4 *)(blk_dst + i * blk_ld + c) = __ldcg((const float4 *)(msrc + (size_t)glob_of_loc(Ip, Jp, i) * np + gcol(c)));
-    }
-    __syncthreads();
-    const int m0 = (warp & 3) * 16, n0 = (warp >> 2) * 32;
-    const bool on_tensor = TENSOR;
-    float acc[4][4];
-    if (fp) {
-        if (on_tensor) product64<false>(Vp, Bk, LDB, m0, n0, acc);  // T = Vt_p * block
-        else product64_fma<false>(Vp, Bk, LDB, m0, n0, acc);
-        if (fq) {
-#pragma unroll
-            for (int nt = 0; nt < 4; ++nt) {
-                const int c = n0 + nt * 8 + 2 * t;
-                *(float2 *)(Tm + (m0 + g) * LDA + c) = make_float2(acc[nt][0], acc[nt][1]);
-                *(float2 *)(Tm + (m0 + g + 8) * LDA + c) = make_float2(acc[nt][2], acc[nt][3]);
-            }
-            __syncthreads();
-        }
-    }
-    if (fq) {                                                    // out = T * Vt_q^T
-        if (on_tensor) product64<true>(Tm, Vq, LDA, m0, n0, acc);
-        else product64_fma<true>(Tm, Vq, LDA, m0, n0, acc);
-    }
-    const int gr0 = glob_of_loc(Ip, Jp, m0 + g), gr1 = glob_of_loc(Ip, Jp, m0 + g + 8);
+    const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
 #pragma unroll
     for (int nt = 0; nt < 4; ++nt) {
-        const int gc = gcol(n0 + nt * 8 + 2 * t);                // gc, gc + 1 are contiguous
-        *(float2 *)(mat + (size_t)gr0 * np + gc) = make_float2(acc[nt][0], acc[nt][1]);
-        *(float2 *)(mat + (size_t)gr1 * np + gc) = make_float2(acc[nt][2], acc[nt][3]);
-        if (gblock && q != p) {                                  // mirror block
-            mat[(size_t)gc * np + gr0] = acc[nt][0]; mat[(size_t)(gc + 1) * np + gr0] = acc[nt][1];
-            mat[(size_t)gc * np + gr1] = acc[nt][2]; mat[(size_t)(gc + 1) * np + gr1] = acc[nt][3];
+        const int c = n0 + nt * 8 + 2 * t;
+        *(float2 *)(dst + (m0 + g) * ld + c) = make_float2(acc[nt][0], acc[nt][1]);
+        *(float2 *)(dst + (m0 + g + 8) * ld + c) = make_float2(acc[nt][2], acc[nt][3]);
+    }
+}
+
+template <bool TENSOR>
+__device__ void g_strip(float *sm, const Seq &sq, const float *Gsrc, float *Gdst, const float *Vbuf, const int *vflag, int step, int p, int q0, int cnt)
+{
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+    const int m0 = (warp & 3) * 16, n0 = (warp >> 2) * 32, np = sq.np;
+    float *Vp = sm, *Vq = sm + BLK * LDA, *Tm = sm + 2 * BLK * LDA, *Bk = sm + 3 * BLK * LDA;
+    const int fp = __ldcg(vflag + p);
+    int Ip, Jp;
+    rr_pair(sq.nb, step, p, Ip, Jp);
+    float4 x[4];
+    auto fetch = [&](int q) {
+        int Iq, Jq;
+        rr_pair(sq.nb, step, q, Iq, Jq);
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            const int f = tid + it * NT, i = f >> 4, c = (f & 15) * 4;
+            x[it] = __ldcg((const float4 *)(Gsrc + (size_t)glob_of_loc(Ip, Jp, i) * np + glob_of_loc(Iq, Jq, c)));
+        }
+    };
+    if (fp) {
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            const int f = tid + it * NT, i = f >> 4, c = (f & 15) * 4;
+            *(float4 *)(Vp + i * LDA + c) = __ldcg((const float4 *)(Vbuf + (size_t)p * BLK * BLK + i * BLK + c));
         }
     }
-    __syncthreads();                                             // tiles are reused by the next item
+    fetch(q0);
+    for (int j = 0; j < cnt; ++j) {
+        const int q = q0 + j, fq = __ldcg(vflag + q);
+        int Iq, Jq;
+        rr_pair(sq.nb, step, q, Iq, Jq);
+        if (!fp && !fq) {                                        // unchanged block: both mirror copies move over
+#pragma unroll
+            for (int it = 0; it < 4; ++it) {
+                const int f = tid + it * NT, i = f >> 4, c = (f & 15) * 4;
+                *(float4 *)(Gdst + (size_t)glob_of_loc(Ip, Jp, i) * np + glob_of_loc(Iq, Jq, c)) = x[it];
+                if (q != p) {
+                    const size_t b = (size_t)glob_of_loc(Iq, Jq, i) * np + glob_of_loc(Ip, Jp, c);
+                    *(float4 *)(Gdst + b) = __ldcg((const float4 *)(Gsrc + b));
+                }
+            }
+            if (j + 1 < cnt) fetch(q + 1);
+            continue;
+        }
+        // the block goes to the B tile when a row transform comes first, else straight to the T tile
+        float *blk_dst = fp ? Bk : Tm;
+        const int blk_ld = fp ? LDB : LDA;
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            const int f = tid + it * NT, i = f >> 4, c = (f & 15) * 4;
+            *(float4 *)(blk_dst + i * blk_ld + c) = x[it];
+            if (fq) *(float4 *)(Vq + i * LDA + c) = __ldcg((const float4 *)(Vbuf + (size_t)q * BLK * BLK + i * BLK + c));
+        }
+        __syncthreads();
+        if (j + 1 < cnt) fetch(q + 1);
+        float acc[4][4];
+        if (fp) {
+            if (TENSOR) product64<false>(Vp, Bk, LDB, m0, n0, acc);  // T = Vt_p * block
+            else product64_fma<false>(Vp, Bk, LDB, m0, n0, acc);
+            if (fq) {
+                store_tile_acc(Tm, LDA, m0, n0, acc);
+                __syncthreads();
+            }
+        }
+        if (fq) {                                                // out = T * Vt_q^T
+            if (TENSOR) product64<true>(Tm, Vq, LDA, m0, n0, acc);
+            else product64_fma<true>(Tm, Vq, LDA, m0, n0, acc);
+        }
+        const int gr0 = glob_of_loc(Ip, Jp, m0 + g), gr1 = glob_of_loc(Ip, Jp, m0 + g + 8);
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+            const int gc = glob_of_loc(Iq, Jq, n0 + nt * 8 + 2 * t);     // gc, gc + 1 are contiguous
+            *(float2 *)(Gdst + (size_t)gr0 * np + gc) = make_float2(acc[nt][0], acc[nt][1]);
+            *(float2 *)(Gdst + (size_t)gr1 * np + gc) = make_float2(acc[nt][2], acc[nt][3]);
+            if (q != p) {                                        // mirror block
+                Gdst[(size_t)gc * np + gr0] = acc[nt][0]; Gdst[(size_t)(gc + 1) * np + gr0] = acc[nt][1];
+                Gdst[(size_t)gc * np + gr1] = acc[nt][2]; Gdst[(size_t)(gc + 1) * np + gr1] = acc[nt][3];
+            }
+        }
+        __syncthreads();                                         // tiles are reused by the next block
+    }
+}
+
+template <bool TENSOR>
+__device__ void wt_strip(float *sm, const Seq &sq, const float *Vbuf, const int *vflag, int step, int p, int c0, int cnt)
+{
+    if (!__ldcg(vflag + p)) return;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+    const int m0 = (warp & 3) * 16, n0 = (warp >> 2) * 32, np = sq.np;
+    float *Vp = sm, *Bk = sm + 3 * BLK * LDA;
+    int Ip, Jp;
+    rr_pair(sq.nb, step, p, Ip, Jp);
+    float4 x[4];
+    auto fetch = [&](int chunk) {
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            const int f = tid + it * NT, i = f >> 4, c = (f & 15) * 4;
+            x[it] = __ldcg((const float4 *)(sq.Wt + (size_t)glob_of_loc(Ip, Jp, i) * np + chunk * BLK + c));
+        }
+    };
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+        const int f = tid + it * NT, i = f >> 4, c = (f & 15) * 4;
+        *(float4 *)(Vp + i * LDA + c) = __ldcg((const float4 *)(Vbuf + (size_t)p * BLK * BLK + i * BLK + c));
+    }
+    fetch(c0);
+    const int gr0 = glob_of_loc(Ip, Jp, m0 + g), gr1 = glob_of_loc(Ip, Jp, m0 + g + 8);
+    for (int j = 0; j < cnt; ++j) {
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            const int f = tid + it * NT, i = f >> 4, c = (f & 15) * 4;
+            *(float4 *)(Bk + i * LDB + c) = x[it];
+        }
+        __syncthreads();
+        if (j + 1 < cnt) fetch(c0 + j + 1);
+        float acc[4][4];
+        if (TENSOR) product64<false>(Vp, Bk, LDB, m0, n0, acc);
+        else product64_fma<false>(Vp, Bk, LDB, m0, n0, acc);
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+            const int gc = (c0 + j) * BLK + n0 + nt * 8 + 2 * t;
+            *(float2 *)(sq.Wt + (size_t)gr0 * np + gc) = make_float2(acc[nt][0], acc[nt][1]);
+            *(float2 *)(sq.Wt + (size_t)gr1 * np + gc) = make_float2(acc[nt][2], acc[nt][3]);
+        }
+        __syncthreads();                                         // the B tile is reused by the next chunk
+    }
+}
+
+// Work items of the update: first the strips of G (row by row of the upper triangle), then the strips of Wt.
+__host__ __device__ __forceinline__ int strips_of_g(int npairs)
+{
+    int n = 0;
+    for (int p = 0; p < npairs; ++p) n += (npairs - p + SEG_G - 1) / SEG_G;
+    return n;
+}
+template <bool TENSOR>
+__device__ void apply_item(float *sm, const Seq &sq, const float *Gsrc, float *Gdst, const float *Vbuf, const int *vflag, int step, int idx, int npairs, int items_g, int nw)
+{
+    if (idx < items_g) {
+        int p = 0;
+        for (;;) {
+            const int n = (npairs - p + SEG_G - 1) / SEG_G;
+            if (idx < n) break;
+            idx -= n; ++p;
+        }
+        const int q0 = p + idx * SEG_G;
+        g_strip<TENSOR>(sm, sq, Gsrc, Gdst, Vbuf, vflag, step, p, q0, min(SEG_G, npairs - q0));
+    } else {
+        idx -= items_g;
+        const int nseg = (nw + SEG_W - 1) / SEG_W, p = idx / nseg, c0 = (idx - p * nseg) * SEG_W;
+        wt_strip<TENSOR>(sm, sq, Vbuf, vflag, step, p, c0, min(SEG_W, nw - c0));
+    }
 }
 
 // ---- the kernel --------------------------------------------------------------------------------
@@ -568,7 +660,8 @@ jacobi_persistent_kernel(const __grid_constant__ Batch batch, float tol_conv, fl
     const Seq &sq = batch.s[si];
     const int rank = (int)blockIdx.x - sq.cta0, tid = threadIdx.x;
     if (rank >= sq.ncta || sq.np <= 0) return;
-    const int npairs = sq.nb / 2, nw = sq.np / BLK, ntri = npairs * (npairs + 1) / 2, total = ntri + npairs * nw;
+    const int npairs = sq.nb / 2, nw = sq.np / BLK;
+    const int items_g = strips_of_g(npairs), total = items_g + npairs * ((nw + SEG_W - 1) / SEG_W);
     const int nsteps = sq.nb - 1;
     int *abort_flag = status + 1;
     unsigned gen = 0, gstep = 0;
@@ -631,7 +724,7 @@ jacobi_persistent_kernel(const __grid_constant__ Batch batch, float tol_conv, fl
             while (t < total) {
                 int tn = 0;
                 if (tid == 0) tn = (int)atomicAdd(sq.sync + 16 + par, 1u);
-                apply_item<TENSOR>(j3sm, sq, Gsrc, Gdst, Vcur, fcur, step, t, npairs, ntri, nw);
+                apply_item<TENSOR>(j3sm, sq, Gsrc, Gdst, Vcur, fcur, step, t, npairs, items_g, nw);
                 __syncthreads();
                 if (tid == 0) ticket_s = tn;
                 __syncthreads();
@@ -701,7 +794,9 @@ static inline atp_status launch(atp_ctx *ctx, Batch &jb, float tol_conv, float t
     int next = 0;
     for (int i = 0; i < jb.count; ++i) {
         Seq &q = jb.s[i];
-        const int npairs = q.nb / 2, items = npairs * (npairs + 1) / 2 + npairs * (q.np / BLK);
+        const int npairs = q.nb / 2;
+        int items = npairs * ((q.np / BLK + SEG_W - 1) / SEG_W);                 // strips of the update
+        for (int pp = 0; pp < npairs; ++pp) items += (npairs - pp + SEG_G - 1) / SEG_G;
         int c = (int)((double)total * ((double)q.np * q.np / wsum));
         c = std::max(1, std::min(c, std::max(items, 1)));
         if (q.np <= 0) c = 1;
