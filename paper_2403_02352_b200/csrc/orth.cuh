@@ -4,7 +4,8 @@
 // Panels of 64 columns, left to right; every panel runs `reps` times through
 //   project   C = Q^T P against the finished columns Q (split over row ranges, partials summed in a fixed order)
 //   update    P <- P - Q C
-//   Gram      S = P^T P accumulated in fp64, scaled, Cholesky-factored and inverted in fp64 (panel_chol.cuh)
+//   Gram      S = P^T P accumulated in fp64, scaled, Cholesky-factored and inverted in fp64 (panel_chol.cuh); from the
+//             second repetition on, when S is within 5e-3 of the identity, the factor comes from a three-term series
 //   apply     P <- P (D^-1 L^-T); columns found dependent are replaced by hash noise, which the next
 //             repetition orthonormalises
 // Two repetitions give orthonormality to working precision (the second also repairs the explicit inverse,
@@ -294,7 +295,8 @@ orth_persistent_kernel(const __grid_constant__ Batch batch, int reps, uint64_t s
             if (rank == 0) {
                 for (int e = tid; e < 4096; e += NT) Gs[e] = ordered_sum(sq.gpart2 + e, 4096, nrange);
                 __syncthreads();
-                chol_invert_64(Gs, w, sq.W, sq.flags);
+                // the panel of a later repetition is nearly orthonormal: a short series replaces the factorisation
+                if (!(rep > 0 && lowdin_64(Gs, w, sA, sq.W, sq.flags))) chol_invert_64(Gs, w, sq.W, sq.flags);
                 __syncthreads();
             }
             barrier();

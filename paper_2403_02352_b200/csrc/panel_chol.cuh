@@ -156,3 +156,65 @@ __device__ __noinline__ void chol_invert_64(const double *Gs, int n, float *rinv
     if (tid < PB) flags[tid] = (tid < n) ? (dep[tid] || !(rs[tid] > 0.0)) : 0;
 }
 
+
+// Orthonormalising factor of a panel that is already close to orthonormal (the second Gram-Schmidt repetition):
+// with the Gram matrix scaled to unit diagonal, D^-1/2 G D^-1/2 = I + E, the symmetric factor
+//   W = D^-1/2 (I - E/2 + 3/8 E^2)          (P W has orthonormal columns up to 5/16 |E|^3)
+// needs one 64^3 product instead of a factorisation and its chain of 64 dependent pivots. Taken only when every
+// diagonal entry is positive and the largest absolute row sum of E is at most LOWDIN_LIMIT (then the neglected
+// term is below 4e-8); otherwise nothing is written and the caller factors the matrix. Returns the decision
+// (block-uniform). Es: a 64 x LDE fp32 tile of shared memory; 256 threads.
+constexpr float LOWDIN_LIMIT = 5e-3f;
+constexpr int LDE = 72;
+__device__ __noinline__ bool lowdin_64(const double *Gs, int n, float *Es, float *rinv, int *flags)
+{
+    __shared__ double rsq[PB];
+    __shared__ float rowsum[PB];
+    const int tid = threadIdx.x;
+    bool bad = false;
+    if (tid < PB) {
+        const double d = Gs[tid * PB + tid];
+        const bool pos = tid < n && d > 0.0;
+        rsq[tid] = pos ? rsqrt(d) : 0.0;
+        rowsum[tid] = 0.f;
+        bad = tid < n && !pos;
+    }
+    __syncthreads();
+    for (int e = tid; e < PB * PB; e += 256) {
+        const int i = e >> 6, j = e & 63;
+        float v = 0.f;
+        if (i < n && j < n && i != j) v = (float)(Gs[e] * rsq[i] * rsq[j]);
+        Es[i * LDE + j] = v;
+        float a = fabsf(v);                                      // row i lies in two warps: 32 columns each
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+        if ((tid & 31) == 0) atomicAdd(&rowsum[i], a);
+    }
+    __syncthreads();
+    if (tid < PB && !(rowsum[tid] <= LOWDIN_LIMIT)) bad = true;
+    if (__syncthreads_or(bad)) return false;
+    // E^2 (E is symmetric): thread (ty, tx) owns the 4 x 4 block at rows 4 ty, columns 4 tx
+    const int tx = tid & 15, ty = tid >> 4;
+    float acc[4][4] = {};
+#pragma unroll 4
+    for (int k = 0; k < PB; ++k) {
+        const float4 a = *(const float4 *)&Es[k * LDE + ty * 4];
+        const float4 b = *(const float4 *)&Es[k * LDE + tx * 4];
+        const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int r = ty * 4 + i, c = tx * 4 + j;
+            float w = 0.f;
+            if (r < n && c < n) w = (float)rsq[r] * ((r == c ? 1.f : 0.f) - 0.5f * Es[r * LDE + c] + 0.375f * acc[i][j]);
+            rinv[r * PB + c] = w;
+        }
+    if (tid < PB) flags[tid] = 0;
+    return true;
+}
