@@ -15,6 +15,7 @@ struct AltSeq {
     const float *v0;               // start vectors of this sequence (r x d, row stride ldv)
     void *U, *Xp;                  // outputs: U (L x r), X' (r x d)
     int L, r, ldu, ldx, ldv;
+    int row0;                      // first row of the sequence in the packed input
 };
 struct AltBatch { AltSeq s[ALT_MAX]; int count; };
 
@@ -33,12 +34,11 @@ __device__ __forceinline__ double block_sum_256(double x, double *red)
 }
 
 template <typename T>
-__global__ void __launch_bounds__(256) alt_copy_kernel(const __grid_constant__ AltBatch batch, const T *X, int ldx_in, int d,
-                                                       const int *row0)
+__global__ void __launch_bounds__(256) alt_copy_kernel(const __grid_constant__ AltBatch batch, const T *X, int ldx_in, int d)
 {
     const AltSeq &q = batch.s[blockIdx.y];
     const size_t n = (size_t)q.L * d;
-    const T *src = X + (size_t)row0[blockIdx.y] * ldx_in;
+    const T *src = X + (size_t)q.row0 * ldx_in;
     for (size_t e = (size_t)blockIdx.x * 256 + threadIdx.x; e < n; e += (size_t)gridDim.x * 256) {
         const int l = (int)(e / d), k = (int)(e - (size_t)l * d);
         q.R[e] = to_f32(src[(size_t)l * ldx_in + k]);
@@ -128,7 +128,6 @@ size_t alternating_workspace_bytes(const std::vector<SeqDims> &sd, int d)
 {
     Arena ar(nullptr, (size_t)-1);
     for (auto &s : sd) { ar.take<float>((size_t)s.L * d); ar.take<float>(s.L); ar.take<float>(d); }
-    ar.take<int>(sd.size());
     return ar.off;
 }
 
@@ -146,12 +145,9 @@ static atp_status alternating_impl(atp_ctx *ctx, const atp_mat *X, const std::ve
         q.U = (T *)U_r->data + (size_t)sd[i].row0 * U_r->ld;
         q.Xp = (T *)X_r->data + (size_t)sd[i].rank0 * X_r->ld;
         q.L = sd[i].L; q.r = sd[i].r; q.ldu = (int)U_r->ld; q.ldx = (int)X_r->ld; q.ldv = (int)V0->ld;
+        q.row0 = sd[i].row0;
     }
-    int *row0_dev = ar.take<int>(sd.size());
     if (ar.overflow) return ATP_ERR_WORKSPACE_TOO_SMALL;
-    std::vector<int> row0(sd.size());
-    for (size_t i = 0; i < sd.size(); ++i) row0[i] = sd[i].row0;
-    ATP_CUDA_OK(ctx, cudaMemcpyAsync(row0_dev, row0.data(), sizeof(int) * sd.size(), cudaMemcpyHostToDevice, ctx->stream));
     for (size_t i0 = 0; i0 < sd.size(); i0 += ALT_MAX) {
         AltBatch b; b.count = (int)std::min<size_t>(ALT_MAX, sd.size() - i0);
         int maxL = 0, maxr = 0;
@@ -160,7 +156,7 @@ static atp_status alternating_impl(atp_ctx *ctx, const atp_mat *X, const std::ve
         const double mat_bytes = [&] { double s = 0; for (int k = 0; k < b.count; ++k) s += (double)b.s[k].L * d * 4; return s; }();
         ATP_KERNEL(ctx, "alt_copy", 0, mat_bytes * (1.0 + sizeof(T) / 4.0));
         alt_copy_kernel<T><<<dim3(std::min(1024, (int)(((size_t)maxL * d + 255) / 256)), b.count), 256, 0, ctx->stream>>>(
-            b, (const T *)X->data, (int)X->ld, d, row0_dev + i0);
+            b, (const T *)X->data, (int)X->ld, d);
         ATP_LAUNCHED(ctx);
         const dim3 grows((maxL + 7) / 8, b.count), gcols((d + 63) / 64, b.count);
         for (int comp = 0; comp < maxr; ++comp) {
