@@ -466,8 +466,10 @@ __device__ void pivot_form(float *sm, const Seq &sq, const float *Gsrc, const fl
 // The update of a step is cut into strips. A strip of G: blocks (p, q0 .. q0 + cnt - 1) of the upper triangle,
 // read from Gsrc and written (with their mirrors) to Gdst, also when neither pair was rotated; a strip of Wt: the
 // rows of pair p, column chunks c0 .. c0 + cnt - 1 of 64, in place. Along a strip Vt_p stays in shared memory and
-// the next block is fetched into registers while the current one is multiplied.
-constexpr int SEG_G = 2, SEG_W = 3;
+// the next block is fetched into registers while the current one is multiplied. Short strips win at r~ = 2112: with
+// 296 CTAs a step has only a few items per CTA, and the last ones to finish set the time of the step (strips of
+// 2 + 3 blocks: 39.9 us per step, 1 + 2: 37.3 us).
+constexpr int SEG_G = 1, SEG_W = 2;
 
 __device__ __forceinline__ void store_tile_acc(float *dst, int ld, int m0, int n0, const float (&acc)[4][4])
 {
