@@ -586,7 +586,7 @@ static void plan_basis(Arena &ar, const std::vector<SeqDims> &sd, int d, int ove
             p.oCpart = ar.take<float>(sc.cpart * 4096); p.oC = ar.take<float>(sc.c * 4096);
             p.oDpart = ar.take<float>(sc.dpart * 4096); p.oW = ar.take<float>(4096);
             p.ogpart = ar.take<double>(sc.gpart * 4096); p.ogpart2 = ar.take<double>((size_t)orth::NRED * 4096);
-            p.flags = ar.take<int>(64); p.osync = ar.take<unsigned>(64);
+            p.flags = ar.take<int>(64); p.osync = ar.take<unsigned>(64 + (size_t)p.ocap);
         }
         p.np = jacobi_padded(rt);
         p.G = ar.take<float>((size_t)p.np * p.np);

@@ -8,6 +8,9 @@
 //             second repetition on, when S is within 5e-3 of the identity, the factor comes from a three-term series
 //   apply     P <- P (D^-1 L^-T); columns found dependent are replaced by hash noise, which the next
 //             repetition orthonormalises
+// With two repetitions (what the extraction asks for) the passes are reordered so that the second projection runs
+// beside the single-CTA factorisation of the first repetition and the first apply folds into the second Gram
+// pass; see the panel program in the kernel.
 // Two repetitions give orthonormality to working precision (the second also repairs the explicit inverse,
 // which is only norm-wise stable). Each sequence owns a group of CTAs; the phases of a panel are separated by
 // the group's barrier (bounded spin, see jacobi3.cuh) instead of kernel boundaries, and every phase is a list
@@ -31,7 +34,8 @@ struct Seq {
     float *Cpart, *C, *Dpart, *W;             // tile scratch (see scratch_tiles)
     double *gpart, *gpart2;
     int *flags;
-    unsigned *sync;                           // 64 words: group barrier (jacobi3.cuh)
+    unsigned *sync;                           // 64 words: group barrier (jacobi3.cuh); then one word per CTA of the
+                                              // group (its SM)
     int cta0, ncta, index;                    // CTA group (on entry to launch(): ncta = the cap the scratch was
                                               // sized for); index of the sequence in its batch (noise stream)
 };
@@ -161,50 +165,115 @@ orth_persistent_kernel(const __grid_constant__ Batch batch, int reps, uint64_t s
     constexpr int P_FINE = TENSOR ? 3 : 0;
     auto barrier = [&]() { alive = j3::group_barrier(sq.sync, ++gen, (unsigned)ncta, abort_flag) && alive; };
 
+    // The CTA that shares an SM with rank 0 (if it belongs to this group) stays out of the work that runs beside
+    // rank 0's factorisation, which is a latency chain and slows down under a busy neighbour.
+    unsigned smid;
+    asm("mov.u32 %0, %%smid;" : "=r"(smid));
+    if (tid == 0) sq.sync[64 + rank] = smid;
+    barrier();
+    __shared__ int mate_s;
+    if (tid == 0) mate_s = 1 << 30;
+    __syncthreads();
+    if (alive) {
+        const unsigned sm0 = __ldcg(sq.sync + 64);
+        for (int r = 1 + tid; r < ncta; r += NT)
+            if (__ldcg(sq.sync + 64 + r) == sm0) atomicMin(&mate_s, r);
+    }
+    __syncthreads();
+    const int mate = mate_s < ncta ? mate_s : -1;
+    const bool overlap = reps == 2 && ncta >= 4;
+    const int nworkers = ncta - 1 - (mate > 0 ? 1 : 0);
+    const int wid = (rank == 0 || rank == mate) ? -1 : rank - 1 - ((mate > 0 && rank > mate) ? 1 : 0);
+
+    // A panel is a short program of four kinds of passes, each written once below:
+    //   PF      project (partial C over row ranges, jobs first, first + stride, ...) and / or, on rank 0, the factor
+    //           of the panel's Gram matrix; SUMUPD  C = ordered sum of the partials, then partial D = Q C;
+    //   GRAM    P -= sum D, optionally P <- P W, written back, Gram matrix in fp64 and its ordered sum;
+    //   APPLY   P <- P W, dependent columns refilled, finished columns also as bf16 hi/lo.
+    // Classic order per repetition: PF(project) SUMUPD GRAM PF(factor) APPLY. With two repetitions the second
+    // projection is taken of the panel BEFORE the first factor is applied ((P - Q Q^T P) W = P W - Q Q^T (P W)), so
+    // it runs beside rank 0's factorisation, and the first APPLY folds into the second GRAM pass:
+    //   PF(project) SUMUPD GRAM | PF(project beside factor) SUMUPD GRAM(with W) | PF(series factor) APPLY.
+    // A panel with dependent columns (their replacements must still be projected) returns to the classic order.
+    enum { OP_PF, OP_SUMUPD, OP_GRAM, OP_APPLY };
     for (int pj = 0; pj < npanel && alive; ++pj) {
         const int j0 = pj * 64, w = min(64, rt - j0), nj = pj;            // nj finished panels
-        for (int rep = 0; rep < reps && alive; ++rep) {
-            int G = 1;
-            if (nj > 0) {
-                // ---- project: partial C[jb] over row ranges
-                const int KS = max(1, min(ntile, (ncta + nj - 1) / nj));
-                const int tper = (ntile + KS - 1) / KS;
-                for (int it = rank; it < nj * KS; it += ncta) {
-                    const int jb = it / KS, ks = it - jb * KS;
-                    float acc[4][4] = {};
-                    const int t0 = ks * tper, t1 = min(ntile, (ks + 1) * tper);
-                    TileRegs ra, rb;
-                    if (t0 < t1) {
-                        fetch_tile(ra, sq.M + (size_t)t0 * 64 * ld + jb * 64, ld, min(64, n - t0 * 64), 64, vec);
-                        fetch_tile(rb, sq.M + (size_t)t0 * 64 * ld + j0, ld, min(64, n - t0 * 64), w, vec);
-                    }
-                    for (int t = t0; t < t1; ++t) {
-                        stash_tile(ra, sA, LDB);
-                        stash_tile(rb, sB, LDB);
-                        __syncthreads();
-                        if (t + 1 < t1) {                                   // next tiles in flight during the product
-                            const int rv = min(64, n - (t + 1) * 64);
-                            fetch_tile(ra, sq.M + (size_t)(t + 1) * 64 * ld + jb * 64, ld, rv, 64, vec);
-                            fetch_tile(rb, sq.M + (size_t)(t + 1) * 64 * ld + j0, ld, rv, w, vec);
+        const int KS = nj > 0 ? max(1, min(ntile, (ncta + nj - 1) / nj)) : 1;
+        const int tper = (ntile + KS - 1) / KS;
+        const int G = nj > 0 ? max(1, min(nj, (ncta + ntile - 1) / ntile)) : 1;
+        const int jper = nj > 0 ? (nj + G - 1) / G : 1;
+        const int nrange = max(1, min(8, ntile / 64)), cper = (ntile + nrange - 1) / nrange;
+        int stage = overlap ? 0 : 30, rep = 0;
+        while (stage >= 0 && alive) {
+            int op = OP_PF, first = -1, stride = 1, arep = 0;
+            bool do_factor = false, series_ok = false, with_w = false, last = false, skip = false;
+            switch (stage) {
+                // overlapped order
+                case 0: op = OP_PF; first = rank; stride = ncta; skip = nj == 0; break;
+                case 1: op = OP_SUMUPD; skip = nj == 0; break;
+                case 2: op = OP_GRAM; break;
+                case 3: op = OP_PF; first = nj > 0 ? wid : -1; stride = nworkers; do_factor = true; break;
+                case 4: op = OP_SUMUPD; skip = nj == 0; break;
+                case 5: op = OP_GRAM; with_w = true; break;
+                case 6: op = OP_PF; do_factor = true; series_ok = true; break;
+                case 7: op = OP_APPLY; arep = 1; last = true; break;
+                // dependent columns found by the first factor: classic remainder
+                case 20: op = OP_APPLY; arep = 0; break;
+                case 21: op = OP_PF; first = rank; stride = ncta; skip = nj == 0; break;
+                case 22: op = OP_SUMUPD; skip = nj == 0; break;
+                case 23: op = OP_GRAM; break;
+                case 24: op = OP_PF; do_factor = true; series_ok = true; break;
+                case 25: op = OP_APPLY; arep = 1; last = true; break;
+                // classic order, any number of repetitions
+                case 30: op = OP_PF; first = rank; stride = ncta; skip = nj == 0; break;
+                case 31: op = OP_SUMUPD; skip = nj == 0; break;
+                case 32: op = OP_GRAM; break;
+                case 33: op = OP_PF; do_factor = true; series_ok = rep > 0; break;
+                default: op = OP_APPLY; arep = rep; last = rep == reps - 1; break;      // 34
+            }
+            if (!skip) switch (op) {
+            case OP_PF: {
+                if (do_factor && rank == 0) {
+                    for (int e = tid; e < 4096; e += NT) Gs[e] = ordered_sum(sq.gpart2 + e, 4096, nrange);
+                    __syncthreads();
+                    // a nearly orthonormal panel gets its factor from a short series instead of the factorisation
+                    if (!(series_ok && lowdin_64(Gs, w, sA, sq.W, sq.flags))) chol_invert_64(Gs, w, sq.W, sq.flags);
+                    __syncthreads();
+                } else if (first >= 0) {
+                    for (int it = first; it < nj * KS; it += stride) {
+                        const int jb = it / KS, ks = it - jb * KS;
+                        float acc[4][4] = {};
+                        const int t0 = ks * tper, t1 = min(ntile, (ks + 1) * tper);
+                        TileRegs ra, rb;
+                        if (t0 < t1) {
+                            fetch_tile(ra, sq.M + (size_t)t0 * 64 * ld + jb * 64, ld, min(64, n - t0 * 64), 64, vec);
+                            fetch_tile(rb, sq.M + (size_t)t0 * 64 * ld + j0, ld, min(64, n - t0 * 64), w, vec);
                         }
-                        tile_mac<P_FINE, true>(sA, LDB, sB, LDB, m0, n0, acc);
-                        __syncthreads();
+                        for (int t = t0; t < t1; ++t) {
+                            stash_tile(ra, sA, LDB);
+                            stash_tile(rb, sB, LDB);
+                            __syncthreads();
+                            if (t + 1 < t1) {                               // next tiles in flight during the product
+                                const int rv = min(64, n - (t + 1) * 64);
+                                fetch_tile(ra, sq.M + (size_t)(t + 1) * 64 * ld + jb * 64, ld, rv, 64, vec);
+                                fetch_tile(rb, sq.M + (size_t)(t + 1) * 64 * ld + j0, ld, rv, w, vec);
+                            }
+                            tile_mac<P_FINE, true>(sA, LDB, sB, LDB, m0, n0, acc);
+                            __syncthreads();
+                        }
+                        store_acc(sq.Cpart + (size_t)it * 4096, 64, m0, n0, acc);
                     }
-                    store_acc(sq.Cpart + (size_t)it * 4096, 64, m0, n0, acc);
                 }
                 barrier();
-                if (!alive) break;
-                // ---- sum the partials in order: C[jb]
-                for (int it = rank; it < nj * 4; it += ncta) {               // a quarter tile per job
+            } break;
+            case OP_SUMUPD: {
+                for (int it = rank; it < nj * 4; it += ncta) {           // a quarter tile per job
                     const int jb = it >> 2;
                     for (int e = (it & 3) * 1024 + tid; e < ((it & 3) + 1) * 1024; e += NT)
                         sq.C[(size_t)jb * 4096 + e] = ordered_sum(sq.Cpart + (size_t)jb * KS * 4096 + e, 4096, KS);
                 }
                 barrier();
                 if (!alive) break;
-                // ---- update: partial D[t][g] = sum over a range of jb of Q[t][:, jb] C[jb]
-                G = max(1, min(nj, (ncta + ntile - 1) / ntile));
-                const int jper = (nj + G - 1) / G;
                 for (int it = rank; it < ntile * G; it += ncta) {
                     const int t = it / G, g = it - t * G;
                     const int rv = min(64, n - t * 64);
@@ -229,110 +298,123 @@ orth_persistent_kernel(const __grid_constant__ Batch batch, int reps, uint64_t s
                     store_acc(sq.Dpart + (size_t)it * 4096, 64, m0, n0, acc);
                 }
                 barrier();
-                if (!alive) break;
-            }
-            // ---- P[t] -= sum_g D[t][g] (fixed order), written back; partial Gram matrix of the tile in fp64
-            for (int t = rank; t < ntile; t += ncta) {
-                const int rv = min(64, n - t * 64);
-                load_tile(sA, LDA, sq.M + (size_t)t * 64 * ld + j0, ld, rv, w, vec);
-                __syncthreads();
-                if (nj > 0) {
-                    for (int e0 = tid; e0 < 4096; e0 += 4 * NT) {                // four elements, 4 G loads in flight
-                        float s[4] = {0.f, 0.f, 0.f, 0.f};
-                        const float *dp = sq.Dpart + (size_t)t * G * 4096 + e0;
-                        for (int g = 0; g < G; ++g) {
-                            float x[4];
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) x[q] = __ldcg(dp + (size_t)g * 4096 + q * NT);
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) s[q] += x[q];
-                        }
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            const int e = e0 + q * NT, r = e >> 6, c = e & 63;
-                            const float v = sA[r * LDA + c] - s[q];
-                            sA[r * LDA + c] = (r < rv && c < w) ? v : 0.f;
-                            if (r < rv && c < w) sq.M[((size_t)t * 64 + r) * ld + j0 + c] = v;
-                        }
-                    }
+            } break;
+            case OP_GRAM: {
+                for (int t = rank; t < ntile; t += ncta) {
+                    const int rv = min(64, n - t * 64);
+                    load_tile(sA, LDA, sq.M + (size_t)t * 64 * ld + j0, ld, rv, w, vec);
+                    if (with_w) load_tile(sB, LDB, sq.W, 64, 64, 64, true);
                     __syncthreads();
-                }
-                const int tx = tid & 15, ty = tid >> 4;
-                double acc[4][4];
+                    if (nj > 0) {
+                        for (int e0 = tid; e0 < 4096; e0 += 4 * NT) {            // four elements, 4 G loads in flight
+                            float sacc[4] = {0.f, 0.f, 0.f, 0.f};
+                            const float *dp = sq.Dpart + (size_t)t * G * 4096 + e0;
+                            for (int g = 0; g < G; ++g) {
+                                float x[4];
 #pragma unroll
-                for (int i = 0; i < 4; ++i)
+                                for (int q = 0; q < 4; ++q) x[q] = __ldcg(dp + (size_t)g * 4096 + q * NT);
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) acc[i][j] = 0.0;
-#pragma unroll 4
-                for (int k = 0; k < 64; ++k) {
-                    const float4 a = *(const float4 *)&sA[k * LDA + ty * 4];
-                    const float4 b = *(const float4 *)&sA[k * LDA + tx * 4];
-                    const double av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+                                for (int q = 0; q < 4; ++q) sacc[q] += x[q];
+                            }
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const int e = e0 + q * NT, r = e >> 6, c = e & 63;
+                                const float v = sA[r * LDA + c] - sacc[q];
+                                sA[r * LDA + c] = (r < rv && c < w) ? v : 0.f;
+                                if (!with_w && r < rv && c < w) sq.M[((size_t)t * 64 + r) * ld + j0 + c] = v;
+                            }
+                        }
+                        __syncthreads();
+                    }
+                    if (with_w) {
+                        float acc[4][4] = {};
+                        tile_mac<P_FINE, false>(sA, LDA, sB, LDB, m0, n0, acc);
+                        __syncthreads();
+                        const int lane = tid & 31, g = lane >> 2, tq = lane & 3;
+#pragma unroll
+                        for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const int r = m0 + g + (i >= 2 ? 8 : 0), c = n0 + nt * 8 + 2 * tq + (i & 1);
+                                const bool in = r < rv && c < w;
+                                sA[r * LDA + c] = in ? acc[nt][i] : 0.f;
+                                if (in) sq.M[((size_t)t * 64 + r) * ld + j0 + c] = acc[nt][i];
+                            }
+                        __syncthreads();
+                    }
+                    const int tx = tid & 15, ty = tid >> 4;
+                    double acc[4][4];
 #pragma unroll
                     for (int i = 0; i < 4; ++i)
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) acc[i][j] = fma(av[i], bv[j], acc[i][j]);
-                }
-                double *dst = sq.gpart + (size_t)t * 4096;
+                        for (int j = 0; j < 4; ++j) acc[i][j] = 0.0;
+#pragma unroll 4
+                    for (int k = 0; k < 64; ++k) {
+                        const float4 a = *(const float4 *)&sA[k * LDA + ty * 4];
+                        const float4 b = *(const float4 *)&sA[k * LDA + tx * 4];
+                        const double av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
-                for (int i = 0; i < 4; ++i)
+                        for (int i = 0; i < 4; ++i)
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) dst[(ty * 4 + i) * 64 + tx * 4 + j] = acc[i][j];
-                __syncthreads();
-            }
-            barrier();
-            if (!alive) break;
-            // ---- ordered sum of the partial Gram matrices: 16 element slices x (up to 8) chunk ranges
-            const int nrange = max(1, min(8, ntile / 64)), cper = (ntile + nrange - 1) / nrange;
-            for (int it = rank; it < 16 * nrange; it += ncta) {
-                const int sl = it & 15, rg = it >> 4, e = sl * 256 + tid;
-                const int c0 = rg * cper, c1 = min(ntile, (rg + 1) * cper);
-                sq.gpart2[(size_t)rg * 4096 + e] = ordered_sum(sq.gpart + (size_t)c0 * 4096 + e, 4096, max(c1 - c0, 0));
-            }
-            barrier();
-            if (!alive) break;
-            // ---- Cholesky factor and its inverse (one CTA)
-            if (rank == 0) {
-                for (int e = tid; e < 4096; e += NT) Gs[e] = ordered_sum(sq.gpart2 + e, 4096, nrange);
-                __syncthreads();
-                // the panel of a later repetition is nearly orthonormal: a short series replaces the factorisation
-                if (!(rep > 0 && lowdin_64(Gs, w, sA, sq.W, sq.flags))) chol_invert_64(Gs, w, sq.W, sq.flags);
-                __syncthreads();
-            }
-            barrier();
-            if (!alive) break;
-            // ---- apply: P[t] <- P[t] W, dependent columns refilled, finished columns also as bf16 hi/lo
-            const bool last = rep == reps - 1;
-            const uint64_t nseed = seed + 7919ull * (uint64_t)(pj * 2 + rep);
-            const float rscale = rsqrtf((float)n * (1.f / 3.f));         // replacement columns of about unit norm
-            for (int t = rank; t < ntile; t += ncta) {
-                const int rv = min(64, n - t * 64);
-                load_tile(sA, LDA, sq.M + (size_t)t * 64 * ld + j0, ld, rv, w, vec);
-                load_tile(sB, LDB, sq.W, 64, 64, 64, true);
-                __syncthreads();
-                float acc[4][4] = {};
-                tile_mac<P_FINE, false>(sA, LDA, sB, LDB, m0, n0, acc);
-                const int lane = tid & 31, g = lane >> 2, tq = lane & 3;
-#pragma unroll
-                for (int nt = 0; nt < 4; ++nt)
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int r = m0 + g + (i >= 2 ? 8 : 0), c = n0 + nt * 8 + 2 * tq + (i & 1);
-                        if (r >= rv || c >= w) continue;
-                        const int grow = t * 64 + r;
-                        float v = acc[nt][i];
-                        if (__ldcg(sq.flags + c))
-                            v = rscale * hash_uniform(nseed, ((uint64_t)sq.index << 40) ^ ((uint64_t)grow << 8) ^ (uint64_t)c);
-                        sq.M[(size_t)grow * ld + j0 + c] = v;
-                        if (last && sq.hi) {
-                            const __nv_bfloat16 h = __float2bfloat16_rn(v);
-                            sq.hi[(size_t)grow * sq.ldh + j0 + c] = h;
-                            sq.lo[(size_t)grow * sq.ldh + j0 + c] = __float2bfloat16_rn(v - __bfloat162float(h));
-                        }
+                            for (int j = 0; j < 4; ++j) acc[i][j] = fma(av[i], bv[j], acc[i][j]);
                     }
-                __syncthreads();
+                    double *dst = sq.gpart + (size_t)t * 4096;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) dst[(ty * 4 + i) * 64 + tx * 4 + j] = acc[i][j];
+                    __syncthreads();
+                }
+                barrier();
+                if (!alive) break;
+                // ordered sum of the partial Gram matrices: 16 element slices x (up to 8) chunk ranges
+                for (int it = rank; it < 16 * nrange; it += ncta) {
+                    const int sl = it & 15, rg = it >> 4, e = sl * 256 + tid;
+                    const int c0 = rg * cper, c1 = min(ntile, (rg + 1) * cper);
+                    sq.gpart2[(size_t)rg * 4096 + e] = ordered_sum(sq.gpart + (size_t)c0 * 4096 + e, 4096, max(c1 - c0, 0));
+                }
+                barrier();
+            } break;
+            default: {                                                   // OP_APPLY
+                const uint64_t nseed = seed + 7919ull * (uint64_t)(pj * 2 + arep);
+                const float rscale = rsqrtf((float)n * (1.f / 3.f));     // replacement columns of about unit norm
+                for (int t = rank; t < ntile; t += ncta) {
+                    const int rv = min(64, n - t * 64);
+                    load_tile(sA, LDA, sq.M + (size_t)t * 64 * ld + j0, ld, rv, w, vec);
+                    load_tile(sB, LDB, sq.W, 64, 64, 64, true);
+                    __syncthreads();
+                    float acc[4][4] = {};
+                    tile_mac<P_FINE, false>(sA, LDA, sB, LDB, m0, n0, acc);
+                    const int lane = tid & 31, g = lane >> 2, tq = lane & 3;
+#pragma unroll
+                    for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int r = m0 + g + (i >= 2 ? 8 : 0), c = n0 + nt * 8 + 2 * tq + (i & 1);
+                            if (r >= rv || c >= w) continue;
+                            const int grow = t * 64 + r;
+                            float v = acc[nt][i];
+                            if (__ldcg(sq.flags + c))
+                                v = rscale * hash_uniform(nseed, ((uint64_t)sq.index << 40) ^ ((uint64_t)grow << 8) ^ (uint64_t)c);
+                            sq.M[(size_t)grow * ld + j0 + c] = v;
+                            if (last && sq.hi) {
+                                const __nv_bfloat16 h = __float2bfloat16_rn(v);
+                                sq.hi[(size_t)grow * sq.ldh + j0 + c] = h;
+                                sq.lo[(size_t)grow * sq.ldh + j0 + c] = __float2bfloat16_rn(v - __bfloat162float(h));
+                            }
+                        }
+                    __syncthreads();
+                }
+                barrier();
+            } break;
             }
-            barrier();
+            // next stage
+            if (stage == 3) {
+                const bool dependent = __syncthreads_or(alive && tid < w && __ldcg(sq.flags + tid) != 0) != 0;
+                stage = dependent ? 20 : 4;
+            } else if (stage == 7 || stage == 25) stage = -1;
+            else if (stage == 34) { ++rep; stage = rep < reps ? 30 : -1; }
+            else ++stage;
         }
     }
     if (rank == 0 && tid == 0 && !alive) raise_status(status, ATP_ERR_TIMEOUT);
