@@ -869,7 +869,7 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
                 const int nsw = pass == 0 ? nsw0 : std::max(1, max_sweeps - nsw0);
                 const float tolc = pass == 0 ? fmaxf(tol_conv, 1e-2f) : tol_conv;
                 // fp32 inputs: the block products stay on the fp32 units (the threshold is below split-precision rounding)
-                if ((st = j3::launch<kBf16>(ctx, jb, tolc, tolc * 0.25f, nsw, pass == 1)) != ATP_OK) return st;
+                if ((st = j3::launch<kBf16>(ctx, jb, tolc, tolc * 0.1f, nsw, pass == 1)) != ATP_OK) return st;
                 if (pass == 0) {
                     // Bt2 = Bt Wt^T (d x r~),  Y2 = Y Wt^T (L x r~);  Wt rows are the eigenvectors
                     if constexpr (kBf16) {

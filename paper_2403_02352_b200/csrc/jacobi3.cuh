@@ -667,6 +667,7 @@ jacobi_persistent_kernel(const __grid_constant__ Batch batch, float tol_conv, fl
     const int nsteps = sq.nb - 1;
     int *abort_flag = status + 1;
     unsigned gen = 0, gstep = 0;
+    int gsel = 0;                                                 // which copy of G is current
     bool converged = false, alive = true;
 
     // rotates the block held in shared memory for pair pr of (sweep, step); publishes to parity par
@@ -698,8 +699,10 @@ jacobi_persistent_kernel(const __grid_constant__ Batch batch, float tol_conv, fl
             const int nstep = step + 1 == nsteps ? 0 : step + 1, nsweep = sweep + (step + 1 == nsteps ? 1 : 0);
             const float *Vcur = sq.Vbuf + (size_t)par * npairs * BLK * BLK;
             const int *fcur = sq.vflag + par * npairs;
-            const float *Gsrc = par ? sq.G2 : sq.G;
-            float *Gdst = par ? sq.G : sq.G2;
+            const float *Gsrc = gsel ? sq.G2 : sq.G;
+            float *Gdst = gsel ? sq.G : sq.G2;
+            // a step in which no pair was rotated leaves the matrix where it is: no update, no copy
+            const bool any_rot = __syncthreads_or(tid < npairs && __ldcg(fcur + tid) != 0) != 0;
             if (rank == 0 && tid == 0) sq.sync[16 + (par ^ 1)] = 0u;      // tickets of the next step
             // 1. pivots of the next step
             if (has_next && rank < npairs) {
@@ -720,9 +723,10 @@ jacobi_persistent_kernel(const __grid_constant__ Batch batch, float tol_conv, fl
                 }
             }
             // 2. the update, by tickets (the next one is requested while a block is processed)
-            if (tid == 0) ticket_s = (int)atomicAdd(sq.sync + 16 + par, 1u);
+            if (tid == 0) ticket_s = any_rot ? (int)atomicAdd(sq.sync + 16 + par, 1u) : total;
             __syncthreads();
             int t = ticket_s;
+            if (any_rot) gsel ^= 1;
             while (t < total) {
                 int tn = 0;
                 if (tid == 0) tn = (int)atomicAdd(sq.sync + 16 + par, 1u);
@@ -738,7 +742,7 @@ jacobi_persistent_kernel(const __grid_constant__ Batch batch, float tol_conv, fl
         const float mo = __uint_as_float(*(volatile unsigned *)(sq.sync + 1 + sweep % 4));
         if (mo <= tol_conv) { converged = true; ++sweep; break; }
     }
-    if (alive && (gstep & 1u)) {                                  // the last update wrote G2: the result goes back to G
+    if (alive && gsel) {                                          // the last update wrote G2: the result goes back to G
         const size_t n4 = (size_t)sq.np * sq.np / 4;
         for (size_t e = (size_t)rank * NT + tid; e < n4; e += (size_t)sq.ncta * NT)
             ((float4 *)sq.G)[e] = __ldcg((const float4 *)sq.G2 + e);
