@@ -13,6 +13,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -282,6 +283,46 @@ def stage_rooflines(w, stage_ms, pk, sbytes):
     return out
 
 
+def run_kernel_linear(args):
+    """Micro-benchmark of the low-rank linear layer (a5: T = X_r W, Y = U_r T, two tcgen05 GEMMs) through the
+    public call, at the shapes of the default workload. One JSON line per shape: algorithmic TFLOP/s
+    (2 r d_in d_out + 2 L r d_out flops over the CUDA-event time of a call, L2 flushed between calls) and the
+    fraction of the measured sustained bf16 peak."""
+    import torch
+    import paper_2403_02352_b200 as atp
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    ctx = atp.Context(0)
+    pk = peaks()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    g = torch.Generator(device=dev); g.manual_seed(args.seed)
+    L, r = 4096, (args.rank or 2048)
+    for name, d_in, d_out in (("W_O", 4096, 4096), ("FFN up", 4096, 11008), ("FFN down", 11008, 4096)):
+        U = (torch.randn(L, r, device=dev, generator=g) / math.sqrt(L)).to(torch.bfloat16)
+        Xr = torch.randn(r, d_in, device=dev, generator=g).to(torch.bfloat16)
+        W = (torch.randn(d_in, d_out, device=dev, generator=g) / math.sqrt(d_in)).to(torch.bfloat16)
+        Y = torch.empty(L, d_out, device=dev, dtype=torch.bfloat16)
+        for _ in range(max(args.warmup, 3)):
+            atp.atp_lowrank_linear(ctx, U, Xr, W, [L], [r], out=Y)
+        times = []
+        for _ in range(args.steps):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); atp.atp_lowrank_linear(ctx, U, Xr, W, [L], [r], out=Y); e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        ctx.poll()
+        ms = float(np.median(times))
+        flops = 2.0 * r * d_in * d_out + 2.0 * L * r * d_out
+        tf = flops / ms / 1e9
+        print(json.dumps({"kernel": "lowrank_linear (gemm_tc x 2)", "shape": name, "L": L, "r": r, "d_in": d_in, "d_out": d_out,
+                          "ms": ms, "tflops": tf, "peak": pk["bf16_tflops"], "frac": tf / pk["bf16_tflops"],
+                          "peak_source": pk["source"], "steps": args.steps, "l2": "flushed between calls"}))
+    ctx.close()
+    return 0
+
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -299,9 +340,13 @@ def main():
     ap.add_argument("--jacobi-inner", type=int, default=0)
     ap.add_argument("--max-sweeps", type=int, default=0)
     ap.add_argument("--no-long-context", action="store_true", help="skip the T(32768)/T(16384) measurement")
+    ap.add_argument("--kernel", default=None, choices=["linear"],
+                    help="micro-benchmark of one stage instead of the layer: linear = the two GEMMs of a low-rank linear layer")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.kernel == "linear":
+        return run_kernel_linear(args)
 
     import torch
     import paper_2403_02352_b200 as atp          # raises if libatp.so is missing: no fallback

@@ -261,22 +261,34 @@ gemm_tc_kernel(const __grid_constant__ Batch batch, GemmEpi epi, int *dev_status
                 const int col0 = n0 + c;
                 if (row < pr.M && col0 < pr.N) {
                     float v[32];
+                    const bool full_chunk = (col0 + 32 <= pr.N);
+                    // the D operand of this thread's 32 columns: eight 16-byte loads in flight instead of 32 scalar ones
+                    const bool d_vec = (epi.kind == EPI_D_MINUS || epi.kind == EPI_SILU_D_MUL) && full_chunk &&
+                                       ((pr.ldd & 3) == 0) && (((size_t)pr.D & 15) == 0);
+                    float dv[32];
+                    if (d_vec) {
+                        const float4 *dp = (const float4 *)(pr.D + (size_t)row * pr.ldd + col0);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const float4 q = __ldg(dp + j);
+                            dv[4 * j] = q.x; dv[4 * j + 1] = q.y; dv[4 * j + 2] = q.z; dv[4 * j + 3] = q.w;
+                        }
+                    }
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
                         float x = __uint_as_float(r[j]);
                         const int col = col0 + j;
                         if (col < pr.N) {
                             switch (epi.kind) {
-                                case EPI_D_MINUS: x = pr.D[(size_t)row * pr.ldd + col] - x; break;
+                                case EPI_D_MINUS: x = (d_vec ? dv[j] : pr.D[(size_t)row * pr.ldd + col]) - x; break;
                                 case EPI_BIAS: if (epi.bias) x += epi.bias[col]; break;
                                 case EPI_BIAS_GELU: if (epi.bias) x += epi.bias[col]; x = gelu_erf_f(x); break;
-                                case EPI_SILU_D_MUL: x = silu_f(pr.D[(size_t)row * pr.ldd + col]) * x; break;
+                                case EPI_SILU_D_MUL: x = silu_f(d_vec ? dv[j] : pr.D[(size_t)row * pr.ldd + col]) * x; break;
                                 default: break;
                             }
                         }
                         v[j] = x;
                     }
-                    const bool full_chunk = (col0 + 32 <= pr.N);
                     if (OUT == OUT_F32) {
                         float *dst = (float *)pr.C + (size_t)row * pr.ldc + col0;
                         if (full_chunk && ((pr.ldc & 3) == 0)) {
