@@ -6,17 +6,18 @@
 // CTAs that loops over sweeps and steps on its own and leaves when its matrix has converged; the
 // CTAs of a group meet at a counter in global memory (bounded spin) instead of at kernel boundaries.
 // Blocks of 32 rows; a step handles n/64 disjoint block pairs (round-robin order) in two phases:
-//   pivot : per pair, the 64 x 64 pivot block is rotated on chip by cyclic Jacobi. The rows live at
-//           64 "positions"; positions (2k, 2k+1) are rotated in every round and a fixed permutation
-//           of the positions between rounds brings new partners together (circle method for the
-//           first step of a sweep, which rotates all pairs of the 64 rows once; a cyclic shift of the
-//           second block's rows in the other steps, which rotates each cross pair once). All
-//           addresses are loop invariants; a round is one thread's instruction stream plus one
-//           block barrier. The accumulated row transform Vt (64 x 64) is published.
+//   pivot : per pair, the 64 x 64 pivot block is rotated on chip by cyclic Jacobi (first step of a sweep: all
+//           2016 pairs of its 64 rows once, in 63 rounds; other steps: the 1024 pairs across its two blocks, in
+//           32 rounds). The block lives in registers (see "pivot phase" below); a round is a rotation per row
+//           pair, two block barriers and a shift of the pairing. The accumulated row transform Vt (64 x 64)
+//           is published. The pivot block of the NEXT step is formed on chip from the matrix before this step's
+//           update (pivot_form), so the chain of pivot solves runs beside the update and never waits for it.
 //   apply : every 64 x 64 block (p, q) of G becomes Vt_p G_pq Vt_q^T (upper triangle computed, mirror
-//           stored), rows of Wt become Vt_p Wt. The 64^3 products run on the tensor cores in split
-//           precision (three TF32 mma products per fp32 product), which keeps fp32 accuracy.
-// G and Wt are stored with a leading dimension padded to a multiple of 64; the padding of G is zero
+//           stored), rows of Wt become Vt_p Wt. The update reads one copy of G and writes the other (G, G2), so
+//           that the pivot CTAs read a matrix nobody writes. The 64^3 products run on the tensor cores in split
+//           precision (three TF32 mma products per fp32 product), which keeps fp32 accuracy; fp32 inputs use the
+//           fp32 units.
+// G, G2 and Wt are stored with a leading dimension padded to a multiple of 64; the padding of G is zero
 // (zero diagonal entries are never rotated), the padding of Wt is the identity.
 #pragma once
 #include "common.cuh"
