@@ -61,9 +61,9 @@ __device__ __forceinline__ void rr_pair(int nb, int step, int t, int &I, int &J)
 }
 
 // Group barrier number `gen` (1, 2, ...) of a group of `ncta` CTAs: every CTA adds one to the arrival
-// counter sync[0]; the last one to arrive publishes `gen` in sync[32] (another cache line, so that
-// the pollers do not slow the arrivals down); the others poll that word. Bounded: returns false when
-// the wait ran out or another CTA flagged an abort.
+// counter sync[0] (release); the last one to arrive publishes `gen` in sync[32] (another cache line, so that
+// the pollers do not slow the arrivals down); the others poll that word (acquire). Bounded: returns false when
+// the wait ran out or another CTA flagged an abort. Data that crosses the barrier is read with L2 loads.
 __device__ __forceinline__ bool group_barrier(unsigned *sync, unsigned gen, unsigned ncta, int *abort_flag,
                                               unsigned limit = SPIN_LIMIT)
 {
@@ -72,21 +72,23 @@ __device__ __forceinline__ bool group_barrier(unsigned *sync, unsigned gen, unsi
     if (threadIdx.x == 0) {
         int ok = 1;
         if (ncta > 1) {
-            __threadfence();
-            const unsigned old = atomicAdd(sync, 1u);
-            volatile unsigned *flag = sync + 32;
+            // release / acquire at GPU scope: the block barrier above orders the CTA's writes before thread 0's
+            // release, the one below orders its acquire before the CTA's later reads
+            unsigned old;
+            asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(old) : "l"(sync) : "memory");
+            unsigned *flag = sync + 32;
             if (old + 1u == gen * ncta) {
-                __threadfence();
-                *flag = gen;
+                asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(flag), "r"(gen) : "memory");
             } else {
                 ok = 0;
                 for (unsigned i = 0; i < limit; ++i) {
-                    if ((int)(*flag - gen) >= 0) { ok = 1; break; }
+                    unsigned v;
+                    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+                    if ((int)(v - gen) >= 0) { ok = 1; break; }
                     if ((i & 1023u) == 1023u && *(volatile int *)abort_flag) break;
                 }
                 if (!ok) *(volatile int *)abort_flag = 1;
             }
-            __threadfence();
         }
         ok_s = ok;
     }
