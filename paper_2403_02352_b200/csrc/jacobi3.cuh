@@ -814,7 +814,7 @@ static inline atp_status launch(atp_ctx *ctx, Batch &jb, float tol_conv, float t
     }
     if (next > total) return ATP_ERR_INVALID_ARG;      // cannot happen: shares sum to at most `total`
     ATP_KERNEL(ctx, "jacobi_init", 0, wsum * 4.0);
-    init_kernel<<<dim3(64, jb.count), 256, 0, ctx->stream>>>(jb, ctx->dev_status);
+    init_kernel<<<dim3(std::max(64, 4 * ctx->sm_count / jb.count), jb.count), 256, 0, ctx->stream>>>(jb, ctx->dev_status);
     ATP_LAUNCHED(ctx);
     int *status = ctx->dev_status;
     int ms = max_sweeps, rn = raise_not_converged ? 1 : 0;
