@@ -539,7 +539,7 @@ __global__ void __launch_bounds__(256) signfix_kernel(const __grid_constant__ Fi
 
 // ------------------------------------------------------------------------------------------------
 struct SeqPlan {
-    SeqDims dims; int rt, np, npanel_L, npanel_d; unsigned *jsync; float *G2, *tpart;
+    SeqDims dims; int rt, np, npanel_L, npanel_d; unsigned *jsync; float *tpart;
     __nv_bfloat16 *Bth, *Btl, *Y2h, *Y2l, *Wth, *Wtl, *Wsh, *Wsl;
     float *oCpart, *oC, *oDpart, *oW; double *ogpart, *ogpart2; unsigned *osync; int ocap;
     __nv_bfloat16 *Yb, *Yl, *Zb, *Zl; float *Y2; float *Y, *Z, *BW, *Wsel, *tsum, *sig, *Cc, *rinv, *G, *Wt, *Vbuf; double *gpart; int *ord, *flags, *conv, *vflag, *needfix; unsigned *maxoff;
@@ -601,7 +601,6 @@ static void plan_basis(Arena &ar, const std::vector<SeqDims> &sd, int d, int ove
             p.Wth = ar.take<__nv_bfloat16>((size_t)p.np * p.np); p.Wtl = ar.take<__nv_bfloat16>((size_t)p.np * p.np);
             p.Wsh = ar.take<__nv_bfloat16>((size_t)std::max(rt, 1) * ldw); p.Wsl = ar.take<__nv_bfloat16>((size_t)std::max(rt, 1) * ldw);
         }
-        p.G2 = ar.take<float>((size_t)p.np * p.np);
         p.jsync = ar.take<unsigned>(64);
         p.needfix = ar.take<int>(std::max(p.dims.r, 1));
         p.maxoff = ar.take<unsigned>(1);
@@ -817,7 +816,7 @@ static atp_status basis_impl(atp_ctx *ctx, const atp_mat *X, const std::vector<S
                 const int ldr = (int)align_up((size_t)std::max(p.rt, 1), 8), ldw = (int)align_up((size_t)std::max(p.dims.r, 1), 8);
                 g.p[k] = GemmProblem{Xb(p), p.Y, p.BW, nullptr, p.rt > 0 ? d : 0, p.rt, p.dims.L, (int)X->ld, p.rt, p.rt, 0};
                 gg.p[k] = GemmProblem{p.BW, p.BW, p.G, nullptr, p.rt, p.rt, p.rt > 0 ? d : 0, p.rt, p.rt, p.np, 0};
-                jb.s[k] = j3::Seq{p.G, p.G2, p.Wt, p.Vbuf, p.vflag, p.jsync, p.rt, p.np, p.np / j3::JB, 0, 0};
+                jb.s[k] = j3::Seq{p.G, p.Wt, p.Vbuf, p.vflag, p.jsync, p.rt, p.np, p.np / j3::JB, 0, 0};
                 fb.s[k] = Fin2Seq{p.G, p.Wt, p.Y, p.sig, p.ord, p.tsum, p.Wsel, p.needfix,
                                   (T *)X_r->data + (size_t)p.dims.rank0 * X_r->ld, (T *)U_r->data + (size_t)p.dims.row0 * U_r->ld,
                                   sigma ? sigma + p.dims.rank0 : nullptr, p.rt, p.dims.r, d, p.dims.L, kBf16 ? ldr : p.rt, (int)X_r->ld, (int)U_r->ld, p.np,

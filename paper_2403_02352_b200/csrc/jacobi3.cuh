@@ -13,11 +13,12 @@
 //           is published. The pivot block of the NEXT step is formed on chip from the matrix before this step's
 //           update (pivot_form), so the chain of pivot solves runs beside the update and never waits for it.
 //   apply : every 64 x 64 block (p, q) of G becomes Vt_p G_pq Vt_q^T (upper triangle computed, mirror
-//           stored), rows of Wt become Vt_p Wt. The update reads one copy of G and writes the other (G, G2), so
-//           that the pivot CTAs read a matrix nobody writes. The 64^3 products run on the tensor cores in split
+//           stored), rows of Wt become Vt_p Wt, both in place. The pivot CTAs of the step read blocks of G as they
+//           were before the update; a counter of fetched pivot blocks holds the first store of every updating
+//           CTA back until they have them on chip. The 64^3 products run on the tensor cores in split
 //           precision (three TF32 mma products per fp32 product), which keeps fp32 accuracy; fp32 inputs use the
 //           fp32 units.
-// G, G2 and Wt are stored with a leading dimension padded to a multiple of 64; the padding of G is zero
+// G and Wt are stored with a leading dimension padded to a multiple of 64; the padding of G is zero
 // (zero diagonal entries are never rotated), the padding of Wt is the identity.
 #pragma once
 #include "common.cuh"
@@ -35,13 +36,11 @@ constexpr int MAXSEQ = 32;        // sequences per launch
 constexpr unsigned SPIN_LIMIT = 1u << 22;
 
 struct Seq {
-    float *G, *G2, *Wt, *Vbuf;    // G, G2, Wt: np x np (ld = np); G2: scratch, the update of a step reads one
-                                  // copy of the matrix and writes the other; Vbuf: 2 x npairs x 64 x 64 (by
-                                  // step parity)
+    float *G, *Wt, *Vbuf;         // G, Wt: np x np (ld = np); Vbuf: 2 x npairs x 64 x 64 (by step parity)
     int *vflag;                   // 2 x npairs: the pair rotated in this step
     unsigned *sync;               // 64 words. [0]: arrivals at the group barrier (monotonic); [32]: last
                                   // barrier completed; [1..4]: largest scaled off-diagonal entry of a
-                                  // sweep, slot sweep % 4; [5]: sweeps used; [16..17]: work tickets of the update, by step parity
+                                  // sweep, slot sweep % 4; [5]: sweeps used; [16..17]: work tickets of the update, [20..21]: pivot blocks fetched, both by step parity
     int n, np, nb;                // size, padded size (multiple of 64), number of 32-row blocks (even)
     int cta0, ncta;               // the group of CTAs that owns this sequence
 };
@@ -402,7 +401,7 @@ __device__ __forceinline__ void product64_fma(const float *As, const float *Bs, 
 // in three 64^3 products: [W1 X11; W2 X22] and W1 X12 first, then the multiplication by [W1; W2]^T from the
 // right. The result lands in As = sm (stride LDP). So the chain of pivot solves never waits for the update.
 template <bool TENSOR>
-__device__ void pivot_form(float *sm, const Seq &sq, const float *Gsrc, const float *Vcur, int step, int p1, int h1, int f1, int p2, int h2, int f2)
+__device__ void pivot_form(float *sm, const Seq &sq, const float *Gsrc, const float *Vcur, int step, int p1, int h1, int f1, int p2, int h2, int f2, unsigned *fetched)
 {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     float *Wc = sm, *S1 = sm + SLOT, *S2 = sm + 2 * SLOT, *S3 = sm + 3 * SLOT;
@@ -424,6 +423,7 @@ __device__ void pivot_form(float *sm, const Seq &sq, const float *Gsrc, const fl
         *(float4 *)(S3 + i * LDB + c) = __ldcg((const float4 *)(Gsrc + r1 + glob_of_loc(I2, J2, c)));
     }
     __syncthreads();
+    if (tid == 0) atomicAdd(fetched, 1u);                       // the old blocks are on chip: the update may overwrite them
     const int m0 = (warp & 3) * 16, n0 = (warp >> 2) * 32;
     const bool up = m0 < JB;
     const bool on_tensor = TENSOR;
@@ -467,8 +467,9 @@ __device__ void pivot_form(float *sm, const Seq &sq, const float *Gsrc, const fl
 }
 
 // The update of a step is cut into strips. A strip of G: blocks (p, q0 .. q0 + cnt - 1) of the upper triangle,
-// read from Gsrc and written (with their mirrors) to Gdst, also when neither pair was rotated; a strip of Wt: the
-// rows of pair p, column chunks c0 .. c0 + cnt - 1 of 64, in place. Along a strip Vt_p stays in shared memory and
+// updated in place together with their mirrors; a strip of Wt: the rows of pair p, column chunks
+// c0 .. c0 + cnt - 1 of 64, in place. The pivot CTAs of the same step read blocks of G as they were before the
+// update: before its first store of a step a CTA makes sure that all of them have fetched theirs (Fetched). Along a strip Vt_p stays in shared memory and
 // the next block is fetched into registers while the current one is multiplied. Short strips win at r~ = 2112: with
 // 296 CTAs a step has only a few items per CTA, and the last ones to finish set the time of the step (strips of
 // 2 + 3 blocks: 39.9 us per step, 1 + 2: 37.3 us).
@@ -485,8 +486,31 @@ __device__ __forceinline__ void store_tile_acc(float *dst, int ld, int m0, int n
     }
 }
 
+struct Fetched {
+    const unsigned *count; unsigned target; int *abort_flag;   // counter of pivot blocks fetched in this step, its final value
+    bool ok;                                                    // already seen complete by this CTA
+};
+// Block-uniform, bounded: false when the wait ran out.
+__device__ bool wait_fetched(Fetched &f)
+{
+    if (f.ok) return true;
+    __shared__ int ok_s;
+    if (threadIdx.x == 0) {
+        int ok = 0;
+        for (unsigned i = 0; i < SPIN_LIMIT; ++i) {
+            if (*(volatile const unsigned *)f.count >= f.target) { ok = 1; break; }
+            if ((i & 1023u) == 1023u && *(volatile int *)f.abort_flag) break;
+        }
+        if (!ok) *(volatile int *)f.abort_flag = 1;
+        ok_s = ok;
+    }
+    __syncthreads();
+    f.ok = ok_s != 0;
+    return f.ok;
+}
+
 template <bool TENSOR>
-__device__ void g_strip(float *sm, const Seq &sq, const float *Gsrc, float *Gdst, const float *Vbuf, const int *vflag, int step, int p, int q0, int cnt)
+__device__ bool g_strip(float *sm, const Seq &sq, float *G, const float *Vbuf, const int *vflag, int step, int p, int q0, int cnt, Fetched &fetched)
 {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     const int m0 = (warp & 3) * 16, n0 = (warp >> 2) * 32, np = sq.np;
@@ -501,7 +525,7 @@ __device__ void g_strip(float *sm, const Seq &sq, const float *Gsrc, float *Gdst
 #pragma unroll
         for (int it = 0; it < 4; ++it) {
             const int f = tid + it * NT, i = f >> 4, c = (f & 15) * 4;
-            x[it] = __ldcg((const float4 *)(Gsrc + (size_t)glob_of_loc(Ip, Jp, i) * np + glob_of_loc(Iq, Jq, c)));
+            x[it] = __ldcg((const float4 *)(G + (size_t)glob_of_loc(Ip, Jp, i) * np + glob_of_loc(Iq, Jq, c)));
         }
     };
     if (fp) {
@@ -516,16 +540,7 @@ __device__ void g_strip(float *sm, const Seq &sq, const float *Gsrc, float *Gdst
         const int q = q0 + j, fq = __ldcg(vflag + q);
         int Iq, Jq;
         rr_pair(sq.nb, step, q, Iq, Jq);
-        if (!fp && !fq) {                                        // unchanged block: both mirror copies move over
-#pragma unroll
-            for (int it = 0; it < 4; ++it) {
-                const int f = tid + it * NT, i = f >> 4, c = (f & 15) * 4;
-                *(float4 *)(Gdst + (size_t)glob_of_loc(Ip, Jp, i) * np + glob_of_loc(Iq, Jq, c)) = x[it];
-                if (q != p) {
-                    const size_t b = (size_t)glob_of_loc(Iq, Jq, i) * np + glob_of_loc(Ip, Jp, c);
-                    *(float4 *)(Gdst + b) = __ldcg((const float4 *)(Gsrc + b));
-                }
-            }
+        if (!fp && !fq) {                                        // unchanged block
             if (j + 1 < cnt) fetch(q + 1);
             continue;
         }
@@ -553,19 +568,21 @@ __device__ void g_strip(float *sm, const Seq &sq, const float *Gsrc, float *Gdst
             if (TENSOR) product64<true>(Tm, Vq, LDA, m0, n0, acc);
             else product64_fma<true>(Tm, Vq, LDA, m0, n0, acc);
         }
+        if (!wait_fetched(fetched)) return false;
         const int gr0 = glob_of_loc(Ip, Jp, m0 + g), gr1 = glob_of_loc(Ip, Jp, m0 + g + 8);
 #pragma unroll
         for (int nt = 0; nt < 4; ++nt) {
             const int gc = glob_of_loc(Iq, Jq, n0 + nt * 8 + 2 * t);     // gc, gc + 1 are contiguous
-            *(float2 *)(Gdst + (size_t)gr0 * np + gc) = make_float2(acc[nt][0], acc[nt][1]);
-            *(float2 *)(Gdst + (size_t)gr1 * np + gc) = make_float2(acc[nt][2], acc[nt][3]);
+            *(float2 *)(G + (size_t)gr0 * np + gc) = make_float2(acc[nt][0], acc[nt][1]);
+            *(float2 *)(G + (size_t)gr1 * np + gc) = make_float2(acc[nt][2], acc[nt][3]);
             if (q != p) {                                        // mirror block
-                Gdst[(size_t)gc * np + gr0] = acc[nt][0]; Gdst[(size_t)(gc + 1) * np + gr0] = acc[nt][1];
-                Gdst[(size_t)gc * np + gr1] = acc[nt][2]; Gdst[(size_t)(gc + 1) * np + gr1] = acc[nt][3];
+                G[(size_t)gc * np + gr0] = acc[nt][0]; G[(size_t)(gc + 1) * np + gr0] = acc[nt][1];
+                G[(size_t)gc * np + gr1] = acc[nt][2]; G[(size_t)(gc + 1) * np + gr1] = acc[nt][3];
             }
         }
         __syncthreads();                                         // tiles are reused by the next block
     }
+    return true;
 }
 
 template <bool TENSOR>
@@ -621,7 +638,7 @@ __host__ __device__ __forceinline__ int strips_of_g(int npairs)
     return n;
 }
 template <bool TENSOR>
-__device__ void apply_item(float *sm, const Seq &sq, const float *Gsrc, float *Gdst, const float *Vbuf, const int *vflag, int step, int idx, int npairs, int items_g, int nw)
+__device__ bool apply_item(float *sm, const Seq &sq, const float *Vbuf, const int *vflag, int step, int idx, int npairs, int items_g, int nw, Fetched &fetched)
 {
     if (idx < items_g) {
         int p = 0;
@@ -631,12 +648,13 @@ __device__ void apply_item(float *sm, const Seq &sq, const float *Gsrc, float *G
             idx -= n; ++p;
         }
         const int q0 = p + idx * SEG_G;
-        g_strip<TENSOR>(sm, sq, Gsrc, Gdst, Vbuf, vflag, step, p, q0, min(SEG_G, npairs - q0));
+        return g_strip<TENSOR>(sm, sq, sq.G, Vbuf, vflag, step, p, q0, min(SEG_G, npairs - q0), fetched);
     } else {
         idx -= items_g;
         const int nseg = (nw + SEG_W - 1) / SEG_W, p = idx / nseg, c0 = (idx - p * nseg) * SEG_W;
         wt_strip<TENSOR>(sm, sq, Vbuf, vflag, step, p, c0, min(SEG_W, nw - c0));
     }
+    return true;
 }
 
 // ---- the kernel --------------------------------------------------------------------------------
@@ -646,8 +664,10 @@ __device__ void apply_item(float *sm, const Seq &sq, const float *Gsrc, float *G
 //   1. the pivot solves of the NEXT step (a few CTAs; this chain of rotation rounds is the critical path), and
 //   2. the update of this step, its blocks handed out by a ticket counter so that the pivot CTAs join in when
 //      they are through,
-// followed by one group barrier. Vt and the rotated-flags are double buffered by step parity, because the
-// pivots of step s+1 publish while the update of step s still reads.
+// followed by one group barrier. The update works in place; before its first store of a step a CTA waits
+// (as a rule not at all: it has a block to load and multiply first) until every pivot CTA has fetched the
+// blocks it forms its pivot block from. Vt and the rotated-flags are double buffered by step parity, because
+// the pivots of step s+1 publish while the update of step s still reads.
 // status[0]: sticky device status word of the context; status[1]: abort flag of bounded waits.
 constexpr int MAXPAIRS = 72;                  // np <= 4608
 
@@ -670,7 +690,6 @@ jacobi_persistent_kernel(const __grid_constant__ Batch batch, float tol_conv, fl
     const int nsteps = sq.nb - 1;
     int *abort_flag = status + 1;
     unsigned gen = 0, gstep = 0;
-    int gsel = 0;                                                 // which copy of G is current
     bool converged = false, alive = true;
 
     // rotates the block held in shared memory for pair pr of (sweep, step); publishes to parity par
@@ -702,11 +721,13 @@ jacobi_persistent_kernel(const __grid_constant__ Batch batch, float tol_conv, fl
             const int nstep = step + 1 == nsteps ? 0 : step + 1, nsweep = sweep + (step + 1 == nsteps ? 1 : 0);
             const float *Vcur = sq.Vbuf + (size_t)par * npairs * BLK * BLK;
             const int *fcur = sq.vflag + par * npairs;
-            const float *Gsrc = gsel ? sq.G2 : sq.G;
-            float *Gdst = gsel ? sq.G : sq.G2;
-            // a step in which no pair was rotated leaves the matrix where it is: no update, no copy
+            // a step in which no pair was rotated needs no update
             const bool any_rot = __syncthreads_or(tid < npairs && __ldcg(fcur + tid) != 0) != 0;
-            if (rank == 0 && tid == 0) sq.sync[16 + (par ^ 1)] = 0u;      // tickets of the next step
+            if (rank == 0 && tid == 0) {                                  // tickets and fetch count of the next step
+                sq.sync[16 + (par ^ 1)] = 0u;
+                sq.sync[20 + (par ^ 1)] = 0u;
+            }
+            Fetched fetched{sq.sync + 20 + par, has_next ? (unsigned)npairs : 0u, abort_flag, false};
             // 1. pivots of the next step
             if (has_next && rank < npairs) {
                 if (tid < npairs) {
@@ -720,8 +741,11 @@ jacobi_persistent_kernel(const __grid_constant__ Batch batch, float tol_conv, fl
                     rr_pair(sq.nb, nstep, pr, I2, J2);
                     const int p1 = pair_of[I2] >> 1, h1 = pair_of[I2] & 1, p2 = pair_of[J2] >> 1, h2 = pair_of[J2] & 1;
                     const int f1 = __ldcg(fcur + p1), f2 = __ldcg(fcur + p2);
-                    if (!f1 && !f2) pivot_load(j3sm, Gsrc, sq.np, I2, J2);
-                    else pivot_form<TENSOR>(j3sm, sq, Gsrc, Vcur, step, p1, h1, f1, p2, h2, f2);
+                    if (!f1 && !f2) {
+                        pivot_load(j3sm, sq.G, sq.np, I2, J2);
+                        __syncthreads();
+                        if (tid == 0) atomicAdd(sq.sync + 20 + par, 1u);
+                    } else pivot_form<TENSOR>(j3sm, sq, sq.G, Vcur, step, p1, h1, f1, p2, h2, f2, sq.sync + 20 + par);
                     pivot_finish(nsweep, nstep, pr, par ^ 1);
                 }
             }
@@ -729,11 +753,10 @@ jacobi_persistent_kernel(const __grid_constant__ Batch batch, float tol_conv, fl
             if (tid == 0) ticket_s = any_rot ? (int)atomicAdd(sq.sync + 16 + par, 1u) : total;
             __syncthreads();
             int t = ticket_s;
-            if (any_rot) gsel ^= 1;
-            while (t < total) {
+            while (t < total && alive) {
                 int tn = 0;
                 if (tid == 0) tn = (int)atomicAdd(sq.sync + 16 + par, 1u);
-                apply_item<TENSOR>(j3sm, sq, Gsrc, Gdst, Vcur, fcur, step, t, npairs, items_g, nw);
+                alive = apply_item<TENSOR>(j3sm, sq, Vcur, fcur, step, t, npairs, items_g, nw, fetched);
                 __syncthreads();
                 if (tid == 0) ticket_s = tn;
                 __syncthreads();
@@ -744,11 +767,6 @@ jacobi_persistent_kernel(const __grid_constant__ Batch batch, float tol_conv, fl
         if (!alive) break;
         const float mo = __uint_as_float(*(volatile unsigned *)(sq.sync + 1 + sweep % 4));
         if (mo <= tol_conv) { converged = true; ++sweep; break; }
-    }
-    if (alive && gsel) {                                          // the last update wrote G2: the result goes back to G
-        const size_t n4 = (size_t)sq.np * sq.np / 4;
-        for (size_t e = (size_t)rank * NT + tid; e < n4; e += (size_t)sq.ncta * NT)
-            ((float4 *)sq.G)[e] = __ldcg((const float4 *)sq.G2 + e);
     }
     if (rank == 0 && tid == 0) {
         if (!alive) raise_status(status, ATP_ERR_TIMEOUT);
