@@ -97,7 +97,7 @@ ALT_INNER = 2        # rounds per component of Algorithm 1, as the paper runs it
 
 # DRAM bytes (read + write) of one launch of the dominant kernels, from one ncu pass on the same command
 # (profiles/ncu_metrics_llama7b_bf16_r2048.md); other workloads / kernels: no capture, null.
-NCU_DRAM_BYTES_PER_LAUNCH = {("llama7b_bf16", 2048, "jacobi_persistent"): 1617.1e6,
+NCU_DRAM_BYTES_PER_LAUNCH = {("llama7b_bf16", 2048, "jacobi_persistent"): 33.7e6,
                              ("llama7b_bf16", 2048, "orth_persistent"): 67.2e6}
 
 
