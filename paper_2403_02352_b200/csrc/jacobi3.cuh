@@ -837,7 +837,8 @@ static inline atp_status launch(atp_ctx *ctx, Batch &jb, float tol_conv, float t
     int *status = ctx->dev_status;
     int ms = max_sweeps, rn = raise_not_converged ? 1 : 0;
     void *args[] = {(void *)&jb, (void *)&tol_conv, (void *)&tol_rot, (void *)&ms, (void *)&rn, (void *)&status};
-    ATP_KERNEL(ctx, "jacobi_persistent", 0, 0);
+    // bytes: one read and one write of G and Wt (what the kernel must move at least; it runs from L2)
+    ATP_KERNEL(ctx, "jacobi_persistent", 0, wsum * 16.0);
     ATP_CUDA_OK(ctx, cudaLaunchCooperativeKernel((const void *)jacobi_persistent_kernel<TENSOR>, dim3(next), dim3(NT), args, SMEM_BYTES, ctx->stream));
     ATP_LAUNCHED(ctx);
     return ATP_OK;

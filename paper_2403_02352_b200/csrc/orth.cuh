@@ -461,7 +461,8 @@ static inline atp_status launch(atp_ctx *ctx, Batch &ob, int reps, uint64_t seed
     ATP_LAUNCHED(ctx);
     int *status = ctx->dev_status;
     void *args[] = {(void *)&ob, (void *)&reps, (void *)&seed, (void *)&status};
-    ATP_KERNEL(ctx, "orth_persistent", 0, 0);
+    // bytes: one read and one write of every iterate
+    ATP_KERNEL(ctx, "orth_persistent", 0, wsum * 8.0);
     ATP_CUDA_OK(ctx, cudaLaunchCooperativeKernel((const void *)orth_persistent_kernel<TENSOR>, dim3(next), dim3(NT), args, SMEM_BYTES, ctx->stream));
     ATP_LAUNCHED(ctx);
     return ATP_OK;
