@@ -25,7 +25,7 @@ struct Problem {
     CUtensorMap ta, ta2, tb, tb2; // ta2 / tb2 only with a split A / B
     void *C; void *C2; const float *D;
     int M, N, K, ldc, ldd;
-    int tile0, tiles_n;          // first linear tile index of this problem, tiles along N
+    int tile0, tiles_n, tiles_m; // first linear tile index of this problem, tiles along N and along M
 };
 struct Batch {
     Problem p[MAX_PROB];
@@ -173,7 +173,11 @@ gemm_tc_kernel(const __grid_constant__ Batch batch, GemmEpi epi, int *dev_status
     for (int i = 1; i < batch.count; ++i) if (tile >= batch.p[i].tile0) pi = i;
     const Problem &pr = batch.p[pi];
     const int lt = tile - pr.tile0;
-    const int m0 = (lt / pr.tiles_n) * BM, n0 = (lt % pr.tiles_n) * BN;
+    // Where N is much larger than M, consecutive CTAs walk along M: they share a tile of the large operand B, and
+    // the operand that is re-read from L2 is the small one, A (a 4096 x 2048 x 11008 product read 1 GB
+    // from DRAM in row-major tile order: its 45 MB B operand was evicted by the streamed epilogue operand).
+    const bool along_m = pr.tiles_n > 2 * pr.tiles_m;
+    const int m0 = (along_m ? lt % pr.tiles_m : lt / pr.tiles_n) * BM, n0 = (along_m ? lt / pr.tiles_m : lt % pr.tiles_n) * BN;
     const int num_kt = (pr.K + BK - 1) / BK;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -401,6 +405,7 @@ static atp_status launch(atp_ctx *ctx, const std::vector<HostProblem> &probs, Ge
             if (!ok) return ATP_ERR_INVALID_ARG;
             p.C = h.C; p.C2 = h.C2; p.D = h.D; p.M = h.M; p.N = h.N; p.K = h.K; p.ldc = h.ldc; p.ldd = h.ldd;
             p.tiles_n = ceil_div(h.N, BN);
+            p.tiles_m = ceil_div(h.M, BM);
             p.tile0 = b.total_tiles;
             b.total_tiles += ceil_div(h.M, BM) * p.tiles_n;
             b.count++;
